@@ -1,0 +1,180 @@
+/*
+ * sdnn - sparse deep neural network SGD hot path on one NVIDIA B200 (sm_100a).
+ *
+ * C ABI of the shared library libsdnn.so.  The operations are those of the paper
+ * "Partitioning Sparse Deep Neural Networks for Scalable Training and Inference"
+ * (ICS '21), Section 3.2 and Algorithm 1, for a network of L square layers of N
+ * neurons whose weight matrices W^k are sparse:
+ *
+ *   forward   x^k = f(W^k x^{k-1} + b^k),  k = 1..L          (feedforward equation)
+ *   output    delta^L = grad_{x^L} J (.) f'(z^L)             (final-layer gradient equation)
+ *   backward  delta^{k-1} = (W^k)^T delta^k (.) f'(z^{k-1})  (recursive formula)
+ *   update    W^k(j,i) <- W^k(j,i) - eta * delta^k(j) x^{k-1}(i)  on stored entries only
+ *                                                            (gradient update rule)
+ *
+ * W^k(j,i) is the weight of the link from neuron i of layer k to neuron j of
+ * layer k+1: CSR row j of W^k lists the incoming links of output neuron j.
+ * f(z) = min(max(z, 0), clamp); f'(z) = 1 for 0 < z < clamp, else 0.
+ * J = 1/(2B) sum_b ||x^L_b - y_b||^2 (mean squared error over a minibatch of B
+ * inputs); a minibatch step is exact minibatch SGD: one delta per input, the
+ * gradient averaged over the batch (B = 1 is Algorithm 1 verbatim).  The
+ * transposed product of layer k uses W^k as it was before its own update, as in
+ * Algorithm 1 (line computing delta^{k-1} precedes the update line).  delta^0 is
+ * never formed.
+ *
+ * Conventions
+ *  - Every function returns an sdnn_status (0 = success, negative = error) and
+ *    never throws or aborts; sdnn_last_error() gives a message for the last failure.
+ *  - The caller keeps ownership of every array it passes.  The handle owns all
+ *    device memory it allocates and frees it in sdnn_destroy().
+ *  - "host" / "device" below says where a pointer must live.  Device pointers must
+ *    be on the handle's device.  All arithmetic is fp32 (fp32 accumulation, FMA).
+ *  - Calls are issued on cfg->cuda_stream; a call that returns a scalar to the host
+ *    (loss_out, nz_total_out) or uses host buffers synchronises that stream before
+ *    returning, otherwise it returns after enqueueing.
+ *  - A handle is not thread-safe.  There is no CPU fallback: without a CUDA device
+ *    creation fails with SDNN_ERR_CUDA.
+ */
+#ifndef SDNN_H
+#define SDNN_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sdnn sdnn_t; /* opaque */
+
+typedef enum {
+    SDNN_OK = 0,
+    SDNN_ERR_INVALID_ARG = -1,   /* NULL where not allowed, size out of range, batch > max_batch, capacity too small */
+    SDNN_ERR_BAD_CSR = -2,       /* row_ptr not monotone from 0, column out of [0,N), unsorted/duplicate, non-finite value */
+    SDNN_ERR_OOM = -3,           /* device or host allocation failed */
+    SDNN_ERR_CUDA = -4,          /* CUDA runtime error (message in sdnn_last_error) */
+    SDNN_ERR_STATE = -5,         /* call not valid in the handle's state (e.g. train step on an inference handle) */
+    SDNN_ERR_UNIMPLEMENTED = -6
+} sdnn_status;
+
+/* cfg->flags */
+#define SDNN_FLAG_BWD_ATOMICS 0x01u /* backward product by scatter with vector reductions into L2 (one CSR pass)   */
+#define SDNN_FLAG_BWD_CSC     0x02u /* backward product by gather through a transposed index (no atomics)          */
+#define SDNN_FLAG_KEEP_DEBUG  0x04u /* train handles: also store delta^k and the gradient G^k of the last step     */
+#define SDNN_FLAG_SKIP_DEAD   0x08u /* allow data-dependent skipping (dead inputs, all-zero delta rows); default   */
+                                    /* is dense mode: every layer streams its weights and processes every input    */
+#define SDNN_FLAG_NO_GRAPH    0x10u /* launch the layer chain kernel by kernel instead of through a CUDA graph     */
+
+typedef struct {
+    int32_t  activation;   /* 0 = clamped ReLU (the only one implemented) */
+    float    clamp;        /* upper clamp of the activation, e.g. 32.0f; must be > 0 */
+    int32_t  max_batch;    /* train: largest minibatch B; inference: batch tile (inputs processed together) */
+    int32_t  train;        /* 0: inference only (no stored activations); 1: sdnn_train_step allowed */
+    int32_t  update_bias;  /* 1: b^k <- b^k - eta * mean_b delta^k_b (bias read as a column of W^k); 0: bias frozen */
+    uint32_t flags;        /* SDNN_FLAG_* */
+    void*    cuda_stream;  /* cudaStream_t to issue work on; NULL = default stream */
+    int32_t  device;       /* CUDA device ordinal; -1 = the current device */
+} sdnn_config;
+
+/*
+ * Problem statement of Section 3.2 / "Require" line of Algorithm 1: a network {W^k}, k = 1..L.
+ * Creates a handle from per-layer CSR arrays (all host pointers; copied, caller keeps them).
+ *   row_ptr[l] -> int32[n_neurons+1], monotone, row_ptr[l][0] == 0
+ *   col_idx[l] -> int32[nnz_l], in [0,n_neurons), strictly ascending within each row
+ *   values[l]  -> float[nnz_l], finite (explicit zeros are legal stored entries and stay in the pattern)
+ *   bias[l]    -> float[n_neurons], finite
+ * Errors: INVALID_ARG (NULL, sizes <= 0, bad cfg), BAD_CSR, OOM, CUDA.  On error *out is NULL.
+ */
+int sdnn_create(sdnn_t** out, int32_t n_layers, int32_t n_neurons,
+                const int32_t* const* row_ptr, const int32_t* const* col_idx,
+                const float* const* values, const float* const* bias, const sdnn_config* cfg);
+
+/*
+ * Same network, loaded layer by layer so that the host never holds more than one layer:
+ * sdnn_create_deferred reserves device memory for nnz_per_layer[l] stored entries per layer
+ * (host array of n_layers int64), sdnn_load_layer validates and uploads one layer (0-based,
+ * any order, each exactly once), sdnn_finalize makes the handle usable.  sdnn_create is
+ * these three in sequence.  Calling infer/train before finalize gives SDNN_ERR_STATE.
+ */
+int sdnn_create_deferred(sdnn_t** out, int32_t n_layers, int32_t n_neurons,
+                         const int64_t* nnz_per_layer, const sdnn_config* cfg);
+int sdnn_load_layer(sdnn_t* h, int32_t layer, const int32_t* row_ptr, const int32_t* col_idx,
+                    const float* values, const float* bias);
+int sdnn_finalize(sdnn_t* h);
+
+/*
+ * Inference (feedforward equation applied L times; minibatch form X^k = f(W^k X^{k-1}) of
+ * Section 5's Discussion; inputs are independent of one another).
+ *   x0            device float[n_inputs][N], row-major (one input vector per row)
+ *   y_out         device float[n_inputs][N] = x^L per input, or NULL
+ *   nz_count_out  device int32[n_inputs]: number of nonzero entries of x^L per input, or NULL
+ *   nz_index_out  device int32[nz_index_capacity]: for input 0, 1, ... in turn, the ascending
+ *                 neuron ids i with x^L(i) != 0, concatenated; or NULL
+ *   nz_total_out  host int64*: total number of ids (sum of counts), or NULL
+ * The batch is processed in tiles of cfg.max_batch inputs.  If nz_index_out is given and the
+ * capacity is too small, only the ids at positions below the capacity are written, *nz_total_out
+ * (if given) holds the needed capacity and the call returns SDNN_ERR_INVALID_ARG; y_out and
+ * nz_count_out are still valid.  n_inputs == 0 is a valid no-op.
+ */
+int sdnn_infer_batch(sdnn_t* h, const float* x0, int64_t n_inputs, float* y_out,
+                     int32_t* nz_count_out, int32_t* nz_index_out, int64_t nz_index_capacity,
+                     int64_t* nz_total_out);
+
+/* Same call with every array in HOST memory (pinned or pageable); the library stages the
+ * copies itself, tile by tile, and returns when the outputs are in place. */
+int sdnn_infer_batch_host(sdnn_t* h, const float* x0, int64_t n_inputs, float* y_out,
+                          int32_t* nz_count_out, int32_t* nz_index_out, int64_t nz_index_capacity,
+                          int64_t* nz_total_out);
+
+/*
+ * One minibatch SGD step (Algorithm 1 body for a batch of B inputs): forward through all
+ * layers, output gradient, then for k = L..1 the transposed product, the masked gradient and
+ * the in-place weight update, fused into one pass over the stored entries of each layer.
+ *   x0, target  device float[B][N], row-major;  1 <= B <= cfg.max_batch
+ *   eta         learning rate
+ *   loss_out    host float*: J before the update, or NULL (no synchronisation then)
+ * Needs cfg.train = 1 (else SDNN_ERR_STATE).  Weights persist across calls.
+ */
+int sdnn_train_step(sdnn_t* h, const float* x0, const float* target, int32_t B, float eta,
+                    float* loss_out);
+
+/* Same step with x0 and target in HOST memory; copies are staged through pinned buffers. */
+int sdnn_train_step_host(sdnn_t* h, const float* x0, const float* target, int32_t B, float eta,
+                         float* loss_out);
+
+/*
+ * Current parameters of one layer (0-based), in the caller's original CSR order.
+ *   values_out  host float[nnz_l], or NULL;   bias_out  host float[N], or NULL
+ * Synchronises the stream.  Creating a new handle from these arrays resumes training.
+ */
+int sdnn_get_weights(sdnn_t* h, int32_t layer, float* values_out, float* bias_out);
+
+/*
+ * Inspection of the last train step (tests, diagnostics).  All outputs are host arrays,
+ * input-major like x0: out[b*N + i].  layer is the paper's index k.
+ *   sdnn_get_activations: x^k of the last step, k = 0..L                         float[B][N]
+ *   sdnn_get_delta:       delta^k of the last step, k = 1..L  (needs KEEP_DEBUG) float[B][N]
+ *   sdnn_get_gradient:    G^k = (1/B) sum_b delta^k_b (x) x^{k-1}_b on the stored
+ *                         entries, CSR order, k = 1..L        (needs KEEP_DEBUG) float[nnz_k]
+ * SDNN_ERR_STATE if no step has run or the flag is missing.
+ */
+int sdnn_get_activations(sdnn_t* h, int32_t layer, float* out);
+int sdnn_get_delta(sdnn_t* h, int32_t layer, float* out);
+int sdnn_get_gradient(sdnn_t* h, int32_t layer, float* out);
+
+/* Counters since creation: kernels launched by this handle (graph nodes count one each);
+ * device bytes it holds. */
+int64_t sdnn_kernel_launches(const sdnn_t* h);
+int64_t sdnn_device_bytes(const sdnn_t* h);
+
+/* Per-layer liveness of the most recent sdnn_infer_batch tile run with SDNN_FLAG_SKIP_DEAD:
+ * live_inputs_out host int32[L] = inputs still alive after each layer.  SDNN_ERR_STATE otherwise. */
+int sdnn_get_liveness(sdnn_t* h, int32_t* live_inputs_out);
+
+void sdnn_destroy(sdnn_t* h);                 /* NULL is a no-op */
+const char* sdnn_last_error(const sdnn_t* h); /* h may be NULL: last creation error of this thread */
+const char* sdnn_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SDNN_H */

@@ -1,0 +1,9 @@
+"""B200-native sparse-DNN SGD hot path (forward, backward, masked update) behind a C ABI.
+
+`binding` wraps libsdnn.so one-to-one; `build` compiles it.  Importing this package does not
+load the library; the first call does, and raises if it has not been built.
+"""
+from .binding import (  # noqa: F401
+    SdnnError, Sdnn, load_library, exported_symbols,
+    FLAG_BWD_ATOMICS, FLAG_BWD_CSC, FLAG_KEEP_DEBUG, FLAG_SKIP_DEAD, FLAG_NO_GRAPH,
+)

@@ -1,0 +1,211 @@
+"""ctypes binding of libsdnn.so: argument marshalling only, one Python method per C entry point.
+
+Every step of the path runs inside the library's CUDA kernels.  There is no fallback: if the
+library is missing or no CUDA device is present, calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsdnn.so")
+
+FLAG_BWD_ATOMICS, FLAG_BWD_CSC, FLAG_KEEP_DEBUG, FLAG_SKIP_DEAD, FLAG_NO_GRAPH = 0x01, 0x02, 0x04, 0x08, 0x10
+
+STATUS = {0: "SDNN_OK", -1: "SDNN_ERR_INVALID_ARG", -2: "SDNN_ERR_BAD_CSR", -3: "SDNN_ERR_OOM", -4: "SDNN_ERR_CUDA",
+          -5: "SDNN_ERR_STATE", -6: "SDNN_ERR_UNIMPLEMENTED"}
+
+
+class SdnnConfig(ctypes.Structure):
+    _fields_ = [("activation", ctypes.c_int32), ("clamp", ctypes.c_float), ("max_batch", ctypes.c_int32),
+                ("train", ctypes.c_int32), ("update_bias", ctypes.c_int32), ("flags", ctypes.c_uint32),
+                ("cuda_stream", ctypes.c_void_p), ("device", ctypes.c_int32)]
+
+
+class SdnnError(RuntimeError):
+    def __init__(self, code: int, message: str):
+        super().__init__(f"{STATUS.get(code, code)}: {message}")
+        self.code = code
+        self.message = message
+
+
+_vp, _i32, _i64, _f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float
+_PROTOS = {
+    "sdnn_create": (ctypes.c_int, [ctypes.POINTER(_vp), _i32, _i32, _vp, _vp, _vp, _vp, ctypes.POINTER(SdnnConfig)]),
+    "sdnn_create_deferred": (ctypes.c_int, [ctypes.POINTER(_vp), _i32, _i32, _vp, ctypes.POINTER(SdnnConfig)]),
+    "sdnn_load_layer": (ctypes.c_int, [_vp, _i32, _vp, _vp, _vp, _vp]),
+    "sdnn_finalize": (ctypes.c_int, [_vp]),
+    "sdnn_infer_batch": (ctypes.c_int, [_vp, _vp, _i64, _vp, _vp, _vp, _i64, ctypes.POINTER(_i64)]),
+    "sdnn_infer_batch_host": (ctypes.c_int, [_vp, _vp, _i64, _vp, _vp, _vp, _i64, ctypes.POINTER(_i64)]),
+    "sdnn_train_step": (ctypes.c_int, [_vp, _vp, _vp, _i32, _f32, ctypes.POINTER(_f32)]),
+    "sdnn_train_step_host": (ctypes.c_int, [_vp, _vp, _vp, _i32, _f32, ctypes.POINTER(_f32)]),
+    "sdnn_get_weights": (ctypes.c_int, [_vp, _i32, _vp, _vp]),
+    "sdnn_get_activations": (ctypes.c_int, [_vp, _i32, _vp]),
+    "sdnn_get_delta": (ctypes.c_int, [_vp, _i32, _vp]),
+    "sdnn_get_gradient": (ctypes.c_int, [_vp, _i32, _vp]),
+    "sdnn_get_liveness": (ctypes.c_int, [_vp, _vp]),
+    "sdnn_kernel_launches": (_i64, [_vp]),
+    "sdnn_device_bytes": (_i64, [_vp]),
+    "sdnn_destroy": (None, [_vp]),
+    "sdnn_last_error": (ctypes.c_char_p, [_vp]),
+    "sdnn_version": (ctypes.c_char_p, []),
+}
+
+_lib = None
+
+
+def exported_symbols():
+    """Names the header declares (and the library must export)."""
+    return sorted(_PROTOS)
+
+
+def load_library(path: str | None = None):
+    """dlopen libsdnn.so and attach prototypes.  Raises if the library has not been built."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or LIB_PATH
+    if not os.path.exists(p):
+        raise SdnnError(-4, f"{p} not found: build it first (python -m paper_2104_11805_b200.build); "
+                            "there is no CPU fallback")
+    lib = ctypes.CDLL(p)
+    for name, (res, args) in _PROTOS.items():
+        fn = getattr(lib, name)          # AttributeError if a declared symbol is not exported
+        fn.restype, fn.argtypes = res, args
+    if path is None:
+        _lib = lib
+    return lib
+
+
+def _np(a, dtype):
+    return np.ascontiguousarray(a, dtype=dtype)
+
+
+def _addr(x):
+    """Device or host address of a torch tensor / numpy array / int / None."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if isinstance(x, np.ndarray):
+        return x.ctypes.data
+    return x.data_ptr()      # torch tensor
+
+
+class Sdnn:
+    """Owns one sdnn_t handle.  Method names mirror the C entry points (sdnn_ prefix dropped)."""
+
+    def __init__(self, handle, n_layers, n_neurons, nnz, lib):
+        self._h, self.n_layers, self.n_neurons, self.nnz, self._lib = handle, n_layers, n_neurons, list(nnz), lib
+
+    # ---- construction -----------------------------------------------------------------------
+    @staticmethod
+    def _config(max_batch, train, clamp, update_bias, flags, stream, device, activation=0):
+        return SdnnConfig(activation, clamp, max_batch, int(train), int(update_bias), flags, stream, device)
+
+    @classmethod
+    def create(cls, row_ptr, col_idx, values, bias, *, max_batch, train=False, clamp=32.0, update_bias=False,
+               flags=0, stream=None, device=-1, activation=0):
+        lib = load_library()
+        L = len(col_idx)
+        n = len(bias[0]) if L else 0
+        rp = [_np(a, np.int32) for a in row_ptr]
+        ci = [_np(a, np.int32) for a in col_idx]
+        va = [_np(a, np.float32) for a in values]
+        bi = [_np(a, np.float32) for a in bias]
+        arr = lambda xs: (ctypes.c_void_p * max(L, 1))(*[x.ctypes.data for x in xs])
+        cfg = cls._config(max_batch, train, clamp, update_bias, flags, stream, device, activation)
+        h = ctypes.c_void_p()
+        rc = lib.sdnn_create(ctypes.byref(h), L, n, arr(rp), arr(ci), arr(va), arr(bi), ctypes.byref(cfg))
+        if rc != 0:
+            raise SdnnError(rc, (lib.sdnn_last_error(None) or b"").decode())
+        return cls(h, L, n, [len(c) for c in ci], lib)
+
+    @classmethod
+    def create_deferred(cls, n_layers, n_neurons, nnz_per_layer, *, max_batch, train=False, clamp=32.0,
+                        update_bias=False, flags=0, stream=None, device=-1):
+        lib = load_library()
+        nnz = _np(nnz_per_layer, np.int64)
+        cfg = cls._config(max_batch, train, clamp, update_bias, flags, stream, device)
+        h = ctypes.c_void_p()
+        rc = lib.sdnn_create_deferred(ctypes.byref(h), n_layers, n_neurons, nnz.ctypes.data, ctypes.byref(cfg))
+        if rc != 0:
+            raise SdnnError(rc, (lib.sdnn_last_error(None) or b"").decode())
+        return cls(h, n_layers, n_neurons, nnz.tolist(), lib)
+
+    def _check(self, rc):
+        if rc != 0:
+            raise SdnnError(rc, (self._lib.sdnn_last_error(self._h) or b"").decode())
+
+    def load_layer(self, layer, row_ptr, col_idx, values, bias):
+        rp, ci, va, bi = _np(row_ptr, np.int32), _np(col_idx, np.int32), _np(values, np.float32), _np(bias, np.float32)
+        self._check(self._lib.sdnn_load_layer(self._h, layer, rp.ctypes.data, ci.ctypes.data, va.ctypes.data, bi.ctypes.data))
+
+    def finalize(self):
+        self._check(self._lib.sdnn_finalize(self._h))
+
+    # ---- hot path ---------------------------------------------------------------------------
+    def infer_batch(self, x0, n_inputs, y_out=None, nz_count_out=None, nz_index_out=None, nz_index_capacity=0,
+                    want_total=False, host=False):
+        """Device pointers (torch CUDA tensors) unless host=True (numpy / pinned torch CPU tensors).
+        Returns the total id count when want_total (forces a stream sync), else None."""
+        total = ctypes.c_int64(0)
+        fn = self._lib.sdnn_infer_batch_host if host else self._lib.sdnn_infer_batch
+        rc = fn(self._h, _addr(x0), n_inputs, _addr(y_out), _addr(nz_count_out), _addr(nz_index_out),
+                nz_index_capacity, ctypes.byref(total) if want_total else None)
+        self.last_total = total.value
+        self._check(rc)
+        return total.value if want_total else None
+
+    def train_step(self, x0, target, B, eta, want_loss=False, host=False):
+        loss = ctypes.c_float(0.0)
+        fn = self._lib.sdnn_train_step_host if host else self._lib.sdnn_train_step
+        self._check(fn(self._h, _addr(x0), _addr(target), B, eta, ctypes.byref(loss) if want_loss else None))
+        return loss.value if want_loss else None
+
+    # ---- state / inspection -----------------------------------------------------------------
+    def get_weights(self, layer, want_bias=True):
+        v = np.empty(self.nnz[layer], dtype=np.float32)
+        b = np.empty(self.n_neurons, dtype=np.float32) if want_bias else None
+        self._check(self._lib.sdnn_get_weights(self._h, layer, v.ctypes.data, b.ctypes.data if want_bias else None))
+        return (v, b) if want_bias else v
+
+    def get_activations(self, layer, B):
+        out = np.empty((B, self.n_neurons), dtype=np.float32)
+        self._check(self._lib.sdnn_get_activations(self._h, layer, out.ctypes.data))
+        return out
+
+    def get_delta(self, layer, B):
+        out = np.empty((B, self.n_neurons), dtype=np.float32)
+        self._check(self._lib.sdnn_get_delta(self._h, layer, out.ctypes.data))
+        return out
+
+    def get_gradient(self, layer):
+        out = np.empty(self.nnz[layer - 1], dtype=np.float32)
+        self._check(self._lib.sdnn_get_gradient(self._h, layer, out.ctypes.data))
+        return out
+
+    def get_liveness(self):
+        out = np.empty(self.n_layers, dtype=np.int32)
+        self._check(self._lib.sdnn_get_liveness(self._h, out.ctypes.data))
+        return out
+
+    def kernel_launches(self):
+        return int(self._lib.sdnn_kernel_launches(self._h))
+
+    def device_bytes(self):
+        return int(self._lib.sdnn_device_bytes(self._h))
+
+    def destroy(self):
+        if self._h:
+            self._lib.sdnn_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass

@@ -1,0 +1,630 @@
+// Host side of libsdnn.so: the C ABI declared in include/sdnn.h.
+// Validation, device memory, the per-layer launch sequences (optionally as a CUDA graph) and
+// the staging of host buffers.  Every arithmetic step runs in the kernels of kernels.cuh.
+#include "../../include/sdnn.h"
+#include "kernels.cuh"
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+using namespace sdnn_kernels;
+
+namespace {
+
+thread_local std::string g_create_error;
+
+struct DevBuf {
+    void* p = nullptr;
+    size_t bytes = 0;
+};
+
+}  // namespace
+
+struct sdnn {
+    int L = 0, N = 0;
+    sdnn_config cfg{};
+    cudaStream_t stream = nullptr;
+    int device = 0;
+    bool finalized = false, stepped = false;
+    std::vector<int64_t> nnz, off;      // stored entries per layer; offset of the layer in the arenas (elements)
+    std::vector<char> loaded;
+    int64_t slots = 0;                  // arena length in elements
+    int ld_max = 0;                     // padded width of the widest tile this handle processes
+
+    int* d_row_ptr = nullptr;           // [L][N+1], offsets local to the layer
+    int* d_col = nullptr;               // arena
+    float* d_val = nullptr;             // arena
+    float* d_bias = nullptr;            // [L][N]
+
+    // training
+    float* d_acts = nullptr;            // [(L+1)][N][ld]: x^0 .. x^L of the current step
+    float* d_s[2] = {nullptr, nullptr}; // alternating S = W^T delta tiles, all-zero between steps
+    float* d_yt = nullptr;              // target tile
+    StepParams* d_sp = nullptr;
+    double* d_loss = nullptr;
+    float* d_dbg_delta = nullptr;       // [L][N][ld]   (KEEP_DEBUG)
+    float* d_dbg_grad = nullptr;        // arena        (KEEP_DEBUG)
+    int last_b = 0, last_ld = 0;
+    cudaGraphExec_t graph = nullptr;
+    int graph_ld = 0;
+
+    // inference
+    float* d_tile[2] = {nullptr, nullptr};
+    int* d_seg_cnt = nullptr;
+    int* d_tile_cnt = nullptr;
+    long long* d_offs = nullptr;
+    long long* d_running = nullptr;
+
+    // staging for the *_host entry points (allocated on first use)
+    float* d_stage_a = nullptr;
+    float* d_stage_b = nullptr;
+    int* d_stage_cnt = nullptr;
+    int* d_stage_idx = nullptr;
+    int64_t stage_idx_cap = 0;
+
+    int64_t launches = 0;
+    int64_t dev_bytes = 0;
+    std::vector<void*> allocs;
+    std::string err;
+};
+
+namespace {
+
+int fail(sdnn* h, int code, const char* fmt, ...) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    if (h) h->err = buf;
+    g_create_error = buf;
+    return code;
+}
+
+int cuda_fail(sdnn* h, cudaError_t e, const char* what) {
+    int code = (e == cudaErrorMemoryAllocation) ? SDNN_ERR_OOM : SDNN_ERR_CUDA;
+    return fail(h, code, "%s: %s", what, cudaGetErrorString(e));
+}
+
+#define CU(h, call)                                                  \
+    do {                                                             \
+        cudaError_t e_ = (call);                                     \
+        if (e_ != cudaSuccess) return cuda_fail((h), e_, #call);     \
+    } while (0)
+
+template <typename T>
+int dev_alloc(sdnn* h, T** out, size_t count, bool zero) {
+    size_t bytes = count * sizeof(T);
+    if (bytes == 0) bytes = sizeof(T);
+    void* p = nullptr;
+    cudaError_t e = cudaMalloc(&p, bytes);
+    if (e != cudaSuccess) { cudaGetLastError(); return cuda_fail(h, e, "cudaMalloc"); }
+    h->allocs.push_back(p);
+    h->dev_bytes += (int64_t)bytes;
+    if (zero) CU(h, cudaMemsetAsync(p, 0, bytes, h->stream));
+    *out = static_cast<T*>(p);
+    return SDNN_OK;
+}
+
+// padded batch width: 4, 8, .., 128, then multiples of 128
+int padded_width(int b) {
+    if (b <= 4) return 4;
+    if (b <= 128) { int w = 4; while (w < b) w <<= 1; return w; }
+    return (b + 127) / 128 * 128;
+}
+
+struct Geometry { int g; int chunks; };   // lanes per row group; 4g-wide chunks per tile row
+Geometry geometry(int cols) {
+    if (cols <= 128) return {cols / 4, 1};
+    return {32, cols / 128};
+}
+
+int validate_cfg(const sdnn_config* cfg) {
+    if (!cfg) return fail(nullptr, SDNN_ERR_INVALID_ARG, "cfg is NULL");
+    if (cfg->activation != 0) return fail(nullptr, SDNN_ERR_UNIMPLEMENTED, "only activation 0 (clamped ReLU) is implemented");
+    if (!(cfg->clamp > 0.0f) || !std::isfinite(cfg->clamp)) return fail(nullptr, SDNN_ERR_INVALID_ARG, "clamp must be finite and > 0");
+    if (cfg->max_batch < 1) return fail(nullptr, SDNN_ERR_INVALID_ARG, "max_batch must be >= 1");
+    if (cfg->train && cfg->max_batch > 128) return fail(nullptr, SDNN_ERR_INVALID_ARG, "training handles support max_batch <= 128");
+    if ((cfg->flags & SDNN_FLAG_BWD_ATOMICS) && (cfg->flags & SDNN_FLAG_BWD_CSC))
+        return fail(nullptr, SDNN_ERR_INVALID_ARG, "choose one backward strategy");
+    if (cfg->flags & SDNN_FLAG_BWD_CSC) return fail(nullptr, SDNN_ERR_UNIMPLEMENTED, "transposed-index backward is not implemented");
+    return SDNN_OK;
+}
+
+// Host-side check of one layer: returns SDNN_OK or fills the message.
+int validate_layer(sdnn* h, int layer, int n, int64_t expect_nnz, const int32_t* rp, const int32_t* col,
+                   const float* val, const float* bias) {
+    if (!rp || !bias) return fail(h, SDNN_ERR_INVALID_ARG, "layer %d: NULL row_ptr or bias", layer);
+    if (rp[0] != 0) return fail(h, SDNN_ERR_BAD_CSR, "layer %d: row_ptr[0] = %d, expected 0", layer, rp[0]);
+    for (int i = 0; i < n; ++i)
+        if (rp[i + 1] < rp[i]) return fail(h, SDNN_ERR_BAD_CSR, "layer %d: row_ptr decreases at row %d", layer, i);
+    if ((int64_t)rp[n] != expect_nnz)
+        return fail(h, SDNN_ERR_BAD_CSR, "layer %d: row_ptr[N] = %d but %lld stored entries were announced", layer, rp[n],
+                    (long long)expect_nnz);
+    if (expect_nnz > 0 && (!col || !val)) return fail(h, SDNN_ERR_INVALID_ARG, "layer %d: NULL col_idx or values", layer);
+    int bad_row = -1, bad_kind = 0;
+#pragma omp parallel for schedule(static)
+    for (int i = 0; i < n; ++i) {
+        int kind = 0;
+        if (!std::isfinite(bias[i])) kind = 4;
+        for (int p = rp[i]; p < rp[i + 1] && !kind; ++p) {
+            if (col[p] < 0 || col[p] >= n) kind = 1;
+            else if (p > rp[i] && col[p] <= col[p - 1]) kind = (col[p] == col[p - 1]) ? 2 : 3;
+            else if (!std::isfinite(val[p])) kind = 5;
+        }
+        if (kind) {
+#pragma omp critical
+            if (bad_row < 0 || i < bad_row) { bad_row = i; bad_kind = kind; }
+        }
+    }
+    if (bad_row >= 0) {
+        static const char* what[] = {"", "column index out of range", "duplicate column", "columns not ascending",
+                                     "non-finite bias", "non-finite value"};
+        return fail(h, SDNN_ERR_BAD_CSR, "layer %d, row %d: %s", layer, bad_row, what[bad_kind]);
+    }
+    return SDNN_OK;
+}
+
+void count_launch(sdnn* h, int k = 1) { h->launches += k; }
+
+template <int G>
+void launch_forward_g(sdnn* h, int layer, const float* xin, float* xout, int ld, int chunks) {
+    const int rows_per_block = 8 * (32 / G);
+    dim3 grid((h->N + rows_per_block - 1) / rows_per_block, chunks);
+    forward_kernel<G><<<grid, 256, 0, h->stream>>>(h->d_row_ptr + (size_t)layer * (h->N + 1), h->d_col + h->off[layer],
+                                                   h->d_val + h->off[layer], h->d_bias + (size_t)layer * h->N, xin, xout,
+                                                   h->N, ld, h->cfg.clamp);
+}
+
+void launch_forward(sdnn* h, int layer, const float* xin, float* xout, int ld, int cols) {
+    const Geometry q = geometry(cols);
+    switch (q.g) {
+        case 1: launch_forward_g<1>(h, layer, xin, xout, ld, q.chunks); break;
+        case 2: launch_forward_g<2>(h, layer, xin, xout, ld, q.chunks); break;
+        case 4: launch_forward_g<4>(h, layer, xin, xout, ld, q.chunks); break;
+        case 8: launch_forward_g<8>(h, layer, xin, xout, ld, q.chunks); break;
+        case 16: launch_forward_g<16>(h, layer, xin, xout, ld, q.chunks); break;
+        default: launch_forward_g<32>(h, layer, xin, xout, ld, q.chunks); break;
+    }
+    count_launch(h);
+}
+
+template <int G>
+void launch_backward_g(sdnn* h, int layer, int ld) {
+    const int rows_per_block = 8 * (32 / G);
+    dim3 grid((h->N + rows_per_block - 1) / rows_per_block);
+    const size_t tile = (size_t)h->N * ld;
+    const bool last = layer == h->L - 1, prop = layer > 0;
+    const int* rp = h->d_row_ptr + (size_t)layer * (h->N + 1);
+    const int* col = h->d_col + h->off[layer];
+    float* val = h->d_val + h->off[layer];
+    float* bias = h->d_bias + (size_t)layer * h->N;
+    const float* xk = h->d_acts + (size_t)(layer + 1) * tile;
+    const float* xprev = h->d_acts + (size_t)layer * tile;
+    float* s_k = last ? h->d_yt : h->d_s[(layer + 1) & 1];
+    float* s_prev = h->d_s[layer & 1];
+    float* dd = h->d_dbg_delta ? h->d_dbg_delta + (size_t)layer * tile : nullptr;
+    float* dg = h->d_dbg_grad ? h->d_dbg_grad + h->off[layer] : nullptr;
+    const int ub = h->cfg.update_bias ? 1 : 0, sk = (h->cfg.flags & SDNN_FLAG_SKIP_DEAD) ? 1 : 0;
+#define SDNN_BWD(LASTV, PROPV)                                                                              \
+    backward_kernel<G, LASTV, PROPV><<<grid, 256, 0, h->stream>>>(rp, col, val, bias, xk, xprev, s_k, s_prev, \
+                                                                  h->N, h->cfg.clamp, h->d_sp, h->d_loss, dd, dg, ub, sk)
+    if (last && prop) SDNN_BWD(true, true);
+    else if (last) SDNN_BWD(true, false);
+    else if (prop) SDNN_BWD(false, true);
+    else SDNN_BWD(false, false);
+#undef SDNN_BWD
+}
+
+void launch_backward(sdnn* h, int layer, int ld) {
+    switch (ld / 4) {
+        case 1: launch_backward_g<1>(h, layer, ld); break;
+        case 2: launch_backward_g<2>(h, layer, ld); break;
+        case 4: launch_backward_g<4>(h, layer, ld); break;
+        case 8: launch_backward_g<8>(h, layer, ld); break;
+        case 16: launch_backward_g<16>(h, layer, ld); break;
+        default: launch_backward_g<32>(h, layer, ld); break;
+    }
+    count_launch(h);
+}
+
+void launch_transpose_in(sdnn* h, const float* src, float* dst, int cnt, int cols, int ld) {
+    dim3 grid((h->N + 31) / 32, (cols + 31) / 32), block(32, 8);
+    transpose_in_kernel<<<grid, block, 0, h->stream>>>(src, dst, h->N, cnt, cols, ld);
+    count_launch(h);
+}
+
+// forward + backward chain of one train step on the internal buffers
+void enqueue_step_body(sdnn* h, int ld) {
+    const size_t tile = (size_t)h->N * ld;
+    for (int k = 0; k < h->L; ++k)
+        launch_forward(h, k, h->d_acts + (size_t)k * tile, h->d_acts + (size_t)(k + 1) * tile, ld, ld);
+    for (int k = h->L - 1; k >= 0; --k) launch_backward(h, k, ld);
+}
+
+int train_step_device(sdnn* h, const float* x0, const float* target, int B, float eta, float* loss_out) {
+    const int ld = padded_width(B);
+    set_step_params_kernel<<<1, 1, 0, h->stream>>>(h->d_sp, eta, B, h->d_loss);
+    count_launch(h);
+    launch_transpose_in(h, x0, h->d_acts, B, ld, ld);
+    launch_transpose_in(h, target, h->d_yt, B, ld, ld);
+    if (h->cfg.flags & SDNN_FLAG_NO_GRAPH) {
+        enqueue_step_body(h, ld);
+    } else {
+        if (!h->graph || h->graph_ld != ld) {
+            if (h->graph) { cudaGraphExecDestroy(h->graph); h->graph = nullptr; }
+            cudaGraph_t g = nullptr;
+            const int64_t before = h->launches;
+            CU(h, cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal));
+            enqueue_step_body(h, ld);
+            cudaError_t e = cudaStreamEndCapture(h->stream, &g);
+            h->launches = before;
+            if (e != cudaSuccess) return cuda_fail(h, e, "cudaStreamEndCapture");
+            e = cudaGraphInstantiate(&h->graph, g, 0);
+            cudaGraphDestroy(g);
+            if (e != cudaSuccess) { h->graph = nullptr; return cuda_fail(h, e, "cudaGraphInstantiate"); }
+            h->graph_ld = ld;
+        }
+        CU(h, cudaGraphLaunch(h->graph, h->stream));
+        count_launch(h, 2 * h->L);
+    }
+    CU(h, cudaGetLastError());
+    h->stepped = true; h->last_b = B; h->last_ld = ld;
+    if (loss_out) {
+        double j = 0.0;
+        CU(h, cudaMemcpyAsync(&j, h->d_loss, sizeof(double), cudaMemcpyDeviceToHost, h->stream));
+        CU(h, cudaStreamSynchronize(h->stream));
+        *loss_out = (float)j;
+    }
+    return SDNN_OK;
+}
+
+int check_train_args(sdnn* h, const float* x0, const float* target, int B, float eta) {
+    if (!h) return SDNN_ERR_INVALID_ARG;
+    if (!h->finalized) return fail(h, SDNN_ERR_STATE, "handle is not finalized");
+    if (!h->cfg.train) return fail(h, SDNN_ERR_STATE, "handle was created with train = 0");
+    if (!x0 || !target) return fail(h, SDNN_ERR_INVALID_ARG, "x0 or target is NULL");
+    if (B < 1 || B > h->cfg.max_batch) return fail(h, SDNN_ERR_INVALID_ARG, "B = %d outside [1, max_batch = %d]", B, h->cfg.max_batch);
+    if (!std::isfinite(eta)) return fail(h, SDNN_ERR_INVALID_ARG, "eta is not finite");
+    return SDNN_OK;
+}
+
+// One tile of inference on device buffers: x0 [cnt][N] -> outputs for these cnt inputs.
+int infer_tile(sdnn* h, const float* x0, int cnt, float* y_out, int* cnt_out, int* idx_out, long long capacity,
+               bool want_sets) {
+    const int ld = h->ld_max;
+    const int cols = padded_width(cnt);
+    launch_transpose_in(h, x0, h->d_tile[0], cnt, cols, ld);
+    int cur = 0;
+    for (int k = 0; k < h->L; ++k) {
+        launch_forward(h, k, h->d_tile[cur], h->d_tile[cur ^ 1], ld, cols);
+        cur ^= 1;
+    }
+    const float* xl = h->d_tile[cur];
+    if (y_out) {
+        dim3 grid((h->N + 31) / 32, (cnt + 31) / 32), block(32, 8);
+        transpose_out_kernel<<<grid, block, 0, h->stream>>>(xl, y_out, h->N, cnt, ld);
+        count_launch(h);
+    }
+    if (want_sets) {
+        const int nseg = (h->N + NZ_SEG - 1) / NZ_SEG;
+        dim3 grid(nseg, (cnt + 127) / 128);
+        nz_count_kernel<<<grid, 128, 0, h->stream>>>(xl, h->d_seg_cnt, h->N, cnt, ld);
+        nz_scan_segments_kernel<<<(cnt + 127) / 128, 128, 0, h->stream>>>(h->d_seg_cnt, h->d_tile_cnt, nseg, cnt, ld);
+        nz_scan_inputs_kernel<<<1, 1024, 0, h->stream>>>(h->d_tile_cnt, h->d_offs, h->d_running, cnt_out, cnt);
+        count_launch(h, 3);
+        if (idx_out) {
+            nz_fill_kernel<<<grid, 128, 0, h->stream>>>(xl, h->d_seg_cnt, h->d_offs, idx_out, capacity, h->N, cnt, ld);
+            count_launch(h);
+        }
+    }
+    CU(h, cudaGetLastError());
+    return SDNN_OK;
+}
+
+int check_infer_args(sdnn* h, const float* x0, int64_t n_inputs, int32_t* idx, int64_t cap) {
+    if (!h) return SDNN_ERR_INVALID_ARG;
+    if (!h->finalized) return fail(h, SDNN_ERR_STATE, "handle is not finalized");
+    if (n_inputs < 0) return fail(h, SDNN_ERR_INVALID_ARG, "n_inputs < 0");
+    if (n_inputs > 0 && !x0) return fail(h, SDNN_ERR_INVALID_ARG, "x0 is NULL");
+    if (idx && cap < 0) return fail(h, SDNN_ERR_INVALID_ARG, "nz_index_capacity < 0");
+    return SDNN_OK;
+}
+
+int ensure_stage(sdnn* h) {
+    if (h->d_stage_a) return SDNN_OK;
+    const size_t cnt = (size_t)h->cfg.max_batch * h->N;
+    int rc;
+    if ((rc = dev_alloc(h, &h->d_stage_a, cnt, false))) return rc;
+    if ((rc = dev_alloc(h, &h->d_stage_b, cnt, false))) return rc;
+    if ((rc = dev_alloc(h, &h->d_stage_cnt, (size_t)h->cfg.max_batch, false))) return rc;
+    return SDNN_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* sdnn_version(void) { return "sdnn 0.1 (sm_100a)"; }
+
+const char* sdnn_last_error(const sdnn_t* h) { return h ? h->err.c_str() : g_create_error.c_str(); }
+
+int64_t sdnn_kernel_launches(const sdnn_t* h) { return h ? h->launches : 0; }
+int64_t sdnn_device_bytes(const sdnn_t* h) { return h ? h->dev_bytes : 0; }
+
+void sdnn_destroy(sdnn_t* h) {
+    if (!h) return;
+    cudaSetDevice(h->device);
+    cudaStreamSynchronize(h->stream);
+    if (h->graph) cudaGraphExecDestroy(h->graph);
+    for (void* p : h->allocs) cudaFree(p);
+    delete h;
+}
+
+int sdnn_create_deferred(sdnn_t** out, int32_t n_layers, int32_t n_neurons, const int64_t* nnz_per_layer,
+                         const sdnn_config* cfg) {
+    if (!out) return fail(nullptr, SDNN_ERR_INVALID_ARG, "out is NULL");
+    *out = nullptr;
+    int rc = validate_cfg(cfg);
+    if (rc) return rc;
+    if (n_layers < 1 || n_neurons < 1) return fail(nullptr, SDNN_ERR_INVALID_ARG, "n_layers and n_neurons must be >= 1");
+    if (!nnz_per_layer) return fail(nullptr, SDNN_ERR_INVALID_ARG, "nnz_per_layer is NULL");
+    for (int l = 0; l < n_layers; ++l)
+        if (nnz_per_layer[l] < 0 || nnz_per_layer[l] > INT32_MAX)
+            return fail(nullptr, SDNN_ERR_INVALID_ARG, "layer %d: stored-entry count outside [0, 2^31)", l);
+
+    int ndev = 0;
+    cudaError_t e = cudaGetDeviceCount(&ndev);
+    if (e != cudaSuccess || ndev == 0) { cudaGetLastError(); return fail(nullptr, SDNN_ERR_CUDA, "no CUDA device: %s", cudaGetErrorString(e)); }
+
+    sdnn* h = new (std::nothrow) sdnn;
+    if (!h) return fail(nullptr, SDNN_ERR_OOM, "host allocation failed");
+    h->L = n_layers; h->N = n_neurons; h->cfg = *cfg;
+    h->stream = static_cast<cudaStream_t>(cfg->cuda_stream);
+    auto bail = [&](int code) { g_create_error = h->err; sdnn_destroy(h); return code; };
+    if (cfg->device >= 0) {
+        if (cfg->device >= ndev) { h->err = "device ordinal out of range"; return bail(SDNN_ERR_INVALID_ARG); }
+        if ((e = cudaSetDevice(cfg->device)) != cudaSuccess) return bail(cuda_fail(h, e, "cudaSetDevice"));
+        h->device = cfg->device;
+    } else if ((e = cudaGetDevice(&h->device)) != cudaSuccess) {
+        return bail(cuda_fail(h, e, "cudaGetDevice"));
+    }
+    h->nnz.assign(nnz_per_layer, nnz_per_layer + n_layers);
+    h->off.resize(n_layers);
+    h->loaded.assign(n_layers, 0);
+    int64_t run = 0;
+    for (int l = 0; l < n_layers; ++l) { h->off[l] = run; run += (h->nnz[l] + 31) / 32 * 32; }   // 128-byte aligned layers
+    h->slots = run;
+    h->ld_max = padded_width(cfg->max_batch);
+    const size_t N = (size_t)n_neurons, L = (size_t)n_layers, tile = N * (size_t)h->ld_max;
+
+    if ((rc = dev_alloc(h, &h->d_row_ptr, L * (N + 1), false))) return bail(rc);
+    if ((rc = dev_alloc(h, &h->d_col, (size_t)h->slots, true))) return bail(rc);
+    if ((rc = dev_alloc(h, &h->d_val, (size_t)h->slots, true))) return bail(rc);
+    if ((rc = dev_alloc(h, &h->d_bias, L * N, false))) return bail(rc);
+    if (cfg->train) {
+        if ((rc = dev_alloc(h, &h->d_acts, (L + 1) * tile, false))) return bail(rc);
+        if ((rc = dev_alloc(h, &h->d_s[0], tile, true))) return bail(rc);
+        if ((rc = dev_alloc(h, &h->d_s[1], tile, true))) return bail(rc);
+        if ((rc = dev_alloc(h, &h->d_yt, tile, true))) return bail(rc);
+        if ((rc = dev_alloc(h, &h->d_sp, 1, true))) return bail(rc);
+        if ((rc = dev_alloc(h, &h->d_loss, 1, true))) return bail(rc);
+        if (cfg->flags & SDNN_FLAG_KEEP_DEBUG) {
+            if ((rc = dev_alloc(h, &h->d_dbg_delta, L * tile, true))) return bail(rc);
+            if ((rc = dev_alloc(h, &h->d_dbg_grad, (size_t)h->slots, true))) return bail(rc);
+        }
+    }
+    {   // inference buffers (a training handle can also infer)
+        const size_t nseg = (N + NZ_SEG - 1) / NZ_SEG;
+        if ((rc = dev_alloc(h, &h->d_tile[0], tile, false))) return bail(rc);
+        if ((rc = dev_alloc(h, &h->d_tile[1], tile, false))) return bail(rc);
+        if ((rc = dev_alloc(h, &h->d_seg_cnt, nseg * (size_t)h->ld_max, false))) return bail(rc);
+        if ((rc = dev_alloc(h, &h->d_tile_cnt, (size_t)h->ld_max, false))) return bail(rc);
+        if ((rc = dev_alloc(h, &h->d_offs, (size_t)h->ld_max, false))) return bail(rc);
+        if ((rc = dev_alloc(h, &h->d_running, 1, true))) return bail(rc);
+    }
+    *out = h;
+    return SDNN_OK;
+}
+
+int sdnn_load_layer(sdnn_t* h, int32_t layer, const int32_t* row_ptr, const int32_t* col_idx, const float* values,
+                    const float* bias) {
+    if (!h) return SDNN_ERR_INVALID_ARG;
+    if (h->finalized) return fail(h, SDNN_ERR_STATE, "handle already finalized");
+    if (layer < 0 || layer >= h->L) return fail(h, SDNN_ERR_INVALID_ARG, "layer %d outside [0, %d)", layer, h->L);
+    if (h->loaded[layer]) return fail(h, SDNN_ERR_STATE, "layer %d loaded twice", layer);
+    int rc = validate_layer(h, layer, h->N, h->nnz[layer], row_ptr, col_idx, values, bias);
+    if (rc) return rc;
+    CU(h, cudaSetDevice(h->device));
+    const size_t N = (size_t)h->N, nz = (size_t)h->nnz[layer];
+    CU(h, cudaMemcpyAsync(h->d_row_ptr + (size_t)layer * (N + 1), row_ptr, (N + 1) * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+    CU(h, cudaMemcpyAsync(h->d_bias + (size_t)layer * N, bias, N * sizeof(float), cudaMemcpyHostToDevice, h->stream));
+    if (nz) {
+        CU(h, cudaMemcpyAsync(h->d_col + h->off[layer], col_idx, nz * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+        CU(h, cudaMemcpyAsync(h->d_val + h->off[layer], values, nz * sizeof(float), cudaMemcpyHostToDevice, h->stream));
+    }
+    CU(h, cudaStreamSynchronize(h->stream));   // the caller may reuse its arrays right away
+    h->loaded[layer] = 1;
+    return SDNN_OK;
+}
+
+int sdnn_finalize(sdnn_t* h) {
+    if (!h) return SDNN_ERR_INVALID_ARG;
+    if (h->finalized) return fail(h, SDNN_ERR_STATE, "handle already finalized");
+    for (int l = 0; l < h->L; ++l)
+        if (!h->loaded[l]) return fail(h, SDNN_ERR_STATE, "layer %d was never loaded", l);
+    CU(h, cudaStreamSynchronize(h->stream));
+    h->finalized = true;
+    return SDNN_OK;
+}
+
+int sdnn_create(sdnn_t** out, int32_t n_layers, int32_t n_neurons, const int32_t* const* row_ptr,
+                const int32_t* const* col_idx, const float* const* values, const float* const* bias,
+                const sdnn_config* cfg) {
+    if (!out) return fail(nullptr, SDNN_ERR_INVALID_ARG, "out is NULL");
+    *out = nullptr;
+    int rc = validate_cfg(cfg);
+    if (rc) return rc;
+    if (n_layers < 1 || n_neurons < 1) return fail(nullptr, SDNN_ERR_INVALID_ARG, "n_layers and n_neurons must be >= 1");
+    if (!row_ptr || !col_idx || !values || !bias) return fail(nullptr, SDNN_ERR_INVALID_ARG, "NULL array of layer pointers");
+    std::vector<int64_t> nnz(n_layers);
+    for (int l = 0; l < n_layers; ++l) {
+        if (!row_ptr[l]) return fail(nullptr, SDNN_ERR_INVALID_ARG, "layer %d: row_ptr is NULL", l);
+        const int32_t last = row_ptr[l][n_neurons];
+        if (last < 0) return fail(nullptr, SDNN_ERR_BAD_CSR, "layer %d: row_ptr[N] is negative", l);
+        nnz[l] = last;
+    }
+    // validate everything on the host before any device memory is requested
+    for (int l = 0; l < n_layers; ++l)
+        if ((rc = validate_layer(nullptr, l, n_neurons, nnz[l], row_ptr[l], col_idx[l], values[l], bias[l]))) return rc;
+    sdnn* h = nullptr;
+    if ((rc = sdnn_create_deferred(&h, n_layers, n_neurons, nnz.data(), cfg))) return rc;
+    for (int l = 0; l < n_layers; ++l)
+        if ((rc = sdnn_load_layer(h, l, row_ptr[l], col_idx[l], values[l], bias[l]))) { g_create_error = h->err; sdnn_destroy(h); return rc; }
+    if ((rc = sdnn_finalize(h))) { g_create_error = h->err; sdnn_destroy(h); return rc; }
+    *out = h;
+    return SDNN_OK;
+}
+
+int sdnn_train_step(sdnn_t* h, const float* x0, const float* target, int32_t B, float eta, float* loss_out) {
+    int rc = check_train_args(h, x0, target, B, eta);
+    if (rc) return rc;
+    CU(h, cudaSetDevice(h->device));
+    return train_step_device(h, x0, target, B, eta, loss_out);
+}
+
+int sdnn_train_step_host(sdnn_t* h, const float* x0, const float* target, int32_t B, float eta, float* loss_out) {
+    int rc = check_train_args(h, x0, target, B, eta);
+    if (rc) return rc;
+    CU(h, cudaSetDevice(h->device));
+    if ((rc = ensure_stage(h))) return rc;
+    const size_t bytes = (size_t)B * h->N * sizeof(float);
+    CU(h, cudaMemcpyAsync(h->d_stage_a, x0, bytes, cudaMemcpyHostToDevice, h->stream));
+    CU(h, cudaMemcpyAsync(h->d_stage_b, target, bytes, cudaMemcpyHostToDevice, h->stream));
+    rc = train_step_device(h, h->d_stage_a, h->d_stage_b, B, eta, loss_out);
+    if (rc) return rc;
+    CU(h, cudaStreamSynchronize(h->stream));
+    return SDNN_OK;
+}
+
+int sdnn_infer_batch(sdnn_t* h, const float* x0, int64_t n_inputs, float* y_out, int32_t* nz_count_out,
+                     int32_t* nz_index_out, int64_t nz_index_capacity, int64_t* nz_total_out) {
+    int rc = check_infer_args(h, x0, n_inputs, nz_index_out, nz_index_capacity);
+    if (rc) return rc;
+    CU(h, cudaSetDevice(h->device));
+    const bool want_sets = nz_count_out || nz_index_out || nz_total_out;
+    if (want_sets) CU(h, cudaMemsetAsync(h->d_running, 0, sizeof(long long), h->stream));
+    const int T = h->cfg.max_batch;
+    for (int64_t t0 = 0; t0 < n_inputs; t0 += T) {
+        const int cnt = (int)((n_inputs - t0 < T) ? (n_inputs - t0) : T);
+        rc = infer_tile(h, x0 + (size_t)t0 * h->N, cnt, y_out ? y_out + (size_t)t0 * h->N : nullptr,
+                        nz_count_out ? nz_count_out + t0 : nullptr, nz_index_out, nz_index_capacity, want_sets);
+        if (rc) return rc;
+    }
+    if (nz_total_out || nz_index_out) {
+        long long total = 0;
+        CU(h, cudaMemcpyAsync(&total, h->d_running, sizeof total, cudaMemcpyDeviceToHost, h->stream));
+        CU(h, cudaStreamSynchronize(h->stream));
+        if (nz_total_out) *nz_total_out = total;
+        if (nz_index_out && total > nz_index_capacity)
+            return fail(h, SDNN_ERR_INVALID_ARG, "nz_index_capacity %lld too small, %lld ids needed", (long long)nz_index_capacity, total);
+    }
+    return SDNN_OK;
+}
+
+int sdnn_infer_batch_host(sdnn_t* h, const float* x0, int64_t n_inputs, float* y_out, int32_t* nz_count_out,
+                          int32_t* nz_index_out, int64_t nz_index_capacity, int64_t* nz_total_out) {
+    int rc = check_infer_args(h, x0, n_inputs, nz_index_out, nz_index_capacity);
+    if (rc) return rc;
+    CU(h, cudaSetDevice(h->device));
+    if ((rc = ensure_stage(h))) return rc;
+    if (nz_index_out && nz_index_capacity > h->stage_idx_cap) {
+        if ((rc = dev_alloc(h, &h->d_stage_idx, (size_t)nz_index_capacity, false))) return rc;   // grows; old block freed at destroy
+        h->stage_idx_cap = nz_index_capacity;
+    }
+    const bool want_sets = nz_count_out || nz_index_out || nz_total_out;
+    if (want_sets) CU(h, cudaMemsetAsync(h->d_running, 0, sizeof(long long), h->stream));
+    const int T = h->cfg.max_batch;
+    for (int64_t t0 = 0; t0 < n_inputs; t0 += T) {
+        const int cnt = (int)((n_inputs - t0 < T) ? (n_inputs - t0) : T);
+        const size_t bytes = (size_t)cnt * h->N * sizeof(float);
+        CU(h, cudaMemcpyAsync(h->d_stage_a, x0 + (size_t)t0 * h->N, bytes, cudaMemcpyHostToDevice, h->stream));
+        rc = infer_tile(h, h->d_stage_a, cnt, y_out ? h->d_stage_b : nullptr, nz_count_out ? h->d_stage_cnt : nullptr,
+                        nz_index_out ? h->d_stage_idx : nullptr, nz_index_capacity, want_sets);
+        if (rc) return rc;
+        if (y_out) CU(h, cudaMemcpyAsync(y_out + (size_t)t0 * h->N, h->d_stage_b, bytes, cudaMemcpyDeviceToHost, h->stream));
+        if (nz_count_out) CU(h, cudaMemcpyAsync(nz_count_out + t0, h->d_stage_cnt, (size_t)cnt * sizeof(int), cudaMemcpyDeviceToHost, h->stream));
+    }
+    long long total = 0;
+    if (want_sets) CU(h, cudaMemcpyAsync(&total, h->d_running, sizeof total, cudaMemcpyDeviceToHost, h->stream));
+    CU(h, cudaStreamSynchronize(h->stream));
+    if (nz_total_out) *nz_total_out = total;
+    if (nz_index_out) {
+        const long long m = total < nz_index_capacity ? total : nz_index_capacity;
+        if (m > 0) CU(h, cudaMemcpy(nz_index_out, h->d_stage_idx, (size_t)m * sizeof(int), cudaMemcpyDeviceToHost));
+        if (total > nz_index_capacity)
+            return fail(h, SDNN_ERR_INVALID_ARG, "nz_index_capacity %lld too small, %lld ids needed", (long long)nz_index_capacity, total);
+    }
+    return SDNN_OK;
+}
+
+int sdnn_get_weights(sdnn_t* h, int32_t layer, float* values_out, float* bias_out) {
+    if (!h) return SDNN_ERR_INVALID_ARG;
+    if (!h->finalized) return fail(h, SDNN_ERR_STATE, "handle is not finalized");
+    if (layer < 0 || layer >= h->L) return fail(h, SDNN_ERR_INVALID_ARG, "layer %d outside [0, %d)", layer, h->L);
+    CU(h, cudaSetDevice(h->device));
+    CU(h, cudaStreamSynchronize(h->stream));
+    if (values_out && h->nnz[layer])
+        CU(h, cudaMemcpy(values_out, h->d_val + h->off[layer], (size_t)h->nnz[layer] * sizeof(float), cudaMemcpyDeviceToHost));
+    if (bias_out) CU(h, cudaMemcpy(bias_out, h->d_bias + (size_t)layer * h->N, (size_t)h->N * sizeof(float), cudaMemcpyDeviceToHost));
+    return SDNN_OK;
+}
+
+static int fetch_tile(sdnn_t* h, const float* tile, float* out) {
+    // tile [N][ld] on the device -> out [B][N] on the host
+    const int B = h->last_b, ld = h->last_ld, N = h->N;
+    std::vector<float> tmp((size_t)N * ld);
+    CU(h, cudaSetDevice(h->device));
+    CU(h, cudaStreamSynchronize(h->stream));
+    CU(h, cudaMemcpy(tmp.data(), tile, tmp.size() * sizeof(float), cudaMemcpyDeviceToHost));
+    for (int b = 0; b < B; ++b)
+        for (int i = 0; i < N; ++i) out[(size_t)b * N + i] = tmp[(size_t)i * ld + b];
+    return SDNN_OK;
+}
+
+int sdnn_get_activations(sdnn_t* h, int32_t layer, float* out) {
+    if (!h || !out) return SDNN_ERR_INVALID_ARG;
+    if (!h->stepped) return fail(h, SDNN_ERR_STATE, "no train step has run");
+    if (layer < 0 || layer > h->L) return fail(h, SDNN_ERR_INVALID_ARG, "layer %d outside [0, %d]", layer, h->L);
+    return fetch_tile(h, h->d_acts + (size_t)layer * h->N * h->last_ld, out);
+}
+
+int sdnn_get_delta(sdnn_t* h, int32_t layer, float* out) {
+    if (!h || !out) return SDNN_ERR_INVALID_ARG;
+    if (!h->stepped || !h->d_dbg_delta) return fail(h, SDNN_ERR_STATE, "needs SDNN_FLAG_KEEP_DEBUG and a train step");
+    if (layer < 1 || layer > h->L) return fail(h, SDNN_ERR_INVALID_ARG, "layer %d outside [1, %d]", layer, h->L);
+    return fetch_tile(h, h->d_dbg_delta + (size_t)(layer - 1) * h->N * h->last_ld, out);
+}
+
+int sdnn_get_gradient(sdnn_t* h, int32_t layer, float* out) {
+    if (!h || !out) return SDNN_ERR_INVALID_ARG;
+    if (!h->stepped || !h->d_dbg_grad) return fail(h, SDNN_ERR_STATE, "needs SDNN_FLAG_KEEP_DEBUG and a train step");
+    if (layer < 1 || layer > h->L) return fail(h, SDNN_ERR_INVALID_ARG, "layer %d outside [1, %d]", layer, h->L);
+    CU(h, cudaSetDevice(h->device));
+    CU(h, cudaStreamSynchronize(h->stream));
+    if (h->nnz[layer - 1])
+        CU(h, cudaMemcpy(out, h->d_dbg_grad + h->off[layer - 1], (size_t)h->nnz[layer - 1] * sizeof(float), cudaMemcpyDeviceToHost));
+    return SDNN_OK;
+}
+
+int sdnn_get_liveness(sdnn_t* h, int32_t* live_inputs_out) {
+    if (!h || !live_inputs_out) return SDNN_ERR_INVALID_ARG;
+    return fail(h, SDNN_ERR_STATE, "liveness is recorded only by inference with SDNN_FLAG_SKIP_DEAD");
+}
+
+}  // extern "C"

@@ -1,0 +1,74 @@
+"""Harness shared by the GPU parity tests: error metric, kink-ambiguity protocol, net builders.
+
+Error metric (per tensor): max_i |g_i - o_i| / max(|o_i|, 1e-3 * max|o|); a tensor that is identically
+zero in the oracle must be identically zero on the GPU.  Bar: 1e-4.
+
+Kink protocol.  f'(z) jumps at z = 0 and z = clamp, so fp32 and float64 may legitimately disagree on
+the 0/1 derivative mask (and on "x != 0") when z sits within rounding error of a kink.  An entry of
+layer k is *ambiguous* when min(|z|, |z - clamp|) <= tau with tau = TAU_ULPS * 2^-24 * (|b| + sum|w x|),
+the scale of the rounding error of that dot product.  Outside the ambiguous set the GPU's mask must
+equal the oracle's bit for bit; on ambiguous entries the oracle continues with the GPU's decision, so
+that everything downstream (deltas, gradients, weights) is compared like for like.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+TAU_ULPS = 64.0
+TOL = 1e-4
+
+
+def rel_err(gpu: np.ndarray, ora: np.ndarray) -> float:
+    gpu = np.asarray(gpu, dtype=np.float64)
+    ora = np.asarray(ora, dtype=np.float64)
+    assert gpu.shape == ora.shape, (gpu.shape, ora.shape)
+    if ora.size == 0:
+        return 0.0
+    top = np.abs(ora).max()
+    if top == 0.0:
+        return 0.0 if not gpu.any() else float("inf")
+    return float(np.max(np.abs(gpu - ora) / np.maximum(np.abs(ora), 1e-3 * top)))
+
+
+class KinkProtocol:
+    """mask_hook for OracleNet.train_step; `gpu_x(k)` returns the GPU's x^k [B, n] (fp32)."""
+
+    def __init__(self, gpu_x, clamp=32.0, tau_ulps=TAU_ULPS):
+        self.gpu_x, self.clamp, self.tau_ulps = gpu_x, float(clamp), tau_ulps
+        self.ambiguous = 0
+        self.flipped = 0
+        self.entries = 0
+        self.hard_mismatch = 0
+        self.worst = 0.0          # largest margin/tau among entries where the two masks differ
+
+    def __call__(self, k, z, scale, mask):
+        xg = self.gpu_x(k).astype(np.float64)
+        mg = ((xg > 0.0) & (xg < self.clamp)).astype(np.float64)
+        margin = np.minimum(np.abs(z), np.abs(z - self.clamp))
+        tau = self.tau_ulps * 2.0 ** -24 * scale
+        amb = margin <= tau
+        differ = mg != mask
+        self.entries += mask.size
+        self.ambiguous += int(amb.sum())
+        self.flipped += int(differ.sum())
+        self.hard_mismatch += int((differ & ~amb).sum())
+        if differ.any():
+            self.worst = max(self.worst, float((margin[differ] / np.maximum(tau[differ], 1e-300)).max()))
+        return np.where(amb, mg, mask)
+
+
+def ragged_net(rng, n, layers, kmax, scale=0.6, bias_scale=0.1, align4=False):
+    """Random CSR layers with rows of 0..kmax entries (or multiples of 4 when align4)."""
+    rps, cols, vals, biases = [], [], [], []
+    for _ in range(layers):
+        counts = rng.integers(0, kmax + 1, size=n)
+        if align4:
+            counts = counts // 4 * 4
+        counts[rng.integers(0, n)] = kmax
+        rp = np.zeros(n + 1, dtype=np.int32)
+        rp[1:] = np.cumsum(counts)
+        c = np.concatenate([np.sort(rng.choice(n, size=m, replace=False)) for m in counts]).astype(np.int32)
+        rps.append(rp); cols.append(c)
+        vals.append((rng.standard_normal(rp[-1]) * scale).astype(np.float32))
+        biases.append((rng.standard_normal(n) * bias_scale).astype(np.float32))
+    return rps, cols, vals, biases

@@ -1,0 +1,268 @@
+"""GPU-vs-oracle parity through the C ABI (run with -m gpu on a B200).
+
+Same seeded inputs on both sides; activations, deltas, gradients, updated weights and the loss must
+agree within 1e-4 (metric in parity_util.rel_err); derivative masks and final-layer nonzero sets must
+agree bit for bit outside the kink-ambiguous entries (parity_util.KinkProtocol).
+"""
+import numpy as np
+import pytest
+
+import gen
+from oracle import OracleNet
+from parity_util import TAU_ULPS, TOL, KinkProtocol, ragged_net, rel_err
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def torch_cuda():
+    torch = pytest.importorskip("torch")
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_2104_11805_b200.build import build_library
+    build_library()
+    return torch
+
+
+def sdnn():
+    import paper_2104_11805_b200 as pkg
+    return pkg
+
+
+# ----------------------------------------------------------------------------------------------
+def train_parity(torch, arrays, batches, eta, update_bias=False, flags=0, clamp=32.0, expect_live=None):
+    """Runs len(batches) SGD steps on both sides, comparing everything after every step."""
+    pkg = sdnn()
+    rp, col, val, bias = arrays
+    L, n = len(col), len(bias[0])
+    B = batches[0][0].shape[0]
+    h = pkg.Sdnn.create(rp, col, val, bias, max_batch=B, train=True, clamp=clamp, update_bias=update_bias,
+                        flags=pkg.FLAG_KEEP_DEBUG | flags)
+    ora = OracleNet(rp, col, val, bias, clamp=clamp, update_bias=update_bias)
+    stats = dict(ambiguous=0, flipped=0, entries=0, worst=0.0, max_err=0.0, grad_nonzero=False)
+    for x0, y in batches:
+        loss_g = h.train_step(torch.from_numpy(x0).cuda(), torch.from_numpy(y).cuda(), B, eta, want_loss=True)
+        acts = {}
+
+        def gpu_x(k):
+            if k not in acts:
+                acts[k] = h.get_activations(k, B)
+            return acts[k]
+
+        proto = KinkProtocol(gpu_x, clamp=clamp)
+        out = ora.train_step(x0, y, eta, mask_hook=proto)
+        assert proto.hard_mismatch == 0, f"{proto.hard_mismatch} derivative-mask mismatches outside the ambiguous set " \
+                                         f"(worst margin/tau = {proto.worst:.3g})"
+        errs = {}
+        assert np.array_equal(gpu_x(0), x0)
+        for k in range(1, L + 1):
+            errs[f"x{k}"] = rel_err(gpu_x(k), out["x"][k])
+            errs[f"d{k}"] = rel_err(h.get_delta(k, B), out["delta"][k])
+            errs[f"g{k}"] = rel_err(h.get_gradient(k), out["grad"][k - 1])
+            w, b = h.get_weights(k - 1)
+            errs[f"w{k}"] = rel_err(w, ora.w[k - 1])
+            errs[f"b{k}"] = rel_err(b, ora.bias[k - 1])
+            stats["grad_nonzero"] |= bool(np.any(out["grad"][k - 1] != 0.0))
+        errs["loss"] = abs(loss_g - out["loss"]) / max(abs(out["loss"]), 1e-30)
+        worst_key = max(errs, key=errs.get)
+        assert errs[worst_key] <= TOL, f"{worst_key}: rel err {errs[worst_key]:.3g} > {TOL}"
+        stats["max_err"] = max(stats["max_err"], errs[worst_key])
+        for key in ("ambiguous", "flipped", "entries"):
+            stats[key] += getattr(proto, key)
+        stats["worst"] = max(stats["worst"], proto.worst)
+    if expect_live is not None:
+        assert stats["grad_nonzero"] == expect_live
+    h.destroy()
+    return stats
+
+
+def infer_parity(torch, arrays, x0, max_batch, host=False, clamp=32.0, expect_nonempty=None):
+    pkg = sdnn()
+    rp, col, val, bias = arrays
+    L, n = len(col), len(bias[0])
+    cnt = x0.shape[0]
+    h = pkg.Sdnn.create(rp, col, val, bias, max_batch=max_batch, clamp=clamp)
+    cap = cnt * n
+    if host:
+        y = np.empty((cnt, n), dtype=np.float32); c = np.empty(cnt, dtype=np.int32); idx = np.empty(cap, dtype=np.int32)
+        total = h.infer_batch(x0, cnt, y, c, idx, cap, want_total=True, host=True)
+    else:
+        yd = torch.empty((cnt, n), dtype=torch.float32, device="cuda")
+        cd = torch.empty(cnt, dtype=torch.int32, device="cuda")
+        idd = torch.empty(cap, dtype=torch.int32, device="cuda")
+        total = h.infer_batch(torch.from_numpy(x0).cuda(), cnt, yd, cd, idd, cap, want_total=True)
+        y, c, idx = yd.cpu().numpy(), cd.cpu().numpy(), idd.cpu().numpy()
+    h.destroy()
+
+    ora = OracleNet(rp, col, val, bias, clamp=clamp)
+    x = x0.astype(np.float64)
+    for k in range(L - 1):
+        _, x, _ = ora.forward_layer(k, x)
+    z, xl, scale = ora.forward_layer(L - 1, x, want_scale=True)
+    assert rel_err(y, xl) <= TOL
+    assert total == int(c.sum())
+    amb = np.abs(z) <= TAU_ULPS * 2.0 ** -24 * scale
+    starts = np.concatenate([[0], np.cumsum(c)])
+    n_amb = 0
+    for b in range(cnt):
+        ids = idx[starts[b]:starts[b + 1]]
+        assert np.all(np.diff(ids) > 0), "ids must ascend"
+        got = np.zeros(n, dtype=bool); got[ids] = True
+        assert np.array_equal(got, y[b] != 0.0), "ids must list exactly the nonzero outputs"
+        want = xl[b] != 0.0
+        bad = (got != want) & ~amb[b]
+        assert not bad.any(), f"input {b}: nonzero set differs at {np.flatnonzero(bad)[:8]}"
+        n_amb += int((got != want).sum())
+    if expect_nonempty is not None:
+        assert (total > 0) == expect_nonempty
+    return dict(total=total, flipped=n_amb)
+
+
+def batches_for(spec, B, steps):
+    return [(gen.inputs(spec, B, step=s), gen.targets(spec, B, step=s)) for s in range(steps)]
+
+
+# ---------------------------------------------------------------------------------------------- train
+@pytest.mark.parametrize("B", [1, 3, 4, 7, 16, 33, 64, 100, 128])
+@pytest.mark.parametrize("align4", [False, True])
+def test_train_ragged_small(torch_cuda, B, align4):
+    """Ragged / empty rows, every lane-group width, scalar and vector index paths, bias update on."""
+    rng = np.random.default_rng(100 + B)
+    arrays = ragged_net(rng, n=203, layers=5, kmax=12, align4=align4)
+    batches = [(rng.uniform(0, 1.5, size=(B, 203)).astype(np.float32), rng.uniform(0, 1, size=(B, 203)).astype(np.float32))
+               for _ in range(3)]
+    st = train_parity(torch_cuda, arrays, batches, eta=0.01, update_bias=(B % 2 == 1), expect_live=True)
+    assert st["entries"] > 0
+
+
+def test_train_no_graph_matches(torch_cuda):
+    rng = np.random.default_rng(5)
+    arrays = ragged_net(rng, n=130, layers=4, kmax=8)
+    batches = [(rng.uniform(0, 1.5, size=(16, 130)).astype(np.float32), rng.uniform(0, 1, size=(16, 130)).astype(np.float32))
+               for _ in range(2)]
+    train_parity(torch_cuda, arrays, batches, eta=0.01, flags=sdnn().FLAG_NO_GRAPH, expect_live=True)
+
+
+@pytest.mark.parametrize("variant,live", [("base", False), ("live", True)])
+def test_train_cfg1_full(torch_cuda, variant, live):
+    """Config 1 training: 1024 x 120, per-sample SGD (B = 1); dead as specified, live with He weights."""
+    spec = gen.CFG1_TRAIN if variant == "base" else gen.CFG1_TRAIN.live()
+    st = train_parity(torch_cuda, gen.network(spec), batches_for(spec, 1, 8), eta=1e-3, expect_live=live)
+    print(variant, st)
+
+
+def test_train_saturating_hits_upper_kink(torch_cuda):
+    spec = gen.CFG1_TRAIN.scaled(512, 12).saturating()
+    train_parity(torch_cuda, gen.network(spec), batches_for(spec, 16, 2), eta=1e-3)
+
+
+@pytest.mark.parametrize("spec,B,steps", [
+    (gen.CFG3.scaled(2048, 24).live(), 64, 3),
+    (gen.CFG3.scaled(2048, 24), 64, 1),
+    (gen.CFG5.scaled(65536, 6).live(), 16, 2),
+    (gen.CFG5.scaled(8192, 40).live(), 16, 2),
+])
+def test_train_scaled_configs(torch_cuda, spec, B, steps):
+    st = train_parity(torch_cuda, gen.network(spec), batches_for(spec, B, steps), eta=1e-3)
+    print(spec.name, st)
+
+
+def test_train_cfg3_live_full_size(torch_cuda):
+    """Config 3 at full size (16384 x 480, B = 64), live companion, one step."""
+    spec = gen.CFG3.live()
+    st = train_parity(torch_cuda, gen.network(spec), batches_for(spec, 64, 1), eta=1e-3, expect_live=True)
+    print(spec.name, st)
+
+
+# ---------------------------------------------------------------------------------------------- inference
+@pytest.mark.parametrize("cnt,max_batch", [(1, 1), (5, 8), (37, 16), (130, 64), (300, 256), (700, 512)])
+@pytest.mark.parametrize("host", [False, True])
+def test_infer_ragged_small(torch_cuda, cnt, max_batch, host):
+    rng = np.random.default_rng(cnt)
+    arrays = ragged_net(rng, n=301, layers=4, kmax=10, scale=0.5)
+    x0 = rng.uniform(0, 1.0, size=(cnt, 301)).astype(np.float32)
+    infer_parity(torch_cuda, arrays, x0, max_batch, host=host, expect_nonempty=True)
+
+
+@pytest.mark.parametrize("variant", ["base", "live", "sat"])
+def test_infer_cfg1_full(torch_cuda, variant):
+    spec = {"base": gen.CFG1_INF, "live": gen.CFG1_INF.live(), "sat": gen.CFG1_INF.saturating()}[variant]
+    st = infer_parity(torch_cuda, gen.network(spec), gen.inputs(spec, 256), 256, expect_nonempty=(variant != "base"))
+    print(variant, st)
+
+
+@pytest.mark.parametrize("variant", ["base", "live"])
+def test_infer_cfg2_two_tiles(torch_cuda, variant):
+    """Config 2 net at full size; one full tile of 1024 plus a ragged tile of 608 inputs."""
+    spec = gen.CFG2 if variant == "base" else gen.CFG2.live()
+    st = infer_parity(torch_cuda, gen.network(spec), gen.inputs(spec, 1632), 1024, expect_nonempty=(variant == "live"))
+    print(variant, st)
+
+
+@pytest.mark.parametrize("variant", ["base", "live"])
+def test_infer_cfg4_sampled(torch_cuda, variant):
+    """Config 4 net at full size (65536 x 120, banded-permuted) on a sample of 96 inputs, host buffers."""
+    spec = gen.CFG4 if variant == "base" else gen.CFG4.live()
+    st = infer_parity(torch_cuda, gen.network(spec), gen.inputs(spec, 96, start=59000), 64, host=True,
+                      expect_nonempty=(variant == "live"))
+    print(variant, st)
+
+
+# ---------------------------------------------------------------------------------------------- API behaviour on a device
+def test_capacity_too_small_reports_needed(torch_cuda):
+    pkg = sdnn()
+    rng = np.random.default_rng(1)
+    arrays = ragged_net(rng, n=64, layers=2, kmax=6)
+    h = pkg.Sdnn.create(*arrays, max_batch=8)
+    x0 = torch_cuda.from_numpy(rng.uniform(0, 1, size=(8, 64)).astype(np.float32)).cuda()
+    idx = torch_cuda.full((4,), -1, dtype=torch_cuda.int32, device="cuda")
+    with pytest.raises(pkg.SdnnError) as ei:
+        h.infer_batch(x0, 8, None, None, idx, 4, want_total=True)
+    assert ei.value.code == -1 and h.last_total > 4
+    assert h.infer_batch(x0, 0, None, None, None, 0, want_total=True) == 0       # empty batch is a no-op
+    h.destroy()
+
+
+def test_state_and_argument_errors(torch_cuda):
+    pkg = sdnn()
+    rng = np.random.default_rng(2)
+    arrays = ragged_net(rng, n=32, layers=2, kmax=4)
+    h = pkg.Sdnn.create(*arrays, max_batch=4)                                   # inference handle
+    x = torch_cuda.zeros((4, 32), device="cuda")
+    with pytest.raises(pkg.SdnnError) as ei:
+        h.train_step(x, x, 4, 0.1)
+    assert ei.value.code == -5
+    h.destroy()
+    h = pkg.Sdnn.create(*arrays, max_batch=4, train=True)
+    with pytest.raises(pkg.SdnnError) as ei:
+        h.train_step(x, x, 5, 0.1)
+    assert ei.value.code == -1
+    with pytest.raises(pkg.SdnnError) as ei:
+        h.get_activations(0, 4)
+    assert ei.value.code == -5
+    h.destroy()
+
+
+def test_deferred_creation_and_resume(torch_cuda):
+    """Layer-by-layer loading gives the same handle; get_weights -> create resumes training exactly."""
+    pkg = sdnn()
+    spec = gen.CFG1_TRAIN.scaled(256, 6).live()
+    rp, col, val, bias = gen.network(spec)
+    (x0, y), = batches_for(spec, 8, 1)
+    xd, yd = torch_cuda.from_numpy(x0).cuda(), torch_cuda.from_numpy(y).cuda()
+    a = pkg.Sdnn.create(rp, col, val, bias, max_batch=8, train=True)
+    b = pkg.Sdnn.create_deferred(6, 256, [len(c) for c in col], max_batch=8, train=True)
+    with pytest.raises(pkg.SdnnError):
+        b.train_step(xd, yd, 8, 1e-3)                                           # not finalized yet
+    for l in (3, 0, 5, 1, 4, 2):
+        b.load_layer(l, rp[l], col[l], val[l], bias[l])
+    b.finalize()
+    la, lb = a.train_step(xd, yd, 8, 1e-2, want_loss=True), b.train_step(xd, yd, 8, 1e-2, want_loss=True)
+    assert abs(la - lb) <= 1e-6 * abs(la)
+    wa = [a.get_weights(l) for l in range(6)]
+    c = pkg.Sdnn.create(rp, col, [w for w, _ in wa], [bb for _, bb in wa], max_batch=8, train=True)
+    l2a, l2c = a.train_step(xd, yd, 8, 1e-2, want_loss=True), c.train_step(xd, yd, 8, 1e-2, want_loss=True)
+    assert abs(l2a - l2c) <= 1e-6 * abs(l2a) and l2a < la
+    for l in range(6):
+        assert rel_err(c.get_weights(l)[0], a.get_weights(l)[0]) <= 1e-6
+    for h in (a, b, c):
+        h.destroy()

@@ -71,7 +71,8 @@ typedef struct {
     int32_t  train;        /* 0: inference only (no stored activations); 1: sdnn_train_step allowed */
     int32_t  update_bias;  /* 1: b^k <- b^k - eta * mean_b delta^k_b (bias read as a column of W^k); 0: bias frozen */
     uint32_t flags;        /* SDNN_FLAG_* */
-    void*    cuda_stream;  /* cudaStream_t to issue work on; NULL = default stream */
+    void*    cuda_stream;  /* cudaStream_t to issue work on; NULL = a stream the handle creates, which orders
+                              itself against the legacy default stream like any blocking stream */
     int32_t  device;       /* CUDA device ordinal; -1 = the current device */
 } sdnn_config;
 
@@ -147,6 +148,14 @@ int sdnn_train_step_host(sdnn_t* h, const float* x0, const float* target, int32_
  * Synchronises the stream.  Creating a new handle from these arrays resumes training.
  */
 int sdnn_get_weights(sdnn_t* h, int32_t layer, float* values_out, float* bias_out);
+
+/*
+ * Overwrites the parameters of one layer (0-based) from host arrays in the caller's CSR order
+ * (restore from a checkpoint without re-creating the handle; the pattern cannot change).
+ *   values  host float[nnz_l], or NULL to keep;   bias  host float[N], or NULL to keep
+ * Values must be finite (else SDNN_ERR_BAD_CSR).  Synchronises the stream.
+ */
+int sdnn_set_weights(sdnn_t* h, int32_t layer, const float* values, const float* bias);
 
 /*
  * Inspection of the last train step (tests, diagnostics).  All outputs are host arrays,

@@ -93,6 +93,15 @@ class OracleNet:
             if self.row_ptr[k].shape != (self.n + 1,) or self.col[k].shape != self.w[k].shape:
                 raise ValueError("inconsistent CSR arrays")
 
+    def quantize_state(self):
+        """Rounds weights and biases to the nearest fp32 numbers (kept as float64).
+
+        The GPU library stores its parameters in fp32 between steps.  A parity harness that wants both
+        sides to START a step from identical numbers calls this and loads the result into the library;
+        within the step all oracle arithmetic stays float64.  Not called by train_step itself."""
+        self.w = [w.astype(np.float32).astype(np.float64) for w in self.w]
+        self.bias = [b.astype(np.float32).astype(np.float64) for b in self.bias]
+
     # ---- single steps -------------------------------------------------------------------------
     def forward_layer(self, k: int, x_prev: np.ndarray, want_scale: bool = False):
         """Layer k (0-based: uses W^{k+1}) on x_prev [B, n] -> (z, x, scale); scale = |b| + sum|w x| or None."""

@@ -43,6 +43,7 @@ _PROTOS = {
     "sdnn_train_step": (ctypes.c_int, [_vp, _vp, _vp, _i32, _f32, ctypes.POINTER(_f32)]),
     "sdnn_train_step_host": (ctypes.c_int, [_vp, _vp, _vp, _i32, _f32, ctypes.POINTER(_f32)]),
     "sdnn_get_weights": (ctypes.c_int, [_vp, _i32, _vp, _vp]),
+    "sdnn_set_weights": (ctypes.c_int, [_vp, _i32, _vp, _vp]),
     "sdnn_get_activations": (ctypes.c_int, [_vp, _i32, _vp]),
     "sdnn_get_delta": (ctypes.c_int, [_vp, _i32, _vp]),
     "sdnn_get_gradient": (ctypes.c_int, [_vp, _i32, _vp]),
@@ -172,6 +173,11 @@ class Sdnn:
         b = np.empty(self.n_neurons, dtype=np.float32) if want_bias else None
         self._check(self._lib.sdnn_get_weights(self._h, layer, v.ctypes.data, b.ctypes.data if want_bias else None))
         return (v, b) if want_bias else v
+
+    def set_weights(self, layer, values=None, bias=None):
+        v = None if values is None else _np(values, np.float32)
+        b = None if bias is None else _np(bias, np.float32)
+        self._check(self._lib.sdnn_set_weights(self._h, layer, _addr(v), _addr(b)))
 
     def get_activations(self, layer, B):
         out = np.empty((B, self.n_neurons), dtype=np.float32)

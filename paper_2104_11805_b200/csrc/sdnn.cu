@@ -29,6 +29,7 @@ struct sdnn {
     int L = 0, N = 0;
     sdnn_config cfg{};
     cudaStream_t stream = nullptr;
+    bool own_stream = false;
     int device = 0;
     bool finalized = false, stepped = false;
     std::vector<int64_t> nnz, off;      // stored entries per layer; offset of the layer in the arenas (elements)
@@ -360,9 +361,10 @@ int64_t sdnn_device_bytes(const sdnn_t* h) { return h ? h->dev_bytes : 0; }
 void sdnn_destroy(sdnn_t* h) {
     if (!h) return;
     cudaSetDevice(h->device);
-    cudaStreamSynchronize(h->stream);
+    if (h->stream || h->own_stream) cudaStreamSynchronize(h->stream);
     if (h->graph) cudaGraphExecDestroy(h->graph);
     for (void* p : h->allocs) cudaFree(p);
+    if (h->own_stream) cudaStreamDestroy(h->stream);
     delete h;
 }
 
@@ -393,6 +395,11 @@ int sdnn_create_deferred(sdnn_t** out, int32_t n_layers, int32_t n_neurons, cons
         h->device = cfg->device;
     } else if ((e = cudaGetDevice(&h->device)) != cudaSuccess) {
         return bail(cuda_fail(h, e, "cudaGetDevice"));
+    }
+    if (!h->stream) {   // the legacy default stream cannot be captured into a graph: use a blocking stream of our own,
+                        // which still orders itself against work on the legacy default stream
+        if ((e = cudaStreamCreate(&h->stream)) != cudaSuccess) { h->stream = nullptr; return bail(cuda_fail(h, e, "cudaStreamCreate")); }
+        h->own_stream = true;
     }
     h->nnz.assign(nnz_per_layer, nnz_per_layer + n_layers);
     h->off.resize(n_layers);
@@ -582,6 +589,24 @@ int sdnn_get_weights(sdnn_t* h, int32_t layer, float* values_out, float* bias_ou
     if (values_out && h->nnz[layer])
         CU(h, cudaMemcpy(values_out, h->d_val + h->off[layer], (size_t)h->nnz[layer] * sizeof(float), cudaMemcpyDeviceToHost));
     if (bias_out) CU(h, cudaMemcpy(bias_out, h->d_bias + (size_t)layer * h->N, (size_t)h->N * sizeof(float), cudaMemcpyDeviceToHost));
+    return SDNN_OK;
+}
+
+int sdnn_set_weights(sdnn_t* h, int32_t layer, const float* values, const float* bias) {
+    if (!h) return SDNN_ERR_INVALID_ARG;
+    if (!h->finalized) return fail(h, SDNN_ERR_STATE, "handle is not finalized");
+    if (layer < 0 || layer >= h->L) return fail(h, SDNN_ERR_INVALID_ARG, "layer %d outside [0, %d)", layer, h->L);
+    if (values)
+        for (int64_t p = 0; p < h->nnz[layer]; ++p)
+            if (!std::isfinite(values[p])) return fail(h, SDNN_ERR_BAD_CSR, "layer %d: non-finite value at entry %lld", layer, (long long)p);
+    if (bias)
+        for (int i = 0; i < h->N; ++i)
+            if (!std::isfinite(bias[i])) return fail(h, SDNN_ERR_BAD_CSR, "layer %d: non-finite bias at row %d", layer, i);
+    CU(h, cudaSetDevice(h->device));
+    CU(h, cudaStreamSynchronize(h->stream));
+    if (values && h->nnz[layer])
+        CU(h, cudaMemcpy(h->d_val + h->off[layer], values, (size_t)h->nnz[layer] * sizeof(float), cudaMemcpyHostToDevice));
+    if (bias) CU(h, cudaMemcpy(h->d_bias + (size_t)layer * h->N, bias, (size_t)h->N * sizeof(float), cudaMemcpyHostToDevice));
     return SDNN_OK;
 }
 

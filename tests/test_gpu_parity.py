@@ -9,7 +9,7 @@ import pytest
 
 import gen
 from oracle import OracleNet
-from parity_util import TAU_ULPS, TOL, KinkProtocol, ragged_net, rel_err
+from parity_util import TAU_ULPS, TOL, KinkProtocol, check_close, ragged_net, rel_err
 
 pytestmark = pytest.mark.gpu
 
@@ -29,8 +29,15 @@ def sdnn():
 
 
 # ----------------------------------------------------------------------------------------------
-def train_parity(torch, arrays, batches, eta, update_bias=False, flags=0, clamp=32.0, expect_live=None):
-    """Runs len(batches) SGD steps on both sides, comparing everything after every step."""
+def train_parity(torch, arrays, batches, eta, update_bias=False, flags=0, clamp=32.0, expect_live=None, sync=True):
+    """Runs len(batches) SGD steps on both sides, comparing everything after every step.
+
+    sync=True: before every step after the first the oracle rounds its parameters to fp32 (the library's
+    storage precision) and they are loaded into the library, so both sides start each step from identical
+    numbers; rounding differences of earlier steps would otherwise be amplified step after step by the
+    training dynamics themselves (observed: x 10 in five steps on the live 1024 x 120 net), which says
+    nothing about one step's arithmetic.  sync=False lets the two trajectories run free (checks that
+    parameters persist across calls)."""
     pkg = sdnn()
     rp, col, val, bias = arrays
     L, n = len(col), len(bias[0])
@@ -39,7 +46,11 @@ def train_parity(torch, arrays, batches, eta, update_bias=False, flags=0, clamp=
                         flags=pkg.FLAG_KEEP_DEBUG | flags)
     ora = OracleNet(rp, col, val, bias, clamp=clamp, update_bias=update_bias)
     stats = dict(ambiguous=0, flipped=0, entries=0, worst=0.0, max_err=0.0, grad_nonzero=False)
-    for x0, y in batches:
+    for step, (x0, y) in enumerate(batches):
+        if sync and step > 0:
+            ora.quantize_state()
+            for l in range(L):
+                h.set_weights(l, ora.w[l], ora.bias[l])
         loss_g = h.train_step(torch.from_numpy(x0).cuda(), torch.from_numpy(y).cuda(), B, eta, want_loss=True)
         acts = {}
 
@@ -55,12 +66,12 @@ def train_parity(torch, arrays, batches, eta, update_bias=False, flags=0, clamp=
         errs = {}
         assert np.array_equal(gpu_x(0), x0)
         for k in range(1, L + 1):
-            errs[f"x{k}"] = rel_err(gpu_x(k), out["x"][k])
-            errs[f"d{k}"] = rel_err(h.get_delta(k, B), out["delta"][k])
-            errs[f"g{k}"] = rel_err(h.get_gradient(k), out["grad"][k - 1])
+            errs[f"x{k}"] = check_close(gpu_x(k), out["x"][k], f"step {step} x^{k}")
+            errs[f"d{k}"] = check_close(h.get_delta(k, B), out["delta"][k], f"step {step} delta^{k}")
+            errs[f"g{k}"] = check_close(h.get_gradient(k), out["grad"][k - 1], f"step {step} G^{k}")
             w, b = h.get_weights(k - 1)
-            errs[f"w{k}"] = rel_err(w, ora.w[k - 1])
-            errs[f"b{k}"] = rel_err(b, ora.bias[k - 1])
+            errs[f"w{k}"] = check_close(w, ora.w[k - 1], f"step {step} W^{k}")
+            errs[f"b{k}"] = check_close(b, ora.bias[k - 1], f"step {step} b^{k}")
             stats["grad_nonzero"] |= bool(np.any(out["grad"][k - 1] != 0.0))
         errs["loss"] = abs(loss_g - out["loss"]) / max(abs(out["loss"]), 1e-30)
         worst_key = max(errs, key=errs.get)
@@ -98,7 +109,7 @@ def infer_parity(torch, arrays, x0, max_batch, host=False, clamp=32.0, expect_no
     for k in range(L - 1):
         _, x, _ = ora.forward_layer(k, x)
     z, xl, scale = ora.forward_layer(L - 1, x, want_scale=True)
-    assert rel_err(y, xl) <= TOL
+    check_close(y, xl, "x^L")
     assert total == int(c.sum())
     amb = np.abs(z) <= TAU_ULPS * 2.0 ** -24 * scale
     starts = np.concatenate([[0], np.cumsum(c)])
@@ -132,6 +143,15 @@ def test_train_ragged_small(torch_cuda, B, align4):
                for _ in range(3)]
     st = train_parity(torch_cuda, arrays, batches, eta=0.01, update_bias=(B % 2 == 1), expect_live=True)
     assert st["entries"] > 0
+
+
+def test_train_free_running_trajectories_stay_close(torch_cuda):
+    """No re-synchronisation between steps: parameters persist inside the handle across calls."""
+    rng = np.random.default_rng(77)
+    arrays = ragged_net(rng, n=150, layers=4, kmax=8)
+    batches = [(rng.uniform(0, 1.5, size=(8, 150)).astype(np.float32), rng.uniform(0, 1, size=(8, 150)).astype(np.float32))
+               for _ in range(4)]
+    train_parity(torch_cuda, arrays, batches, eta=0.005, sync=False, expect_live=True)
 
 
 def test_train_no_graph_matches(torch_cuda):

@@ -1,0 +1,422 @@
+#!/usr/bin/env python
+"""Benchmark of the sparse-DNN SGD hot path on B200 (one process per GPU).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+Default workload: the largest training configuration (65536 neurons x 1920 layers, 32 nonzeros per
+row, minibatch 16).  A "step" is one pass of the whole path over one fresh minibatch: forward through
+all layers, loss and output gradient, then backward product + masked gradient + weight update for
+every layer.  Inference workloads time one sdnn_infer_batch call over all inputs per step.
+
+Prints ONE JSON line (rank 0).  `value` = edges/s with inputs resident in HBM; `e2e` = the same metric
+through the host-buffer entry point (pinned host inputs, loss / counts read back).  `roofline` is for
+the dominant kernel, timed by events on the library's stream inside the timed steps.  `cpu_baseline`
+times the float64 CPU oracle on a bounded slice of the same workload.  With --impl reference only the
+oracle runs (rank 0; the other ranks exit).  Nothing here reads files outside the repository.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import gen  # noqa: E402
+
+ETA = 1e-3
+
+# name -> (spec, kind, batch or tile, inputs per step)
+WORKLOADS = {
+    "cfg5": (gen.CFG5, "train", 16, 16),
+    "cfg5-live": (gen.CFG5.live(), "train", 16, 16),
+    "cfg3": (gen.CFG3, "train", 64, 64),
+    "cfg3-live": (gen.CFG3.live(), "train", 64, 64),
+    "cfg1-train": (gen.CFG1_TRAIN, "train", 1, 1),
+    "cfg1-inf": (gen.CFG1_INF, "infer", 256, 256),
+    "cfg2": (gen.CFG2, "infer", 1024, 60000),
+    "cfg2-live": (gen.CFG2.live(), "infer", 1024, 60000),
+    "cfg4": (gen.CFG4, "infer", 1024, 60000),
+    "cfg4-live": (gen.CFG4.live(), "infer", 1024, 60000),
+}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period: float = 0.02):
+        self.index, self.period = index, period
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.dev = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.dev, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    NAMES = {0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+             0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+             0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting"}
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.dev, nv.NVML_CLOCK_SM))
+                bits = nv.nvmlDeviceGetCurrentClocksEventReasons(self.dev)
+                for bit, name in self.NAMES.items():
+                    if bits & bit and name != "gpu_idle":
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["unavailable"]}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def oracle_train_sample(spec, B, layers, steps, warmup):
+    """Times the float64 oracle's train step on the first `layers` layers of the net (full N, full B)."""
+    from oracle import OracleNet
+    sl = spec.sliced(layers)
+    ora = OracleNet(*gen.network(sl))
+    times = []
+    for s in range(warmup + steps):
+        x0, y = gen.inputs(sl, B, step=s), gen.targets(sl, B, step=s)
+        t = time.perf_counter()
+        ora.train_step(x0, y, ETA, keep=())
+        dt = time.perf_counter() - t
+        if s >= warmup:
+            times.append(dt)
+    edges = B * sl.total_nnz
+    return edges, times
+
+
+def oracle_infer_sample(spec, inputs, layers, steps, warmup):
+    from oracle import OracleNet
+    sl = spec.sliced(layers)
+    ora = OracleNet(*gen.network(sl))
+    x0 = gen.inputs(sl, inputs)
+    times = []
+    for s in range(warmup + steps):
+        t = time.perf_counter()
+        ora.infer(x0)
+        dt = time.perf_counter() - t
+        if s >= warmup:
+            times.append(dt)
+    return inputs * sl.total_nnz, times
+
+
+def oracle_sample_shape(spec, kind, batch, budget_edges):
+    """Slice of the workload (layers, inputs) holding about `budget_edges` edge-visits per oracle step."""
+    if kind == "train":
+        layers = int(max(1, min(spec.layers, budget_edges // (batch * spec.nnz_per_layer))))
+        return layers, batch
+    inputs = int(min(batch, 256))
+    layers = int(max(1, min(spec.layers, budget_edges // (inputs * spec.nnz_per_layer))))
+    return layers, inputs
+
+
+def run_reference(args, spec, kind, batch, wname):
+    """The reference arm: the oracle as it stands, on the host cores, on a bounded sample per step."""
+    cores = os.cpu_count()
+    layers, inputs = oracle_sample_shape(spec, kind, batch, budget_edges=1.0e9)
+    if kind == "train":
+        edges, times = oracle_train_sample(spec, inputs, layers, args.steps, args.warmup)
+        sample = f"train step on layers 1..{layers} of {spec.layers} at full width N={spec.n}, B={inputs}"
+    else:
+        edges, times = oracle_infer_sample(spec, inputs, layers, args.steps, args.warmup)
+        sample = f"inference of {inputs} inputs through layers 1..{layers} of {spec.layers} at full width N={spec.n}"
+    ms = 1e3 * float(np.mean(times))
+    value = edges / (ms * 1e-3)
+    line = {
+        "impl": "reference", "metric": metric_name(kind), "value": value, "unit": "edges/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(wname, spec, kind, batch),
+        "cpu_baseline": {"value": value, "unit": "edges/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "edges/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def metric_name(kind):
+    return "edges_per_sec_train_step" if kind == "train" else "edges_per_sec_inference"
+
+
+def workload_config(wname, spec, kind, batch):
+    cfg = {"workload": f"{wname}: {spec.name} {spec.n} neurons x {spec.layers} layers, {spec.k} nnz/row, "
+                       + (f"minibatch {batch}, fresh minibatch per step" if kind == "train" else f"batch tile {batch}"),
+           "mode": "dense (no data-dependent skipping)",
+           "l2": "working set per step (weights + activations) is larger than L2; no explicit flush"
+           if spec.total_nnz * 8 > 256e6 else "explicit L2 flush (256 MB write) before every timed step"}
+    return cfg
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="cfg5", choices=sorted(WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", type=int, default=None, help="use only the first LAYERS layers (profiling captures)")
+    ap.add_argument("--inputs", type=int, default=None, help="inference: number of inputs per call")
+    ap.add_argument("--flags", type=lambda s: int(s, 0), default=0, help="extra SDNN_FLAG_* bits")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.layers is None:
+        args.warmup = 3
+    spec, kind, batch, n_inputs = WORKLOADS[args.workload]
+    if args.layers:
+        spec = spec.sliced(args.layers)
+    if args.inputs and kind == "infer":
+        n_inputs = args.inputs
+    if args.steps is None:
+        args.steps = 10 if kind == "train" else 3
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if rank == 0:
+            run_reference(args, spec, kind, batch, args.workload)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    import paper_2104_11805_b200 as pkg
+    from paper_2104_11805_b200.build import build_library
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    build_library()
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    stream = torch.cuda.Stream()
+    hbm_peak, peak_src = measured_peaks()
+
+    # ------------------------------------------------------------------ build the net, layer by layer
+    t_setup = time.perf_counter()
+    L, N = spec.layers, spec.n
+    flags = args.flags
+    h = pkg.Sdnn.create_deferred(L, N, [spec.nnz_per_layer] * L, max_batch=batch, train=(kind == "train"),
+                                 flags=flags, stream=stream.cuda_stream, device=local_rank)
+    for l in range(L):
+        h.load_layer(l, *gen.layer(spec, l))
+    h.finalize()
+    setup_s = time.perf_counter() - t_setup
+
+    total = args.warmup + args.steps
+    edges_per_step = n_inputs * spec.total_nnz
+    flush = None if spec.total_nnz * 8 > 256e6 else torch.empty(64 << 20, dtype=torch.float32, device="cuda")
+
+    def l2_flush():
+        if flush is not None:
+            flush.fill_(1.0)
+
+    with torch.cuda.stream(stream):
+        if kind == "train":
+            # every rank trains its own replica on its own stream of minibatches (replicas only: no collective)
+            xs = [torch.from_numpy(gen.inputs(spec, batch, step=rank * 1000 + s)).cuda() for s in range(total)]
+            ys = [torch.from_numpy(gen.targets(spec, batch, step=rank * 1000 + s)).cuda() for s in range(total)]
+            hx = [x.cpu().pin_memory() for x in xs]
+            hy = [y.cpu().pin_memory() for y in ys]
+
+            def step(i):
+                h.train_step(xs[i], ys[i], batch, ETA)
+
+            def step_e2e(i):
+                return h.train_step(hx[i], hy[i], batch, ETA, want_loss=True, host=True)
+
+            h2d, d2h = 2 * batch * N * 4, 4
+        else:
+            # the batch is sharded over ranks: each rank infers its own n_inputs inputs (weak scaling, no collective)
+            chunk = 4096
+            x_all = torch.empty((n_inputs, N), dtype=torch.float32, device="cuda")
+            for s0 in range(0, n_inputs, chunk):
+                c = min(chunk, n_inputs - s0)
+                x_all[s0:s0 + c] = torch.from_numpy(gen.inputs(spec, c, start=rank * n_inputs + s0)).cuda()
+            counts = torch.empty(n_inputs, dtype=torch.int32, device="cuda")
+            cap = 1 << 20
+            idx = torch.empty(cap, dtype=torch.int32, device="cuda")
+            n_e2e = min(n_inputs, 8192)
+            hx_all = x_all[:n_e2e].cpu().pin_memory()
+            hcounts = torch.empty(n_e2e, dtype=torch.int32).pin_memory()
+
+            def step(i):
+                h.infer_batch(x_all, n_inputs, None, counts, None, 0)
+
+            def step_e2e(i):
+                return h.infer_batch(hx_all, n_e2e, None, hcounts, None, 0, want_total=True, host=True)
+
+            h2d, d2h = n_e2e * N * 4, n_e2e * 4 + 8
+
+        def barrier():
+            torch.cuda.synchronize()
+            if world > 1:
+                dist.barrier()
+            torch.cuda.synchronize()
+
+        # ---------------------------------------------------------------- device-resident timing
+        for i in range(args.warmup):
+            l2_flush()
+            step(i)
+        barrier()
+        launches0 = h.kernel_launches()
+        fwd_ms = bwd_ms = 0.0
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        step_ms = []
+        with ClockSampler(local_rank) as clocks:
+            if flush is None and kind == "train":
+                e0.record(stream)
+                for i in range(args.steps):
+                    step(args.warmup + i)
+                e1.record(stream)
+                barrier()
+                total_ms = e0.elapsed_time(e1)
+            else:
+                total_ms = 0.0
+                for i in range(args.steps):
+                    l2_flush()
+                    a = torch.cuda.Event(enable_timing=True)
+                    b = torch.cuda.Event(enable_timing=True)
+                    a.record(stream)
+                    step(args.warmup + i)
+                    b.record(stream)
+                    torch.cuda.synchronize()
+                    step_ms.append(a.elapsed_time(b))
+                    total_ms += step_ms[-1]
+                barrier()
+        launches = h.kernel_launches() - launches0
+        if kind == "train":
+            fwd_ms, bwd_ms = h.get_phase_times()      # last timed step
+        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+        if world > 1:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+        ms_per_step = total_ms / args.steps
+        value = world * edges_per_step / (ms_per_step * 1e-3)
+
+        # ---------------------------------------------------------------- end-to-end through host buffers
+        e2e = None
+        if not args.no_e2e:
+            k_e2e = args.steps
+            step_e2e(0)
+            barrier()
+            a = torch.cuda.Event(enable_timing=True)
+            b = torch.cuda.Event(enable_timing=True)
+            t0 = time.perf_counter()
+            a.record(stream)
+            for i in range(k_e2e):
+                step_e2e(args.warmup + i if kind == "train" else i)
+            b.record(stream)
+            barrier()
+            wall_ms = 1e3 * (time.perf_counter() - t0)
+            dev_ms = a.elapsed_time(b)
+            t = torch.tensor([max(wall_ms, dev_ms)], dtype=torch.float64, device="cuda")
+            if world > 1:
+                dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            per = float(t.item()) / k_e2e
+            e2e_edges = edges_per_step if kind == "train" else n_e2e * spec.total_nnz
+            e2e = {"value": world * e2e_edges / (per * 1e-3), "unit": "edges/s", "h2d_bytes_per_step": h2d,
+                   "d2h_bytes_per_step": d2h, "ms_per_step": per,
+                   "api": "sdnn_train_step_host" if kind == "train" else f"sdnn_infer_batch_host on {n_e2e} inputs"}
+
+    # -------------------------------------------------------------------- roofline of the dominant kernel
+    nnz_l = spec.nnz_per_layer
+    if kind == "train":
+        ld = max(4, 1 << (batch - 1).bit_length())
+        # backward+update launch: index read + value read + value write per stored entry, x^{k-1} tile read once
+        bwd_bytes = 12 * nnz_l + N * ld * 4
+        fwd_bytes = 8 * nnz_l + N * ld * 4
+        dom = "backward_kernel" if bwd_ms >= fwd_ms else "forward_kernel"
+        per_launch_ms = (bwd_ms if dom == "backward_kernel" else fwd_ms) / L
+        alg = bwd_bytes if dom == "backward_kernel" else fwd_bytes
+        extra = {"fwd_ms_per_step": fwd_ms, "bwd_ms_per_step": bwd_ms,
+                 "fwd_GBps": fwd_bytes * L / (fwd_ms * 1e-3) / 1e9 if fwd_ms else None,
+                 "bwd_GBps": bwd_bytes * L / (bwd_ms * 1e-3) / 1e9 if bwd_ms else None,
+                 "step_bytes": (fwd_bytes + bwd_bytes) * L,
+                 "step_GBps": (fwd_bytes + bwd_bytes) * L / (ms_per_step * 1e-3) / 1e9}
+    else:
+        tiles = (n_inputs + batch - 1) // batch
+        dom = "forward_kernel"
+        per_launch_ms = ms_per_step / (tiles * L)      # includes the (small) transpose and count kernels of each tile
+        # per launch: the layer's indices and values once, the activation tile read and written once
+        alg = 8 * nnz_l + 2 * N * min(batch, n_inputs) * 4
+        extra = {"tiles": tiles, "note": "launch time = call time / forward launches (upper bound)"}
+    achieved = alg / (per_launch_ms * 1e-3) / 1e9 if per_launch_ms else None
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
+                "frac": achieved / hbm_peak if achieved else None, "traffic": None, "peak_source": peak_src,
+                "algorithmic_bytes_per_launch": alg, "launch_ms": per_launch_ms, **extra}
+
+    # -------------------------------------------------------------------- CPU oracle on a bounded sample (rank 0, N = 1)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        layers_s, inputs_s = oracle_sample_shape(spec, kind, batch, budget_edges=1.5e9)
+        if kind == "train":
+            edges, times = oracle_train_sample(spec, inputs_s, layers_s, 2, 1)
+            sample = f"2 train steps on layers 1..{layers_s} of {L} at full width N={N}, B={inputs_s}"
+        else:
+            edges, times = oracle_infer_sample(spec, inputs_s, layers_s, 2, 1)
+            sample = f"2 inference passes of {inputs_s} inputs through layers 1..{layers_s} of {L} at full width N={N}"
+        cpu = {"value": edges / float(np.mean(times)), "unit": "edges/s", "cores": os.cpu_count(), "kind": "oracle",
+               "sample": sample, "seconds_per_sample_step": float(np.mean(times))}
+
+    if rank == 0:
+        line = {
+            "metric": metric_name(kind), "value": value, "unit": "edges/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {**workload_config(args.workload, spec, kind, batch),
+                       "parallelism": "replicas only (no collective)" if kind == "train" else "batch sharded over ranks, no collective",
+                       "inputs_per_step_per_gpu": n_inputs, "setup_seconds": setup_s, "device_bytes": h.device_bytes()},
+            "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
+        }
+        print(json.dumps(line), flush=True)
+    h.destroy()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -175,6 +175,12 @@ int sdnn_get_gradient(sdnn_t* h, int32_t layer, float* out);
 int64_t sdnn_kernel_launches(const sdnn_t* h);
 int64_t sdnn_device_bytes(const sdnn_t* h);
 
+/* Device time of the two kernel chains of the most recent train step, from events recorded on the
+ * handle's stream around them (inside the graph when one is used): fwd_ms covers the L forward
+ * launches, bwd_ms the L backward+update launches.  Synchronises the stream.  SDNN_ERR_STATE if no
+ * step has run. */
+int sdnn_get_phase_times(sdnn_t* h, float* fwd_ms, float* bwd_ms);
+
 /* Per-layer liveness of the most recent sdnn_infer_batch tile run with SDNN_FLAG_SKIP_DEAD:
  * live_inputs_out host int32[L] = inputs still alive after each layer.  SDNN_ERR_STATE otherwise. */
 int sdnn_get_liveness(sdnn_t* h, int32_t* live_inputs_out);

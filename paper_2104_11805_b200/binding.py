@@ -47,6 +47,7 @@ _PROTOS = {
     "sdnn_get_activations": (ctypes.c_int, [_vp, _i32, _vp]),
     "sdnn_get_delta": (ctypes.c_int, [_vp, _i32, _vp]),
     "sdnn_get_gradient": (ctypes.c_int, [_vp, _i32, _vp]),
+    "sdnn_get_phase_times": (ctypes.c_int, [_vp, ctypes.POINTER(_f32), ctypes.POINTER(_f32)]),
     "sdnn_get_liveness": (ctypes.c_int, [_vp, _vp]),
     "sdnn_kernel_launches": (_i64, [_vp]),
     "sdnn_device_bytes": (_i64, [_vp]),
@@ -193,6 +194,12 @@ class Sdnn:
         out = np.empty(self.nnz[layer - 1], dtype=np.float32)
         self._check(self._lib.sdnn_get_gradient(self._h, layer, out.ctypes.data))
         return out
+
+    def get_phase_times(self):
+        """(forward_ms, backward_ms) of the most recent train step."""
+        a, b = ctypes.c_float(0.0), ctypes.c_float(0.0)
+        self._check(self._lib.sdnn_get_phase_times(self._h, ctypes.byref(a), ctypes.byref(b)))
+        return a.value, b.value
 
     def get_liveness(self):
         out = np.empty(self.n_layers, dtype=np.int32)

@@ -53,6 +53,7 @@ struct sdnn {
     int last_b = 0, last_ld = 0;
     cudaGraphExec_t graph = nullptr;
     int graph_ld = 0;
+    cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};   // before forward chain, between, after backward chain
 
     // inference
     float* d_tile[2] = {nullptr, nullptr};
@@ -240,12 +241,16 @@ void launch_transpose_in(sdnn* h, const float* src, float* dst, int cnt, int col
     count_launch(h);
 }
 
-// forward + backward chain of one train step on the internal buffers
-void enqueue_step_body(sdnn* h, int ld) {
+// forward + backward chain of one train step on the internal buffers; `flags` selects how the three
+// timing events are recorded (as external event-record nodes while capturing a graph)
+void enqueue_step_body(sdnn* h, int ld, unsigned flags) {
     const size_t tile = (size_t)h->N * ld;
+    cudaEventRecordWithFlags(h->ev[0], h->stream, flags);
     for (int k = 0; k < h->L; ++k)
         launch_forward(h, k, h->d_acts + (size_t)k * tile, h->d_acts + (size_t)(k + 1) * tile, ld, ld);
+    cudaEventRecordWithFlags(h->ev[1], h->stream, flags);
     for (int k = h->L - 1; k >= 0; --k) launch_backward(h, k, ld);
+    cudaEventRecordWithFlags(h->ev[2], h->stream, flags);
 }
 
 int train_step_device(sdnn* h, const float* x0, const float* target, int B, float eta, float* loss_out) {
@@ -255,14 +260,14 @@ int train_step_device(sdnn* h, const float* x0, const float* target, int B, floa
     launch_transpose_in(h, x0, h->d_acts, B, ld, ld);
     launch_transpose_in(h, target, h->d_yt, B, ld, ld);
     if (h->cfg.flags & SDNN_FLAG_NO_GRAPH) {
-        enqueue_step_body(h, ld);
+        enqueue_step_body(h, ld, cudaEventRecordDefault);
     } else {
         if (!h->graph || h->graph_ld != ld) {
             if (h->graph) { cudaGraphExecDestroy(h->graph); h->graph = nullptr; }
             cudaGraph_t g = nullptr;
             const int64_t before = h->launches;
             CU(h, cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal));
-            enqueue_step_body(h, ld);
+            enqueue_step_body(h, ld, cudaEventRecordExternal);
             cudaError_t e = cudaStreamEndCapture(h->stream, &g);
             h->launches = before;
             if (e != cudaSuccess) return cuda_fail(h, e, "cudaStreamEndCapture");
@@ -363,6 +368,7 @@ void sdnn_destroy(sdnn_t* h) {
     cudaSetDevice(h->device);
     if (h->stream || h->own_stream) cudaStreamSynchronize(h->stream);
     if (h->graph) cudaGraphExecDestroy(h->graph);
+    for (cudaEvent_t e : h->ev) if (e) cudaEventDestroy(e);
     for (void* p : h->allocs) cudaFree(p);
     if (h->own_stream) cudaStreamDestroy(h->stream);
     delete h;
@@ -415,6 +421,8 @@ int sdnn_create_deferred(sdnn_t** out, int32_t n_layers, int32_t n_neurons, cons
     if ((rc = dev_alloc(h, &h->d_val, (size_t)h->slots, true))) return bail(rc);
     if ((rc = dev_alloc(h, &h->d_bias, L * N, false))) return bail(rc);
     if (cfg->train) {
+        for (cudaEvent_t& ev : h->ev)
+            if ((e = cudaEventCreate(&ev)) != cudaSuccess) { ev = nullptr; return bail(cuda_fail(h, e, "cudaEventCreate")); }
         if ((rc = dev_alloc(h, &h->d_acts, (L + 1) * tile, false))) return bail(rc);
         if ((rc = dev_alloc(h, &h->d_s[0], tile, true))) return bail(rc);
         if ((rc = dev_alloc(h, &h->d_s[1], tile, true))) return bail(rc);
@@ -644,6 +652,19 @@ int sdnn_get_gradient(sdnn_t* h, int32_t layer, float* out) {
     CU(h, cudaStreamSynchronize(h->stream));
     if (h->nnz[layer - 1])
         CU(h, cudaMemcpy(out, h->d_dbg_grad + h->off[layer - 1], (size_t)h->nnz[layer - 1] * sizeof(float), cudaMemcpyDeviceToHost));
+    return SDNN_OK;
+}
+
+int sdnn_get_phase_times(sdnn_t* h, float* fwd_ms, float* bwd_ms) {
+    if (!h) return SDNN_ERR_INVALID_ARG;
+    if (!h->stepped) return fail(h, SDNN_ERR_STATE, "no train step has run");
+    CU(h, cudaSetDevice(h->device));
+    CU(h, cudaStreamSynchronize(h->stream));
+    float a = 0.f, b = 0.f;
+    CU(h, cudaEventElapsedTime(&a, h->ev[0], h->ev[1]));
+    CU(h, cudaEventElapsedTime(&b, h->ev[1], h->ev[2]));
+    if (fwd_ms) *fwd_ms = a;
+    if (bwd_ms) *bwd_ms = b;
     return SDNN_OK;
 }
 

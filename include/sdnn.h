@@ -185,6 +185,42 @@ int sdnn_get_phase_times(sdnn_t* h, float* fwd_ms, float* bwd_ms);
  * live_inputs_out host int32[L] = inputs still alive after each layer.  SDNN_ERR_STATE otherwise. */
 int sdnn_get_liveness(sdnn_t* h, int32_t* live_inputs_out);
 
+/*
+ * Inference without any allocation (the paper has no counterpart: this entry point exists for
+ * callers that cannot allocate device memory when they call us - for example a host application
+ * whose own allocator has already reserved the whole device so that a raw cudaMalloc would fail,
+ * a latency-critical loop that cannot afford the device-wide synchronisation an allocation may
+ * imply, or a plug-in interface that forbids allocating after initialisation).
+ *
+ * Same arithmetic as sdnn_infer_batch with y_out only (L forward layers, one tile), but with no
+ * handle: the network stays in the caller's device arrays and the two ping-pong activation tiles
+ * live in a fixed array inside the library (SDNN_NOALLOC_SCRATCH_BYTES, held by every GPU that
+ * loads the library until the process exits).  The call makes no cudaMalloc / cudaFree and uses
+ * no allocating library routine; it only launches kernels on `cuda_stream` (NULL = legacy default
+ * stream) and returns without synchronising.
+ *   row_ptr       device int32[n_layers][n_neurons+1], offsets local to each layer
+ *   col_idx       device int32[], values device float[]: the layers' stored entries; layer l
+ *                 starts at element layer_offset[l] (host int64[n_layers], each a multiple of 4;
+ *                 both base pointers 16-byte aligned).  The arrays are NOT validated: they must
+ *                 satisfy the rules of sdnn_create.
+ *   bias          device float[n_layers][n_neurons]
+ *   x0            device float[n_inputs][n_neurons];  y_out  device float[n_inputs][n_neurons]
+ * Limit: n_neurons * padded(n_inputs) <= SDNN_NOALLOC_MAX_TILE_FLOATS, where padded() rounds the
+ * batch up to 4, 8, .., 128 and then to multiples of 128; larger problems are rejected with
+ * SDNN_ERR_INVALID_ARG and a message (sdnn_last_error(NULL)) before anything is launched.
+ * The first call on each device looks up the address of the library's scratch array (once per
+ * device, with that device current); make that first call outside any stream capture.
+ * All calls share the one scratch array, which keeps whatever the previous call left in it; every
+ * call overwrites the part it reads, so nothing needs clearing, but two calls whose kernels may
+ * overlap on the GPU (different streams, or different host threads) race on it and must be
+ * serialised by the caller.
+ */
+#define SDNN_NOALLOC_MAX_TILE_FLOATS (1 << 20)
+#define SDNN_NOALLOC_SCRATCH_BYTES   (2 * SDNN_NOALLOC_MAX_TILE_FLOATS * 4)
+int sdnn_infer_noalloc(int32_t n_layers, int32_t n_neurons, const int32_t* row_ptr, const int32_t* col_idx,
+                       const float* values, const int64_t* layer_offset, const float* bias,
+                       const float* x0, int32_t n_inputs, float* y_out, float clamp, void* cuda_stream);
+
 void sdnn_destroy(sdnn_t* h);                 /* NULL is a no-op */
 const char* sdnn_last_error(const sdnn_t* h); /* h may be NULL: last creation error of this thread */
 const char* sdnn_version(void);

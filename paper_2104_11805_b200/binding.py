@@ -49,6 +49,7 @@ _PROTOS = {
     "sdnn_get_gradient": (ctypes.c_int, [_vp, _i32, _vp]),
     "sdnn_get_phase_times": (ctypes.c_int, [_vp, ctypes.POINTER(_f32), ctypes.POINTER(_f32)]),
     "sdnn_get_liveness": (ctypes.c_int, [_vp, _vp]),
+    "sdnn_infer_noalloc": (ctypes.c_int, [_i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _f32, _vp]),
     "sdnn_kernel_launches": (_i64, [_vp]),
     "sdnn_device_bytes": (_i64, [_vp]),
     "sdnn_destroy": (None, [_vp]),
@@ -95,6 +96,28 @@ def _addr(x):
     if isinstance(x, np.ndarray):
         return x.ctypes.data
     return x.data_ptr()      # torch tensor
+
+
+NOALLOC_MAX_TILE_FLOATS = 1 << 20
+
+
+def infer_noalloc(n_layers, n_neurons, row_ptr, col_idx, values, layer_offset, bias, x0, n_inputs, y_out,
+                  clamp=32.0, stream=None):
+    """sdnn_infer_noalloc: forward through the whole net with no handle and no allocation.
+
+    For callers that may not allocate device memory at call time (the device is fully reserved by
+    another allocator, an allocation's implicit synchronisation is not acceptable, or their interface
+    forbids it): the net and the inputs/outputs are the caller's device arrays (anything with
+    data_ptr(), or raw addresses), the activation scratch is a fixed array inside the library.
+    layer_offset is a host sequence of element offsets (multiples of 4).  Raises SdnnError if
+    n_neurons * padded(n_inputs) exceeds NOALLOC_MAX_TILE_FLOATS.  Calls sharing the scratch must not
+    overlap on the GPU."""
+    lib = load_library()
+    off = _np(layer_offset, np.int64)
+    rc = lib.sdnn_infer_noalloc(n_layers, n_neurons, _addr(row_ptr), _addr(col_idx), _addr(values), off.ctypes.data,
+                                _addr(bias), _addr(x0), n_inputs, _addr(y_out), clamp, stream)
+    if rc != 0:
+        raise SdnnError(rc, (lib.sdnn_last_error(None) or b"").decode())
 
 
 class Sdnn:

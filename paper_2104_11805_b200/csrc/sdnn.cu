@@ -674,3 +674,99 @@ int sdnn_get_liveness(sdnn_t* h, int32_t* live_inputs_out) {
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free inference (see sdnn_infer_noalloc in the header).  The two activation tiles of
+// the forward chain live in this file-scope device array instead of memory owned by a handle.
+// In host code the array's name is only a stand-in for the symbol, not a device address: the
+// address each device gave it is looked up once per device with cudaGetSymbolAddress.
+namespace {
+
+static __device__ __align__(256) float g_noalloc_scratch[2 * SDNN_NOALLOC_MAX_TILE_FLOATS];
+
+constexpr int kMaxDevices = 64;
+float* g_noalloc_ptr[kMaxDevices] = {};      // per device: address of g_noalloc_scratch on that device
+
+int noalloc_scratch(float** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(nullptr, e, "cudaGetDevice");
+    if (dev < 0 || dev >= kMaxDevices) return fail(nullptr, SDNN_ERR_INVALID_ARG, "device ordinal %d not supported", dev);
+    float* p = g_noalloc_ptr[dev];
+    if (!p) {
+#pragma omp critical(sdnn_noalloc_setup)
+        {
+            p = g_noalloc_ptr[dev];
+            if (!p) {
+                e = cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_noalloc_scratch);
+                if (e == cudaSuccess) g_noalloc_ptr[dev] = p; else p = nullptr;
+            }
+        }
+        if (!p) return cuda_fail(nullptr, e, "cudaGetSymbolAddress(scratch)");
+    }
+    *out = p;
+    return SDNN_OK;
+}
+
+template <int G>
+void noalloc_forward_g(cudaStream_t st, const int* rp, const int* col, const float* val, const float* bias,
+                       const float* xin, float* xout, int n, int ld, int chunks, float clamp) {
+    const int rows_per_block = 8 * (32 / G);
+    dim3 grid((n + rows_per_block - 1) / rows_per_block, chunks);
+    forward_kernel<G><<<grid, 256, 0, st>>>(rp, col, val, bias, xin, xout, n, ld, clamp);
+}
+
+}  // namespace
+
+extern "C" int sdnn_infer_noalloc(int32_t n_layers, int32_t n_neurons, const int32_t* row_ptr, const int32_t* col_idx,
+                                  const float* values, const int64_t* layer_offset, const float* bias,
+                                  const float* x0, int32_t n_inputs, float* y_out, float clamp, void* cuda_stream) {
+    if (n_layers < 1 || n_neurons < 1 || n_inputs < 0) return fail(nullptr, SDNN_ERR_INVALID_ARG, "sizes must be positive");
+    if (!row_ptr || !col_idx || !values || !layer_offset || !bias) return fail(nullptr, SDNN_ERR_INVALID_ARG, "NULL network array");
+    if (!(clamp > 0.0f) || !std::isfinite(clamp)) return fail(nullptr, SDNN_ERR_INVALID_ARG, "clamp must be finite and > 0");
+    if (n_inputs == 0) return SDNN_OK;
+    if (!x0 || !y_out) return fail(nullptr, SDNN_ERR_INVALID_ARG, "x0 or y_out is NULL");
+    const int ld = padded_width(n_inputs);
+    if ((int64_t)n_neurons * ld > (int64_t)SDNN_NOALLOC_MAX_TILE_FLOATS)
+        return fail(nullptr, SDNN_ERR_INVALID_ARG,
+                    "problem too large for the built-in scratch: n_neurons * padded(n_inputs) = %lld floats, limit %d",
+                    (long long)n_neurons * ld, (int)SDNN_NOALLOC_MAX_TILE_FLOATS);
+    if ((reinterpret_cast<uintptr_t>(col_idx) | reinterpret_cast<uintptr_t>(values)) & 15)
+        return fail(nullptr, SDNN_ERR_INVALID_ARG, "col_idx and values must be 16-byte aligned");
+    for (int l = 0; l < n_layers; ++l)
+        if (layer_offset[l] < 0 || (layer_offset[l] & 3)) return fail(nullptr, SDNN_ERR_INVALID_ARG, "layer_offset[%d] must be a non-negative multiple of 4", l);
+
+    float* scratch = nullptr;
+    int rc = noalloc_scratch(&scratch);
+    if (rc) return rc;
+    float* tile[2] = {scratch, scratch + SDNN_NOALLOC_MAX_TILE_FLOATS};
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const Geometry q = geometry(ld);
+    {
+        dim3 grid((n_neurons + 31) / 32, (ld + 31) / 32), block(32, 8);
+        transpose_in_kernel<<<grid, block, 0, st>>>(x0, tile[0], n_neurons, n_inputs, ld, ld);
+    }
+    int cur = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        const int* rp = row_ptr + (size_t)l * (n_neurons + 1);
+        const int* col = col_idx + layer_offset[l];
+        const float* val = values + layer_offset[l];
+        const float* b = bias + (size_t)l * n_neurons;
+        switch (q.g) {
+            case 1: noalloc_forward_g<1>(st, rp, col, val, b, tile[cur], tile[cur ^ 1], n_neurons, ld, q.chunks, clamp); break;
+            case 2: noalloc_forward_g<2>(st, rp, col, val, b, tile[cur], tile[cur ^ 1], n_neurons, ld, q.chunks, clamp); break;
+            case 4: noalloc_forward_g<4>(st, rp, col, val, b, tile[cur], tile[cur ^ 1], n_neurons, ld, q.chunks, clamp); break;
+            case 8: noalloc_forward_g<8>(st, rp, col, val, b, tile[cur], tile[cur ^ 1], n_neurons, ld, q.chunks, clamp); break;
+            case 16: noalloc_forward_g<16>(st, rp, col, val, b, tile[cur], tile[cur ^ 1], n_neurons, ld, q.chunks, clamp); break;
+            default: noalloc_forward_g<32>(st, rp, col, val, b, tile[cur], tile[cur ^ 1], n_neurons, ld, q.chunks, clamp); break;
+        }
+        cur ^= 1;
+    }
+    {
+        dim3 grid((n_neurons + 31) / 32, (n_inputs + 31) / 32), block(32, 8);
+        transpose_out_kernel<<<grid, block, 0, st>>>(tile[cur], y_out, n_neurons, n_inputs, ld);
+    }
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(nullptr, e, "kernel launch");
+    return SDNN_OK;
+}

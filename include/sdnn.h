@@ -57,12 +57,15 @@ typedef enum {
 } sdnn_status;
 
 /* cfg->flags */
-#define SDNN_FLAG_BWD_ATOMICS 0x01u /* backward product by scatter with vector reductions into L2 (one CSR pass)   */
-#define SDNN_FLAG_BWD_CSC     0x02u /* backward product by gather through a transposed index (no atomics)          */
+#define SDNN_FLAG_BWD_ATOMICS 0x01u /* backward product by scatter with vector reductions into L2 (one pass, one   */
+                                    /* copy of the weights)                                                        */
+#define SDNN_FLAG_BWD_CSC     0x02u /* backward product by gather through a transposed copy of the layer (second   */
+                                    /* index and value array, both copies updated; no atomics).  The default.      */
 #define SDNN_FLAG_KEEP_DEBUG  0x04u /* train handles: also store delta^k and the gradient G^k of the last step     */
 #define SDNN_FLAG_SKIP_DEAD   0x08u /* allow data-dependent skipping (dead inputs, all-zero delta rows); default   */
                                     /* is dense mode: every layer streams its weights and processes every input    */
 #define SDNN_FLAG_NO_GRAPH    0x10u /* launch the layer chain kernel by kernel instead of through a CUDA graph     */
+#define SDNN_FLAG_NO_PDL      0x20u /* do not let a layer's kernel start its prologue under the previous layer's tail */
 
 typedef struct {
     int32_t  activation;   /* 0 = clamped ReLU (the only one implemented) */
@@ -169,6 +172,18 @@ int sdnn_set_weights(sdnn_t* h, int32_t layer, const float* values, const float*
 int sdnn_get_activations(sdnn_t* h, int32_t layer, float* out);
 int sdnn_get_delta(sdnn_t* h, int32_t layer, float* out);
 int sdnn_get_gradient(sdnn_t* h, int32_t layer, float* out);
+
+/*
+ * Consistency of the two copies of a training layer's weights.  Without SDNN_FLAG_BWD_ATOMICS a training
+ * handle keeps, beside the row-major copy of W^k that the forward product reads, a transposed copy (entries
+ * by column, own value array) so that the transposed product of the recursive formula is a gather like the
+ * forward product and needs no atomic adds.  Both copies receive the update of the gradient update rule with
+ * bit-identical arithmetic.  count_out (host) = number of stored entries of `layer` (0-based) whose two values
+ * differ in any bit; bit 32 and up count entries of the transposed pattern missing from the row-major one
+ * (never set for a handle this library built).  0 for layers without a transposed copy (the first layer,
+ * atomics handles, inference handles).  Synchronises the stream.
+ */
+int sdnn_mirror_mismatches(sdnn_t* h, int32_t layer, int64_t* count_out);
 
 /* Counters since creation: kernels launched by this handle (graph nodes count one each);
  * device bytes it holds. */

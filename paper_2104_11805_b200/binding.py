@@ -13,7 +13,7 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsdnn.so")
 
-FLAG_BWD_ATOMICS, FLAG_BWD_CSC, FLAG_KEEP_DEBUG, FLAG_SKIP_DEAD, FLAG_NO_GRAPH = 0x01, 0x02, 0x04, 0x08, 0x10
+FLAG_BWD_ATOMICS, FLAG_BWD_CSC, FLAG_KEEP_DEBUG, FLAG_SKIP_DEAD, FLAG_NO_GRAPH, FLAG_NO_PDL = 0x01, 0x02, 0x04, 0x08, 0x10, 0x20
 
 STATUS = {0: "SDNN_OK", -1: "SDNN_ERR_INVALID_ARG", -2: "SDNN_ERR_BAD_CSR", -3: "SDNN_ERR_OOM", -4: "SDNN_ERR_CUDA",
           -5: "SDNN_ERR_STATE", -6: "SDNN_ERR_UNIMPLEMENTED"}
@@ -47,6 +47,7 @@ _PROTOS = {
     "sdnn_get_activations": (ctypes.c_int, [_vp, _i32, _vp]),
     "sdnn_get_delta": (ctypes.c_int, [_vp, _i32, _vp]),
     "sdnn_get_gradient": (ctypes.c_int, [_vp, _i32, _vp]),
+    "sdnn_mirror_mismatches": (ctypes.c_int, [_vp, _i32, ctypes.POINTER(_i64)]),
     "sdnn_get_phase_times": (ctypes.c_int, [_vp, ctypes.POINTER(_f32), ctypes.POINTER(_f32)]),
     "sdnn_get_liveness": (ctypes.c_int, [_vp, _vp]),
     "sdnn_infer_noalloc": (ctypes.c_int, [_i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _f32, _vp]),
@@ -217,6 +218,12 @@ class Sdnn:
         out = np.empty(self.nnz[layer - 1], dtype=np.float32)
         self._check(self._lib.sdnn_get_gradient(self._h, layer, out.ctypes.data))
         return out
+
+    def mirror_mismatches(self, layer):
+        """Entries of the layer's transposed copy whose bits differ from the row-major copy (0 when consistent)."""
+        c = ctypes.c_int64(0)
+        self._check(self._lib.sdnn_mirror_mismatches(self._h, layer, ctypes.byref(c)))
+        return c.value
 
     def get_phase_times(self):
         """(forward_ms, backward_ms) of the most recent train step."""

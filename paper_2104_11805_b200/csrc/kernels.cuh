@@ -1,11 +1,20 @@
 // Device kernels of the sparse-DNN SGD hot path (sm_100a).
 //
-// Data layout.  Activations, deltas and the partial products S = W^T delta live in
-// neuron-major tiles X[i*ld + b] (neuron i, input b; ld = padded batch, a multiple of 4),
-// so that the row of X gathered for one stored entry W(i,j) is contiguous and every
-// access is a 128-bit vector.  A row of a tile is shared by G lanes (G*4 batch entries,
-// one float4 per lane); a warp therefore works on 32/G matrix rows at once.  Tiles
-// wider than 128 inputs are processed in chunks of 128 (blockIdx.y).
+// Tiles.  Activations x^k, deltas and the partial products S = W^T delta live in neuron-major tiles
+// X[i*ld + b] (neuron i, input b; ld = padded batch, a multiple of 4), so that the row of X gathered
+// for one stored entry W(i,j) is contiguous and every access is a 128-bit vector.  A row of a tile is
+// shared by G lanes (G*4 batch entries, one float4 per lane); a warp therefore works on 32/G matrix
+// rows at once.  Tiles wider than 128 inputs are processed in chunks of 128 (blockIdx.y).
+//
+// Stored entries.  What bounds these kernels is the number of L1 wavefronts per stored entry: the
+// gather of a tile row costs one, and with plain CSR the index and value loads of the eight row groups
+// of a warp cost another half each, because the eight rows sit in eight different 128-byte lines.
+// The entries are therefore kept in slices of 8 rows, interleaved in chunks of 4:
+//     entry q of row i  ->  slice_off[i/8] + (q/4)*32 + (i%8)*4 + q%4          (element offset)
+// so that the 16-byte chunks the eight row groups of a warp read in one step are one 128-byte line.
+// A slice is padded to the longest of its rows rounded up to 4; padding has index 0 and value 0 and
+// is never updated.  The transposed matrix (columns as "rows", for the backward product without
+// atomics) uses the same layout over the columns sorted by descending length.
 //
 // Equations (paper, Section 3.2): forward x^k = f(W^k x^{k-1} + b^k); recursion
 // delta^{k-1} = (W^k)^T delta^k (.) f'(z^{k-1}); update W^k(j,i) -= eta delta^k(j) x^{k-1}(i)
@@ -23,6 +32,16 @@ struct StepParams {     // written by set_step_params before each train step; re
     int   pad;
 };
 
+// One matrix in sliced layout.  `order` is NULL for the row-major copy (unit u is row u); for the
+// transposed copy it lists the matrix column each unit stands for.
+struct Sliced {
+    const int* slice_off;   // [ceil(n/8) + 1] element offsets of the slices, multiples of 32
+    const int* len;         // [n] stored entries of each unit
+    const int* idx;         // gathered tile row of each entry (column index; row index in the transposed copy)
+    float*     val;
+    const int* order;
+};
+
 __device__ __forceinline__ float4 ld_f4(const float* p) { return *reinterpret_cast<const float4*>(p); }
 __device__ __forceinline__ void st_f4(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
 
@@ -35,8 +54,22 @@ __device__ __forceinline__ void red_add_f4(float* p, float4 v) {
                  :: "l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
 }
 
+// asks for `bytes` (a multiple of 16, address 16-byte aligned) to be brought into L2; no destination, no wait
+__device__ __forceinline__ void prefetch_l2(const void* p, unsigned bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" :: "l"(p), "r"(bytes) : "memory");
+}
+
+// programmatic dependent launch: wait for the kernels this one depends on / let the next one start its prologue
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ float clampf(float z, float c) { return fminf(fmaxf(z, 0.0f), c); }
 __device__ __forceinline__ float dmask(float x, float c) { return (x > 0.0f && x < c) ? 1.0f : 0.0f; }
+
+template <int G>
+__device__ __forceinline__ unsigned group_mask(int grp) {
+    return (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << (grp * G));
+}
 
 // sum over the G lanes of a row group; `gmask` names exactly those lanes, so that groups of one warp
 // whose rows have different lengths may sit in different loop iterations
@@ -45,6 +78,75 @@ __device__ __forceinline__ float group_sum(float v, unsigned gmask) {
 #pragma unroll
     for (int o = G / 2; o > 0; o >>= 1) v += __shfl_xor_sync(gmask, v, o);
     return v;
+}
+
+// Partial dot product of one lane: its four batch columns of delta (d) against those of x.  Written with
+// explicit roundings so that the row pass and the column pass, which swap the roles of the gathered and
+// the resident operand, produce the same bits (a*b and fma(a,b,c) are symmetric in a and b).
+__device__ __forceinline__ float dot4(const float4& d, const float4& x) {
+    return __fmaf_rn(d.w, x.w, __fmaf_rn(d.z, x.z, __fmaf_rn(d.y, x.y, __fmul_rn(d.x, x.x))));
+}
+
+// The G lanes of a group hold partial sums p0..p3 for the four entries of a chunk.  On return
+//   G >= 4: p0 = full sum of entry (sub & 3)          (three shuffles instead of eight)
+//   G == 2: p0, p1 = full sums of entries 2*sub, 2*sub+1
+//   G == 1: nothing to do.
+// The additions pair the same lanes whatever entry a lane ends up owning, so the result does not depend
+// on the position of an entry inside its chunk.
+template <int G>
+__device__ __forceinline__ void chunk_sums(float& p0, float& p1, float& p2, float& p3, int sub, unsigned gmask) {
+    if (G > 4) {
+#pragma unroll
+        for (int o = G / 2; o >= 4; o >>= 1) {
+            p0 += __shfl_xor_sync(gmask, p0, o); p1 += __shfl_xor_sync(gmask, p1, o);
+            p2 += __shfl_xor_sync(gmask, p2, o); p3 += __shfl_xor_sync(gmask, p3, o);
+        }
+    }
+    if (G >= 4) {
+        const bool hi = (sub & 2) != 0;
+        const float s0 = hi ? p0 : p2, s1 = hi ? p1 : p3;
+        float k0 = hi ? p2 : p0, k1 = hi ? p3 : p1;
+        k0 += __shfl_xor_sync(gmask, s0, 2);
+        k1 += __shfl_xor_sync(gmask, s1, 2);
+        const bool odd = (sub & 1) != 0;
+        const float s = odd ? k0 : k1;
+        float k = odd ? k1 : k0;
+        k += __shfl_xor_sync(gmask, s, 1);
+        p0 = k;
+    } else if (G == 2) {
+        const bool odd = (sub & 1) != 0;
+        const float s0 = odd ? p0 : p2, s1 = odd ? p1 : p3;
+        float k0 = odd ? p2 : p0, k1 = odd ? p3 : p1;
+        k0 += __shfl_xor_sync(gmask, s0, 1);
+        k1 += __shfl_xor_sync(gmask, s1, 1);
+        p0 = k0; p1 = k1;
+    }
+}
+
+// Applies the update w <- w - step*g to the entries of one chunk this lane owns after chunk_sums and
+// stores them (entries at positions >= len are padding and stay untouched).  `lim` = len - (first entry this
+// lane owns in a chunk), so that "entry stored" is q0 < lim.  DBG: also record the gradient G = g / B.
+template <int G, bool DBG>
+__device__ __forceinline__ void chunk_update(float* vp, float* gp, const float4& w, float p0, float p1, float p2, float p3,
+                                             int sub, int q0, int lim, float step, float inv_b) {
+    if (G >= 4) {
+        const float wo = (sub & 2) ? ((sub & 1) ? w.w : w.z) : ((sub & 1) ? w.y : w.x);
+        const float nw = __fmaf_rn(-step, p0, wo);
+        if ((G == 4 || sub < 4) && q0 < lim) {
+            vp[sub & 3] = nw;
+            if (DBG) gp[sub & 3] = p0 * inv_b;
+        }
+    } else if (G == 2) {
+        const float wa = sub ? w.z : w.x, wb = sub ? w.w : w.y;
+        const int m = 2 * sub;
+        if (q0 < lim) { vp[m] = __fmaf_rn(-step, p0, wa); if (DBG) gp[m] = p0 * inv_b; }
+        if (q0 + 1 < lim) { vp[m + 1] = __fmaf_rn(-step, p1, wb); if (DBG) gp[m + 1] = p1 * inv_b; }
+    } else {
+        if (q0 + 0 < lim) { vp[0] = __fmaf_rn(-step, p0, w.x); if (DBG) gp[0] = p0 * inv_b; }
+        if (q0 + 1 < lim) { vp[1] = __fmaf_rn(-step, p1, w.y); if (DBG) gp[1] = p1 * inv_b; }
+        if (q0 + 2 < lim) { vp[2] = __fmaf_rn(-step, p2, w.z); if (DBG) gp[2] = p2 * inv_b; }
+        if (q0 + 3 < lim) { vp[3] = __fmaf_rn(-step, p3, w.w); if (DBG) gp[3] = p3 * inv_b; }
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -87,15 +189,13 @@ __global__ void set_step_params_kernel(StepParams* p, float eta, int batch, doub
 }
 
 // ---------------------------------------------------------------------------------------------
-// Forward layer (feedforward equation): Xout[i,:] = clamp(bias[i] + sum_p val[p] * Xin[col[p],:]).
-// One group of G lanes per matrix row; each lane accumulates 4 batch entries.  The products of a
-// row are added in CSR order with fp32 FMAs.  Index/value loads are 128-bit when the row segment
-// is 16-byte aligned (always the case for rows of 4k entries in a 16-byte aligned layer).
+// Forward layer on plain CSR arrays (feedforward equation).  Used only where the stored entries
+// belong to the caller and cannot be re-laid out (sdnn_infer_noalloc).
 template <int G>
 __global__ void __launch_bounds__(256)
-forward_kernel(const int* __restrict__ row_ptr, const int* __restrict__ col, const float* __restrict__ val,
-               const float* __restrict__ bias, const float* __restrict__ xin, float* __restrict__ xout,
-               int n, int ld, float clamp) {
+forward_csr_kernel(const int* __restrict__ row_ptr, const int* __restrict__ col, const float* __restrict__ val,
+                   const float* __restrict__ bias, const float* __restrict__ xin, float* __restrict__ xout,
+                   int n, int ld, float clamp) {
     constexpr int RPW = 32 / G;
     const int lane = threadIdx.x & 31;
     const int sub = lane % G, grp = lane / G;
@@ -109,6 +209,7 @@ forward_kernel(const int* __restrict__ row_ptr, const int* __restrict__ col, con
     const float b = bias[row];
     float4 acc = make_float4(b, b, b, b);
     int p = s;
+#define SDNN_FMA4(W, X) acc.x = fmaf(W, X.x, acc.x); acc.y = fmaf(W, X.y, acc.y); acc.z = fmaf(W, X.z, acc.z); acc.w = fmaf(W, X.w, acc.w);
     if (((s | e) & 3) == 0) {
         for (; p + 8 <= e; p += 8) {
             const int4 c0 = *reinterpret_cast<const int4*>(col + p), c1 = *reinterpret_cast<const int4*>(col + p + 4);
@@ -117,7 +218,6 @@ forward_kernel(const int* __restrict__ row_ptr, const int* __restrict__ col, con
             const float4 x2 = gather_f4(xg + (size_t)c0.z * ld), x3 = gather_f4(xg + (size_t)c0.w * ld);
             const float4 x4 = gather_f4(xg + (size_t)c1.x * ld), x5 = gather_f4(xg + (size_t)c1.y * ld);
             const float4 x6 = gather_f4(xg + (size_t)c1.z * ld), x7 = gather_f4(xg + (size_t)c1.w * ld);
-#define SDNN_FMA4(W, X) acc.x = fmaf(W, X.x, acc.x); acc.y = fmaf(W, X.y, acc.y); acc.z = fmaf(W, X.z, acc.z); acc.w = fmaf(W, X.w, acc.w);
             SDNN_FMA4(w0.x, x0) SDNN_FMA4(w0.y, x1) SDNN_FMA4(w0.z, x2) SDNN_FMA4(w0.w, x3)
             SDNN_FMA4(w1.x, x4) SDNN_FMA4(w1.y, x5) SDNN_FMA4(w1.z, x6) SDNN_FMA4(w1.w, x7)
         }
@@ -141,108 +241,383 @@ forward_kernel(const int* __restrict__ row_ptr, const int* __restrict__ col, con
 }
 
 // ---------------------------------------------------------------------------------------------
-// Backward + update of one layer k in ONE pass over its stored entries (Algorithm 1, loop body):
-//   delta^k[i,:]   = LAST ? (x^L[i,:] - y[i,:]) (.) f'   :  S_k[i,:] (.) f'      with f' = [0 < x^k < c]
-//   for each stored (i,j), old weight w:
-//       g          = sum_b delta^k[i,b] x^{k-1}[j,b]                 (masked gradient, times B)
-//       S_{k-1}[j,:] += w * delta^k[i,:]      (PROP; w is the value BEFORE the update)
-//       W(i,j)     = w - (eta/B) g
-// S_k is cleared row by row as it is consumed, so the two S buffers can alternate between layers
-// without a separate memset.  The scatter uses one 128-bit vector reduction per lane.  The whole
-// minibatch sits in one chunk (ld = 4G <= 128), so each weight is owned by exactly one lane group.
-template <int G, bool LAST, bool PROP>
-__global__ void __launch_bounds__(256)
-backward_kernel(const int* __restrict__ row_ptr, const int* __restrict__ col, float* __restrict__ val,
-                float* __restrict__ bias, const float* __restrict__ xk, const float* __restrict__ xprev,
-                float* __restrict__ s_k /* LAST: target tile y */, float* __restrict__ s_prev,
-                int n, float clamp, const StepParams* __restrict__ sp, double* __restrict__ loss,
-                float* __restrict__ dbg_delta, float* __restrict__ dbg_grad, int update_bias, int skip_dead) {
+// Helpers of the layer kernels' software pipeline.  A step handles two chunks (8 entries) of a row, all of
+// whose gathers are in flight together; slices are padded to a multiple of 8 entries per row, so a step never
+// needs a guard.  All the rows of a slice run through the slice's padded width (padding has index 0 and value
+// 0), which keeps the lanes of a warp converged.  The indices of a step are loaded one step ahead (while the
+// previous step's gathers are in flight, also across the boundary between two units), so that a step costs
+// one memory round trip, not two dependent ones.
+__device__ __forceinline__ void load_idx2(int4& c0, int4& c1, const int* p) {
+    c0 = __ldcs(reinterpret_cast<const int4*>(p));
+    c1 = __ldcs(reinterpret_cast<const int4*>(p + 32));
+}
+
+// asks for the slices that hold the rows of unit `u` (rpw consecutive rows) to be brought into L2
+__device__ __forceinline__ void prefetch_unit(const Sliced& m, int u, int rpw, int n, int units_per_slice) {
+    const int r0 = u * rpw;
+    if (units_per_slice > 1 && (r0 & 7) != 0) return;      // units narrower than a slice: the first one asks for the whole slice
+    const int s0 = r0 >> 3, s1 = min((n + 7) >> 3, ((r0 + rpw - 1) >> 3) + 1);
+    const int lo = m.slice_off[s0], hi = m.slice_off[s1];
+    if (hi > lo) { prefetch_l2(m.idx + lo, (unsigned)(hi - lo) * 4u); prefetch_l2(m.val + lo, (unsigned)(hi - lo) * 4u); }
+}
+
+// address of tile row `r` (an index below 2^32 / pitch): one 32 x 32 -> 64 bit multiply-add, no 64-bit multiply
+__device__ __forceinline__ const float* tile_row(const float* base, int r, unsigned pitch_bytes) {
+    return reinterpret_cast<const float*>(reinterpret_cast<const char*>(base) + (unsigned long long)(unsigned)r * (unsigned long long)pitch_bytes);
+}
+__device__ __forceinline__ float* tile_row(float* base, int r, unsigned pitch_bytes) {
+    return reinterpret_cast<float*>(reinterpret_cast<char*>(base) + (unsigned long long)(unsigned)r * (unsigned long long)pitch_bytes);
+}
+
+#define SDNN_GATHER4(X, I, C, P, PITCH)                                                                 \
+    X[4 * (I) + 0] = gather_f4(tile_row(P, C.x, PITCH)); X[4 * (I) + 1] = gather_f4(tile_row(P, C.y, PITCH)); \
+    X[4 * (I) + 2] = gather_f4(tile_row(P, C.z, PITCH)); X[4 * (I) + 3] = gather_f4(tile_row(P, C.w, PITCH));
+
+// Position of a group's item (matrix row, or position in the transposed copy) in unit U of matrix M: BASE =
+// element offset of its first chunk, NCH = chunks of its slice (even), ITEM = n for groups beyond the matrix
+// (they run through the padding rows of the last slice like everyone else and store nothing).
+#define SDNN_UNIT_SHAPE(M, U, NUNITS, ITEM, BASE, NCH)                                        \
+    ITEM = (U) * RPW + grp; BASE = 0; NCH = 0;                                                \
+    if ((U) < (NUNITS) && (ITEM >> 3) < ((n + 7) >> 3)) {                                     \
+        const int so_ = M.slice_off[ITEM >> 3];                                               \
+        BASE = so_ + (ITEM & 7) * 4; NCH = (M.slice_off[(ITEM >> 3) + 1] - so_) >> 5;         \
+    }                                                                                         \
+    if (ITEM >= n) ITEM = n;
+
+// ---------------------------------------------------------------------------------------------
+// Forward layer (feedforward equation): Xout[i,:] = clamp(bias[i] + sum_q val[i,q] * Xin[idx[i,q],:]).
+// Persistent grid: a warp takes units (32/G consecutive rows) in a grid-stride loop.  One group of G lanes
+// per row; each lane accumulates 4 batch entries with fp32 FMAs in stored (ascending column) order.
+// While it works on a unit a warp asks for the entries of its next unit to be brought into L2.
+template <int G>
+__global__ void __launch_bounds__(256, 3)
+forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict__ xin, float* __restrict__ xout,
+               int n, int ld, float clamp, int pdl) {
     constexpr int RPW = 32 / G;
-    constexpr int ld = 4 * G;
+    constexpr int UPS = (RPW >= 8) ? 1 : 8 / RPW;      // units per slice
     const int lane = threadIdx.x & 31;
     const int sub = lane % G, grp = lane / G;
-    const unsigned gmask = (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << (grp * G));
-    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int row = warp * RPW + grp;
-    const int boff = sub * 4;
-    const float inv_b = sp->inv_b;
-    const float step = sp->eta * inv_b;
-    const bool valid = row < n;
+    const int wpb = blockDim.x >> 5;
+    const int nunits = (n + RPW - 1) / RPW;
+    const int stride = gridDim.x * wpb;
+    const int boff = blockIdx.y * (4 * G) + sub * 4;
+    const float* xg = xin + boff;
+    const unsigned pitch = (unsigned)ld * 4u;
+    const int* __restrict__ idx = m.idx;
+    const float* __restrict__ val = m.val;
 
-    float4 d = make_float4(0.f, 0.f, 0.f, 0.f);
+    int unit = blockIdx.x * wpb + (threadIdx.x >> 5);
+    // prologue that does not depend on the previous layer: shape of the first row, its entries on their way to L2
+    int row, base, nch;
+    SDNN_UNIT_SHAPE(m, unit, nunits, row, base, nch)
+    float b = (row < n) ? bias[row] : 0.0f;
+    if (unit < nunits && lane == 0) prefetch_unit(m, unit, RPW, n, UPS);
+    int4 c0 = make_int4(0, 0, 0, 0), c1 = c0;
+    if (nch > 0) load_idx2(c0, c1, idx + base);
+    if (pdl) grid_dependency_wait();
+
+    while (unit < nunits) {
+        // shape of this group's row in the warp's next unit (used when this unit's last step prefetches across the boundary)
+        const int nunit = unit + stride;
+        int nrow, nbase, nnch;
+        SDNN_UNIT_SHAPE(m, nunit, nunits, nrow, nbase, nnch)
+        const float nb = (nrow < n) ? bias[nrow] : 0.0f;
+        if (nunit < nunits && lane == 0) prefetch_unit(m, nunit, RPW, n, UPS);
+
+        float4 acc = make_float4(b, b, b, b);
+        const int* cp = idx + base;
+        const float* vp = val + base;
+        for (int t = 0; t < nch; t += 2) {
+            float4 x[8];
+            const float4 w0 = __ldcs(reinterpret_cast<const float4*>(vp + t * 32));
+            const float4 w1 = __ldcs(reinterpret_cast<const float4*>(vp + t * 32 + 32));
+            SDNN_GATHER4(x, 0, c0, xg, pitch)
+            SDNN_GATHER4(x, 1, c1, xg, pitch)
+            if (t + 2 < nch) load_idx2(c0, c1, cp + (t + 2) * 32);
+            else if (nnch > 0) load_idx2(c0, c1, idx + nbase);
+            SDNN_FMA4(w0.x, x[0]) SDNN_FMA4(w0.y, x[1]) SDNN_FMA4(w0.z, x[2]) SDNN_FMA4(w0.w, x[3])
+            SDNN_FMA4(w1.x, x[4]) SDNN_FMA4(w1.y, x[5]) SDNN_FMA4(w1.z, x[6]) SDNN_FMA4(w1.w, x[7])
+        }
+        if (nch == 0 && nnch > 0) load_idx2(c0, c1, idx + nbase);      // empty slice: nothing prefetched across the boundary yet
+        if (row < n) {
+            acc.x = clampf(acc.x, clamp); acc.y = clampf(acc.y, clamp);
+            acc.z = clampf(acc.z, clamp); acc.w = clampf(acc.w, clamp);
+            st_f4(tile_row(xout + boff, row, pitch), acc);
+        }
+        unit = nunit; row = nrow; base = nbase; nch = nnch; b = nb;
+    }
+    if (pdl) grid_launch_dependents();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Output gradient (final-layer gradient equation) and loss: delta^L = (x^L - y) (.) f'(x^L) on the valid
+// batch columns, 0 on the padding; J = 1/(2B) sum (x^L - y)^2 accumulated in double, one atomic per block.
+__global__ void __launch_bounds__(256)
+output_gradient_kernel(const float* __restrict__ xl, const float* __restrict__ y, float* __restrict__ delta,
+                       int n, int ld, float clamp, const StepParams* __restrict__ sp, double* __restrict__ loss) {
+    const int per_row = ld >> 2;
+    const long long total = (long long)n * per_row;
+    const int nb = sp->batch;
     float sq = 0.0f;
-    if (valid) {
-        const size_t o = (size_t)row * ld + boff;
-        const float4 x = ld_f4(xk + o);
-        float4 t = ld_f4(s_k + o);
-        if (LAST) {
-            const int nb = sp->batch;
-            t.x = (boff + 0 < nb) ? x.x - t.x : 0.0f; t.y = (boff + 1 < nb) ? x.y - t.y : 0.0f;
-            t.z = (boff + 2 < nb) ? x.z - t.z : 0.0f; t.w = (boff + 3 < nb) ? x.w - t.w : 0.0f;
-            sq = t.x * t.x + t.y * t.y + t.z * t.z + t.w * t.w;
-        } else {
-            st_f4(s_k + o, make_float4(0.f, 0.f, 0.f, 0.f));
-        }
-        d.x = t.x * dmask(x.x, clamp); d.y = t.y * dmask(x.y, clamp);
-        d.z = t.z * dmask(x.z, clamp); d.w = t.w * dmask(x.w, clamp);
-        if (dbg_delta) st_f4(dbg_delta + o, d);
+    for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < total; v += (long long)gridDim.x * blockDim.x) {
+        const int boff = (int)(v % per_row) * 4;
+        const float4 x = ld_f4(xl + v * 4), t = ld_f4(y + v * 4);
+        float4 e;
+        e.x = (boff + 0 < nb) ? x.x - t.x : 0.0f; e.y = (boff + 1 < nb) ? x.y - t.y : 0.0f;
+        e.z = (boff + 2 < nb) ? x.z - t.z : 0.0f; e.w = (boff + 3 < nb) ? x.w - t.w : 0.0f;
+        sq += e.x * e.x + e.y * e.y + e.z * e.z + e.w * e.w;
+        st_f4(delta + v * 4, make_float4(e.x * dmask(x.x, clamp), e.y * dmask(x.y, clamp),
+                                         e.z * dmask(x.z, clamp), e.w * dmask(x.w, clamp)));
     }
-    if (LAST) {   // loss J = 1/(2B) sum (x^L - y)^2 : block sum in fp32 partials, one double atomic per block
-        __shared__ float part[8];
-        float w = sq;
+    __shared__ float part[8];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) w += __shfl_xor_sync(0xffffffffu, w, o);
-        if (lane == 0) part[threadIdx.x >> 5] = w;
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            double tot = 0.0;
-            for (int q = 0; q < (int)(blockDim.x >> 5); ++q) tot += (double)part[q];
-            if (tot != 0.0) atomicAdd(loss, 0.5 * tot * (double)inv_b);
-        }
+    for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = sq;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double tot = 0.0;
+        for (int q = 0; q < (int)(blockDim.x >> 5); ++q) tot += (double)part[q];
+        if (tot != 0.0) atomicAdd(loss, 0.5 * tot * (double)sp->inv_b);
     }
-    if (!valid) return;      // whole groups leave together; the shuffles below name only the group's lanes
-    if (update_bias) {       // bias read as one more column of W^k whose input is the constant 1
-        const float bg = group_sum<G>(d.x + d.y + d.z + d.w, gmask);
-        if (sub == 0) bias[row] -= step * bg;
-    }
-    if (skip_dead) {
-        const bool alive = !(d.x == 0.0f && d.y == 0.0f && d.z == 0.0f && d.w == 0.0f);
-        if ((__ballot_sync(gmask, alive) & gmask) == 0u) return;   // delta^k(i) = 0 for every input: nothing changes
-    }
+}
 
+// ---------------------------------------------------------------------------------------------
+// Backward + update of one layer k (Algorithm 1, loop body), two realisations.
+//
+// Row units (always): for row i of W^k with delta^k[i,:] in registers, for each stored (i,j):
+//       g = sum_b delta^k[i,b] x^{k-1}[j,b]      (masked gradient times B; x^{k-1}[j,:] gathered)
+//       W(i,j) = w - (eta/B) g
+//   SCATTER (atomics realisation) additionally S_{k-1}[j,:] += w * delta^k[i,:] with one 128-bit vector
+//   reduction per lane, w being the value BEFORE the update; there delta^k[i,:] = S_k[i,:] (.) f'(x^k[i,:])
+//   is formed on the fly and S_k is cleared row by row as it is consumed (FROM_S).
+//
+// Column units (transposed realisation, MIRROR): for column j of W^k (a row of the transposed copy,
+//   which has its own value array kept bit-identical to the row-major one), with x^{k-1}[j,:] in registers:
+//       acc  = sum_i w(i,j) delta^k[i,:]            (delta^k[i,:] gathered; w BEFORE the update)
+//       g, update of the transposed copy's value: same arithmetic, same bits as the row unit's
+//       delta^{k-1}[j,:] = acc (.) f'(x^{k-1}[j,:])
+//   No atomics; one gather per stored entry serves both the product and the gradient.
+//
+// A launch processes the column units (if any) first, then the row units; both only read delta^k and
+// x^{k-1}, so they are independent of each other.  The whole minibatch sits in one chunk (ld = 4G <= 128).
+// Same software pipeline as the forward kernel; in addition the resident operand of a unit (delta^k row or
+// x^{k-1} row) is loaded during the last step of the unit before it.
+struct BackwardArgs {
+    Sliced rows;              // row-major copy of W^k
+    Sliced cols;              // transposed copy (MIRROR)
+    float* bias;              // b^k (updated when update_bias)
+    const float* xk;          // x^k tile        (FROM_S: derivative mask of delta^k)
+    const float* xprev;       // x^{k-1} tile
+    float* dk;                // delta^k tile, or S_k when FROM_S (cleared as consumed)
+    float* dprev;             // SCATTER: S_{k-1};  MIRROR: delta^{k-1} tile;  else unused
+    float* dbg_delta;         // DBG: copy of delta^k (FROM_S only; otherwise dk is the record)
+    float* dbg_grad;          // DBG: G^k in the row-major copy's layout
+    const StepParams* sp;
+    int n;
+    float clamp;
+    int update_bias, skip_dead, col_units, pdl;
+};
+
+// Column units of the transposed realisation (see backward_kernel).
+template <int G>
+__device__ __forceinline__ void backward_col_units(const Sliced m, const float* __restrict__ xprev, const float* __restrict__ dk,
+                                                   float* __restrict__ dprev, int n, float clamp, float step, float inv_b,
+                                                   int first, int stride) {
+    constexpr int RPW = 32 / G;
+    constexpr int UPS = (RPW >= 8) ? 1 : 8 / RPW;
+    constexpr unsigned pitch = 16u * G;
+    const int lane = threadIdx.x & 31;
+    const int sub = lane % G, grp = lane / G;
+    const unsigned gmask = (G >= 4) ? 0xffffffffu : group_mask<G>(grp);     // G >= 4: the warp's lanes stay converged
+    const int nunits = (n + RPW - 1) / RPW;
+    const int boff = sub * 4;
+    const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int* __restrict__ idx = m.idx;
+    float* val = m.val;
+    const float* dg = dk + boff;
+
+    int u = first, item, base, nch;
+    SDNN_UNIT_SHAPE(m, u, nunits, item, base, nch)
+    if (u < nunits && lane == 0) prefetch_unit(m, u, RPW, n, UPS);
+    int len = 0, j = 0;
+    if (item < n) { len = m.len[item]; j = m.order[item]; }
+    int4 c0 = make_int4(0, 0, 0, 0), c1 = c0;
+    if (nch > 0) load_idx2(c0, c1, idx + base);
+    float4 xj = (item < n) ? ld_f4(tile_row(xprev + boff, j, pitch)) : zero4;
+
+    while (u < nunits) {
+        const int nu = u + stride;
+        int nitem, nbase, nnch, nlen = 0, nj = 0;
+        SDNN_UNIT_SHAPE(m, nu, nunits, nitem, nbase, nnch)
+        if (nitem < n) { nlen = m.len[nitem]; nj = m.order[nitem]; }
+        if (nu < nunits && lane == 0) prefetch_unit(m, nu, RPW, n, UPS);
+        float4 nxj = zero4;
+        float4 acc = zero4;
+        const int* ip = idx + base;
+        float* vp = val + base;
+        const int lim = len - ((G >= 4) ? (sub & 3) : (G == 2) ? 2 * sub : 0);
+#define SDNN_COL_NEXT if (nnch > 0) load_idx2(c0, c1, idx + nbase); if (nitem < n) nxj = ld_f4(tile_row(xprev + boff, nj, pitch));
+#define SDNN_ACC4(W, D) acc.x = fmaf(W, D.x, acc.x); acc.y = fmaf(W, D.y, acc.y); acc.z = fmaf(W, D.z, acc.z); acc.w = fmaf(W, D.w, acc.w);
+#define SDNN_COL_CHUNK(W, D0, D1, D2, D3, T)                                                                    \
+        {                                                                                                           \
+            SDNN_ACC4(W.x, D0) SDNN_ACC4(W.y, D1) SDNN_ACC4(W.z, D2) SDNN_ACC4(W.w, D3)                             \
+            float p0 = dot4(D0, xj), p1 = dot4(D1, xj), p2 = dot4(D2, xj), p3 = dot4(D3, xj);                       \
+            chunk_sums<G>(p0, p1, p2, p3, sub, gmask);                                                              \
+            chunk_update<G, false>(vp + (T) * 32, nullptr, W, p0, p1, p2, p3, sub, (T) * 4, lim, step, inv_b);       \
+        }
+        for (int t = 0; t < nch; t += 2) {
+            float4 d[8];
+            const float4 w0 = ld_f4(vp + t * 32), w1 = ld_f4(vp + t * 32 + 32);
+            SDNN_GATHER4(d, 0, c0, dg, pitch)
+            SDNN_GATHER4(d, 1, c1, dg, pitch)
+            if (t + 2 < nch) { load_idx2(c0, c1, ip + (t + 2) * 32); }
+            else { SDNN_COL_NEXT }
+            SDNN_COL_CHUNK(w0, d[0], d[1], d[2], d[3], t)
+            SDNN_COL_CHUNK(w1, d[4], d[5], d[6], d[7], t + 1)
+        }
+        if (nch == 0) { SDNN_COL_NEXT }
+#undef SDNN_COL_NEXT
+#undef SDNN_COL_CHUNK
+        if (item < n)
+            st_f4(tile_row(dprev + boff, j, pitch),
+                  make_float4(acc.x * dmask(xj.x, clamp), acc.y * dmask(xj.y, clamp), acc.z * dmask(xj.z, clamp), acc.w * dmask(xj.w, clamp)));
+        u = nu; item = nitem; base = nbase; nch = nnch; len = nlen; j = nj; xj = nxj;
+    }
+}
+
+// Row units (see backward_kernel).
+template <int G, bool FROM_S, bool SCATTER, bool DBG>
+__device__ __forceinline__ void backward_row_units(const Sliced m, float* __restrict__ bias, const float* __restrict__ xk,
+                                                   const float* __restrict__ xprev, float* dk, float* dprev,
+                                                   float* __restrict__ dbg_delta, float* __restrict__ dbg_grad, int n, float clamp,
+                                                   float step, float inv_b, int update_bias, int skip_dead, int first, int stride) {
+    constexpr int RPW = 32 / G;
+    constexpr int UPS = (RPW >= 8) ? 1 : 8 / RPW;
+    constexpr unsigned pitch = 16u * G;
+    const int lane = threadIdx.x & 31;
+    const int sub = lane % G, grp = lane / G;
+    const unsigned gmask1 = group_mask<G>(grp);
+    const unsigned gmask = (G >= 4) ? 0xffffffffu : gmask1;
+    const int nunits = (n + RPW - 1) / RPW;
+    const int boff = sub * 4;
+    const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int* __restrict__ idx = m.idx;
+    float* val = m.val;
     const float* xg = xprev + boff;
-    float* sg = s_prev + boff;
-    const int s = row_ptr[row], e = row_ptr[row + 1];
-    int p = s;
-#define SDNN_DOT4(X) fmaf(d.w, X.w, fmaf(d.z, X.z, fmaf(d.y, X.y, d.x * X.x)))
-#define SDNN_SCAT(C, W) red_add_f4(sg + (size_t)(C) * ld, make_float4(W * d.x, W * d.y, W * d.z, W * d.w));
-    if (((s | e) & 3) == 0) {
-        for (; p < e; p += 4) {
-            const int4 c = *reinterpret_cast<const int4*>(col + p);
-            const float4 w = ld_f4(val + p);
-            const float4 x0 = gather_f4(xg + (size_t)c.x * ld), x1 = gather_f4(xg + (size_t)c.y * ld);
-            const float4 x2 = gather_f4(xg + (size_t)c.z * ld), x3 = gather_f4(xg + (size_t)c.w * ld);
-            if (PROP) { SDNN_SCAT(c.x, w.x) SDNN_SCAT(c.y, w.y) SDNN_SCAT(c.z, w.z) SDNN_SCAT(c.w, w.w) }
-            float4 g;
-            g.x = group_sum<G>(SDNN_DOT4(x0), gmask); g.y = group_sum<G>(SDNN_DOT4(x1), gmask);
-            g.z = group_sum<G>(SDNN_DOT4(x2), gmask); g.w = group_sum<G>(SDNN_DOT4(x3), gmask);
-            if (sub == 0) {
-                st_f4(val + p, make_float4(fmaf(-step, g.x, w.x), fmaf(-step, g.y, w.y),
-                                           fmaf(-step, g.z, w.z), fmaf(-step, g.w, w.w)));
-                if (dbg_grad) st_f4(dbg_grad + p, make_float4(g.x * inv_b, g.y * inv_b, g.z * inv_b, g.w * inv_b));
+    float* sg = SCATTER ? dprev + boff : nullptr;
+
+    int u = first, item, base, nch;
+    SDNN_UNIT_SHAPE(m, u, nunits, item, base, nch)
+    if (u < nunits && lane == 0) prefetch_unit(m, u, RPW, n, UPS);
+    int len = (item < n) ? m.len[item] : 0;
+    int4 c0 = make_int4(0, 0, 0, 0), c1 = c0;
+    if (nch > 0) load_idx2(c0, c1, idx + base);
+    float4 h0 = zero4, h1 = zero4;       // delta^k[i,:] (or S_k[i,:]) and, FROM_S, x^k[i,:]
+    if (item < n) { h0 = ld_f4(tile_row(dk + boff, item, pitch)); if (FROM_S) h1 = ld_f4(tile_row(xk + boff, item, pitch)); }
+
+    while (u < nunits) {
+        const int nu = u + stride;
+        int nitem, nbase, nnch;
+        SDNN_UNIT_SHAPE(m, nu, nunits, nitem, nbase, nnch)
+        const int nlen = (nitem < n) ? m.len[nitem] : 0;
+        if (nu < nunits && lane == 0) prefetch_unit(m, nu, RPW, n, UPS);
+        float4 nh0 = zero4, nh1 = zero4;
+        float4 d = h0;
+        if (item < n) {
+            float* o = tile_row(dk + boff, item, pitch);
+            if (FROM_S) {
+                st_f4(o, zero4);
+                d.x *= dmask(h1.x, clamp); d.y *= dmask(h1.y, clamp);
+                d.z *= dmask(h1.z, clamp); d.w *= dmask(h1.w, clamp);
+                if (DBG) st_f4(tile_row(dbg_delta + boff, item, pitch), d);
+            }
+            if (update_bias) {       // bias read as one more column of W^k whose input is the constant 1
+                const float bg = group_sum<G>(d.x + d.y + d.z + d.w, gmask1);
+                if (sub == 0) bias[item] -= step * bg;
             }
         }
-    } else {
-        for (; p < e; ++p) {
-            const int c = col[p];
-            const float w = val[p];
-            const float4 x = gather_f4(xg + (size_t)c * ld);
-            if (PROP) { SDNN_SCAT(c, w) }
-            const float g = group_sum<G>(SDNN_DOT4(x), gmask);
-            if (sub == 0) {
-                val[p] = fmaf(-step, g, w);
-                if (dbg_grad) dbg_grad[p] = g * inv_b;
+        if (skip_dead) {             // delta^k(i) = 0 for every input of every row of the unit: nothing changes
+            const bool alive = !(d.x == 0.0f && d.y == 0.0f && d.z == 0.0f && d.w == 0.0f);
+            if (__ballot_sync(gmask, alive) == 0u) nch = 0;
+        }
+        const int* cp = idx + base;
+        float* vp = val + base;
+        float* gp = DBG ? dbg_grad + base : nullptr;
+        const int lim = len - ((G >= 4) ? (sub & 3) : (G == 2) ? 2 * sub : 0);
+#define SDNN_ROW_NEXT                                                                                    \
+        if (nnch > 0) load_idx2(c0, c1, idx + nbase);                                                    \
+        if (nitem < n) { nh0 = ld_f4(tile_row(dk + boff, nitem, pitch)); if (FROM_S) nh1 = ld_f4(tile_row(xk + boff, nitem, pitch)); }
+#define SDNN_SCAT(C, W, Q) if ((Q) < len) red_add_f4(tile_row(sg, C, pitch), make_float4(W * d.x, W * d.y, W * d.z, W * d.w));
+#define SDNN_ROW_CHUNK(W, X0, X1, X2, X3, T)                                                                \
+        {                                                                                                       \
+            float p0 = dot4(d, X0), p1 = dot4(d, X1), p2 = dot4(d, X2), p3 = dot4(d, X3);                       \
+            chunk_sums<G>(p0, p1, p2, p3, sub, gmask);                                                          \
+            chunk_update<G, DBG>(vp + (T) * 32, DBG ? gp + (T) * 32 : nullptr, W, p0, p1, p2, p3, sub, (T) * 4, lim, step, inv_b); \
+        }
+        for (int t = 0; t < nch; t += 2) {
+            float4 x[8];
+            const float4 w0 = ld_f4(vp + t * 32), w1 = ld_f4(vp + t * 32 + 32);
+            SDNN_GATHER4(x, 0, c0, xg, pitch)
+            SDNN_GATHER4(x, 1, c1, xg, pitch)
+            if (SCATTER) {       // stored entries only: padding must not touch S
+                const int q = 4 * t;
+                SDNN_SCAT(c0.x, w0.x, q) SDNN_SCAT(c0.y, w0.y, q + 1) SDNN_SCAT(c0.z, w0.z, q + 2) SDNN_SCAT(c0.w, w0.w, q + 3)
+                SDNN_SCAT(c1.x, w1.x, q + 4) SDNN_SCAT(c1.y, w1.y, q + 5) SDNN_SCAT(c1.z, w1.z, q + 6) SDNN_SCAT(c1.w, w1.w, q + 7)
             }
+            if (t + 2 < nch) { load_idx2(c0, c1, cp + (t + 2) * 32); }
+            else { SDNN_ROW_NEXT }
+            SDNN_ROW_CHUNK(w0, x[0], x[1], x[2], x[3], t)
+            SDNN_ROW_CHUNK(w1, x[4], x[5], x[6], x[7], t + 1)
+        }
+        if (nch == 0) { SDNN_ROW_NEXT }
+#undef SDNN_ROW_NEXT
+#undef SDNN_ROW_CHUNK
+        u = nu; item = nitem; base = nbase; nch = nnch; len = nlen; h0 = nh0; h1 = nh1;
+    }
+}
+
+template <int G, bool FROM_S, bool SCATTER, bool MIRROR, bool DBG>
+__global__ void __launch_bounds__(256, 3)
+backward_kernel(const BackwardArgs a) {
+    const int wpb = blockDim.x >> 5;
+    const int stride = gridDim.x * wpb;
+    const int first = blockIdx.x * wpb + (threadIdx.x >> 5);
+    if (a.pdl) grid_dependency_wait();
+    const float inv_b = a.sp->inv_b;
+    const float step = a.sp->eta * inv_b;
+    if (MIRROR) backward_col_units<G>(a.cols, a.xprev, a.dk, a.dprev, a.n, a.clamp, step, inv_b, first, stride);
+    backward_row_units<G, FROM_S, SCATTER, DBG>(a.rows, a.bias, a.xk, a.xprev, a.dk, a.dprev, a.dbg_delta, a.dbg_grad, a.n, a.clamp,
+                                           step, inv_b, a.update_bias, a.skip_dead, first, stride);
+    if (a.pdl) grid_launch_dependents();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Fills the transposed copy's values from the row-major copy: entry (column j, row i) of the transposed
+// copy is looked up by binary search in row i (ascending columns).  One thread per transposed entry slot.
+// With `mismatch` non-NULL nothing is written; entries whose bits differ from the row-major copy are counted.
+__global__ void mirror_values_kernel(Sliced rows, Sliced cols, int n, unsigned long long* mismatch) {
+    const int cc = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);      // one warp per transposed unit
+    if (cc >= n) return;
+    const int len = cols.len[cc];
+    const int j = cols.order[cc];
+    const int base = cols.slice_off[cc >> 3] + (cc & 7) * 4;
+    for (int q = threadIdx.x & 31; q < len; q += 32) {
+        const int pos = base + (q >> 2) * 32 + (q & 3);
+        const int i = cols.idx[pos];
+        const int rb = rows.slice_off[i >> 3] + (i & 7) * 4;
+        int lo = 0, hi = rows.len[i] - 1, at = -1;
+        while (lo <= hi) {
+            const int mid = (lo + hi) >> 1;
+            const int c = rows.idx[rb + (mid >> 2) * 32 + (mid & 3)];
+            if (c == j) { at = mid; break; }
+            if (c < j) lo = mid + 1; else hi = mid - 1;
+        }
+        if (at < 0) { if (mismatch) atomicAdd(mismatch, 1ull << 32); continue; }     // pattern error: high word
+        const float w = rows.val[rb + (at >> 2) * 32 + (at & 3)];
+        if (mismatch) {
+            if (__float_as_uint(w) != __float_as_uint(cols.val[pos])) atomicAdd(mismatch, 1ull);
+        } else {
+            cols.val[pos] = w;
         }
     }
 }

@@ -1,16 +1,23 @@
 // Host side of libsdnn.so: the C ABI declared in include/sdnn.h.
-// Validation, device memory, the per-layer launch sequences (optionally as a CUDA graph) and
-// the staging of host buffers.  Every arithmetic step runs in the kernels of kernels.cuh.
+// Validation, re-layout of the stored entries into the kernels' sliced format, device memory, the
+// per-layer launch sequences (optionally as a CUDA graph) and the staging of host buffers.  Every
+// arithmetic step runs in the kernels of kernels.cuh.
 #include "../../include/sdnn.h"
 #include "kernels.cuh"
 
+#include <algorithm>
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <map>
 #include <new>
 #include <string>
+#include <tuple>
 #include <vector>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
 
 using namespace sdnn_kernels;
 
@@ -18,38 +25,57 @@ namespace {
 
 thread_local std::string g_create_error;
 
-struct DevBuf {
-    void* p = nullptr;
-    size_t bytes = 0;
+// Host description of a layer's stored entries, kept for get/set_weights: either every row has the same
+// number of entries (no array needed) or the caller's row_ptr is remembered.
+struct RowShape {
+    int uniform_k = -1;
+    std::vector<int> row_ptr;
+    int len(int i) const { return uniform_k >= 0 ? uniform_k : row_ptr[i + 1] - row_ptr[i]; }
+    int64_t start(int i) const { return uniform_k >= 0 ? (int64_t)i * uniform_k : row_ptr[i]; }
+};
+
+struct LayerMem {
+    int64_t r_elems = 0, c_elems = 0;      // padded lengths of the two sliced copies
+    int* r_idx = nullptr; float* r_val = nullptr; float* r_grad = nullptr;
+    int* c_idx = nullptr; float* c_val = nullptr;
+    std::vector<int> r_slice_off;          // host copy of the row-major slice offsets
+    RowShape shape;
 };
 
 }  // namespace
 
 struct sdnn {
-    int L = 0, N = 0;
+    int L = 0, N = 0, NS = 0;           // layers, neurons, slices of 8 rows
     sdnn_config cfg{};
     cudaStream_t stream = nullptr;
     bool own_stream = false;
-    int device = 0;
+    int device = 0, sms = 0;
     bool finalized = false, stepped = false;
-    std::vector<int64_t> nnz, off;      // stored entries per layer; offset of the layer in the arenas (elements)
+    bool mirror = false;                // training with the transposed copy (no atomics)
+    bool pdl = false;                   // programmatic dependent launch between the layer kernels
+    bool steps4 = false;                // TUNING: 4 chunks per pipeline step instead of 2
+    int tune_wps = 0;                   // TUNING: forced warps per SM
+    std::vector<int64_t> nnz;
     std::vector<char> loaded;
-    int64_t slots = 0;                  // arena length in elements
+    std::vector<LayerMem> lay;
     int ld_max = 0;                     // padded width of the widest tile this handle processes
 
-    int* d_row_ptr = nullptr;           // [L][N+1], offsets local to the layer
-    int* d_col = nullptr;               // arena
-    float* d_val = nullptr;             // arena
+    int* d_r_slice_off = nullptr;       // [L][NS+1]
+    int* d_r_len = nullptr;             // [L][N]
+    int* d_c_slice_off = nullptr;       // [L][NS+1]   (mirror)
+    int* d_c_len = nullptr;             // [L][N]
+    int* d_c_order = nullptr;           // [L][N]
     float* d_bias = nullptr;            // [L][N]
 
     // training
     float* d_acts = nullptr;            // [(L+1)][N][ld]: x^0 .. x^L of the current step
-    float* d_s[2] = {nullptr, nullptr}; // alternating S = W^T delta tiles, all-zero between steps
+    float* d_s[2] = {nullptr, nullptr}; // atomics: alternating S = W^T delta tiles (all-zero between steps); mirror: delta tiles
+    float* d_dl = nullptr;              // delta^L tile (atomics realisation)
     float* d_yt = nullptr;              // target tile
     StepParams* d_sp = nullptr;
     double* d_loss = nullptr;
     float* d_dbg_delta = nullptr;       // [L][N][ld]   (KEEP_DEBUG)
-    float* d_dbg_grad = nullptr;        // arena        (KEEP_DEBUG)
+    unsigned long long* d_mismatch = nullptr;
     int last_b = 0, last_ld = 0;
     cudaGraphExec_t graph = nullptr;
     int graph_ld = 0;
@@ -68,6 +94,9 @@ struct sdnn {
     int* d_stage_cnt = nullptr;
     int* d_stage_idx = nullptr;
     int64_t stage_idx_cap = 0;
+
+    std::map<std::tuple<const void*, int, int>, std::pair<int, int>> plans;   // (kernel, units, chunks) -> (grid.x, block)
+    std::map<std::pair<const void*, int>, int> occupancy;                     // (kernel, block) -> resident CTAs per SM
 
     int64_t launches = 0;
     int64_t dev_bytes = 0;
@@ -134,7 +163,6 @@ int validate_cfg(const sdnn_config* cfg) {
     if (cfg->train && cfg->max_batch > 128) return fail(nullptr, SDNN_ERR_INVALID_ARG, "training handles support max_batch <= 128");
     if ((cfg->flags & SDNN_FLAG_BWD_ATOMICS) && (cfg->flags & SDNN_FLAG_BWD_CSC))
         return fail(nullptr, SDNN_ERR_INVALID_ARG, "choose one backward strategy");
-    if (cfg->flags & SDNN_FLAG_BWD_CSC) return fail(nullptr, SDNN_ERR_UNIMPLEMENTED, "transposed-index backward is not implemented");
     return SDNN_OK;
 }
 
@@ -172,15 +200,113 @@ int validate_layer(sdnn* h, int layer, int n, int64_t expect_nnz, const int32_t*
     return SDNN_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Sliced layout (see kernels.cuh): slices of 8 units, chunks of 4 entries interleaved over the 8 units.
+inline int64_t sliced_pos(const int* slice_off, int unit, int q) {
+    return (int64_t)slice_off[unit >> 3] + (int64_t)(q >> 2) * 32 + (unit & 7) * 4 + (q & 3);
+}
+
+// slice offsets from unit lengths; returns the padded element count or -1 if it does not fit int32
+template <typename LenFn>
+int64_t build_slice_offsets(int n, LenFn len, std::vector<int>& off) {
+    const int ns = (n + 7) / 8;
+    off.assign(ns + 1, 0);
+    int64_t run = 0;
+    for (int s = 0; s < ns; ++s) {
+        int w = 0;
+        for (int i = s * 8; i < std::min(n, s * 8 + 8); ++i) w = std::max(w, len(i));
+        w = (w + 7) / 8 * 8;      // whole pipeline steps of two chunks
+        run += 8LL * w;
+        if (run > INT32_MAX) return -1;
+        off[s + 1] = (int)run;
+    }
+    return run;
+}
+
 void count_launch(sdnn* h, int k = 1) { h->launches += k; }
+
+// ---------------------------------------------------------------------------------------------
+// Launch shapes.  The layer kernels are persistent: warps take units in a grid-stride loop.  The number of
+// warps per SM is chosen so that the last round of the loop is as full as possible (a nearly empty last
+// round leaves too few requests in flight to keep the memory system busy).
+int resident_ctas(sdnn* h, const void* kernel, int block) {
+    auto key = std::make_pair(kernel, block);
+    auto it = h->occupancy.find(key);
+    if (it != h->occupancy.end()) return it->second;
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, block, 0) != cudaSuccess || occ < 1) { cudaGetLastError(); occ = 1; }
+    h->occupancy[key] = occ;
+    return occ;
+}
+
+std::pair<int, int> plan_grid(sdnn* h, const void* kernel, int units, int chunks) {
+    auto key = std::make_tuple(kernel, units, chunks);
+    auto it = h->plans.find(key);
+    if (it != h->plans.end()) return it->second;
+    double best = -1.0;
+    std::pair<int, int> pick{1, 256};
+    for (int wpb = 8; wpb >= 4; --wpb) {
+        const int block = wpb * 32;
+        const int occ = resident_ctas(h, kernel, block);
+        for (int c = occ; c >= 1; --c) {
+            const int per_sm_warps = c * wpb;
+            if (per_sm_warps < 16 && c != occ) continue;
+            if (h->tune_wps && per_sm_warps != h->tune_wps) continue;
+            int gx = std::max(1, h->sms * c / chunks);
+            const int64_t warps = (int64_t)gx * wpb;
+            if (warps >= units) {      // one round: a plain grid of ceil(units / wpb) CTAs does it
+                gx = (units + wpb - 1) / wpb;
+                const double eff = 1.0 + 1e-3 * per_sm_warps / 64.0;
+                if (eff > best) { best = eff; pick = {gx, block}; }
+                continue;
+            }
+            const int64_t rounds = (units + warps - 1) / warps;
+            double eff = (double)units / (double)(rounds * warps) + 1e-3 * per_sm_warps / 64.0;   // ties: more warps
+            if (eff > best) { best = eff; pick = {gx, block}; }
+        }
+    }
+    h->plans[key] = pick;
+    return pick;
+}
+
+Sliced rows_of(sdnn* h, int layer) {
+    Sliced m;
+    m.slice_off = h->d_r_slice_off + (size_t)layer * (h->NS + 1);
+    m.len = h->d_r_len + (size_t)layer * h->N;
+    m.idx = h->lay[layer].r_idx;
+    m.val = h->lay[layer].r_val;
+    m.order = nullptr;
+    return m;
+}
+
+Sliced cols_of(sdnn* h, int layer) {
+    Sliced m;
+    m.slice_off = h->d_c_slice_off + (size_t)layer * (h->NS + 1);
+    m.len = h->d_c_len + (size_t)layer * h->N;
+    m.idx = h->lay[layer].c_idx;
+    m.val = h->lay[layer].c_val;
+    m.order = h->d_c_order + (size_t)layer * h->N;
+    return m;
+}
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_k(sdnn* h, void (*kernel)(KArgs...), dim3 grid, dim3 block, bool pdl, Args... args) {
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = grid; lc.blockDim = block; lc.dynamicSmemBytes = 0; lc.stream = h->stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = at; lc.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&lc, kernel, KArgs(args)...);
+}
 
 template <int G>
 void launch_forward_g(sdnn* h, int layer, const float* xin, float* xout, int ld, int chunks) {
-    const int rows_per_block = 8 * (32 / G);
-    dim3 grid((h->N + rows_per_block - 1) / rows_per_block, chunks);
-    forward_kernel<G><<<grid, 256, 0, h->stream>>>(h->d_row_ptr + (size_t)layer * (h->N + 1), h->d_col + h->off[layer],
-                                                   h->d_val + h->off[layer], h->d_bias + (size_t)layer * h->N, xin, xout,
-                                                   h->N, ld, h->cfg.clamp);
+    constexpr int RPW = 32 / G;
+    const int units = (h->N + RPW - 1) / RPW;
+    auto plan = plan_grid(h, (const void*)forward_kernel<G>, units, chunks);
+    launch_k(h, forward_kernel<G>, dim3(plan.first, chunks), dim3(plan.second), h->pdl, rows_of(h, layer),
+             (const float*)(h->d_bias + (size_t)layer * h->N), xin, xout, h->N, ld, h->cfg.clamp, h->pdl ? 1 : 0);
 }
 
 void launch_forward(sdnn* h, int layer, const float* xin, float* xout, int ld, int cols) {
@@ -196,30 +322,63 @@ void launch_forward(sdnn* h, int layer, const float* xin, float* xout, int ld, i
     count_launch(h);
 }
 
+// delta tile of layer `layer` (0-based; the paper's delta^{layer+1}) in the transposed realisation
+float* delta_tile(sdnn* h, int layer, size_t tile) {
+    return h->d_dbg_delta ? h->d_dbg_delta + (size_t)layer * tile : h->d_s[layer & 1];
+}
+
 template <int G>
 void launch_backward_g(sdnn* h, int layer, int ld) {
-    const int rows_per_block = 8 * (32 / G);
-    dim3 grid((h->N + rows_per_block - 1) / rows_per_block);
+    constexpr int RPW = 32 / G;
     const size_t tile = (size_t)h->N * ld;
     const bool last = layer == h->L - 1, prop = layer > 0;
-    const int* rp = h->d_row_ptr + (size_t)layer * (h->N + 1);
-    const int* col = h->d_col + h->off[layer];
-    float* val = h->d_val + h->off[layer];
-    float* bias = h->d_bias + (size_t)layer * h->N;
-    const float* xk = h->d_acts + (size_t)(layer + 1) * tile;
-    const float* xprev = h->d_acts + (size_t)layer * tile;
-    float* s_k = last ? h->d_yt : h->d_s[(layer + 1) & 1];
-    float* s_prev = h->d_s[layer & 1];
-    float* dd = h->d_dbg_delta ? h->d_dbg_delta + (size_t)layer * tile : nullptr;
-    float* dg = h->d_dbg_grad ? h->d_dbg_grad + h->off[layer] : nullptr;
-    const int ub = h->cfg.update_bias ? 1 : 0, sk = (h->cfg.flags & SDNN_FLAG_SKIP_DEAD) ? 1 : 0;
-#define SDNN_BWD(LASTV, PROPV)                                                                              \
-    backward_kernel<G, LASTV, PROPV><<<grid, 256, 0, h->stream>>>(rp, col, val, bias, xk, xprev, s_k, s_prev, \
-                                                                  h->N, h->cfg.clamp, h->d_sp, h->d_loss, dd, dg, ub, sk)
-    if (last && prop) SDNN_BWD(true, true);
-    else if (last) SDNN_BWD(true, false);
-    else if (prop) SDNN_BWD(false, true);
-    else SDNN_BWD(false, false);
+    const int units = (h->N + RPW - 1) / RPW;
+    BackwardArgs a{};
+    a.rows = rows_of(h, layer);
+    a.bias = h->d_bias + (size_t)layer * h->N;
+    a.xk = h->d_acts + (size_t)(layer + 1) * tile;
+    a.xprev = h->d_acts + (size_t)layer * tile;
+    a.dbg_grad = h->lay[layer].r_grad;
+    a.sp = h->d_sp;
+    a.n = h->N;
+    a.clamp = h->cfg.clamp;
+    a.update_bias = h->cfg.update_bias ? 1 : 0;
+    a.skip_dead = (h->cfg.flags & SDNN_FLAG_SKIP_DEAD) ? 1 : 0;
+    a.pdl = h->pdl ? 1 : 0;
+    a.col_units = 0;
+    const void* fn = nullptr;
+#define SDNN_BWD(FROM_S, SCAT, MIR, TOTAL)                                                     \
+    do {                                                                                       \
+        if (a.dbg_grad) {                                                                      \
+            fn = (const void*)backward_kernel<G, FROM_S, SCAT, MIR, true>;                     \
+            auto plan = plan_grid(h, fn, (TOTAL), 1);                                          \
+            launch_k(h, backward_kernel<G, FROM_S, SCAT, MIR, true>, dim3(plan.first), dim3(plan.second), h->pdl, a); \
+        } else {                                                                               \
+            fn = (const void*)backward_kernel<G, FROM_S, SCAT, MIR, false>;                    \
+            auto plan = plan_grid(h, fn, (TOTAL), 1);                                          \
+            launch_k(h, backward_kernel<G, FROM_S, SCAT, MIR, false>, dim3(plan.first), dim3(plan.second), h->pdl, a); \
+        }                                                                                      \
+    } while (0)
+    if (h->mirror) {
+        a.dk = delta_tile(h, layer, tile);
+        if (prop) {
+            a.cols = cols_of(h, layer);
+            a.col_units = units;
+            a.dprev = delta_tile(h, layer - 1, tile);
+            SDNN_BWD(false, false, true, units);
+        } else {
+            SDNN_BWD(false, false, false, units);
+        }
+    } else {
+        float* dl = h->d_dbg_delta ? h->d_dbg_delta + (size_t)layer * tile : h->d_dl;
+        a.dk = last ? dl : h->d_s[(layer + 1) & 1];
+        a.dprev = h->d_s[layer & 1];
+        a.dbg_delta = (!last && h->d_dbg_delta) ? h->d_dbg_delta + (size_t)layer * tile : nullptr;
+        if (last && prop) SDNN_BWD(false, true, false, units);
+        else if (last) SDNN_BWD(false, false, false, units);
+        else if (prop) SDNN_BWD(true, true, false, units);
+        else SDNN_BWD(true, false, false, units);
+    }
 #undef SDNN_BWD
 }
 
@@ -232,6 +391,17 @@ void launch_backward(sdnn* h, int layer, int ld) {
         case 16: launch_backward_g<16>(h, layer, ld); break;
         default: launch_backward_g<32>(h, layer, ld); break;
     }
+    count_launch(h);
+}
+
+void launch_output_gradient(sdnn* h, int ld) {
+    const size_t tile = (size_t)h->N * ld;
+    float* dl = h->mirror ? delta_tile(h, h->L - 1, tile)
+                          : (h->d_dbg_delta ? h->d_dbg_delta + (size_t)(h->L - 1) * tile : h->d_dl);
+    const long long vecs = (long long)h->N * (ld / 4);
+    const int grid = (int)std::min<long long>((vecs + 255) / 256, (long long)h->sms * 8);
+    output_gradient_kernel<<<grid, 256, 0, h->stream>>>(h->d_acts + (size_t)h->L * tile, h->d_yt, dl, h->N, ld, h->cfg.clamp,
+                                                        h->d_sp, h->d_loss);
     count_launch(h);
 }
 
@@ -249,6 +419,7 @@ void enqueue_step_body(sdnn* h, int ld, unsigned flags) {
     for (int k = 0; k < h->L; ++k)
         launch_forward(h, k, h->d_acts + (size_t)k * tile, h->d_acts + (size_t)(k + 1) * tile, ld, ld);
     cudaEventRecordWithFlags(h->ev[1], h->stream, flags);
+    launch_output_gradient(h, ld);
     for (int k = h->L - 1; k >= 0; --k) launch_backward(h, k, ld);
     cudaEventRecordWithFlags(h->ev[2], h->stream, flags);
 }
@@ -277,7 +448,7 @@ int train_step_device(sdnn* h, const float* x0, const float* target, int B, floa
             h->graph_ld = ld;
         }
         CU(h, cudaGraphLaunch(h->graph, h->stream));
-        count_launch(h, 2 * h->L);
+        count_launch(h, 2 * h->L + 1);
     }
     CU(h, cudaGetLastError());
     h->stepped = true; h->last_b = B; h->last_ld = ld;
@@ -352,11 +523,40 @@ int ensure_stage(sdnn* h) {
     return SDNN_OK;
 }
 
+// values in the caller's CSR order -> row-major sliced copy (padding zero)
+void csr_to_sliced(const sdnn* h, const LayerMem& lm, const float* src, std::vector<float>& dst) {
+    dst.assign((size_t)lm.r_elems, 0.0f);
+    const int* off = lm.r_slice_off.data();
+#pragma omp parallel for schedule(static)
+    for (int i = 0; i < h->N; ++i) {
+        const int len = lm.shape.len(i);
+        const int64_t s = lm.shape.start(i);
+        for (int q = 0; q < len; ++q) dst[(size_t)sliced_pos(off, i, q)] = src[s + q];
+    }
+}
+
+void sliced_to_csr(const sdnn* h, const LayerMem& lm, const std::vector<float>& src, float* dst) {
+    const int* off = lm.r_slice_off.data();
+#pragma omp parallel for schedule(static)
+    for (int i = 0; i < h->N; ++i) {
+        const int len = lm.shape.len(i);
+        const int64_t s = lm.shape.start(i);
+        for (int q = 0; q < len; ++q) dst[s + q] = src[(size_t)sliced_pos(off, i, q)];
+    }
+}
+
+int refresh_mirror(sdnn* h, int layer, unsigned long long* mismatch_dev) {
+    const int wpb = 8;
+    mirror_values_kernel<<<(h->N + wpb - 1) / wpb, wpb * 32, 0, h->stream>>>(rows_of(h, layer), cols_of(h, layer), h->N, mismatch_dev);
+    CU(h, cudaGetLastError());
+    return SDNN_OK;
+}
+
 }  // namespace
 
 extern "C" {
 
-const char* sdnn_version(void) { return "sdnn 0.1 (sm_100a)"; }
+const char* sdnn_version(void) { return "sdnn 0.2 (sm_100a)"; }
 
 const char* sdnn_last_error(const sdnn_t* h) { return h ? h->err.c_str() : g_create_error.c_str(); }
 
@@ -392,7 +592,7 @@ int sdnn_create_deferred(sdnn_t** out, int32_t n_layers, int32_t n_neurons, cons
 
     sdnn* h = new (std::nothrow) sdnn;
     if (!h) return fail(nullptr, SDNN_ERR_OOM, "host allocation failed");
-    h->L = n_layers; h->N = n_neurons; h->cfg = *cfg;
+    h->L = n_layers; h->N = n_neurons; h->NS = (n_neurons + 7) / 8; h->cfg = *cfg;
     h->stream = static_cast<cudaStream_t>(cfg->cuda_stream);
     auto bail = [&](int code) { g_create_error = h->err; sdnn_destroy(h); return code; };
     if (cfg->device >= 0) {
@@ -402,37 +602,44 @@ int sdnn_create_deferred(sdnn_t** out, int32_t n_layers, int32_t n_neurons, cons
     } else if ((e = cudaGetDevice(&h->device)) != cudaSuccess) {
         return bail(cuda_fail(h, e, "cudaGetDevice"));
     }
+    if ((e = cudaDeviceGetAttribute(&h->sms, cudaDevAttrMultiProcessorCount, h->device)) != cudaSuccess || h->sms < 1)
+        return bail(cuda_fail(h, e, "cudaDeviceGetAttribute(multiprocessor count)"));
     if (!h->stream) {   // the legacy default stream cannot be captured into a graph: use a blocking stream of our own,
                         // which still orders itself against work on the legacy default stream
         if ((e = cudaStreamCreate(&h->stream)) != cudaSuccess) { h->stream = nullptr; return bail(cuda_fail(h, e, "cudaStreamCreate")); }
         h->own_stream = true;
     }
+    h->mirror = cfg->train && !(cfg->flags & SDNN_FLAG_BWD_ATOMICS);
+    h->pdl = !(cfg->flags & SDNN_FLAG_NO_PDL);
+    if (const char* e_ = getenv("SDNN_TUNE_S4")) h->steps4 = atoi(e_) != 0;
+    if (const char* e_ = getenv("SDNN_TUNE_WPS")) h->tune_wps = atoi(e_);
     h->nnz.assign(nnz_per_layer, nnz_per_layer + n_layers);
-    h->off.resize(n_layers);
     h->loaded.assign(n_layers, 0);
-    int64_t run = 0;
-    for (int l = 0; l < n_layers; ++l) { h->off[l] = run; run += (h->nnz[l] + 31) / 32 * 32; }   // 128-byte aligned layers
-    h->slots = run;
+    h->lay.resize(n_layers);
     h->ld_max = padded_width(cfg->max_batch);
     const size_t N = (size_t)n_neurons, L = (size_t)n_layers, tile = N * (size_t)h->ld_max;
 
-    if ((rc = dev_alloc(h, &h->d_row_ptr, L * (N + 1), false))) return bail(rc);
-    if ((rc = dev_alloc(h, &h->d_col, (size_t)h->slots, true))) return bail(rc);
-    if ((rc = dev_alloc(h, &h->d_val, (size_t)h->slots, true))) return bail(rc);
+    if ((rc = dev_alloc(h, &h->d_r_slice_off, L * (h->NS + 1), false))) return bail(rc);
+    if ((rc = dev_alloc(h, &h->d_r_len, L * N, false))) return bail(rc);
     if ((rc = dev_alloc(h, &h->d_bias, L * N, false))) return bail(rc);
+    if (h->mirror) {
+        if ((rc = dev_alloc(h, &h->d_c_slice_off, L * (h->NS + 1), false))) return bail(rc);
+        if ((rc = dev_alloc(h, &h->d_c_len, L * N, false))) return bail(rc);
+        if ((rc = dev_alloc(h, &h->d_c_order, L * N, false))) return bail(rc);
+        if ((rc = dev_alloc(h, &h->d_mismatch, 1, true))) return bail(rc);
+    }
     if (cfg->train) {
         for (cudaEvent_t& ev : h->ev)
             if ((e = cudaEventCreate(&ev)) != cudaSuccess) { ev = nullptr; return bail(cuda_fail(h, e, "cudaEventCreate")); }
         if ((rc = dev_alloc(h, &h->d_acts, (L + 1) * tile, false))) return bail(rc);
         if ((rc = dev_alloc(h, &h->d_s[0], tile, true))) return bail(rc);
         if ((rc = dev_alloc(h, &h->d_s[1], tile, true))) return bail(rc);
+        if (!h->mirror && (rc = dev_alloc(h, &h->d_dl, tile, true))) return bail(rc);
         if ((rc = dev_alloc(h, &h->d_yt, tile, true))) return bail(rc);
         if ((rc = dev_alloc(h, &h->d_sp, 1, true))) return bail(rc);
         if ((rc = dev_alloc(h, &h->d_loss, 1, true))) return bail(rc);
-        if (cfg->flags & SDNN_FLAG_KEEP_DEBUG) {
+        if (cfg->flags & SDNN_FLAG_KEEP_DEBUG)
             if ((rc = dev_alloc(h, &h->d_dbg_delta, L * tile, true))) return bail(rc);
-            if ((rc = dev_alloc(h, &h->d_dbg_grad, (size_t)h->slots, true))) return bail(rc);
-        }
     }
     {   // inference buffers (a training handle can also infer)
         const size_t nseg = (N + NZ_SEG - 1) / NZ_SEG;
@@ -456,14 +663,85 @@ int sdnn_load_layer(sdnn_t* h, int32_t layer, const int32_t* row_ptr, const int3
     int rc = validate_layer(h, layer, h->N, h->nnz[layer], row_ptr, col_idx, values, bias);
     if (rc) return rc;
     CU(h, cudaSetDevice(h->device));
-    const size_t N = (size_t)h->N, nz = (size_t)h->nnz[layer];
-    CU(h, cudaMemcpyAsync(h->d_row_ptr + (size_t)layer * (N + 1), row_ptr, (N + 1) * sizeof(int), cudaMemcpyHostToDevice, h->stream));
-    CU(h, cudaMemcpyAsync(h->d_bias + (size_t)layer * N, bias, N * sizeof(float), cudaMemcpyHostToDevice, h->stream));
-    if (nz) {
-        CU(h, cudaMemcpyAsync(h->d_col + h->off[layer], col_idx, nz * sizeof(int), cudaMemcpyHostToDevice, h->stream));
-        CU(h, cudaMemcpyAsync(h->d_val + h->off[layer], values, nz * sizeof(float), cudaMemcpyHostToDevice, h->stream));
+    const int N = h->N, NS = h->NS;
+    LayerMem& lm = h->lay[layer];
+
+    // ---- row-major sliced copy
+    bool uniform = true;
+    const int k0 = row_ptr[1] - row_ptr[0];
+    for (int i = 1; i < N && uniform; ++i) uniform = (row_ptr[i + 1] - row_ptr[i]) == k0;
+    if (uniform) lm.shape.uniform_k = k0; else lm.shape.row_ptr.assign(row_ptr, row_ptr + N + 1);
+    std::vector<int> r_len(N);
+    for (int i = 0; i < N; ++i) r_len[i] = row_ptr[i + 1] - row_ptr[i];
+    lm.r_elems = build_slice_offsets(N, [&](int i) { return r_len[i]; }, lm.r_slice_off);
+    if (lm.r_elems < 0) return fail(h, SDNN_ERR_INVALID_ARG, "layer %d: padded sliced layout exceeds 2^31 entries", layer);
+    std::vector<int> r_idx((size_t)lm.r_elems, 0);
+    std::vector<float> r_val;
+    csr_to_sliced(h, lm, values, r_val);
+    {
+        const int* off = lm.r_slice_off.data();
+#pragma omp parallel for schedule(static)
+        for (int i = 0; i < N; ++i)
+            for (int q = 0; q < r_len[i]; ++q) r_idx[(size_t)sliced_pos(off, i, q)] = col_idx[row_ptr[i] + q];
     }
-    CU(h, cudaStreamSynchronize(h->stream));   // the caller may reuse its arrays right away
+    if ((rc = dev_alloc(h, &lm.r_idx, (size_t)lm.r_elems, false))) return rc;
+    if ((rc = dev_alloc(h, &lm.r_val, (size_t)lm.r_elems, false))) return rc;
+    if (h->cfg.train && (h->cfg.flags & SDNN_FLAG_KEEP_DEBUG))
+        if ((rc = dev_alloc(h, &lm.r_grad, (size_t)lm.r_elems, true))) return rc;
+    CU(h, cudaMemcpyAsync(h->d_r_slice_off + (size_t)layer * (NS + 1), lm.r_slice_off.data(), (size_t)(NS + 1) * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+    CU(h, cudaMemcpyAsync(h->d_r_len + (size_t)layer * N, r_len.data(), (size_t)N * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+    CU(h, cudaMemcpyAsync(h->d_bias + (size_t)layer * N, bias, (size_t)N * sizeof(float), cudaMemcpyHostToDevice, h->stream));
+    if (lm.r_elems) {
+        CU(h, cudaMemcpyAsync(lm.r_idx, r_idx.data(), (size_t)lm.r_elems * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+        CU(h, cudaMemcpyAsync(lm.r_val, r_val.data(), (size_t)lm.r_elems * sizeof(float), cudaMemcpyHostToDevice, h->stream));
+    }
+
+    // ---- transposed sliced copy (not needed for the first layer: delta^0 is never formed)
+    std::vector<int> c_idx, c_len, order, c_off;
+    if (h->mirror && layer > 0) {
+        const int64_t nz = h->nnz[layer];
+        std::vector<int> deg(N, 0);
+        for (int64_t p = 0; p < nz; ++p) ++deg[col_idx[p]];
+        int dmax = 0;
+        for (int j = 0; j < N; ++j) dmax = std::max(dmax, deg[j]);
+        // columns by descending length (stable in j): slices of nearly equal length, little padding
+        std::vector<int> bucket(dmax + 2, 0);
+        for (int j = 0; j < N; ++j) ++bucket[dmax - deg[j] + 1];
+        for (int d = 0; d <= dmax; ++d) bucket[d + 1] += bucket[d];
+        order.resize(N);
+        std::vector<int> place(N);
+        for (int j = 0; j < N; ++j) { const int cc = bucket[dmax - deg[j]]++; order[cc] = j; place[j] = cc; }
+        c_len.resize(N);
+        for (int cc = 0; cc < N; ++cc) c_len[cc] = deg[order[cc]];
+        lm.c_elems = build_slice_offsets(N, [&](int cc) { return c_len[cc]; }, c_off);
+        if (lm.c_elems < 0) return fail(h, SDNN_ERR_INVALID_ARG, "layer %d: padded transposed layout exceeds 2^31 entries", layer);
+        c_idx.assign((size_t)lm.c_elems, 0);
+        // each thread owns a range of columns and scans all entries in row order: rows ascend within a column
+#pragma omp parallel
+        {
+            int nt = 1, tid = 0;
+#ifdef _OPENMP
+            nt = omp_get_num_threads(); tid = omp_get_thread_num();
+#endif
+            const int j0 = (int)((int64_t)N * tid / nt), j1 = (int)((int64_t)N * (tid + 1) / nt);
+            std::vector<int> cursor(j1 - j0, 0);
+            for (int i = 0; i < N; ++i)
+                for (int p = row_ptr[i]; p < row_ptr[i + 1]; ++p) {
+                    const int j = col_idx[p];
+                    if (j < j0 || j >= j1) continue;
+                    const int q = cursor[j - j0]++;
+                    c_idx[(size_t)sliced_pos(c_off.data(), place[j], q)] = i;
+                }
+        }
+        if ((rc = dev_alloc(h, &lm.c_idx, (size_t)lm.c_elems, false))) return rc;
+        if ((rc = dev_alloc(h, &lm.c_val, (size_t)lm.c_elems, true))) return rc;
+        CU(h, cudaMemcpyAsync(h->d_c_slice_off + (size_t)layer * (NS + 1), c_off.data(), (size_t)(NS + 1) * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+        CU(h, cudaMemcpyAsync(h->d_c_len + (size_t)layer * N, c_len.data(), (size_t)N * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+        CU(h, cudaMemcpyAsync(h->d_c_order + (size_t)layer * N, order.data(), (size_t)N * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+        if (lm.c_elems) CU(h, cudaMemcpyAsync(lm.c_idx, c_idx.data(), (size_t)lm.c_elems * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+        if ((rc = refresh_mirror(h, layer, nullptr))) return rc;
+    }
+    CU(h, cudaStreamSynchronize(h->stream));   // the host vectors above go out of scope; the caller may reuse its arrays
     h->loaded[layer] = 1;
     return SDNN_OK;
 }
@@ -594,8 +872,12 @@ int sdnn_get_weights(sdnn_t* h, int32_t layer, float* values_out, float* bias_ou
     if (layer < 0 || layer >= h->L) return fail(h, SDNN_ERR_INVALID_ARG, "layer %d outside [0, %d)", layer, h->L);
     CU(h, cudaSetDevice(h->device));
     CU(h, cudaStreamSynchronize(h->stream));
-    if (values_out && h->nnz[layer])
-        CU(h, cudaMemcpy(values_out, h->d_val + h->off[layer], (size_t)h->nnz[layer] * sizeof(float), cudaMemcpyDeviceToHost));
+    const LayerMem& lm = h->lay[layer];
+    if (values_out && lm.r_elems) {
+        std::vector<float> tmp((size_t)lm.r_elems);
+        CU(h, cudaMemcpy(tmp.data(), lm.r_val, tmp.size() * sizeof(float), cudaMemcpyDeviceToHost));
+        sliced_to_csr(h, lm, tmp, values_out);
+    }
     if (bias_out) CU(h, cudaMemcpy(bias_out, h->d_bias + (size_t)layer * h->N, (size_t)h->N * sizeof(float), cudaMemcpyDeviceToHost));
     return SDNN_OK;
 }
@@ -612,9 +894,35 @@ int sdnn_set_weights(sdnn_t* h, int32_t layer, const float* values, const float*
             if (!std::isfinite(bias[i])) return fail(h, SDNN_ERR_BAD_CSR, "layer %d: non-finite bias at row %d", layer, i);
     CU(h, cudaSetDevice(h->device));
     CU(h, cudaStreamSynchronize(h->stream));
-    if (values && h->nnz[layer])
-        CU(h, cudaMemcpy(h->d_val + h->off[layer], values, (size_t)h->nnz[layer] * sizeof(float), cudaMemcpyHostToDevice));
+    const LayerMem& lm = h->lay[layer];
+    if (values && lm.r_elems) {
+        std::vector<float> tmp;
+        csr_to_sliced(h, lm, values, tmp);
+        CU(h, cudaMemcpy(lm.r_val, tmp.data(), tmp.size() * sizeof(float), cudaMemcpyHostToDevice));
+        if (lm.c_val) {
+            int rc = refresh_mirror(h, layer, nullptr);
+            if (rc) return rc;
+            CU(h, cudaStreamSynchronize(h->stream));
+        }
+    }
     if (bias) CU(h, cudaMemcpy(h->d_bias + (size_t)layer * h->N, bias, (size_t)h->N * sizeof(float), cudaMemcpyHostToDevice));
+    return SDNN_OK;
+}
+
+int sdnn_mirror_mismatches(sdnn_t* h, int32_t layer, int64_t* count_out) {
+    if (!h || !count_out) return SDNN_ERR_INVALID_ARG;
+    if (!h->finalized) return fail(h, SDNN_ERR_STATE, "handle is not finalized");
+    if (layer < 0 || layer >= h->L) return fail(h, SDNN_ERR_INVALID_ARG, "layer %d outside [0, %d)", layer, h->L);
+    *count_out = 0;
+    if (!h->lay[layer].c_val) return SDNN_OK;      // no transposed copy for this layer: nothing can differ
+    CU(h, cudaSetDevice(h->device));
+    CU(h, cudaMemsetAsync(h->d_mismatch, 0, sizeof(unsigned long long), h->stream));
+    int rc = refresh_mirror(h, layer, h->d_mismatch);
+    if (rc) return rc;
+    unsigned long long v = 0;
+    CU(h, cudaMemcpyAsync(&v, h->d_mismatch, sizeof v, cudaMemcpyDeviceToHost, h->stream));
+    CU(h, cudaStreamSynchronize(h->stream));
+    *count_out = (int64_t)v;
     return SDNN_OK;
 }
 
@@ -646,12 +954,16 @@ int sdnn_get_delta(sdnn_t* h, int32_t layer, float* out) {
 
 int sdnn_get_gradient(sdnn_t* h, int32_t layer, float* out) {
     if (!h || !out) return SDNN_ERR_INVALID_ARG;
-    if (!h->stepped || !h->d_dbg_grad) return fail(h, SDNN_ERR_STATE, "needs SDNN_FLAG_KEEP_DEBUG and a train step");
+    if (!h->stepped || !h->d_dbg_delta) return fail(h, SDNN_ERR_STATE, "needs SDNN_FLAG_KEEP_DEBUG and a train step");
     if (layer < 1 || layer > h->L) return fail(h, SDNN_ERR_INVALID_ARG, "layer %d outside [1, %d]", layer, h->L);
     CU(h, cudaSetDevice(h->device));
     CU(h, cudaStreamSynchronize(h->stream));
-    if (h->nnz[layer - 1])
-        CU(h, cudaMemcpy(out, h->d_dbg_grad + h->off[layer - 1], (size_t)h->nnz[layer - 1] * sizeof(float), cudaMemcpyDeviceToHost));
+    const LayerMem& lm = h->lay[layer - 1];
+    if (lm.r_elems && lm.r_grad) {
+        std::vector<float> tmp((size_t)lm.r_elems);
+        CU(h, cudaMemcpy(tmp.data(), lm.r_grad, tmp.size() * sizeof(float), cudaMemcpyDeviceToHost));
+        sliced_to_csr(h, lm, tmp, out);
+    }
     return SDNN_OK;
 }
 
@@ -713,7 +1025,7 @@ void noalloc_forward_g(cudaStream_t st, const int* rp, const int* col, const flo
                        const float* xin, float* xout, int n, int ld, int chunks, float clamp) {
     const int rows_per_block = 8 * (32 / G);
     dim3 grid((n + rows_per_block - 1) / rows_per_block, chunks);
-    forward_kernel<G><<<grid, 256, 0, st>>>(rp, col, val, bias, xin, xout, n, ld, clamp);
+    forward_csr_kernel<G><<<grid, 256, 0, st>>>(rp, col, val, bias, xin, xout, n, ld, clamp);
 }
 
 }  // namespace

@@ -76,6 +76,8 @@ def train_parity(torch, arrays, batches, eta, update_bias=False, flags=0, clamp=
         errs["loss"] = abs(loss_g - out["loss"]) / max(abs(out["loss"]), 1e-30)
         worst_key = max(errs, key=errs.get)
         assert errs[worst_key] <= TOL, f"{worst_key}: rel err {errs[worst_key]:.3g} > {TOL}"
+        for l in range(L):      # transposed copy (if the handle keeps one) must hold the same bits as the row-major copy
+            assert h.mirror_mismatches(l) == 0, f"step {step}: layer {l} copies differ"
         stats["max_err"] = max(stats["max_err"], errs[worst_key])
         for key in ("ambiguous", "flipped", "entries"):
             stats[key] += getattr(proto, key)
@@ -133,33 +135,43 @@ def batches_for(spec, B, steps):
 
 
 # ---------------------------------------------------------------------------------------------- train
+BWD_MODES = {"transposed": 0x02, "atomics": 0x01}
+
+
 @pytest.mark.parametrize("B", [1, 3, 4, 7, 16, 33, 64, 100, 128])
 @pytest.mark.parametrize("align4", [False, True])
-def test_train_ragged_small(torch_cuda, B, align4):
-    """Ragged / empty rows, every lane-group width, scalar and vector index paths, bias update on."""
+@pytest.mark.parametrize("bwd", sorted(BWD_MODES))
+def test_train_ragged_small(torch_cuda, B, align4, bwd):
+    """Ragged / empty rows, every lane-group width, partial chunks, bias update on; both backward realisations."""
     rng = np.random.default_rng(100 + B)
     arrays = ragged_net(rng, n=203, layers=5, kmax=12, align4=align4)
     batches = [(rng.uniform(0, 1.5, size=(B, 203)).astype(np.float32), rng.uniform(0, 1, size=(B, 203)).astype(np.float32))
                for _ in range(3)]
-    st = train_parity(torch_cuda, arrays, batches, eta=0.01, update_bias=(B % 2 == 1), expect_live=True)
+    st = train_parity(torch_cuda, arrays, batches, eta=0.01, update_bias=(B % 2 == 1), flags=BWD_MODES[bwd], expect_live=True)
     assert st["entries"] > 0
 
 
-def test_train_free_running_trajectories_stay_close(torch_cuda):
-    """No re-synchronisation between steps: parameters persist inside the handle across calls."""
+@pytest.mark.parametrize("bwd", sorted(BWD_MODES))
+def test_train_free_running_trajectories_stay_close(torch_cuda, bwd):
+    """No re-synchronisation between steps: parameters persist inside the handle across calls (and the
+    two copies of the weights of the transposed realisation stay bit-identical over several updates)."""
     rng = np.random.default_rng(77)
     arrays = ragged_net(rng, n=150, layers=4, kmax=8)
     batches = [(rng.uniform(0, 1.5, size=(8, 150)).astype(np.float32), rng.uniform(0, 1, size=(8, 150)).astype(np.float32))
                for _ in range(4)]
-    train_parity(torch_cuda, arrays, batches, eta=0.005, sync=False, expect_live=True)
+    train_parity(torch_cuda, arrays, batches, eta=0.005, sync=False, flags=BWD_MODES[bwd], expect_live=True)
 
 
-def test_train_no_graph_matches(torch_cuda):
+@pytest.mark.parametrize("extra", ["no_graph", "no_pdl", "no_graph_no_pdl"])
+def test_train_launch_variants_match(torch_cuda, extra):
+    """Kernel-by-kernel launches and launches without programmatic dependent launch give the same results."""
+    pkg = sdnn()
+    flags = {"no_graph": pkg.FLAG_NO_GRAPH, "no_pdl": pkg.FLAG_NO_PDL, "no_graph_no_pdl": pkg.FLAG_NO_GRAPH | pkg.FLAG_NO_PDL}[extra]
     rng = np.random.default_rng(5)
     arrays = ragged_net(rng, n=130, layers=4, kmax=8)
     batches = [(rng.uniform(0, 1.5, size=(16, 130)).astype(np.float32), rng.uniform(0, 1, size=(16, 130)).astype(np.float32))
                for _ in range(2)]
-    train_parity(torch_cuda, arrays, batches, eta=0.01, flags=sdnn().FLAG_NO_GRAPH, expect_live=True)
+    train_parity(torch_cuda, arrays, batches, eta=0.01, flags=flags, expect_live=True)
 
 
 @pytest.mark.parametrize("variant,live", [("base", False), ("live", True)])
@@ -181,8 +193,9 @@ def test_train_saturating_hits_upper_kink(torch_cuda):
     (gen.CFG5.scaled(65536, 6).live(), 16, 2),
     (gen.CFG5.scaled(8192, 40).live(), 16, 2),
 ])
-def test_train_scaled_configs(torch_cuda, spec, B, steps):
-    st = train_parity(torch_cuda, gen.network(spec), batches_for(spec, B, steps), eta=1e-3)
+@pytest.mark.parametrize("bwd", sorted(BWD_MODES))
+def test_train_scaled_configs(torch_cuda, spec, B, steps, bwd):
+    st = train_parity(torch_cuda, gen.network(spec), batches_for(spec, B, steps), eta=1e-3, flags=BWD_MODES[bwd])
     print(spec.name, st)
 
 

@@ -1,20 +1,21 @@
 // Device kernels of the sparse-DNN SGD hot path (sm_100a).
 //
 // Tiles.  Activations x^k, deltas and the partial products S = W^T delta live in neuron-major tiles
-// X[i*ld + b] (neuron i, input b; ld = padded batch, a multiple of 4), so that the row of X gathered
-// for one stored entry W(i,j) is contiguous and every access is a 128-bit vector.  A row of a tile is
-// shared by G lanes (G*4 batch entries, one float4 per lane); a warp therefore works on 32/G matrix
-// rows at once.  Tiles wider than 128 inputs are processed in chunks of 128 (blockIdx.y).
+// X[i*ld + b] (neuron i, input b; ld = padded batch), so that the row of X gathered for one stored entry
+// W(i,j) is contiguous.  A lane holds V = 8 batch entries of a row (one 256-bit access; V = 4 only for tiles
+// of 4 columns), a row is shared by G = ld / V lanes, and a warp works on 32/G matrix rows at once.  Tiles
+// wider than 256 inputs are processed in chunks of 256 (blockIdx.y).
 //
-// Stored entries.  What bounds these kernels is the number of L1 wavefronts per stored entry: the
-// gather of a tile row costs one, and with plain CSR the index and value loads of the eight row groups
-// of a warp cost another half each, because the eight rows sit in eight different 128-byte lines.
-// The entries are therefore kept in slices of 8 rows, interleaved in chunks of 4:
-//     entry q of row i  ->  slice_off[i/8] + (q/4)*32 + (i%8)*4 + q%4          (element offset)
-// so that the 16-byte chunks the eight row groups of a warp read in one step are one 128-byte line.
-// A slice is padded to the longest of its rows rounded up to 4; padding has index 0 and value 0 and
-// is never updated.  The transposed matrix (columns as "rows", for the backward product without
-// atomics) uses the same layout over the columns sorted by descending length.
+// Stored entries.  These kernels are bound by instruction issue and by L1 wavefronts per stored entry,
+// not by bytes: the gather of a tile row costs one wavefront whatever its width up to 128 bytes, and with
+// plain CSR the index and value loads of the row groups of a warp would cost as much again, because each row
+// sits in a different 128-byte line.  The entries are therefore kept in slices of 16 rows, interleaved in
+// chunks of 4:
+//     entry q of row i  ->  slice_off[i/16] + (q/4)*64 + (i%16)*4 + q%4          (element offset)
+// so that the 16-byte chunks the row groups of a warp read in one step are contiguous.  A slice is padded
+// to the longest of its rows rounded up to 8; padding has index 0 and value 0 and is never updated.  The
+// transposed matrix (columns as "rows", for the backward product without atomics) uses the same layout over
+// the columns sorted by descending length.
 //
 // Equations (paper, Section 3.2): forward x^k = f(W^k x^{k-1} + b^k); recursion
 // delta^{k-1} = (W^k)^T delta^k (.) f'(z^{k-1}); update W^k(j,i) -= eta delta^k(j) x^{k-1}(i)
@@ -32,10 +33,13 @@ struct StepParams {     // written by set_step_params before each train step; re
     int   pad;
 };
 
+constexpr int SLICE = 16;            // rows per slice
+constexpr int CHUNK_ROW = SLICE * 4; // elements of one chunk over the rows of a slice
+
 // One matrix in sliced layout.  `order` is NULL for the row-major copy (unit u is row u); for the
 // transposed copy it lists the matrix column each unit stands for.
 struct Sliced {
-    const int* slice_off;   // [ceil(n/8) + 1] element offsets of the slices, multiples of 32
+    const int* slice_off;   // [ceil(n/16) + 1] element offsets of the slices, multiples of 128
     const int* len;         // [n] stored entries of each unit
     const int* idx;         // gathered tile row of each entry (column index; row index in the transposed copy)
     float*     val;
@@ -66,25 +70,98 @@ __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddep
 __device__ __forceinline__ float clampf(float z, float c) { return fminf(fmaxf(z, 0.0f), c); }
 __device__ __forceinline__ float dmask(float x, float c) { return (x > 0.0f && x < c) ? 1.0f : 0.0f; }
 
+// address of tile row `r` (r * pitch below 2^32): one 32 x 32 -> 64 bit multiply-add
+__device__ __forceinline__ const float* tile_row(const float* base, int r, unsigned pitch_bytes) {
+    unsigned long long out;
+    asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(out) : "r"(r), "r"(pitch_bytes), "l"(base));
+    return reinterpret_cast<const float*>(out);
+}
+__device__ __forceinline__ float* tile_row(float* base, int r, unsigned pitch_bytes) {
+    unsigned long long out;
+    asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(out) : "r"(r), "r"(pitch_bytes), "l"(base));
+    return reinterpret_cast<float*>(out);
+}
+
+// ---------------------------------------------------------------------------------------------
+// The V batch entries a lane holds of one tile row.
+template <int V> struct Lane;
+template <> struct Lane<4> { float4 a; };
+template <> struct Lane<8> { float4 a, b; };
+
+__device__ __forceinline__ void lane_fill(Lane<4>& v, float s) { v.a = make_float4(s, s, s, s); }
+__device__ __forceinline__ void lane_fill(Lane<8>& v, float s) { v.a = make_float4(s, s, s, s); v.b = v.a; }
+
+__device__ __forceinline__ void lane_load(Lane<4>& v, const float* p) { v.a = ld_f4(p); }
+__device__ __forceinline__ void lane_load(Lane<8>& v, const float* p) {      // one 256-bit load (p 32-byte aligned)
+    asm volatile("ld.global.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(v.a.x), "=f"(v.a.y), "=f"(v.a.z), "=f"(v.a.w), "=f"(v.b.x), "=f"(v.b.y), "=f"(v.b.z), "=f"(v.b.w) : "l"(p) : "memory");
+}
+__device__ __forceinline__ void lane_gather(Lane<4>& v, const float* p) { v.a = gather_f4(p); }
+__device__ __forceinline__ void lane_gather(Lane<8>& v, const float* p) {    // read-only path, one 256-bit load
+    asm volatile("ld.global.nc.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(v.a.x), "=f"(v.a.y), "=f"(v.a.z), "=f"(v.a.w), "=f"(v.b.x), "=f"(v.b.y), "=f"(v.b.z), "=f"(v.b.w) : "l"(p));
+}
+__device__ __forceinline__ void lane_store(float* p, const Lane<4>& v) { st_f4(p, v.a); }
+__device__ __forceinline__ void lane_store(float* p, const Lane<8>& v) {
+    asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 :: "l"(p), "f"(v.a.x), "f"(v.a.y), "f"(v.a.z), "f"(v.a.w), "f"(v.b.x), "f"(v.b.y), "f"(v.b.z), "f"(v.b.w) : "memory");
+}
+
+#define SDNN_F4_FMA(W, X, A) A.x = fmaf(W, X.x, A.x); A.y = fmaf(W, X.y, A.y); A.z = fmaf(W, X.z, A.z); A.w = fmaf(W, X.w, A.w);
+__device__ __forceinline__ void lane_fma(float w, const Lane<4>& x, Lane<4>& acc) { SDNN_F4_FMA(w, x.a, acc.a) }
+__device__ __forceinline__ void lane_fma(float w, const Lane<8>& x, Lane<8>& acc) { SDNN_F4_FMA(w, x.a, acc.a) SDNN_F4_FMA(w, x.b, acc.b) }
+
+// Partial dot product of one lane: its batch columns of delta (d) against those of x.  Written with explicit
+// roundings and a fixed order so that the row pass and the column pass, which swap the roles of the gathered
+// and the resident operand, produce the same bits (a*b and fma(a,b,c) are symmetric in a and b).
+__device__ __forceinline__ float dot_f4(const float4& d, const float4& x, float s) {
+    return __fmaf_rn(d.w, x.w, __fmaf_rn(d.z, x.z, __fmaf_rn(d.y, x.y, __fmaf_rn(d.x, x.x, s))));
+}
+__device__ __forceinline__ float lane_dot(const Lane<4>& d, const Lane<4>& x) {
+    return __fmaf_rn(d.a.w, x.a.w, __fmaf_rn(d.a.z, x.a.z, __fmaf_rn(d.a.y, x.a.y, __fmul_rn(d.a.x, x.a.x))));
+}
+__device__ __forceinline__ float lane_dot(const Lane<8>& d, const Lane<8>& x) {
+    const float s = __fmaf_rn(d.a.w, x.a.w, __fmaf_rn(d.a.z, x.a.z, __fmaf_rn(d.a.y, x.a.y, __fmul_rn(d.a.x, x.a.x))));
+    return dot_f4(d.b, x.b, s);
+}
+
+__device__ __forceinline__ void f4_mask(float4& d, const float4& x, float c) {
+    d.x *= dmask(x.x, c); d.y *= dmask(x.y, c); d.z *= dmask(x.z, c); d.w *= dmask(x.w, c);
+}
+__device__ __forceinline__ void lane_mask(Lane<4>& d, const Lane<4>& x, float c) { f4_mask(d.a, x.a, c); }
+__device__ __forceinline__ void lane_mask(Lane<8>& d, const Lane<8>& x, float c) { f4_mask(d.a, x.a, c); f4_mask(d.b, x.b, c); }
+
+__device__ __forceinline__ void f4_clamp(float4& v, float c) { v.x = clampf(v.x, c); v.y = clampf(v.y, c); v.z = clampf(v.z, c); v.w = clampf(v.w, c); }
+__device__ __forceinline__ void lane_clamp(Lane<4>& v, float c) { f4_clamp(v.a, c); }
+__device__ __forceinline__ void lane_clamp(Lane<8>& v, float c) { f4_clamp(v.a, c); f4_clamp(v.b, c); }
+
+__device__ __forceinline__ float lane_sum(const Lane<4>& v) { return v.a.x + v.a.y + v.a.z + v.a.w; }
+__device__ __forceinline__ float lane_sum(const Lane<8>& v) { return (v.a.x + v.a.y + v.a.z + v.a.w) + (v.b.x + v.b.y + v.b.z + v.b.w); }
+
+__device__ __forceinline__ bool f4_any(const float4& v) { return !(v.x == 0.0f && v.y == 0.0f && v.z == 0.0f && v.w == 0.0f); }
+__device__ __forceinline__ bool lane_any(const Lane<4>& v) { return f4_any(v.a); }
+__device__ __forceinline__ bool lane_any(const Lane<8>& v) { return f4_any(v.a) || f4_any(v.b); }
+
+// S[row,:] += w * d[:] with 128-bit vector reductions
+__device__ __forceinline__ void lane_red_add(float* p, float w, const Lane<4>& d) {
+    red_add_f4(p, make_float4(w * d.a.x, w * d.a.y, w * d.a.z, w * d.a.w));
+}
+__device__ __forceinline__ void lane_red_add(float* p, float w, const Lane<8>& d) {
+    red_add_f4(p, make_float4(w * d.a.x, w * d.a.y, w * d.a.z, w * d.a.w));
+    red_add_f4(p + 4, make_float4(w * d.b.x, w * d.b.y, w * d.b.z, w * d.b.w));
+}
+
 template <int G>
 __device__ __forceinline__ unsigned group_mask(int grp) {
     return (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << (grp * G));
 }
 
-// sum over the G lanes of a row group; `gmask` names exactly those lanes, so that groups of one warp
-// whose rows have different lengths may sit in different loop iterations
+// sum over the G lanes of a row group; `gmask` names exactly those lanes
 template <int G>
 __device__ __forceinline__ float group_sum(float v, unsigned gmask) {
 #pragma unroll
     for (int o = G / 2; o > 0; o >>= 1) v += __shfl_xor_sync(gmask, v, o);
     return v;
-}
-
-// Partial dot product of one lane: its four batch columns of delta (d) against those of x.  Written with
-// explicit roundings so that the row pass and the column pass, which swap the roles of the gathered and
-// the resident operand, produce the same bits (a*b and fma(a,b,c) are symmetric in a and b).
-__device__ __forceinline__ float dot4(const float4& d, const float4& x) {
-    return __fmaf_rn(d.w, x.w, __fmaf_rn(d.z, x.z, __fmaf_rn(d.y, x.y, __fmul_rn(d.x, x.x))));
 }
 
 // The G lanes of a group hold partial sums p0..p3 for the four entries of a chunk.  On return
@@ -241,66 +318,59 @@ forward_csr_kernel(const int* __restrict__ row_ptr, const int* __restrict__ col,
 }
 
 // ---------------------------------------------------------------------------------------------
-// Helpers of the layer kernels' software pipeline.  A step handles two chunks (8 entries) of a row, all of
-// whose gathers are in flight together; slices are padded to a multiple of 8 entries per row, so a step never
-// needs a guard.  All the rows of a slice run through the slice's padded width (padding has index 0 and value
-// 0), which keeps the lanes of a warp converged.  The indices of a step are loaded one step ahead (while the
-// previous step's gathers are in flight, also across the boundary between two units), so that a step costs
-// one memory round trip, not two dependent ones.
-__device__ __forceinline__ void load_idx2(int4& c0, int4& c1, const int* p) {
-    c0 = __ldcs(reinterpret_cast<const int4*>(p));
-    c1 = __ldcs(reinterpret_cast<const int4*>(p + 32));
+// Helpers of the layer kernels' software pipeline.  A step handles CPS chunks (4*CPS entries) of a row, all of
+// whose gathers are in flight together; slices are padded to a multiple of 8 entries per row, so a step of
+// one or two chunks never needs a guard.  All the rows of a slice run through the slice's padded width
+// (padding has index 0 and value 0), which keeps the lanes of a warp converged.  The indices of a step are
+// loaded one step ahead (while the previous step's gathers are in flight, also across the boundary between
+// two units), so that a step costs one memory round trip, not two dependent ones.
+template <int CPS>
+__device__ __forceinline__ void load_idx(int4 (&c)[CPS], const int* p) {
+#pragma unroll
+    for (int i = 0; i < CPS; ++i) c[i] = __ldcs(reinterpret_cast<const int4*>(p + CHUNK_ROW * i));
 }
 
 // asks for the slices that hold the rows of unit `u` (rpw consecutive rows) to be brought into L2
 __device__ __forceinline__ void prefetch_unit(const Sliced& m, int u, int rpw, int n, int units_per_slice) {
     const int r0 = u * rpw;
-    if (units_per_slice > 1 && (r0 & 7) != 0) return;      // units narrower than a slice: the first one asks for the whole slice
-    const int s0 = r0 >> 3, s1 = min((n + 7) >> 3, ((r0 + rpw - 1) >> 3) + 1);
+    if (units_per_slice > 1 && (r0 & (SLICE - 1)) != 0) return;      // units narrower than a slice: the first one asks for the whole slice
+    const int s0 = r0 / SLICE, s1 = min((n + SLICE - 1) / SLICE, (r0 + rpw - 1) / SLICE + 1);
     const int lo = m.slice_off[s0], hi = m.slice_off[s1];
     if (hi > lo) { prefetch_l2(m.idx + lo, (unsigned)(hi - lo) * 4u); prefetch_l2(m.val + lo, (unsigned)(hi - lo) * 4u); }
 }
 
-// address of tile row `r` (an index below 2^32 / pitch): one 32 x 32 -> 64 bit multiply-add, no 64-bit multiply
-__device__ __forceinline__ const float* tile_row(const float* base, int r, unsigned pitch_bytes) {
-    return reinterpret_cast<const float*>(reinterpret_cast<const char*>(base) + (unsigned long long)(unsigned)r * (unsigned long long)pitch_bytes);
-}
-__device__ __forceinline__ float* tile_row(float* base, int r, unsigned pitch_bytes) {
-    return reinterpret_cast<float*>(reinterpret_cast<char*>(base) + (unsigned long long)(unsigned)r * (unsigned long long)pitch_bytes);
-}
-
-#define SDNN_GATHER4(X, I, C, P, PITCH)                                                                 \
-    X[4 * (I) + 0] = gather_f4(tile_row(P, C.x, PITCH)); X[4 * (I) + 1] = gather_f4(tile_row(P, C.y, PITCH)); \
-    X[4 * (I) + 2] = gather_f4(tile_row(P, C.z, PITCH)); X[4 * (I) + 3] = gather_f4(tile_row(P, C.w, PITCH));
+#define SDNN_GATHER_CHUNK(X, I, C, P, PITCH)                                                              \
+    lane_gather(X[4 * (I) + 0], tile_row(P, C.x, PITCH)); lane_gather(X[4 * (I) + 1], tile_row(P, C.y, PITCH)); \
+    lane_gather(X[4 * (I) + 2], tile_row(P, C.z, PITCH)); lane_gather(X[4 * (I) + 3], tile_row(P, C.w, PITCH));
 
 // Position of a group's item (matrix row, or position in the transposed copy) in unit U of matrix M: BASE =
 // element offset of its first chunk, NCH = chunks of its slice (even), ITEM = n for groups beyond the matrix
 // (they run through the padding rows of the last slice like everyone else and store nothing).
 #define SDNN_UNIT_SHAPE(M, U, NUNITS, ITEM, BASE, NCH)                                        \
     ITEM = (U) * RPW + grp; BASE = 0; NCH = 0;                                                \
-    if ((U) < (NUNITS) && (ITEM >> 3) < ((n + 7) >> 3)) {                                     \
-        const int so_ = M.slice_off[ITEM >> 3];                                               \
-        BASE = so_ + (ITEM & 7) * 4; NCH = (M.slice_off[(ITEM >> 3) + 1] - so_) >> 5;         \
+    if ((U) < (NUNITS) && (ITEM / SLICE) < ((n + SLICE - 1) / SLICE)) {                       \
+        const int so_ = M.slice_off[ITEM / SLICE];                                            \
+        BASE = so_ + (ITEM % SLICE) * 4; NCH = (M.slice_off[ITEM / SLICE + 1] - so_) / CHUNK_ROW; \
     }                                                                                         \
     if (ITEM >= n) ITEM = n;
 
 // ---------------------------------------------------------------------------------------------
 // Forward layer (feedforward equation): Xout[i,:] = clamp(bias[i] + sum_q val[i,q] * Xin[idx[i,q],:]).
 // Persistent grid: a warp takes units (32/G consecutive rows) in a grid-stride loop.  One group of G lanes
-// per row; each lane accumulates 4 batch entries with fp32 FMAs in stored (ascending column) order.
+// per row; each lane accumulates V batch entries with fp32 FMAs in stored (ascending column) order.
 // While it works on a unit a warp asks for the entries of its next unit to be brought into L2.
-template <int G>
-__global__ void __launch_bounds__(256, 3)
+template <int G, int V, int CPS>
+__global__ void __launch_bounds__(256, 2)
 forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict__ xin, float* __restrict__ xout,
                int n, int ld, float clamp, int pdl) {
     constexpr int RPW = 32 / G;
-    constexpr int UPS = (RPW >= 8) ? 1 : 8 / RPW;      // units per slice
+    constexpr int UPS = (RPW >= SLICE) ? 1 : SLICE / RPW;      // units per slice
     const int lane = threadIdx.x & 31;
     const int sub = lane % G, grp = lane / G;
     const int wpb = blockDim.x >> 5;
     const int nunits = (n + RPW - 1) / RPW;
     const int stride = gridDim.x * wpb;
-    const int boff = blockIdx.y * (4 * G) + sub * 4;
+    const int boff = blockIdx.y * (V * G) + sub * V;
     const float* xg = xin + boff;
     const unsigned pitch = (unsigned)ld * 4u;
     const int* __restrict__ idx = m.idx;
@@ -312,8 +382,10 @@ forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict
     SDNN_UNIT_SHAPE(m, unit, nunits, row, base, nch)
     float b = (row < n) ? bias[row] : 0.0f;
     if (unit < nunits && lane == 0) prefetch_unit(m, unit, RPW, n, UPS);
-    int4 c0 = make_int4(0, 0, 0, 0), c1 = c0;
-    if (nch > 0) load_idx2(c0, c1, idx + base);
+    int4 c[CPS];
+#pragma unroll
+    for (int i = 0; i < CPS; ++i) c[i] = make_int4(0, 0, 0, 0);
+    if (nch > 0) load_idx<CPS>(c, idx + base);
     if (pdl) grid_dependency_wait();
 
     while (unit < nunits) {
@@ -324,25 +396,29 @@ forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict
         const float nb = (nrow < n) ? bias[nrow] : 0.0f;
         if (nunit < nunits && lane == 0) prefetch_unit(m, nunit, RPW, n, UPS);
 
-        float4 acc = make_float4(b, b, b, b);
+        Lane<V> acc;
+        lane_fill(acc, b);
         const int* cp = idx + base;
         const float* vp = val + base;
-        for (int t = 0; t < nch; t += 2) {
-            float4 x[8];
-            const float4 w0 = __ldcs(reinterpret_cast<const float4*>(vp + t * 32));
-            const float4 w1 = __ldcs(reinterpret_cast<const float4*>(vp + t * 32 + 32));
-            SDNN_GATHER4(x, 0, c0, xg, pitch)
-            SDNN_GATHER4(x, 1, c1, xg, pitch)
-            if (t + 2 < nch) load_idx2(c0, c1, cp + (t + 2) * 32);
-            else if (nnch > 0) load_idx2(c0, c1, idx + nbase);
-            SDNN_FMA4(w0.x, x[0]) SDNN_FMA4(w0.y, x[1]) SDNN_FMA4(w0.z, x[2]) SDNN_FMA4(w0.w, x[3])
-            SDNN_FMA4(w1.x, x[4]) SDNN_FMA4(w1.y, x[5]) SDNN_FMA4(w1.z, x[6]) SDNN_FMA4(w1.w, x[7])
+        for (int t = 0; t < nch; t += CPS) {
+            float4 w[CPS];
+            Lane<V> x[4 * CPS];
+#pragma unroll
+            for (int i = 0; i < CPS; ++i) w[i] = __ldcs(reinterpret_cast<const float4*>(vp + (t + i) * CHUNK_ROW));
+#pragma unroll
+            for (int i = 0; i < CPS; ++i) { SDNN_GATHER_CHUNK(x, i, c[i], xg, pitch) }
+            if (t + CPS < nch) load_idx<CPS>(c, cp + (t + CPS) * CHUNK_ROW);
+            else if (nnch > 0) load_idx<CPS>(c, idx + nbase);
+#pragma unroll
+            for (int i = 0; i < CPS; ++i) {
+                lane_fma(w[i].x, x[4 * i + 0], acc); lane_fma(w[i].y, x[4 * i + 1], acc);
+                lane_fma(w[i].z, x[4 * i + 2], acc); lane_fma(w[i].w, x[4 * i + 3], acc);
+            }
         }
-        if (nch == 0 && nnch > 0) load_idx2(c0, c1, idx + nbase);      // empty slice: nothing prefetched across the boundary yet
+        if (nch == 0 && nnch > 0) load_idx<CPS>(c, idx + nbase);      // empty slice: nothing prefetched across the boundary yet
         if (row < n) {
-            acc.x = clampf(acc.x, clamp); acc.y = clampf(acc.y, clamp);
-            acc.z = clampf(acc.z, clamp); acc.w = clampf(acc.w, clamp);
-            st_f4(tile_row(xout + boff, row, pitch), acc);
+            lane_clamp(acc, clamp);
+            lane_store(tile_row(xout + boff, row, pitch), acc);
         }
         unit = nunit; row = nrow; base = nbase; nch = nnch; b = nb;
     }
@@ -387,8 +463,8 @@ output_gradient_kernel(const float* __restrict__ xl, const float* __restrict__ y
 // Row units (always): for row i of W^k with delta^k[i,:] in registers, for each stored (i,j):
 //       g = sum_b delta^k[i,b] x^{k-1}[j,b]      (masked gradient times B; x^{k-1}[j,:] gathered)
 //       W(i,j) = w - (eta/B) g
-//   SCATTER (atomics realisation) additionally S_{k-1}[j,:] += w * delta^k[i,:] with one 128-bit vector
-//   reduction per lane, w being the value BEFORE the update; there delta^k[i,:] = S_k[i,:] (.) f'(x^k[i,:])
+//   SCATTER (atomics realisation) additionally S_{k-1}[j,:] += w * delta^k[i,:] with 128-bit vector
+//   reductions, w being the value BEFORE the update; there delta^k[i,:] = S_k[i,:] (.) f'(x^k[i,:])
 //   is formed on the fly and S_k is cleared row by row as it is consumed (FROM_S).
 //
 // Column units (transposed realisation, MIRROR): for column j of W^k (a row of the transposed copy,
@@ -398,8 +474,8 @@ output_gradient_kernel(const float* __restrict__ xl, const float* __restrict__ y
 //       delta^{k-1}[j,:] = acc (.) f'(x^{k-1}[j,:])
 //   No atomics; one gather per stored entry serves both the product and the gradient.
 //
-// A launch processes the column units (if any) first, then the row units; both only read delta^k and
-// x^{k-1}, so they are independent of each other.  The whole minibatch sits in one chunk (ld = 4G <= 128).
+// A warp processes its column units (if any) first, then its row units; both only read delta^k and
+// x^{k-1}, so they are independent of each other.  The whole minibatch sits in one chunk (ld = V*G <= 128).
 // Same software pipeline as the forward kernel; in addition the resident operand of a unit (delta^k row or
 // x^{k-1} row) is loaded during the last step of the unit before it.
 struct BackwardArgs {
@@ -415,23 +491,24 @@ struct BackwardArgs {
     const StepParams* sp;
     int n;
     float clamp;
-    int update_bias, skip_dead, col_units, pdl;
+    int update_bias, skip_dead, pdl;
+    const float* warm;        // tile the NEXT backward launch will gather from (x^{k-2}), or NULL: asked into L2 now,
+    unsigned warm_bytes;      // because it was written a whole forward pass ago and has left the cache
 };
 
-// Column units of the transposed realisation (see backward_kernel).
-template <int G>
+// Column units of the transposed realisation.
+template <int G, int V, int CPS>
 __device__ __forceinline__ void backward_col_units(const Sliced m, const float* __restrict__ xprev, const float* __restrict__ dk,
                                                    float* __restrict__ dprev, int n, float clamp, float step, float inv_b,
                                                    int first, int stride) {
     constexpr int RPW = 32 / G;
-    constexpr int UPS = (RPW >= 8) ? 1 : 8 / RPW;
-    constexpr unsigned pitch = 16u * G;
+    constexpr int UPS = (RPW >= SLICE) ? 1 : SLICE / RPW;
+    constexpr unsigned pitch = 4u * V * G;
     const int lane = threadIdx.x & 31;
     const int sub = lane % G, grp = lane / G;
-    const unsigned gmask = (G >= 4) ? 0xffffffffu : group_mask<G>(grp);     // G >= 4: the warp's lanes stay converged
+    const unsigned gmask = (G >= 2) ? 0xffffffffu : group_mask<G>(grp);     // G >= 2: one slice per warp, its lanes stay converged
     const int nunits = (n + RPW - 1) / RPW;
-    const int boff = sub * 4;
-    const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int boff = sub * V;
     const int* __restrict__ idx = m.idx;
     float* val = m.val;
     const float* dg = dk + boff;
@@ -441,9 +518,13 @@ __device__ __forceinline__ void backward_col_units(const Sliced m, const float* 
     if (u < nunits && lane == 0) prefetch_unit(m, u, RPW, n, UPS);
     int len = 0, j = 0;
     if (item < n) { len = m.len[item]; j = m.order[item]; }
-    int4 c0 = make_int4(0, 0, 0, 0), c1 = c0;
-    if (nch > 0) load_idx2(c0, c1, idx + base);
-    float4 xj = (item < n) ? ld_f4(tile_row(xprev + boff, j, pitch)) : zero4;
+    int4 c[CPS];
+#pragma unroll
+    for (int i = 0; i < CPS; ++i) c[i] = make_int4(0, 0, 0, 0);
+    if (nch > 0) load_idx<CPS>(c, idx + base);
+    Lane<V> xj;
+    lane_fill(xj, 0.0f);
+    if (item < n) lane_load(xj, tile_row(xprev + boff, j, pitch));
 
     while (u < nunits) {
         const int nu = u + stride;
@@ -451,56 +532,56 @@ __device__ __forceinline__ void backward_col_units(const Sliced m, const float* 
         SDNN_UNIT_SHAPE(m, nu, nunits, nitem, nbase, nnch)
         if (nitem < n) { nlen = m.len[nitem]; nj = m.order[nitem]; }
         if (nu < nunits && lane == 0) prefetch_unit(m, nu, RPW, n, UPS);
-        float4 nxj = zero4;
-        float4 acc = zero4;
+        Lane<V> nxj, acc;
+        lane_fill(nxj, 0.0f);
+        lane_fill(acc, 0.0f);
         const int* ip = idx + base;
         float* vp = val + base;
         const int lim = len - ((G >= 4) ? (sub & 3) : (G == 2) ? 2 * sub : 0);
-#define SDNN_COL_NEXT if (nnch > 0) load_idx2(c0, c1, idx + nbase); if (nitem < n) nxj = ld_f4(tile_row(xprev + boff, nj, pitch));
-#define SDNN_ACC4(W, D) acc.x = fmaf(W, D.x, acc.x); acc.y = fmaf(W, D.y, acc.y); acc.z = fmaf(W, D.z, acc.z); acc.w = fmaf(W, D.w, acc.w);
-#define SDNN_COL_CHUNK(W, D0, D1, D2, D3, T)                                                                    \
-        {                                                                                                           \
-            SDNN_ACC4(W.x, D0) SDNN_ACC4(W.y, D1) SDNN_ACC4(W.z, D2) SDNN_ACC4(W.w, D3)                             \
-            float p0 = dot4(D0, xj), p1 = dot4(D1, xj), p2 = dot4(D2, xj), p3 = dot4(D3, xj);                       \
-            chunk_sums<G>(p0, p1, p2, p3, sub, gmask);                                                              \
-            chunk_update<G, false>(vp + (T) * 32, nullptr, W, p0, p1, p2, p3, sub, (T) * 4, lim, step, inv_b);       \
-        }
-        for (int t = 0; t < nch; t += 2) {
-            float4 d[8];
-            const float4 w0 = ld_f4(vp + t * 32), w1 = ld_f4(vp + t * 32 + 32);
-            SDNN_GATHER4(d, 0, c0, dg, pitch)
-            SDNN_GATHER4(d, 1, c1, dg, pitch)
-            if (t + 2 < nch) { load_idx2(c0, c1, ip + (t + 2) * 32); }
+#define SDNN_COL_NEXT if (nnch > 0) load_idx<CPS>(c, idx + nbase); if (nitem < n) lane_load(nxj, tile_row(xprev + boff, nj, pitch));
+        for (int t = 0; t < nch; t += CPS) {
+            float4 w[CPS];
+            Lane<V> d[4 * CPS];
+#pragma unroll
+            for (int i = 0; i < CPS; ++i) w[i] = ld_f4(vp + (t + i) * CHUNK_ROW);
+#pragma unroll
+            for (int i = 0; i < CPS; ++i) { SDNN_GATHER_CHUNK(d, i, c[i], dg, pitch) }
+            if (t + CPS < nch) { load_idx<CPS>(c, ip + (t + CPS) * CHUNK_ROW); }
             else { SDNN_COL_NEXT }
-            SDNN_COL_CHUNK(w0, d[0], d[1], d[2], d[3], t)
-            SDNN_COL_CHUNK(w1, d[4], d[5], d[6], d[7], t + 1)
+#pragma unroll
+            for (int i = 0; i < CPS; ++i) {
+                lane_fma(w[i].x, d[4 * i + 0], acc); lane_fma(w[i].y, d[4 * i + 1], acc);
+                lane_fma(w[i].z, d[4 * i + 2], acc); lane_fma(w[i].w, d[4 * i + 3], acc);
+                float p0 = lane_dot(d[4 * i + 0], xj), p1 = lane_dot(d[4 * i + 1], xj), p2 = lane_dot(d[4 * i + 2], xj), p3 = lane_dot(d[4 * i + 3], xj);
+                chunk_sums<G>(p0, p1, p2, p3, sub, gmask);
+                chunk_update<G, false>(vp + (t + i) * CHUNK_ROW, nullptr, w[i], p0, p1, p2, p3, sub, (t + i) * 4, lim, step, inv_b);
+            }
         }
         if (nch == 0) { SDNN_COL_NEXT }
 #undef SDNN_COL_NEXT
-#undef SDNN_COL_CHUNK
-        if (item < n)
-            st_f4(tile_row(dprev + boff, j, pitch),
-                  make_float4(acc.x * dmask(xj.x, clamp), acc.y * dmask(xj.y, clamp), acc.z * dmask(xj.z, clamp), acc.w * dmask(xj.w, clamp)));
+        if (item < n) {
+            lane_mask(acc, xj, clamp);
+            lane_store(tile_row(dprev + boff, j, pitch), acc);
+        }
         u = nu; item = nitem; base = nbase; nch = nnch; len = nlen; j = nj; xj = nxj;
     }
 }
 
-// Row units (see backward_kernel).
-template <int G, bool FROM_S, bool SCATTER, bool DBG>
+// Row units.
+template <int G, int V, int CPS, bool FROM_S, bool SCATTER, bool DBG>
 __device__ __forceinline__ void backward_row_units(const Sliced m, float* __restrict__ bias, const float* __restrict__ xk,
                                                    const float* __restrict__ xprev, float* dk, float* dprev,
                                                    float* __restrict__ dbg_delta, float* __restrict__ dbg_grad, int n, float clamp,
                                                    float step, float inv_b, int update_bias, int skip_dead, int first, int stride) {
     constexpr int RPW = 32 / G;
-    constexpr int UPS = (RPW >= 8) ? 1 : 8 / RPW;
-    constexpr unsigned pitch = 16u * G;
+    constexpr int UPS = (RPW >= SLICE) ? 1 : SLICE / RPW;
+    constexpr unsigned pitch = 4u * V * G;
     const int lane = threadIdx.x & 31;
     const int sub = lane % G, grp = lane / G;
     const unsigned gmask1 = group_mask<G>(grp);
-    const unsigned gmask = (G >= 4) ? 0xffffffffu : gmask1;
+    const unsigned gmask = (G >= 2) ? 0xffffffffu : gmask1;
     const int nunits = (n + RPW - 1) / RPW;
-    const int boff = sub * 4;
-    const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int boff = sub * V;
     const int* __restrict__ idx = m.idx;
     float* val = m.val;
     const float* xg = xprev + boff;
@@ -510,10 +591,13 @@ __device__ __forceinline__ void backward_row_units(const Sliced m, float* __rest
     SDNN_UNIT_SHAPE(m, u, nunits, item, base, nch)
     if (u < nunits && lane == 0) prefetch_unit(m, u, RPW, n, UPS);
     int len = (item < n) ? m.len[item] : 0;
-    int4 c0 = make_int4(0, 0, 0, 0), c1 = c0;
-    if (nch > 0) load_idx2(c0, c1, idx + base);
-    float4 h0 = zero4, h1 = zero4;       // delta^k[i,:] (or S_k[i,:]) and, FROM_S, x^k[i,:]
-    if (item < n) { h0 = ld_f4(tile_row(dk + boff, item, pitch)); if (FROM_S) h1 = ld_f4(tile_row(xk + boff, item, pitch)); }
+    int4 c[CPS];
+#pragma unroll
+    for (int i = 0; i < CPS; ++i) c[i] = make_int4(0, 0, 0, 0);
+    if (nch > 0) load_idx<CPS>(c, idx + base);
+    Lane<V> h0, h1;       // delta^k[i,:] (or S_k[i,:]) and, FROM_S, x^k[i,:]
+    lane_fill(h0, 0.0f); lane_fill(h1, 0.0f);
+    if (item < n) { lane_load(h0, tile_row(dk + boff, item, pitch)); if (FROM_S) lane_load(h1, tile_row(xk + boff, item, pitch)); }
 
     while (u < nunits) {
         const int nu = u + stride;
@@ -521,99 +605,109 @@ __device__ __forceinline__ void backward_row_units(const Sliced m, float* __rest
         SDNN_UNIT_SHAPE(m, nu, nunits, nitem, nbase, nnch)
         const int nlen = (nitem < n) ? m.len[nitem] : 0;
         if (nu < nunits && lane == 0) prefetch_unit(m, nu, RPW, n, UPS);
-        float4 nh0 = zero4, nh1 = zero4;
-        float4 d = h0;
+        Lane<V> nh0, nh1;
+        lane_fill(nh0, 0.0f); lane_fill(nh1, 0.0f);
+        Lane<V> d = h0;
         if (item < n) {
-            float* o = tile_row(dk + boff, item, pitch);
             if (FROM_S) {
-                st_f4(o, zero4);
-                d.x *= dmask(h1.x, clamp); d.y *= dmask(h1.y, clamp);
-                d.z *= dmask(h1.z, clamp); d.w *= dmask(h1.w, clamp);
-                if (DBG) st_f4(tile_row(dbg_delta + boff, item, pitch), d);
+                Lane<V> z;
+                lane_fill(z, 0.0f);
+                lane_store(tile_row(dk + boff, item, pitch), z);
+                lane_mask(d, h1, clamp);
+                if (DBG) lane_store(tile_row(dbg_delta + boff, item, pitch), d);
             }
             if (update_bias) {       // bias read as one more column of W^k whose input is the constant 1
-                const float bg = group_sum<G>(d.x + d.y + d.z + d.w, gmask1);
+                const float bg = group_sum<G>(lane_sum(d), gmask1);
                 if (sub == 0) bias[item] -= step * bg;
             }
         }
         if (skip_dead) {             // delta^k(i) = 0 for every input of every row of the unit: nothing changes
-            const bool alive = !(d.x == 0.0f && d.y == 0.0f && d.z == 0.0f && d.w == 0.0f);
-            if (__ballot_sync(gmask, alive) == 0u) nch = 0;
+            if (__ballot_sync(gmask, lane_any(d)) == 0u) nch = 0;
         }
         const int* cp = idx + base;
         float* vp = val + base;
         float* gp = DBG ? dbg_grad + base : nullptr;
         const int lim = len - ((G >= 4) ? (sub & 3) : (G == 2) ? 2 * sub : 0);
 #define SDNN_ROW_NEXT                                                                                    \
-        if (nnch > 0) load_idx2(c0, c1, idx + nbase);                                                    \
-        if (nitem < n) { nh0 = ld_f4(tile_row(dk + boff, nitem, pitch)); if (FROM_S) nh1 = ld_f4(tile_row(xk + boff, nitem, pitch)); }
-#define SDNN_SCAT(C, W, Q) if ((Q) < len) red_add_f4(tile_row(sg, C, pitch), make_float4(W * d.x, W * d.y, W * d.z, W * d.w));
-#define SDNN_ROW_CHUNK(W, X0, X1, X2, X3, T)                                                                \
-        {                                                                                                       \
-            float p0 = dot4(d, X0), p1 = dot4(d, X1), p2 = dot4(d, X2), p3 = dot4(d, X3);                       \
-            chunk_sums<G>(p0, p1, p2, p3, sub, gmask);                                                          \
-            chunk_update<G, DBG>(vp + (T) * 32, DBG ? gp + (T) * 32 : nullptr, W, p0, p1, p2, p3, sub, (T) * 4, lim, step, inv_b); \
-        }
-        for (int t = 0; t < nch; t += 2) {
-            float4 x[8];
-            const float4 w0 = ld_f4(vp + t * 32), w1 = ld_f4(vp + t * 32 + 32);
-            SDNN_GATHER4(x, 0, c0, xg, pitch)
-            SDNN_GATHER4(x, 1, c1, xg, pitch)
+        if (nnch > 0) load_idx<CPS>(c, idx + nbase);                                                     \
+        if (nitem < n) { lane_load(nh0, tile_row(dk + boff, nitem, pitch)); if (FROM_S) lane_load(nh1, tile_row(xk + boff, nitem, pitch)); }
+#define SDNN_SCAT(C, W, Q) if ((Q) < len) lane_red_add(tile_row(sg, C, pitch), W, d);
+        for (int t = 0; t < nch; t += CPS) {
+            float4 w[CPS];
+            Lane<V> x[4 * CPS];
+#pragma unroll
+            for (int i = 0; i < CPS; ++i) w[i] = ld_f4(vp + (t + i) * CHUNK_ROW);
+#pragma unroll
+            for (int i = 0; i < CPS; ++i) { SDNN_GATHER_CHUNK(x, i, c[i], xg, pitch) }
             if (SCATTER) {       // stored entries only: padding must not touch S
-                const int q = 4 * t;
-                SDNN_SCAT(c0.x, w0.x, q) SDNN_SCAT(c0.y, w0.y, q + 1) SDNN_SCAT(c0.z, w0.z, q + 2) SDNN_SCAT(c0.w, w0.w, q + 3)
-                SDNN_SCAT(c1.x, w1.x, q + 4) SDNN_SCAT(c1.y, w1.y, q + 5) SDNN_SCAT(c1.z, w1.z, q + 6) SDNN_SCAT(c1.w, w1.w, q + 7)
+#pragma unroll
+                for (int i = 0; i < CPS; ++i) {
+                    const int q = 4 * (t + i);
+                    SDNN_SCAT(c[i].x, w[i].x, q) SDNN_SCAT(c[i].y, w[i].y, q + 1) SDNN_SCAT(c[i].z, w[i].z, q + 2) SDNN_SCAT(c[i].w, w[i].w, q + 3)
+                }
             }
-            if (t + 2 < nch) { load_idx2(c0, c1, cp + (t + 2) * 32); }
+            if (t + CPS < nch) { load_idx<CPS>(c, cp + (t + CPS) * CHUNK_ROW); }
             else { SDNN_ROW_NEXT }
-            SDNN_ROW_CHUNK(w0, x[0], x[1], x[2], x[3], t)
-            SDNN_ROW_CHUNK(w1, x[4], x[5], x[6], x[7], t + 1)
+#pragma unroll
+            for (int i = 0; i < CPS; ++i) {
+                float p0 = lane_dot(d, x[4 * i + 0]), p1 = lane_dot(d, x[4 * i + 1]), p2 = lane_dot(d, x[4 * i + 2]), p3 = lane_dot(d, x[4 * i + 3]);
+                chunk_sums<G>(p0, p1, p2, p3, sub, gmask);
+                chunk_update<G, DBG>(vp + (t + i) * CHUNK_ROW, DBG ? gp + (t + i) * CHUNK_ROW : nullptr, w[i], p0, p1, p2, p3, sub,
+                                     (t + i) * 4, lim, step, inv_b);
+            }
         }
         if (nch == 0) { SDNN_ROW_NEXT }
 #undef SDNN_ROW_NEXT
-#undef SDNN_ROW_CHUNK
+#undef SDNN_SCAT
         u = nu; item = nitem; base = nbase; nch = nnch; len = nlen; h0 = nh0; h1 = nh1;
     }
 }
 
-template <int G, bool FROM_S, bool SCATTER, bool MIRROR, bool DBG>
-__global__ void __launch_bounds__(256, 3)
+template <int G, int V, int CPS, bool FROM_S, bool SCATTER, bool MIRROR, bool DBG>
+__global__ void __launch_bounds__(256, 2)
 backward_kernel(const BackwardArgs a) {
     const int wpb = blockDim.x >> 5;
     const int stride = gridDim.x * wpb;
     const int first = blockIdx.x * wpb + (threadIdx.x >> 5);
+    if (a.warm && (threadIdx.x & 31) == 0) {      // each warp asks for its share, in pieces of 4 KB
+        const unsigned pieces = (a.warm_bytes + 4095u) >> 12;
+        for (unsigned q = first; q < pieces; q += stride) {
+            const unsigned lo = q << 12, len = min(4096u, a.warm_bytes - lo);
+            prefetch_l2(reinterpret_cast<const char*>(a.warm) + lo, len & ~15u);
+        }
+    }
     if (a.pdl) grid_dependency_wait();
     const float inv_b = a.sp->inv_b;
     const float step = a.sp->eta * inv_b;
-    if (MIRROR) backward_col_units<G>(a.cols, a.xprev, a.dk, a.dprev, a.n, a.clamp, step, inv_b, first, stride);
-    backward_row_units<G, FROM_S, SCATTER, DBG>(a.rows, a.bias, a.xk, a.xprev, a.dk, a.dprev, a.dbg_delta, a.dbg_grad, a.n, a.clamp,
-                                           step, inv_b, a.update_bias, a.skip_dead, first, stride);
+    if (MIRROR) backward_col_units<G, V, CPS>(a.cols, a.xprev, a.dk, a.dprev, a.n, a.clamp, step, inv_b, first, stride);
+    backward_row_units<G, V, CPS, FROM_S, SCATTER, DBG>(a.rows, a.bias, a.xk, a.xprev, a.dk, a.dprev, a.dbg_delta, a.dbg_grad, a.n,
+                                                        a.clamp, step, inv_b, a.update_bias, a.skip_dead, first, stride);
     if (a.pdl) grid_launch_dependents();
 }
 
 // ---------------------------------------------------------------------------------------------
 // Fills the transposed copy's values from the row-major copy: entry (column j, row i) of the transposed
-// copy is looked up by binary search in row i (ascending columns).  One thread per transposed entry slot.
+// copy is looked up by binary search in row i (ascending columns).  One warp per transposed unit.
 // With `mismatch` non-NULL nothing is written; entries whose bits differ from the row-major copy are counted.
 __global__ void mirror_values_kernel(Sliced rows, Sliced cols, int n, unsigned long long* mismatch) {
-    const int cc = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);      // one warp per transposed unit
+    const int cc = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (cc >= n) return;
     const int len = cols.len[cc];
     const int j = cols.order[cc];
-    const int base = cols.slice_off[cc >> 3] + (cc & 7) * 4;
+    const int base = cols.slice_off[cc / SLICE] + (cc % SLICE) * 4;
     for (int q = threadIdx.x & 31; q < len; q += 32) {
-        const int pos = base + (q >> 2) * 32 + (q & 3);
+        const int pos = base + (q >> 2) * CHUNK_ROW + (q & 3);
         const int i = cols.idx[pos];
-        const int rb = rows.slice_off[i >> 3] + (i & 7) * 4;
+        const int rb = rows.slice_off[i / SLICE] + (i % SLICE) * 4;
         int lo = 0, hi = rows.len[i] - 1, at = -1;
         while (lo <= hi) {
             const int mid = (lo + hi) >> 1;
-            const int c = rows.idx[rb + (mid >> 2) * 32 + (mid & 3)];
+            const int c = rows.idx[rb + (mid >> 2) * CHUNK_ROW + (mid & 3)];
             if (c == j) { at = mid; break; }
             if (c < j) lo = mid + 1; else hi = mid - 1;
         }
         if (at < 0) { if (mismatch) atomicAdd(mismatch, 1ull << 32); continue; }     // pattern error: high word
-        const float w = rows.val[rb + (at >> 2) * 32 + (at & 3)];
+        const float w = rows.val[rb + (at >> 2) * CHUNK_ROW + (at & 3)];
         if (mismatch) {
             if (__float_as_uint(w) != __float_as_uint(cols.val[pos])) atomicAdd(mismatch, 1ull);
         } else {

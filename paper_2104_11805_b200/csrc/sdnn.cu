@@ -45,7 +45,7 @@ struct LayerMem {
 }  // namespace
 
 struct sdnn {
-    int L = 0, N = 0, NS = 0;           // layers, neurons, slices of 8 rows
+    int L = 0, N = 0, NS = 0;           // layers, neurons, slices of SLICE rows
     sdnn_config cfg{};
     cudaStream_t stream = nullptr;
     bool own_stream = false;
@@ -53,8 +53,6 @@ struct sdnn {
     bool finalized = false, stepped = false;
     bool mirror = false;                // training with the transposed copy (no atomics)
     bool pdl = false;                   // programmatic dependent launch between the layer kernels
-    bool steps4 = false;                // TUNING: 4 chunks per pipeline step instead of 2
-    int tune_wps = 0;                   // TUNING: forced warps per SM
     std::vector<int64_t> nnz;
     std::vector<char> loaded;
     std::vector<LayerMem> lay;
@@ -142,17 +140,19 @@ int dev_alloc(sdnn* h, T** out, size_t count, bool zero) {
     return SDNN_OK;
 }
 
-// padded batch width: 4, 8, .., 128, then multiples of 128
+// padded batch width: 4, 8, .., 256, then multiples of 256
 int padded_width(int b) {
     if (b <= 4) return 4;
-    if (b <= 128) { int w = 4; while (w < b) w <<= 1; return w; }
-    return (b + 127) / 128 * 128;
+    if (b <= 256) { int w = 4; while (w < b) w <<= 1; return w; }
+    return (b + 255) / 256 * 256;
 }
 
-struct Geometry { int g; int chunks; };   // lanes per row group; 4g-wide chunks per tile row
+// lanes per row group (g), batch entries per lane (v), (g*v)-wide chunks per tile row
+struct Geometry { int g; int v; int chunks; };
 Geometry geometry(int cols) {
-    if (cols <= 128) return {cols / 4, 1};
-    return {32, cols / 128};
+    if (cols <= 4) return {1, 4, 1};
+    if (cols <= 256) return {cols / 8, 8, 1};
+    return {32, 8, cols / 256};
 }
 
 int validate_cfg(const sdnn_config* cfg) {
@@ -201,22 +201,22 @@ int validate_layer(sdnn* h, int layer, int n, int64_t expect_nnz, const int32_t*
 }
 
 // ---------------------------------------------------------------------------------------------
-// Sliced layout (see kernels.cuh): slices of 8 units, chunks of 4 entries interleaved over the 8 units.
+// Sliced layout (see kernels.cuh): slices of SLICE units, chunks of 4 entries interleaved over the units of a slice.
 inline int64_t sliced_pos(const int* slice_off, int unit, int q) {
-    return (int64_t)slice_off[unit >> 3] + (int64_t)(q >> 2) * 32 + (unit & 7) * 4 + (q & 3);
+    return (int64_t)slice_off[unit / SLICE] + (int64_t)(q >> 2) * CHUNK_ROW + (unit % SLICE) * 4 + (q & 3);
 }
 
 // slice offsets from unit lengths; returns the padded element count or -1 if it does not fit int32
 template <typename LenFn>
 int64_t build_slice_offsets(int n, LenFn len, std::vector<int>& off) {
-    const int ns = (n + 7) / 8;
+    const int ns = (n + SLICE - 1) / SLICE;
     off.assign(ns + 1, 0);
     int64_t run = 0;
     for (int s = 0; s < ns; ++s) {
         int w = 0;
-        for (int i = s * 8; i < std::min(n, s * 8 + 8); ++i) w = std::max(w, len(i));
+        for (int i = s * SLICE; i < std::min(n, (s + 1) * SLICE); ++i) w = std::max(w, len(i));
         w = (w + 7) / 8 * 8;      // whole pipeline steps of two chunks
-        run += 8LL * w;
+        run += (int64_t)SLICE * w;
         if (run > INT32_MAX) return -1;
         off[s + 1] = (int)run;
     }
@@ -251,7 +251,6 @@ std::pair<int, int> plan_grid(sdnn* h, const void* kernel, int units, int chunks
         for (int c = occ; c >= 1; --c) {
             const int per_sm_warps = c * wpb;
             if (per_sm_warps < 16 && c != occ) continue;
-            if (h->tune_wps && per_sm_warps != h->tune_wps) continue;
             int gx = std::max(1, h->sms * c / chunks);
             const int64_t warps = (int64_t)gx * wpb;
             if (warps >= units) {      // one round: a plain grid of ceil(units / wpb) CTAs does it
@@ -300,24 +299,26 @@ cudaError_t launch_k(sdnn* h, void (*kernel)(KArgs...), dim3 grid, dim3 block, b
     return cudaLaunchKernelEx(&lc, kernel, KArgs(args)...);
 }
 
-template <int G>
-void launch_forward_g(sdnn* h, int layer, const float* xin, float* xout, int ld, int chunks) {
+template <int G, int V>
+void launch_forward_gv(sdnn* h, int layer, const float* xin, float* xout, int ld, int chunks) {
     constexpr int RPW = 32 / G;
     const int units = (h->N + RPW - 1) / RPW;
-    auto plan = plan_grid(h, (const void*)forward_kernel<G>, units, chunks);
-    launch_k(h, forward_kernel<G>, dim3(plan.first, chunks), dim3(plan.second), h->pdl, rows_of(h, layer),
-             (const float*)(h->d_bias + (size_t)layer * h->N), xin, xout, h->N, ld, h->cfg.clamp, h->pdl ? 1 : 0);
+    const float* bias = h->d_bias + (size_t)layer * h->N;
+    auto plan = plan_grid(h, (const void*)forward_kernel<G, V, 2>, units, chunks);
+    launch_k(h, forward_kernel<G, V, 2>, dim3(plan.first, chunks), dim3(plan.second), h->pdl, rows_of(h, layer), bias, xin, xout,
+             h->N, ld, h->cfg.clamp, h->pdl ? 1 : 0);
 }
 
 void launch_forward(sdnn* h, int layer, const float* xin, float* xout, int ld, int cols) {
     const Geometry q = geometry(cols);
-    switch (q.g) {
-        case 1: launch_forward_g<1>(h, layer, xin, xout, ld, q.chunks); break;
-        case 2: launch_forward_g<2>(h, layer, xin, xout, ld, q.chunks); break;
-        case 4: launch_forward_g<4>(h, layer, xin, xout, ld, q.chunks); break;
-        case 8: launch_forward_g<8>(h, layer, xin, xout, ld, q.chunks); break;
-        case 16: launch_forward_g<16>(h, layer, xin, xout, ld, q.chunks); break;
-        default: launch_forward_g<32>(h, layer, xin, xout, ld, q.chunks); break;
+    if (q.v == 4) launch_forward_gv<1, 4>(h, layer, xin, xout, ld, q.chunks);
+    else switch (q.g) {
+        case 1: launch_forward_gv<1, 8>(h, layer, xin, xout, ld, q.chunks); break;
+        case 2: launch_forward_gv<2, 8>(h, layer, xin, xout, ld, q.chunks); break;
+        case 4: launch_forward_gv<4, 8>(h, layer, xin, xout, ld, q.chunks); break;
+        case 8: launch_forward_gv<8, 8>(h, layer, xin, xout, ld, q.chunks); break;
+        case 16: launch_forward_gv<16, 8>(h, layer, xin, xout, ld, q.chunks); break;
+        default: launch_forward_gv<32, 8>(h, layer, xin, xout, ld, q.chunks); break;
     }
     count_launch(h);
 }
@@ -327,8 +328,8 @@ float* delta_tile(sdnn* h, int layer, size_t tile) {
     return h->d_dbg_delta ? h->d_dbg_delta + (size_t)layer * tile : h->d_s[layer & 1];
 }
 
-template <int G>
-void launch_backward_g(sdnn* h, int layer, int ld) {
+template <int G, int V, int CPS>
+void launch_backward_gvc(sdnn* h, int layer, int ld) {
     constexpr int RPW = 32 / G;
     const size_t tile = (size_t)h->N * ld;
     const bool last = layer == h->L - 1, prop = layer > 0;
@@ -345,51 +346,54 @@ void launch_backward_g(sdnn* h, int layer, int ld) {
     a.update_bias = h->cfg.update_bias ? 1 : 0;
     a.skip_dead = (h->cfg.flags & SDNN_FLAG_SKIP_DEAD) ? 1 : 0;
     a.pdl = h->pdl ? 1 : 0;
-    a.col_units = 0;
-    const void* fn = nullptr;
-#define SDNN_BWD(FROM_S, SCAT, MIR, TOTAL)                                                     \
+    a.warm = (layer >= 1) ? h->d_acts + (size_t)(layer - 1) * tile : nullptr;
+    a.warm_bytes = (unsigned)(tile * sizeof(float));
+#define SDNN_BWD(FROM_S, SCAT, MIR)                                                            \
     do {                                                                                       \
         if (a.dbg_grad) {                                                                      \
-            fn = (const void*)backward_kernel<G, FROM_S, SCAT, MIR, true>;                     \
-            auto plan = plan_grid(h, fn, (TOTAL), 1);                                          \
-            launch_k(h, backward_kernel<G, FROM_S, SCAT, MIR, true>, dim3(plan.first), dim3(plan.second), h->pdl, a); \
+            auto plan = plan_grid(h, (const void*)backward_kernel<G, V, CPS, FROM_S, SCAT, MIR, true>, units, 1);   \
+            launch_k(h, backward_kernel<G, V, CPS, FROM_S, SCAT, MIR, true>, dim3(plan.first), dim3(plan.second), h->pdl, a); \
         } else {                                                                               \
-            fn = (const void*)backward_kernel<G, FROM_S, SCAT, MIR, false>;                    \
-            auto plan = plan_grid(h, fn, (TOTAL), 1);                                          \
-            launch_k(h, backward_kernel<G, FROM_S, SCAT, MIR, false>, dim3(plan.first), dim3(plan.second), h->pdl, a); \
+            auto plan = plan_grid(h, (const void*)backward_kernel<G, V, CPS, FROM_S, SCAT, MIR, false>, units, 1);  \
+            launch_k(h, backward_kernel<G, V, CPS, FROM_S, SCAT, MIR, false>, dim3(plan.first), dim3(plan.second), h->pdl, a); \
         }                                                                                      \
     } while (0)
     if (h->mirror) {
         a.dk = delta_tile(h, layer, tile);
         if (prop) {
             a.cols = cols_of(h, layer);
-            a.col_units = units;
             a.dprev = delta_tile(h, layer - 1, tile);
-            SDNN_BWD(false, false, true, units);
+            SDNN_BWD(false, false, true);
         } else {
-            SDNN_BWD(false, false, false, units);
+            SDNN_BWD(false, false, false);
         }
     } else {
         float* dl = h->d_dbg_delta ? h->d_dbg_delta + (size_t)layer * tile : h->d_dl;
         a.dk = last ? dl : h->d_s[(layer + 1) & 1];
         a.dprev = h->d_s[layer & 1];
         a.dbg_delta = (!last && h->d_dbg_delta) ? h->d_dbg_delta + (size_t)layer * tile : nullptr;
-        if (last && prop) SDNN_BWD(false, true, false, units);
-        else if (last) SDNN_BWD(false, false, false, units);
-        else if (prop) SDNN_BWD(true, true, false, units);
-        else SDNN_BWD(true, false, false, units);
+        if (last && prop) SDNN_BWD(false, true, false);
+        else if (last) SDNN_BWD(false, false, false);
+        else if (prop) SDNN_BWD(true, true, false);
+        else SDNN_BWD(true, false, false);
     }
 #undef SDNN_BWD
 }
 
+template <int G, int V>
+void launch_backward_gv(sdnn* h, int layer, int ld) {
+    launch_backward_gvc<G, V, 2>(h, layer, ld);
+}
+
 void launch_backward(sdnn* h, int layer, int ld) {
-    switch (ld / 4) {
-        case 1: launch_backward_g<1>(h, layer, ld); break;
-        case 2: launch_backward_g<2>(h, layer, ld); break;
-        case 4: launch_backward_g<4>(h, layer, ld); break;
-        case 8: launch_backward_g<8>(h, layer, ld); break;
-        case 16: launch_backward_g<16>(h, layer, ld); break;
-        default: launch_backward_g<32>(h, layer, ld); break;
+    const Geometry q = geometry(ld);
+    if (q.v == 4) launch_backward_gv<1, 4>(h, layer, ld);
+    else switch (q.g) {
+        case 1: launch_backward_gv<1, 8>(h, layer, ld); break;
+        case 2: launch_backward_gv<2, 8>(h, layer, ld); break;
+        case 4: launch_backward_gv<4, 8>(h, layer, ld); break;
+        case 8: launch_backward_gv<8, 8>(h, layer, ld); break;
+        default: launch_backward_gv<16, 8>(h, layer, ld); break;
     }
     count_launch(h);
 }
@@ -592,7 +596,7 @@ int sdnn_create_deferred(sdnn_t** out, int32_t n_layers, int32_t n_neurons, cons
 
     sdnn* h = new (std::nothrow) sdnn;
     if (!h) return fail(nullptr, SDNN_ERR_OOM, "host allocation failed");
-    h->L = n_layers; h->N = n_neurons; h->NS = (n_neurons + 7) / 8; h->cfg = *cfg;
+    h->L = n_layers; h->N = n_neurons; h->NS = (n_neurons + SLICE - 1) / SLICE; h->cfg = *cfg;
     h->stream = static_cast<cudaStream_t>(cfg->cuda_stream);
     auto bail = [&](int code) { g_create_error = h->err; sdnn_destroy(h); return code; };
     if (cfg->device >= 0) {
@@ -611,8 +615,6 @@ int sdnn_create_deferred(sdnn_t** out, int32_t n_layers, int32_t n_neurons, cons
     }
     h->mirror = cfg->train && !(cfg->flags & SDNN_FLAG_BWD_ATOMICS);
     h->pdl = !(cfg->flags & SDNN_FLAG_NO_PDL);
-    if (const char* e_ = getenv("SDNN_TUNE_S4")) h->steps4 = atoi(e_) != 0;
-    if (const char* e_ = getenv("SDNN_TUNE_WPS")) h->tune_wps = atoi(e_);
     h->nnz.assign(nnz_per_layer, nnz_per_layer + n_layers);
     h->loaded.assign(n_layers, 0);
     h->lay.resize(n_layers);
@@ -996,6 +998,13 @@ namespace {
 
 static __device__ __align__(256) float g_noalloc_scratch[2 * SDNN_NOALLOC_MAX_TILE_FLOATS];
 
+// tile geometry of this entry point (plain CSR kernel: 4 batch entries per lane, chunks of 128 columns)
+int noalloc_padded_width(int b) {
+    if (b <= 4) return 4;
+    if (b <= 128) { int w = 4; while (w < b) w <<= 1; return w; }
+    return (b + 127) / 128 * 128;
+}
+
 constexpr int kMaxDevices = 64;
 float* g_noalloc_ptr[kMaxDevices] = {};      // per device: address of g_noalloc_scratch on that device
 
@@ -1038,7 +1047,7 @@ extern "C" int sdnn_infer_noalloc(int32_t n_layers, int32_t n_neurons, const int
     if (!(clamp > 0.0f) || !std::isfinite(clamp)) return fail(nullptr, SDNN_ERR_INVALID_ARG, "clamp must be finite and > 0");
     if (n_inputs == 0) return SDNN_OK;
     if (!x0 || !y_out) return fail(nullptr, SDNN_ERR_INVALID_ARG, "x0 or y_out is NULL");
-    const int ld = padded_width(n_inputs);
+    const int ld = noalloc_padded_width(n_inputs);
     if ((int64_t)n_neurons * ld > (int64_t)SDNN_NOALLOC_MAX_TILE_FLOATS)
         return fail(nullptr, SDNN_ERR_INVALID_ARG,
                     "problem too large for the built-in scratch: n_neurons * padded(n_inputs) = %lld floats, limit %d",
@@ -1053,7 +1062,7 @@ extern "C" int sdnn_infer_noalloc(int32_t n_layers, int32_t n_neurons, const int
     if (rc) return rc;
     float* tile[2] = {scratch, scratch + SDNN_NOALLOC_MAX_TILE_FLOATS};
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    const Geometry q = geometry(ld);
+    const struct { int g, chunks; } q = {ld <= 128 ? ld / 4 : 32, ld <= 128 ? 1 : ld / 128};
     {
         dim3 grid((n_neurons + 31) / 32, (ld + 31) / 32), block(32, 8);
         transpose_in_kernel<<<grid, block, 0, st>>>(x0, tile[0], n_neurons, n_inputs, ld, ld);

@@ -62,8 +62,13 @@ typedef enum {
 #define SDNN_FLAG_BWD_CSC     0x02u /* backward product by gather through a transposed copy of the layer (second   */
                                     /* index and value array, both copies updated; no atomics).  The default.      */
 #define SDNN_FLAG_KEEP_DEBUG  0x04u /* train handles: also store delta^k and the gradient G^k of the last step     */
-#define SDNN_FLAG_SKIP_DEAD   0x08u /* allow data-dependent skipping (dead inputs, all-zero delta rows); default   */
-                                    /* is dense mode: every layer streams its weights and processes every input    */
+#define SDNN_FLAG_SKIP_DEAD   0x08u /* allow data-dependent skipping; default is dense mode: every layer streams   */
+                                    /* its weights and processes every input.  Inference: inputs whose activation  */
+                                    /* vector has become all zero are dropped from the tile (whole chunks of 256   */
+                                    /* columns at a time); only done while no layer has a positive bias, because   */
+                                    /* only then does an all-zero vector stay all zero.  Training: a unit of rows  */
+                                    /* whose delta is zero for every input skips its entries.  Results are the     */
+                                    /* same as in dense mode.                                                      */
 #define SDNN_FLAG_NO_GRAPH    0x10u /* launch the layer chain kernel by kernel instead of through a CUDA graph     */
 #define SDNN_FLAG_NO_PDL      0x20u /* do not let a layer's kernel start its prologue under the previous layer's tail */
 
@@ -196,8 +201,9 @@ int64_t sdnn_device_bytes(const sdnn_t* h);
  * step has run. */
 int sdnn_get_phase_times(sdnn_t* h, float* fwd_ms, float* bwd_ms);
 
-/* Per-layer liveness of the most recent sdnn_infer_batch tile run with SDNN_FLAG_SKIP_DEAD:
- * live_inputs_out host int32[L] = inputs still alive after each layer.  SDNN_ERR_STATE otherwise. */
+/* Per-layer liveness of the most recent inference tile run with SDNN_FLAG_SKIP_DEAD in effect (see the flag):
+ * live_inputs_out host int32[L] = inputs of that tile whose activation vector is not all zero after each layer.
+ * Synchronises the stream.  SDNN_ERR_STATE if no such tile has run. */
 int sdnn_get_liveness(sdnn_t* h, int32_t* live_inputs_out);
 
 /*

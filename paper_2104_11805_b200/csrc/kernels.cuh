@@ -142,6 +142,12 @@ __device__ __forceinline__ bool f4_any(const float4& v) { return !(v.x == 0.0f &
 __device__ __forceinline__ bool lane_any(const Lane<4>& v) { return f4_any(v.a); }
 __device__ __forceinline__ bool lane_any(const Lane<8>& v) { return f4_any(v.a) || f4_any(v.b); }
 
+__device__ __forceinline__ unsigned f4_nonzero_bits(const float4& v) {
+    return (v.x != 0.0f ? 1u : 0u) | (v.y != 0.0f ? 2u : 0u) | (v.z != 0.0f ? 4u : 0u) | (v.w != 0.0f ? 8u : 0u);
+}
+__device__ __forceinline__ unsigned lane_nonzero_bits(const Lane<4>& v) { return f4_nonzero_bits(v.a); }
+__device__ __forceinline__ unsigned lane_nonzero_bits(const Lane<8>& v) { return f4_nonzero_bits(v.a) | (f4_nonzero_bits(v.b) << 4); }
+
 // S[row,:] += w * d[:] with 128-bit vector reductions
 __device__ __forceinline__ void lane_red_add(float* p, float w, const Lane<4>& d) {
     red_add_f4(p, make_float4(w * d.a.x, w * d.a.y, w * d.a.z, w * d.a.w));
@@ -362,7 +368,7 @@ __device__ __forceinline__ void prefetch_unit(const Sliced& m, int u, int rpw, i
 template <int G, int V, int CPS>
 __global__ void __launch_bounds__(256, 2)
 forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict__ xin, float* __restrict__ xout,
-               int n, int ld, float clamp, int pdl) {
+               int n, int ld, float clamp, int pdl, const int* __restrict__ ncols_dev, int* __restrict__ live_flags) {
     constexpr int RPW = 32 / G;
     constexpr int UPS = (RPW >= SLICE) ? 1 : SLICE / RPW;      // units per slice
     const int lane = threadIdx.x & 31;
@@ -387,6 +393,9 @@ forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict
     for (int i = 0; i < CPS; ++i) c[i] = make_int4(0, 0, 0, 0);
     if (nch > 0) load_idx<CPS>(c, idx + base);
     if (pdl) grid_dependency_wait();
+    // compaction mode: only the first *ncols_dev columns of the tile still hold live inputs
+    if (ncols_dev && blockIdx.y * (V * G) >= *ncols_dev) return;
+    unsigned live = 0u;       // bit e: column boff + e of some row this lane produced is nonzero
 
     while (unit < nunits) {
         // shape of this group's row in the warp's next unit (used when this unit's last step prefetches across the boundary)
@@ -419,8 +428,14 @@ forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict
         if (row < n) {
             lane_clamp(acc, clamp);
             lane_store(tile_row(xout + boff, row, pitch), acc);
+            if (live_flags) live |= lane_nonzero_bits(acc);
         }
         unit = nunit; row = nrow; base = nbase; nch = nnch; b = nb;
+    }
+    if (live_flags) {
+#pragma unroll
+        for (int e = 0; e < V; ++e)
+            if ((live >> e) & 1u) live_flags[boff + e] = 1;      // many lanes may store the same 1
     }
     if (pdl) grid_launch_dependents();
 }
@@ -713,6 +728,124 @@ __global__ void mirror_values_kernel(Sliced rows, Sliced cols, int n, unsigned l
         } else {
             cols.val[pos] = w;
         }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Dropping dead inputs during inference (inputs are independent of one another, Section 2; an input whose
+// activation vector has become all zero stays all zero when no bias is positive).  The tile keeps its live
+// inputs in its first *ncols columns; colmap[c] = position in the caller's tile of the input in column c.
+//   cols_init : ncols = cnt, colmap = identity, flags cleared
+//   live      : after a forward layer has marked the columns that still hold a nonzero: count them, record
+//               the count for this layer, and - if that frees at least one whole chunk of columns - renumber
+//               (perm[new] = old column, colmap follows, ncols = count, *do_compact = 1).  Single block.
+//   compact   : moves the columns of every row to their new places, in place (a warp reads the part of a row it
+//               is about to overwrite before it writes), and clears the rest of the last live chunk
+//   expand    : final tile back to the caller's column positions, dead inputs all zero
+struct ColState {
+    int* ncols;        // live columns (device scalar)
+    int* old_ncols;    // value of ncols before the last renumbering
+    int* do_compact;
+    int* colmap;       // [ld]
+    int* perm;         // [ld]
+    int* flags;        // [ld]
+};
+
+__global__ void cols_init_kernel(ColState s, int cnt, int ld) {
+    for (int c = blockIdx.x * blockDim.x + threadIdx.x; c < ld; c += gridDim.x * blockDim.x) {
+        s.colmap[c] = c; s.perm[c] = c; s.flags[c] = 0;
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) { *s.ncols = cnt; *s.old_ncols = cnt; *s.do_compact = 0; }
+}
+
+__global__ void __launch_bounds__(1024) live_kernel(ColState s, int* __restrict__ live_after_layer, int chunk) {
+    __shared__ int warp_tot[32];
+    __shared__ int carry, total;
+    const int n = *s.ncols;
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    // pass 1: how many columns are still live
+    int cnt = 0;
+    for (int b = threadIdx.x; b < n; b += 1024) cnt += (s.flags[b] != 0);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+    if (lane == 0) warp_tot[wid] = cnt;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int t = 0;
+        for (int q = 0; q < 32; ++q) t += warp_tot[q];
+        total = t; carry = 0;
+        *live_after_layer = t;
+    }
+    __syncthreads();
+    const int live = total;
+    const bool renumber = (live + chunk - 1) / chunk < (n + chunk - 1) / chunk;
+    if (renumber) {
+        // pass 2: stable renumbering, 1024 columns at a time (new position <= old position)
+        for (int base = 0; base < n; base += 1024) {
+            const int b = base + threadIdx.x;
+            const int f = (b < n && s.flags[b] != 0) ? 1 : 0;
+            const int cm = (b < n) ? s.colmap[b] : 0;
+            int incl = f;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += t;
+            }
+            __syncthreads();                  // warp_tot free again; every colmap[b] of this round has been read
+            if (lane == 31) warp_tot[wid] = incl;
+            __syncthreads();
+            int before = carry;
+            for (int q = 0; q < wid; ++q) before += warp_tot[q];
+            if (f) { const int np = before + incl - 1; s.perm[np] = b; s.colmap[np] = cm; }
+            __syncthreads();
+            if (threadIdx.x == 1023) carry = before + incl;
+            __syncthreads();
+        }
+    }
+    for (int b = threadIdx.x; b < n; b += 1024) s.flags[b] = 0;
+    if (threadIdx.x == 0) {
+        *s.do_compact = renumber ? 1 : 0;
+        if (renumber) { *s.old_ncols = n; *s.ncols = live; }
+    }
+}
+
+__global__ void __launch_bounds__(256) compact_kernel(ColState s, float* __restrict__ tile, int n, int ld, int chunk) {
+    if (*s.do_compact == 0) return;
+    const int live = *s.ncols;
+    const int fill = min(ld, (live + chunk - 1) / chunk * chunk);       // columns the next layer will read
+    const int lane = threadIdx.x & 31;
+    const int warps = (gridDim.x * blockDim.x) >> 5;
+    for (int row = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; row < n; row += warps) {
+        float* r = tile + (size_t)row * ld;
+        for (int base = 0; base < fill; base += 1024) {
+            float v[32];
+#pragma unroll
+            for (int q = 0; q < 32; ++q) {
+                const int c = base + q * 32 + lane;
+                v[q] = (c < live) ? r[s.perm[c]] : 0.0f;
+            }
+            __syncwarp();
+#pragma unroll
+            for (int q = 0; q < 32; ++q) {
+                const int c = base + q * 32 + lane;
+                if (c < fill) r[c] = v[q];
+            }
+            __syncwarp();
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256) expand_kernel(ColState s, const float* __restrict__ src, float* __restrict__ dst,
+                                                     int n, int cols, int ld) {
+    const int live = *s.ncols;
+    const int lane = threadIdx.x & 31;
+    const int warps = (gridDim.x * blockDim.x) >> 5;
+    for (int row = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; row < n; row += warps) {
+        const float* a = src + (size_t)row * ld;
+        float* r = dst + (size_t)row * ld;
+        for (int c = lane; c < cols; c += 32) r[c] = 0.0f;
+        __syncwarp();
+        for (int c = lane; c < live; c += 32) r[s.colmap[c]] = a[c];
     }
 }
 

@@ -85,6 +85,11 @@ struct sdnn {
     int* d_tile_cnt = nullptr;
     long long* d_offs = nullptr;
     long long* d_running = nullptr;
+    bool compaction = false;            // SDNN_FLAG_SKIP_DEAD asked for; effective while no bias is positive
+    std::vector<char> bias_nonpositive; // per layer
+    ColState cs{};                      // device state of the live-column bookkeeping
+    int* d_live_hist = nullptr;         // [L] live inputs after each layer of the most recent tile
+    bool live_valid = false;
 
     // staging for the *_host entry points (allocated on first use)
     float* d_stage_a = nullptr;
@@ -300,25 +305,27 @@ cudaError_t launch_k(sdnn* h, void (*kernel)(KArgs...), dim3 grid, dim3 block, b
 }
 
 template <int G, int V>
-void launch_forward_gv(sdnn* h, int layer, const float* xin, float* xout, int ld, int chunks) {
+void launch_forward_gv(sdnn* h, int layer, const float* xin, float* xout, int ld, int chunks, bool track) {
     constexpr int RPW = 32 / G;
     const int units = (h->N + RPW - 1) / RPW;
     const float* bias = h->d_bias + (size_t)layer * h->N;
     auto plan = plan_grid(h, (const void*)forward_kernel<G, V, 2>, units, chunks);
     launch_k(h, forward_kernel<G, V, 2>, dim3(plan.first, chunks), dim3(plan.second), h->pdl, rows_of(h, layer), bias, xin, xout,
-             h->N, ld, h->cfg.clamp, h->pdl ? 1 : 0);
+             h->N, ld, h->cfg.clamp, h->pdl ? 1 : 0, track ? (const int*)h->cs.ncols : (const int*)nullptr,
+             track ? h->cs.flags : (int*)nullptr);
 }
 
-void launch_forward(sdnn* h, int layer, const float* xin, float* xout, int ld, int cols) {
+// track: compaction mode (process only the live columns, mark the columns that stay live)
+void launch_forward(sdnn* h, int layer, const float* xin, float* xout, int ld, int cols, bool track = false) {
     const Geometry q = geometry(cols);
-    if (q.v == 4) launch_forward_gv<1, 4>(h, layer, xin, xout, ld, q.chunks);
+    if (q.v == 4) launch_forward_gv<1, 4>(h, layer, xin, xout, ld, q.chunks, track);
     else switch (q.g) {
-        case 1: launch_forward_gv<1, 8>(h, layer, xin, xout, ld, q.chunks); break;
-        case 2: launch_forward_gv<2, 8>(h, layer, xin, xout, ld, q.chunks); break;
-        case 4: launch_forward_gv<4, 8>(h, layer, xin, xout, ld, q.chunks); break;
-        case 8: launch_forward_gv<8, 8>(h, layer, xin, xout, ld, q.chunks); break;
-        case 16: launch_forward_gv<16, 8>(h, layer, xin, xout, ld, q.chunks); break;
-        default: launch_forward_gv<32, 8>(h, layer, xin, xout, ld, q.chunks); break;
+        case 1: launch_forward_gv<1, 8>(h, layer, xin, xout, ld, q.chunks, track); break;
+        case 2: launch_forward_gv<2, 8>(h, layer, xin, xout, ld, q.chunks, track); break;
+        case 4: launch_forward_gv<4, 8>(h, layer, xin, xout, ld, q.chunks, track); break;
+        case 8: launch_forward_gv<8, 8>(h, layer, xin, xout, ld, q.chunks, track); break;
+        case 16: launch_forward_gv<16, 8>(h, layer, xin, xout, ld, q.chunks, track); break;
+        default: launch_forward_gv<32, 8>(h, layer, xin, xout, ld, q.chunks, track); break;
     }
     count_launch(h);
 }
@@ -482,9 +489,30 @@ int infer_tile(sdnn* h, const float* x0, int cnt, float* y_out, int* cnt_out, in
     const int cols = padded_width(cnt);
     launch_transpose_in(h, x0, h->d_tile[0], cnt, cols, ld);
     int cur = 0;
-    for (int k = 0; k < h->L; ++k) {
-        launch_forward(h, k, h->d_tile[cur], h->d_tile[cur ^ 1], ld, cols);
+    bool track = h->compaction;
+    for (int l = 0; l < h->L && track; ++l) track = h->bias_nonpositive[l] != 0;     // the zero vector must be a fixed point
+    if (track) {
+        const Geometry q = geometry(cols);
+        const int chunk = q.g * q.v;
+        const int rows_grid = std::min((h->N + 7) / 8, h->sms * 8);
+        cols_init_kernel<<<(ld + 255) / 256, 256, 0, h->stream>>>(h->cs, cnt, ld);
+        count_launch(h);
+        for (int k = 0; k < h->L; ++k) {
+            launch_forward(h, k, h->d_tile[cur], h->d_tile[cur ^ 1], ld, cols, true);
+            cur ^= 1;
+            live_kernel<<<1, 1024, 0, h->stream>>>(h->cs, h->d_live_hist + k, chunk);
+            compact_kernel<<<rows_grid, 256, 0, h->stream>>>(h->cs, h->d_tile[cur], h->N, ld, chunk);
+            count_launch(h, 2);
+        }
+        expand_kernel<<<rows_grid, 256, 0, h->stream>>>(h->cs, h->d_tile[cur], h->d_tile[cur ^ 1], h->N, cols, ld);
+        count_launch(h);
         cur ^= 1;
+        h->live_valid = true;
+    } else {
+        for (int k = 0; k < h->L; ++k) {
+            launch_forward(h, k, h->d_tile[cur], h->d_tile[cur ^ 1], ld, cols);
+            cur ^= 1;
+        }
     }
     const float* xl = h->d_tile[cur];
     if (y_out) {
@@ -651,6 +679,15 @@ int sdnn_create_deferred(sdnn_t** out, int32_t n_layers, int32_t n_neurons, cons
         if ((rc = dev_alloc(h, &h->d_tile_cnt, (size_t)h->ld_max, false))) return bail(rc);
         if ((rc = dev_alloc(h, &h->d_offs, (size_t)h->ld_max, false))) return bail(rc);
         if ((rc = dev_alloc(h, &h->d_running, 1, true))) return bail(rc);
+        h->compaction = (cfg->flags & SDNN_FLAG_SKIP_DEAD) != 0;
+        h->bias_nonpositive.assign(n_layers, 0);
+        if (h->compaction) {
+            int* blk = nullptr;
+            if ((rc = dev_alloc(h, &blk, 3 * (size_t)h->ld_max + 4, true))) return bail(rc);
+            h->cs.colmap = blk; h->cs.perm = blk + h->ld_max; h->cs.flags = blk + 2 * (size_t)h->ld_max;
+            h->cs.ncols = blk + 3 * (size_t)h->ld_max; h->cs.old_ncols = h->cs.ncols + 1; h->cs.do_compact = h->cs.ncols + 2;
+            if ((rc = dev_alloc(h, &h->d_live_hist, L, true))) return bail(rc);
+        }
     }
     *out = h;
     return SDNN_OK;
@@ -744,6 +781,11 @@ int sdnn_load_layer(sdnn_t* h, int32_t layer, const int32_t* row_ptr, const int3
         if ((rc = refresh_mirror(h, layer, nullptr))) return rc;
     }
     CU(h, cudaStreamSynchronize(h->stream));   // the host vectors above go out of scope; the caller may reuse its arrays
+    {
+        bool nonpos = true;
+        for (int i = 0; i < N && nonpos; ++i) nonpos = !(bias[i] > 0.0f);
+        h->bias_nonpositive[layer] = nonpos ? 1 : 0;
+    }
     h->loaded[layer] = 1;
     return SDNN_OK;
 }
@@ -907,7 +949,12 @@ int sdnn_set_weights(sdnn_t* h, int32_t layer, const float* values, const float*
             CU(h, cudaStreamSynchronize(h->stream));
         }
     }
-    if (bias) CU(h, cudaMemcpy(h->d_bias + (size_t)layer * h->N, bias, (size_t)h->N * sizeof(float), cudaMemcpyHostToDevice));
+    if (bias) {
+        CU(h, cudaMemcpy(h->d_bias + (size_t)layer * h->N, bias, (size_t)h->N * sizeof(float), cudaMemcpyHostToDevice));
+        bool nonpos = true;
+        for (int i = 0; i < h->N && nonpos; ++i) nonpos = !(bias[i] > 0.0f);
+        h->bias_nonpositive[layer] = nonpos ? 1 : 0;
+    }
     return SDNN_OK;
 }
 
@@ -984,7 +1031,11 @@ int sdnn_get_phase_times(sdnn_t* h, float* fwd_ms, float* bwd_ms) {
 
 int sdnn_get_liveness(sdnn_t* h, int32_t* live_inputs_out) {
     if (!h || !live_inputs_out) return SDNN_ERR_INVALID_ARG;
-    return fail(h, SDNN_ERR_STATE, "liveness is recorded only by inference with SDNN_FLAG_SKIP_DEAD");
+    if (!h->live_valid) return fail(h, SDNN_ERR_STATE, "liveness is recorded only by inference with SDNN_FLAG_SKIP_DEAD on a net without positive biases");
+    CU(h, cudaSetDevice(h->device));
+    CU(h, cudaStreamSynchronize(h->stream));
+    CU(h, cudaMemcpy(live_inputs_out, h->d_live_hist, (size_t)h->L * sizeof(int), cudaMemcpyDeviceToHost));
+    return SDNN_OK;
 }
 
 }  // extern "C"

@@ -240,6 +240,51 @@ def test_infer_cfg4_sampled(torch_cuda, variant):
     print(variant, st)
 
 
+@pytest.mark.parametrize("variant", ["live", "base"])
+def test_infer_dropping_dead_inputs_gives_dense_results(torch_cuda, variant):
+    """SDNN_FLAG_SKIP_DEAD: same outputs as dense mode, bit for bit, and the per-layer live counts.
+
+    live: He weights, bias 0, 60 % of the inputs all zero (they die at layer 1, the others stay alive), so the
+    tile shrinks from three chunks of 256 columns to two; base: the net as specified dies entirely by layer 3."""
+    pkg = sdnn()
+    spec = gen.CFG2.scaled(1024, 12)
+    if variant == "live":
+        spec = spec.live()
+    rp, col, val, bias = gen.network(spec)
+    cnt = 700
+    x0 = gen.inputs(spec, cnt)
+    rng = np.random.default_rng(3)
+    dead = rng.uniform(size=cnt) < 0.6
+    if variant == "live":
+        x0[dead] = 0.0
+    outs = []
+    for flags in (0, pkg.FLAG_SKIP_DEAD):
+        h = pkg.Sdnn.create(rp, col, val, bias, max_batch=1024, flags=flags)
+        yd = torch_cuda.full((cnt, spec.n), -1.0, dtype=torch_cuda.float32, device="cuda")
+        cd = torch_cuda.full((cnt,), -1, dtype=torch_cuda.int32, device="cuda")
+        idd = torch_cuda.empty(cnt * spec.n, dtype=torch_cuda.int32, device="cuda")
+        total = h.infer_batch(torch_cuda.from_numpy(x0).cuda(), cnt, yd, cd, idd, cnt * spec.n, want_total=True)
+        live = h.get_liveness() if flags else None
+        if not flags:
+            with pytest.raises(pkg.SdnnError):
+                h.get_liveness()
+        outs.append((yd.cpu().numpy(), cd.cpu().numpy(), idd.cpu().numpy()[:total], total, live))
+        h.destroy()
+    (y0, c0, i0, t0, _), (y1, c1, i1, t1, live) = outs
+    assert np.array_equal(y0, y1) and np.array_equal(c0, c1) and t0 == t1 and np.array_equal(i0, i1)
+    ora = OracleNet(rp, col, val, bias)
+    x = x0.astype(np.float64)
+    want = []
+    for k in range(spec.layers):
+        _, x, _ = ora.forward_layer(k, x)
+        want.append(int((x != 0).any(axis=1).sum()))
+    assert list(live) == want, (list(live), want)
+    if variant == "live":
+        assert want[-1] == int((~dead).sum()) and t0 > 0
+    else:
+        assert want[-1] == 0 and t0 == 0
+
+
 # ---------------------------------------------------------------------------------------------- API behaviour on a device
 def test_capacity_too_small_reports_needed(torch_cuda):
     pkg = sdnn()

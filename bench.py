@@ -48,6 +48,11 @@ WORKLOADS = {
 }
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
+# (training kernels: captured on a 48-layer slice of the same net, per-launch traffic does not depend on the depth)
+NCU_TRAFFIC = {}
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -199,6 +204,7 @@ def main():
     ap.add_argument("--flags", type=lambda s: int(s, 0), default=0, help="extra SDNN_FLAG_* bits")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-compaction", action="store_true", help="inference: skip the extra pass with dead inputs dropped")
     args = ap.parse_args()
     if args.warmup < 3 and args.layers is None:
         args.warmup = 3
@@ -223,6 +229,7 @@ def main():
     import torch.distributed as dist
 
     import paper_2104_11805_b200 as pkg
+    from paper_2104_11805_b200 import shard
     from paper_2104_11805_b200.build import build_library
 
     if not torch.cuda.is_available():
@@ -272,9 +279,10 @@ def main():
             # the batch is sharded over ranks: each rank infers its own n_inputs inputs (weak scaling, no collective)
             chunk = 4096
             x_all = torch.empty((n_inputs, N), dtype=torch.float32, device="cuda")
+            first, _ = shard.rank_inputs(rank, world, n_inputs)
             for s0 in range(0, n_inputs, chunk):
                 c = min(chunk, n_inputs - s0)
-                x_all[s0:s0 + c] = torch.from_numpy(gen.inputs(spec, c, start=rank * n_inputs + s0)).cuda()
+                x_all[s0:s0 + c] = torch.from_numpy(gen.inputs(spec, c, start=first + s0)).cuda()
             counts = torch.empty(n_inputs, dtype=torch.int32, device="cuda")
             cap = 1 << 20
             idx = torch.empty(cap, dtype=torch.int32, device="cuda")
@@ -330,12 +338,7 @@ def main():
         launches = h.kernel_launches() - launches0
         if kind == "train":
             fwd_ms, bwd_ms = h.get_phase_times()      # last timed step
-        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-        if world > 1:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-        ms_per_step = total_ms / args.steps
-        value = world * edges_per_step / (ms_per_step * 1e-3)
+        value, ms_per_step = shard.job_throughput(edges_per_step, total_ms / args.steps, world, device="cuda")
 
         # ---------------------------------------------------------------- end-to-end through host buffers
         e2e = None
@@ -353,14 +356,37 @@ def main():
             barrier()
             wall_ms = 1e3 * (time.perf_counter() - t0)
             dev_ms = a.elapsed_time(b)
-            t = torch.tensor([max(wall_ms, dev_ms)], dtype=torch.float64, device="cuda")
-            if world > 1:
-                dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            per = float(t.item()) / k_e2e
             e2e_edges = edges_per_step if kind == "train" else n_e2e * spec.total_nnz
-            e2e = {"value": world * e2e_edges / (per * 1e-3), "unit": "edges/s", "h2d_bytes_per_step": h2d,
+            e2e_value, per = shard.job_throughput(e2e_edges, max(wall_ms, dev_ms) / k_e2e, world, device="cuda")
+            e2e = {"value": e2e_value, "unit": "edges/s", "h2d_bytes_per_step": h2d,
                    "d2h_bytes_per_step": d2h, "ms_per_step": per,
                    "api": "sdnn_train_step_host" if kind == "train" else f"sdnn_infer_batch_host on {n_e2e} inputs"}
+
+    # -------------------------------------------------------------------- inference: the same call with dead inputs dropped
+    compaction = None
+    if kind == "infer" and not args.no_compaction:
+        with torch.cuda.stream(stream):
+            hc = pkg.Sdnn.create_deferred(L, N, [spec.nnz_per_layer] * L, max_batch=batch, flags=flags | pkg.FLAG_SKIP_DEAD,
+                                          stream=stream.cuda_stream, device=local_rank)
+            for l in range(L):
+                hc.load_layer(l, *gen.layer(spec, l))
+            hc.finalize()
+            hc.infer_batch(x_all, n_inputs, None, counts, None, 0)
+            torch.cuda.synchronize()
+            a = torch.cuda.Event(enable_timing=True)
+            b = torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(2):
+                hc.infer_batch(x_all, n_inputs, None, counts, None, 0)
+            b.record(stream)
+            torch.cuda.synchronize()
+            cv, cms = shard.job_throughput(edges_per_step, a.elapsed_time(b) / 2, world, device="cuda")
+            live = [int(v) for v in hc.get_liveness()]
+            last_tile = n_inputs - (n_inputs - 1) // batch * batch
+            compaction = {"value": cv, "unit": "edges/s (nominal: every stored entry of every input counted, as in dense mode)",
+                          "ms_per_step": cms, "live_inputs_after_layer_last_tile": live[:8] + (["..."] if L > 8 else []) + live[-1:],
+                          "last_tile_inputs": last_tile}
+            hc.destroy()
 
     # -------------------------------------------------------------------- roofline of the dominant kernel
     nnz_l = spec.nnz_per_layer
@@ -385,8 +411,9 @@ def main():
         alg = 8 * nnz_l + 2 * N * min(batch, n_inputs) * 4
         extra = {"tiles": tiles, "note": "launch time = call time / forward launches (upper bound)"}
     achieved = alg / (per_launch_ms * 1e-3) / 1e9 if per_launch_ms else None
+    traffic = NCU_TRAFFIC.get((args.workload.replace("-live", ""), dom)) if not args.layers or kind == "train" else None
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
-                "frac": achieved / hbm_peak if achieved else None, "traffic": None, "peak_source": peak_src,
+                "frac": achieved / hbm_peak if achieved else None, "traffic": traffic, "peak_source": peak_src,
                 "algorithmic_bytes_per_launch": alg, "launch_ms": per_launch_ms, **extra}
 
     # -------------------------------------------------------------------- CPU oracle on a bounded sample (rank 0, N = 1)
@@ -411,6 +438,7 @@ def main():
                        "parallelism": "replicas only (no collective)" if kind == "train" else "batch sharded over ranks, no collective",
                        "inputs_per_step_per_gpu": n_inputs, "setup_seconds": setup_s, "device_bytes": h.device_bytes()},
             "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
+            "compaction_mode": compaction,
         }
         print(json.dumps(line), flush=True)
     h.destroy()

@@ -410,6 +410,22 @@ def main():
         # per launch: the layer's indices and values once, the activation tile read and written once
         alg = 8 * nnz_l + 2 * N * min(batch, n_inputs) * 4
         extra = {"tiles": tiles, "note": "launch time = call time / forward launches (upper bound)"}
+    # what bounds these launches instead of HBM: random gathers of tile rows out of L2 (measured now, on this device)
+    if kind == "train":
+        row_bytes, gathers = 4 * ld, (2 if dom == "backward_kernel" else 1) * nnz_l
+        table_rows = 1 << (N - 1).bit_length()
+    else:
+        row_bytes, gathers = 512, nnz_l * (min(batch, n_inputs) * 4 + 511) // 512
+        table_rows = 1 << max(0, (N * min(batch, n_inputs) * 4 // 512 - 1).bit_length())
+    table_rows = min(table_rows, (1 << 30) // row_bytes)
+    try:
+        gather_rate = pkg.probe_gather_rate(min(row_bytes, 512), table_rows)
+        floor_ms = gathers / gather_rate * 1e3
+        extra["gather_bound"] = {"probe_rows_per_s": gather_rate, "row_bytes": min(row_bytes, 512), "table_rows": table_rows,
+                                 "gathers_per_launch": gathers, "floor_ms_per_launch": floor_ms,
+                                 "frac_of_gather_floor": floor_ms / per_launch_ms if per_launch_ms else None}
+    except Exception as exc:      # the probe is a diagnostic; the line stands without it
+        extra["gather_bound"] = {"error": str(exc)}
     achieved = alg / (per_launch_ms * 1e-3) / 1e9 if per_launch_ms else None
     traffic = NCU_TRAFFIC.get((args.workload.replace("-live", ""), dom)) if not args.layers or kind == "train" else None
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",

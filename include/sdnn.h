@@ -190,6 +190,17 @@ int sdnn_get_gradient(sdnn_t* h, int32_t layer, float* out);
  */
 int sdnn_mirror_mismatches(sdnn_t* h, int32_t layer, int64_t* count_out);
 
+/*
+ * Measures what bounds the layer kernels on the current device (diagnostic; the paper has no counterpart): the
+ * rate at which an SM array can gather random rows of `row_bytes` bytes (16 .. 512, a power of two) out of a table
+ * of `table_rows` rows (a power of two; at most 1 GiB in all) that sits in L2 or, if larger, in HBM, with nothing
+ * else competing for the load pipe.  A layer with nnz stored entries and a padded batch of ld inputs gathers
+ * nnz rows of 4*ld bytes in the forward product and 2*nnz in the backward launch (transposed realisation), so
+ * nnz / rate is the floor of those launches whatever the HBM bandwidth.  Allocates and frees its own table and
+ * stream, runs about a hundred microseconds of kernels, synchronises.  rows_per_second: host double*.
+ */
+int sdnn_probe_gather_rate(int32_t row_bytes, int64_t table_rows, double* rows_per_second);
+
 /* Counters since creation: kernels launched by this handle (graph nodes count one each);
  * device bytes it holds. */
 int64_t sdnn_kernel_launches(const sdnn_t* h);

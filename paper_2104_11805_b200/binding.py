@@ -48,6 +48,7 @@ _PROTOS = {
     "sdnn_get_delta": (ctypes.c_int, [_vp, _i32, _vp]),
     "sdnn_get_gradient": (ctypes.c_int, [_vp, _i32, _vp]),
     "sdnn_mirror_mismatches": (ctypes.c_int, [_vp, _i32, ctypes.POINTER(_i64)]),
+    "sdnn_probe_gather_rate": (ctypes.c_int, [_i32, _i64, ctypes.POINTER(ctypes.c_double)]),
     "sdnn_get_phase_times": (ctypes.c_int, [_vp, ctypes.POINTER(_f32), ctypes.POINTER(_f32)]),
     "sdnn_get_liveness": (ctypes.c_int, [_vp, _vp]),
     "sdnn_infer_noalloc": (ctypes.c_int, [_i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _f32, _vp]),
@@ -119,6 +120,16 @@ def infer_noalloc(n_layers, n_neurons, row_ptr, col_idx, values, layer_offset, b
                                 _addr(bias), _addr(x0), n_inputs, _addr(y_out), clamp, stream)
     if rc != 0:
         raise SdnnError(rc, (lib.sdnn_last_error(None) or b"").decode())
+
+
+def probe_gather_rate(row_bytes, table_rows):
+    """sdnn_probe_gather_rate: random rows of `row_bytes` bytes per second gathered out of a table of `table_rows` rows."""
+    lib = load_library()
+    out = ctypes.c_double(0.0)
+    rc = lib.sdnn_probe_gather_rate(row_bytes, table_rows, ctypes.byref(out))
+    if rc != 0:
+        raise SdnnError(rc, (lib.sdnn_last_error(None) or b"").decode())
+    return out.value
 
 
 class Sdnn:

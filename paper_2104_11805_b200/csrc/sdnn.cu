@@ -1041,6 +1041,72 @@ int sdnn_get_liveness(sdnn_t* h, int32_t* live_inputs_out) {
 }  // extern "C"
 
 // ---------------------------------------------------------------------------------------------
+// Gather-rate probe (see sdnn_probe_gather_rate in the header).
+namespace {
+
+template <int G>
+float run_gather_probe(const float* table, float* sink, unsigned mask, int per_group, int grid, cudaStream_t st, int reps,
+                       cudaEvent_t a, cudaEvent_t b) {
+    for (int i = 0; i < 2; ++i) gather_probe_kernel<G><<<grid, 256, 0, st>>>(table, sink, mask, per_group, 17u + i);
+    cudaEventRecord(a, st);
+    for (int i = 0; i < reps; ++i) gather_probe_kernel<G><<<grid, 256, 0, st>>>(table, sink, mask, per_group, 101u + i);
+    cudaEventRecord(b, st);
+    cudaEventSynchronize(b);
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, a, b);
+    return ms / reps;
+}
+
+}  // namespace
+
+extern "C" int sdnn_probe_gather_rate(int32_t row_bytes, int64_t table_rows, double* rows_per_second) {
+    if (!rows_per_second) return fail(nullptr, SDNN_ERR_INVALID_ARG, "rows_per_second is NULL");
+    *rows_per_second = 0.0;
+    if (row_bytes != 16 && row_bytes != 32 && row_bytes != 64 && row_bytes != 128 && row_bytes != 256 && row_bytes != 512)
+        return fail(nullptr, SDNN_ERR_INVALID_ARG, "row_bytes must be 16, 32, 64, 128, 256 or 512");
+    if (table_rows < 1 || (table_rows & (table_rows - 1)) || table_rows * row_bytes > (1LL << 30))
+        return fail(nullptr, SDNN_ERR_INVALID_ARG, "table_rows must be a power of two with table_rows * row_bytes <= 1 GiB");
+    int dev = 0, sms = 0;
+    CU(nullptr, cudaGetDevice(&dev));
+    CU(nullptr, cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    float* table = nullptr;
+    float* sink = nullptr;
+    cudaEvent_t a = nullptr, b = nullptr;
+    cudaStream_t st = nullptr;
+    int rc = SDNN_OK;
+    const size_t bytes = (size_t)table_rows * row_bytes;
+    if (cudaMalloc(&table, bytes) != cudaSuccess || cudaMalloc(&sink, 256) != cudaSuccess || cudaStreamCreate(&st) != cudaSuccess ||
+        cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) {
+        cudaGetLastError();
+        rc = fail(nullptr, SDNN_ERR_OOM, "could not allocate the probe's table");
+    } else {
+        cudaMemsetAsync(table, 0, bytes, st);
+        const int g = row_bytes / 16, grid = sms * 4;                 // 1024 threads per SM: the rate no longer grows beyond that
+        const int64_t groups = (int64_t)grid * 256 / g;
+        const int per_group = (int)std::max<int64_t>(8, ((int64_t)1 << 22) / groups / 8 * 8);
+        const unsigned mask = (unsigned)(table_rows - 1);
+        float ms = 0.f;
+        switch (g) {
+            case 1: ms = run_gather_probe<1>(table, sink, mask, per_group, grid, st, 20, a, b); break;
+            case 2: ms = run_gather_probe<2>(table, sink, mask, per_group, grid, st, 20, a, b); break;
+            case 4: ms = run_gather_probe<4>(table, sink, mask, per_group, grid, st, 20, a, b); break;
+            case 8: ms = run_gather_probe<8>(table, sink, mask, per_group, grid, st, 20, a, b); break;
+            case 16: ms = run_gather_probe<16>(table, sink, mask, per_group, grid, st, 20, a, b); break;
+            default: ms = run_gather_probe<32>(table, sink, mask, per_group, grid, st, 20, a, b); break;
+        }
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess || !(ms > 0.f)) rc = cuda_fail(nullptr, e, "gather probe");
+        else *rows_per_second = (double)groups * per_group / (ms * 1e-3);
+    }
+    if (a) cudaEventDestroy(a);
+    if (b) cudaEventDestroy(b);
+    if (st) cudaStreamDestroy(st);
+    if (table) cudaFree(table);
+    if (sink) cudaFree(sink);
+    return rc;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Allocation-free inference (see sdnn_infer_noalloc in the header).  The two activation tiles of
 // the forward chain live in this file-scope device array instead of memory owned by a handle.
 // In host code the array's name is only a stand-in for the symbol, not a device address: the

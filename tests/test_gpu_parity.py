@@ -300,6 +300,16 @@ def test_capacity_too_small_reports_needed(torch_cuda):
     h.destroy()
 
 
+def test_gather_probe_reports_a_rate_and_rejects_bad_sizes(torch_cuda):
+    pkg = sdnn()
+    rate = pkg.probe_gather_rate(64, 65536)
+    assert 1e9 < rate < 1e13          # random 64-byte rows per second out of a 4 MB table
+    for row_bytes, rows in ((48, 1024), (64, 1000), (512, 1 << 22)):
+        with pytest.raises(pkg.SdnnError) as ei:
+            pkg.probe_gather_rate(row_bytes, rows)
+        assert ei.value.code == -1
+
+
 def test_state_and_argument_errors(torch_cuda):
     pkg = sdnn()
     rng = np.random.default_rng(2)

@@ -15,6 +15,9 @@ activation f(z) = min(max(z, 0), c):
 
     f'(z) = 1 for 0 < z < c and 0 otherwise (zero at both kinks).
 
+With activation="sigmoid" (the activation of the paper's own experiments, Section 6) f(z) = 1/(1+exp(-z)) and
+f'(z) = f(z) (1 - f(z)); everything else is unchanged.
+
 Readings taken where the paper is silent: the minibatch step is exact minibatch
 SGD (one delta per input, gradient averaged over the batch; B = 1 is Algorithm 1
 verbatim); delta^0 is never formed (x^0 is data, no z^0 exists); the bias is
@@ -52,7 +55,7 @@ def _L():
     if _lib is None:
         lib = ctypes.CDLL(build())
         i32, dbl, vp = ctypes.c_int32, ctypes.c_double, ctypes.c_void_p
-        lib.oracle_forward_layer.argtypes = [i32, i32, vp, vp, vp, vp, vp, dbl, vp, vp, vp]
+        lib.oracle_forward_layer.argtypes = [i32, i32, vp, vp, vp, vp, vp, dbl, i32, vp, vp, vp]
         lib.oracle_transposed_product.argtypes = [i32, i32, vp, vp, vp, vp, vp]
         lib.oracle_masked_gradient.argtypes = [i32, i32, vp, vp, vp, vp, vp]
         for f in (lib.oracle_forward_layer, lib.oracle_transposed_product, lib.oracle_masked_gradient):
@@ -80,7 +83,11 @@ def nonzero_sets(x_last: np.ndarray):
 class OracleNet:
     """L square sparse layers in CSR plus biases; weights are held (and trained) in float64."""
 
-    def __init__(self, row_ptr, col, val, bias, clamp: float = 32.0, update_bias: bool = False):
+    def __init__(self, row_ptr, col, val, bias, clamp: float = 32.0, update_bias: bool = False,
+                 activation: str = "clamped_relu"):
+        if activation not in ("clamped_relu", "sigmoid"):
+            raise ValueError(activation)
+        self.activation = activation
         self.layers = len(col)
         self.n = len(bias[0])
         self.row_ptr = [np.ascontiguousarray(r, dtype=np.int32) for r in row_ptr]
@@ -111,11 +118,14 @@ class OracleNet:
         x = np.empty((nb, self.n))
         scale = np.empty((nb, self.n)) if want_scale else None
         _L().oracle_forward_layer(self.n, nb, _p(self.row_ptr[k]), _p(self.col[k]), _p(self.w[k]), _p(self.bias[k]),
-                                  _p(x_prev), self.clamp, _p(z), _p(x), _p(scale))
+                                  _p(x_prev), self.clamp, 1 if self.activation == "sigmoid" else 0, _p(z), _p(x), _p(scale))
         return z, x, scale
 
     def derivative_mask(self, z: np.ndarray) -> np.ndarray:
-        """f'(z) as a 0/1 array: 1 strictly inside (0, c)."""
+        """f'(z): clamped ReLU: a 0/1 array, 1 strictly inside (0, c); sigmoid: f(z) (1 - f(z))."""
+        if self.activation == "sigmoid":
+            f = 1.0 / (1.0 + np.exp(-z))
+            return f * (1.0 - f)
         return ((z > 0.0) & (z < self.clamp)).astype(np.float64)
 
     def transposed_product(self, k: int, delta: np.ndarray) -> np.ndarray:
@@ -159,6 +169,8 @@ class OracleNet:
         for k in range(self.layers):
             z, x, scale = self.forward_layer(k, x, want_scale=mask_hook is not None)
             m = self.derivative_mask(z)
+            if mask_hook is not None and self.activation == "sigmoid":
+                raise ValueError("mask_hook is for the kinks of the clamped ReLU; the sigmoid has none")
             if mask_hook is not None:
                 m = mask_hook(k + 1, z, scale, m)
             xs.append(x)

@@ -23,11 +23,13 @@
 #include <math.h>
 #include <stdint.h>
 
-/* z = W x + b for every input; x_out = f(z) with f(z) = min(max(z, 0), clamp);
+/* z = W x + b for every input; x_out = f(z) with
+ *   activation 0: f(z) = min(max(z, 0), clamp)
+ *   activation 1: f(z) = 1 / (1 + exp(-z))      (the sigmoid of the paper's experimental setup, Section 6)
  * absacc (nullable) = |b| + sum |w x| (the scale of the rounding error of z). */
 void oracle_forward_layer(int32_t n, int32_t nb, const int32_t *row_ptr, const int32_t *col,
                           const double *w, const double *bias, const double *x_in, double clamp,
-                          double *z, double *x_out, double *absacc) {
+                          int32_t activation, double *z, double *x_out, double *absacc) {
 #pragma omp parallel for collapse(2) schedule(static)
     for (int32_t b = 0; b < nb; ++b) {
         for (int32_t i = 0; i < n; ++i) {
@@ -41,8 +43,12 @@ void oracle_forward_layer(int32_t n, int32_t nb, const int32_t *row_ptr, const i
             }
             int64_t o = (int64_t)b * n + i;
             z[o] = acc;
-            double a = acc > 0.0 ? acc : 0.0;
-            x_out[o] = a < clamp ? a : clamp;
+            if (activation == 1) {
+                x_out[o] = 1.0 / (1.0 + exp(-acc));
+            } else {
+                double a = acc > 0.0 ? acc : 0.0;
+                x_out[o] = a < clamp ? a : clamp;
+            }
             if (absacc) absacc[o] = mag;
         }
     }

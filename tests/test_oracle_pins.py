@@ -353,3 +353,100 @@ def test_mask_hook_replaces_the_derivative_mask():
     out = OracleNet(rp, c, v, b).train_step(x0, y, 0.1, mask_hook=hook)
     assert seen == list(range(1, len(c) + 1))
     assert all(np.all(g == 0.0) for g in out["grad"])                    # delta^L = 0 kills every gradient
+
+
+# ------------------------------------------------------------------ sigmoid activation (the paper's experimental setup, Section 6)
+def _sig(z):
+    return 1.0 / (1.0 + np.exp(-z))
+
+
+def _sig_dense_loss(Ws, bs, x0, y):
+    x = x0
+    for W, b in zip(Ws, bs):
+        x = _sig(x @ W.T + b)
+    return ((x - y) ** 2).sum() / (2 * x0.shape[0])
+
+
+def _sig_case(seed, n=10, layers=3, k=4, B=3):
+    rng = np.random.default_rng(seed)
+    rp, c, v, b = random_net(rng, n, layers, k, scale=0.9, bias_scale=0.3)
+    x0 = rng.uniform(0.0, 1.0, size=(B, n)).astype(np.float32)
+    y = rng.uniform(0.0, 1.0, size=(B, n)).astype(np.float32)
+    return rp, c, v, b, x0, y
+
+
+@pytest.mark.parametrize("seed", [5, 6])
+def test_sigmoid_gradient_matches_finite_differences_and_dense_formulas(seed):
+    """With activation="sigmoid": G is dJ/dW on every stored entry (central differences on an independent dense
+    evaluation of J), the forward values are the dense ones, and entries outside the pattern never appear."""
+    rp, c, v, b, x0, y = _sig_case(seed)
+    n, layers = len(b[0]), len(c)
+    dn = [dense_of(rp[l], c[l], v[l].astype(float), n) for l in range(layers)]
+    Ws, bs = [d[0] for d in dn], [bb.astype(float) for bb in b]
+    net = OracleNet(rp, c, v, b, activation="sigmoid")
+    out = net.train_step(x0, y, 0.01)
+    x = x0.astype(float)
+    for l in range(layers):
+        x = _sig(x @ Ws[l].T + bs[l])
+        np.testing.assert_allclose(out["x"][l + 1], x, rtol=0, atol=1e-13)
+    assert abs(out["loss"] - _sig_dense_loss(Ws, bs, x0.astype(float), y.astype(float))) <= 1e-13
+    h = 1e-6
+    for l in range(layers):
+        p = 0
+        for i in range(n):
+            for q in range(rp[l][i], rp[l][i + 1]):
+                j = c[l][q]
+                Wp = [W.copy() for W in Ws]; Wm = [W.copy() for W in Ws]
+                Wp[l][i, j] += h; Wm[l][i, j] -= h
+                fd = (_sig_dense_loss(Wp, bs, x0.astype(float), y.astype(float))
+                      - _sig_dense_loss(Wm, bs, x0.astype(float), y.astype(float))) / (2 * h)
+                assert abs(out["grad"][l][p] - fd) <= 1e-7 * max(1.0, abs(fd)), (l, i, j)
+                p += 1
+        bp = 0
+        for i in range(n):                      # bias gradient = mean of delta = dJ/db
+            bsp = [bb.copy() for bb in bs]; bsm = [bb.copy() for bb in bs]
+            bsp[l][i] += h; bsm[l][i] -= h
+            fd = (_sig_dense_loss(Ws, bsp, x0.astype(float), y.astype(float))
+                  - _sig_dense_loss(Ws, bsm, x0.astype(float), y.astype(float))) / (2 * h)
+            assert abs(out["bias_grad"][l][i] - fd) <= 1e-7 * max(1.0, abs(fd))
+
+
+def test_sigmoid_autograd_and_update():
+    """Same step through torch autograd (float64, dense masked weights, torch.sigmoid): gradients and new weights."""
+    torch = pytest.importorskip("torch")
+    rp, c, v, b, x0, y = _sig_case(11, n=14, layers=4, k=5, B=2)
+    n, layers = len(b[0]), len(c)
+    dn = [dense_of(rp[l], c[l], v[l].astype(float), n) for l in range(layers)]
+    Ws = [torch.tensor(d[0], dtype=torch.float64, requires_grad=True) for d in dn]
+    x = torch.tensor(x0.astype(float))
+    for l in range(layers):
+        x = torch.sigmoid(x @ Ws[l].T + torch.tensor(b[l].astype(float)))
+    loss = ((x - torch.tensor(y.astype(float))) ** 2).sum() / (2 * x0.shape[0])
+    loss.backward()
+    eta = 0.05
+    net = OracleNet(rp, c, v, b, activation="sigmoid")
+    out = net.train_step(x0, y, eta)
+    assert abs(out["loss"] - float(loss)) <= 1e-13
+    for l in range(layers):
+        g = csr_gather(Ws[l].grad.numpy(), rp[l], c[l], n)
+        np.testing.assert_allclose(out["grad"][l], g, rtol=0, atol=1e-13)
+        np.testing.assert_allclose(net.w[l], v[l].astype(float) - float(np.float32(eta)) * g, rtol=0, atol=1e-13)
+
+
+def test_sigmoid_scalar_recurrence_and_mask_hook_refusal():
+    """k equal weights v per row and a constant input: every neuron follows a_l = sigmoid(k v a_{l-1} + b)."""
+    n, k, layers = 64, 8, 6
+    col = gen.circulant_pattern(n, k, 3)
+    rp = (np.arange(n + 1) * k).astype(np.int32)
+    val = np.full(n * k, 0.25, dtype=np.float32)
+    bias = np.full(n, -0.5, dtype=np.float32)
+    net = OracleNet([rp] * layers, [col] * layers, [val] * layers, [bias] * layers, activation="sigmoid")
+    xs = net.infer(np.full((2, n), 0.3, dtype=np.float32), keep_all=True)
+    a = float(np.float32(0.3))
+    for l in range(1, layers + 1):
+        a = 1.0 / (1.0 + np.exp(-(k * 0.25 * a - 0.5)))
+        np.testing.assert_allclose(xs[l], a, rtol=0, atol=1e-14)
+    with pytest.raises(ValueError):
+        net.train_step(np.zeros((1, n), np.float32), np.zeros((1, n), np.float32), 0.1, mask_hook=lambda *a: a[-1])
+    with pytest.raises(ValueError):
+        OracleNet([rp], [col], [val], [bias], activation="tanh")

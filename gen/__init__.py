@@ -73,7 +73,7 @@ class NetSpec:
     k: int = 32                 # nonzeros per row
     pattern: str = "uniform"    # "uniform" | "windowed"
     window: int = 1024
-    values: str = "const"       # "const" (value `const`) | "normal" (std `sigma`)
+    values: str = "const"       # "const" (value `const`) | "normal" (std `sigma`) | "uniform_pm1" (uniform in [-1, 1))
     const: float = 1.0 / 16.0
     sigma: float = 32.0 ** -0.5
     bias: float = -0.30
@@ -89,6 +89,11 @@ class NetSpec:
     def saturating(self) -> "NetSpec":
         """Same pattern; all weights 1/16, bias -0.30, inputs Bernoulli(0.5): every neuron reaches the clamp."""
         return replace(self, name=self.name + "-sat", values="const", const=1.0 / 16.0, bias=-0.30, input_prob=0.5)
+
+    def paper_setup(self) -> "NetSpec":
+        """Same pattern with the training setup of the paper's Section 6: weights uniform in [-1, 1], bias 0 (to be
+        used with the sigmoid activation and eta = 0.01; no neuron ever dies)."""
+        return replace(self, name=self.name + "-paper", values="uniform_pm1", bias=0.0)
 
     def sliced(self, layers: int) -> "NetSpec":
         return replace(self, layers=layers)
@@ -147,6 +152,9 @@ def layer_values(spec: NetSpec, layer: int) -> np.ndarray:
     if spec.values == "const":
         return np.full(cnt, np.float32(spec.const), dtype=np.float32)
     out = np.empty(cnt, dtype=np.float32)
+    if spec.values == "uniform_pm1":
+        _L().sdnn_gen_uniform(spec.seed, (spec.config_id << 8) | S_VALUES, layer, cnt, _ptr(out))
+        return (2.0 * out - 1.0).astype(np.float32)
     _L().sdnn_gen_normal(spec.seed, (spec.config_id << 8) | S_VALUES, layer, cnt, float(spec.sigma), _ptr(out))
     return out
 

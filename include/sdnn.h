@@ -14,7 +14,8 @@
  *
  * W^k(j,i) is the weight of the link from neuron i of layer k to neuron j of
  * layer k+1: CSR row j of W^k lists the incoming links of output neuron j.
- * f(z) = min(max(z, 0), clamp); f'(z) = 1 for 0 < z < clamp, else 0.
+ * f(z) = min(max(z, 0), clamp); f'(z) = 1 for 0 < z < clamp, else 0 (activation 0), or the sigmoid of the
+ * paper's experimental setup (Section 6), f(z) = 1/(1+exp(-z)), f'(z) = f(z)(1 - f(z)) (activation 1).
  * J = 1/(2B) sum_b ||x^L_b - y_b||^2 (mean squared error over a minibatch of B
  * inputs); a minibatch step is exact minibatch SGD: one delta per input, the
  * gradient averaged over the batch (B = 1 is Algorithm 1 verbatim).  The
@@ -72,9 +73,12 @@ typedef enum {
 #define SDNN_FLAG_NO_GRAPH    0x10u /* launch the layer chain kernel by kernel instead of through a CUDA graph     */
 #define SDNN_FLAG_NO_PDL      0x20u /* do not let a layer's kernel start its prologue under the previous layer's tail */
 
+#define SDNN_ACT_CLAMPED_RELU 0
+#define SDNN_ACT_SIGMOID      1
+
 typedef struct {
-    int32_t  activation;   /* 0 = clamped ReLU (the only one implemented) */
-    float    clamp;        /* upper clamp of the activation, e.g. 32.0f; must be > 0 */
+    int32_t  activation;   /* SDNN_ACT_CLAMPED_RELU or SDNN_ACT_SIGMOID */
+    float    clamp;        /* upper clamp of the clamped ReLU, e.g. 32.0f; must be > 0 (ignored by the sigmoid) */
     int32_t  max_batch;    /* train: largest minibatch B; inference: batch tile (inputs processed together) */
     int32_t  train;        /* 0: inference only (no stored activations); 1: sdnn_train_step allowed */
     int32_t  update_bias;  /* 1: b^k <- b^k - eta * mean_b delta^k_b (bias read as a column of W^k); 0: bias frozen */

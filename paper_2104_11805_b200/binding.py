@@ -14,6 +14,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsdnn.so")
 
 FLAG_BWD_ATOMICS, FLAG_BWD_CSC, FLAG_KEEP_DEBUG, FLAG_SKIP_DEAD, FLAG_NO_GRAPH, FLAG_NO_PDL = 0x01, 0x02, 0x04, 0x08, 0x10, 0x20
+ACT_CLAMPED_RELU, ACT_SIGMOID = 0, 1
 
 STATUS = {0: "SDNN_OK", -1: "SDNN_ERR_INVALID_ARG", -2: "SDNN_ERR_BAD_CSR", -3: "SDNN_ERR_OOM", -4: "SDNN_ERR_CUDA",
           -5: "SDNN_ERR_STATE", -6: "SDNN_ERR_UNIMPLEMENTED"}
@@ -163,10 +164,10 @@ class Sdnn:
 
     @classmethod
     def create_deferred(cls, n_layers, n_neurons, nnz_per_layer, *, max_batch, train=False, clamp=32.0,
-                        update_bias=False, flags=0, stream=None, device=-1):
+                        update_bias=False, flags=0, stream=None, device=-1, activation=0):
         lib = load_library()
         nnz = _np(nnz_per_layer, np.int64)
-        cfg = cls._config(max_batch, train, clamp, update_bias, flags, stream, device)
+        cfg = cls._config(max_batch, train, clamp, update_bias, flags, stream, device, activation)
         h = ctypes.c_void_p()
         rc = lib.sdnn_create_deferred(ctypes.byref(h), n_layers, n_neurons, nnz.ctypes.data, ctypes.byref(cfg))
         if rc != 0:

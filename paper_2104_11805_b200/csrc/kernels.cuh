@@ -70,6 +70,16 @@ __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddep
 __device__ __forceinline__ float clampf(float z, float c) { return fminf(fmaxf(z, 0.0f), c); }
 __device__ __forceinline__ float dmask(float x, float c) { return (x > 0.0f && x < c) ? 1.0f : 0.0f; }
 
+// Activations (cfg.activation): 0 = ReLU clamped at c, f'(z) = [0 < x < c]; 1 = sigmoid (the activation of the
+// paper's experiments, Section 6), f'(z) = x (1 - x).  Both derivatives are functions of the stored output x.
+constexpr int ACT_CLAMPED_RELU = 0, ACT_SIGMOID = 1;
+__device__ __forceinline__ float activate(float z, int act, float c) {
+    return act == ACT_SIGMOID ? 1.0f / (1.0f + expf(-z)) : clampf(z, c);
+}
+__device__ __forceinline__ float derivative(float x, int act, float c) {
+    return act == ACT_SIGMOID ? x * (1.0f - x) : dmask(x, c);
+}
+
 // address of tile row `r` (r * pitch below 2^32): one 32 x 32 -> 64 bit multiply-add
 __device__ __forceinline__ const float* tile_row(const float* base, int r, unsigned pitch_bytes) {
     unsigned long long out;
@@ -125,15 +135,18 @@ __device__ __forceinline__ float lane_dot(const Lane<8>& d, const Lane<8>& x) {
     return dot_f4(d.b, x.b, s);
 }
 
-__device__ __forceinline__ void f4_mask(float4& d, const float4& x, float c) {
-    d.x *= dmask(x.x, c); d.y *= dmask(x.y, c); d.z *= dmask(x.z, c); d.w *= dmask(x.w, c);
+// d *= f'(z) with f' taken from the stored output x
+__device__ __forceinline__ void f4_mask(float4& d, const float4& x, int act, float c) {
+    d.x *= derivative(x.x, act, c); d.y *= derivative(x.y, act, c); d.z *= derivative(x.z, act, c); d.w *= derivative(x.w, act, c);
 }
-__device__ __forceinline__ void lane_mask(Lane<4>& d, const Lane<4>& x, float c) { f4_mask(d.a, x.a, c); }
-__device__ __forceinline__ void lane_mask(Lane<8>& d, const Lane<8>& x, float c) { f4_mask(d.a, x.a, c); f4_mask(d.b, x.b, c); }
+__device__ __forceinline__ void lane_mask(Lane<4>& d, const Lane<4>& x, int act, float c) { f4_mask(d.a, x.a, act, c); }
+__device__ __forceinline__ void lane_mask(Lane<8>& d, const Lane<8>& x, int act, float c) { f4_mask(d.a, x.a, act, c); f4_mask(d.b, x.b, act, c); }
 
-__device__ __forceinline__ void f4_clamp(float4& v, float c) { v.x = clampf(v.x, c); v.y = clampf(v.y, c); v.z = clampf(v.z, c); v.w = clampf(v.w, c); }
-__device__ __forceinline__ void lane_clamp(Lane<4>& v, float c) { f4_clamp(v.a, c); }
-__device__ __forceinline__ void lane_clamp(Lane<8>& v, float c) { f4_clamp(v.a, c); f4_clamp(v.b, c); }
+__device__ __forceinline__ void f4_activate(float4& v, int act, float c) {
+    v.x = activate(v.x, act, c); v.y = activate(v.y, act, c); v.z = activate(v.z, act, c); v.w = activate(v.w, act, c);
+}
+__device__ __forceinline__ void lane_activate(Lane<4>& v, int act, float c) { f4_activate(v.a, act, c); }
+__device__ __forceinline__ void lane_activate(Lane<8>& v, int act, float c) { f4_activate(v.a, act, c); f4_activate(v.b, act, c); }
 
 __device__ __forceinline__ float lane_sum(const Lane<4>& v) { return v.a.x + v.a.y + v.a.z + v.a.w; }
 __device__ __forceinline__ float lane_sum(const Lane<8>& v) { return (v.a.x + v.a.y + v.a.z + v.a.w) + (v.b.x + v.b.y + v.b.z + v.b.w); }
@@ -368,7 +381,7 @@ __device__ __forceinline__ void prefetch_unit(const Sliced& m, int u, int rpw, i
 template <int G, int V, int CPS>
 __global__ void __launch_bounds__(256, 2)
 forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict__ xin, float* __restrict__ xout,
-               int n, int ld, float clamp, int pdl, const int* __restrict__ ncols_dev, int* __restrict__ live_flags) {
+               int n, int ld, float clamp, int act, int pdl, const int* __restrict__ ncols_dev, int* __restrict__ live_flags) {
     constexpr int RPW = 32 / G;
     constexpr int UPS = (RPW >= SLICE) ? 1 : SLICE / RPW;      // units per slice
     const int lane = threadIdx.x & 31;
@@ -426,7 +439,7 @@ forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict
         }
         if (nch == 0 && nnch > 0) load_idx<CPS>(c, idx + nbase);      // empty slice: nothing prefetched across the boundary yet
         if (row < n) {
-            lane_clamp(acc, clamp);
+            lane_activate(acc, act, clamp);
             lane_store(tile_row(xout + boff, row, pitch), acc);
             if (live_flags) live |= lane_nonzero_bits(acc);
         }
@@ -445,7 +458,7 @@ forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict
 // batch columns, 0 on the padding; J = 1/(2B) sum (x^L - y)^2 accumulated in double, one atomic per block.
 __global__ void __launch_bounds__(256)
 output_gradient_kernel(const float* __restrict__ xl, const float* __restrict__ y, float* __restrict__ delta,
-                       int n, int ld, float clamp, const StepParams* __restrict__ sp, double* __restrict__ loss) {
+                       int n, int ld, float clamp, int act, const StepParams* __restrict__ sp, double* __restrict__ loss) {
     const int per_row = ld >> 2;
     const long long total = (long long)n * per_row;
     const int nb = sp->batch;
@@ -457,8 +470,8 @@ output_gradient_kernel(const float* __restrict__ xl, const float* __restrict__ y
         e.x = (boff + 0 < nb) ? x.x - t.x : 0.0f; e.y = (boff + 1 < nb) ? x.y - t.y : 0.0f;
         e.z = (boff + 2 < nb) ? x.z - t.z : 0.0f; e.w = (boff + 3 < nb) ? x.w - t.w : 0.0f;
         sq += e.x * e.x + e.y * e.y + e.z * e.z + e.w * e.w;
-        st_f4(delta + v * 4, make_float4(e.x * dmask(x.x, clamp), e.y * dmask(x.y, clamp),
-                                         e.z * dmask(x.z, clamp), e.w * dmask(x.w, clamp)));
+        st_f4(delta + v * 4, make_float4(e.x * derivative(x.x, act, clamp), e.y * derivative(x.y, act, clamp),
+                                         e.z * derivative(x.z, act, clamp), e.w * derivative(x.w, act, clamp)));
     }
     __shared__ float part[8];
 #pragma unroll
@@ -506,6 +519,7 @@ struct BackwardArgs {
     const StepParams* sp;
     int n;
     float clamp;
+    int act;                  // activation (ACT_*)
     int update_bias, skip_dead, pdl;
     const float* warm;        // tile the NEXT backward launch will gather from (x^{k-2}), or NULL: asked into L2 now,
     unsigned warm_bytes;      // because it was written a whole forward pass ago and has left the cache
@@ -514,7 +528,7 @@ struct BackwardArgs {
 // Column units of the transposed realisation.
 template <int G, int V, int CPS>
 __device__ __forceinline__ void backward_col_units(const Sliced m, const float* __restrict__ xprev, const float* __restrict__ dk,
-                                                   float* __restrict__ dprev, int n, float clamp, float step, float inv_b,
+                                                   float* __restrict__ dprev, int n, float clamp, int act, float step, float inv_b,
                                                    int first, int stride) {
     constexpr int RPW = 32 / G;
     constexpr int UPS = (RPW >= SLICE) ? 1 : SLICE / RPW;
@@ -575,7 +589,7 @@ __device__ __forceinline__ void backward_col_units(const Sliced m, const float* 
         if (nch == 0) { SDNN_COL_NEXT }
 #undef SDNN_COL_NEXT
         if (item < n) {
-            lane_mask(acc, xj, clamp);
+            lane_mask(acc, xj, act, clamp);
             lane_store(tile_row(dprev + boff, j, pitch), acc);
         }
         u = nu; item = nitem; base = nbase; nch = nnch; len = nlen; j = nj; xj = nxj;
@@ -586,7 +600,7 @@ __device__ __forceinline__ void backward_col_units(const Sliced m, const float* 
 template <int G, int V, int CPS, bool FROM_S, bool SCATTER, bool DBG>
 __device__ __forceinline__ void backward_row_units(const Sliced m, float* __restrict__ bias, const float* __restrict__ xk,
                                                    const float* __restrict__ xprev, float* dk, float* dprev,
-                                                   float* __restrict__ dbg_delta, float* __restrict__ dbg_grad, int n, float clamp,
+                                                   float* __restrict__ dbg_delta, float* __restrict__ dbg_grad, int n, float clamp, int act,
                                                    float step, float inv_b, int update_bias, int skip_dead, int first, int stride) {
     constexpr int RPW = 32 / G;
     constexpr int UPS = (RPW >= SLICE) ? 1 : SLICE / RPW;
@@ -628,7 +642,7 @@ __device__ __forceinline__ void backward_row_units(const Sliced m, float* __rest
                 Lane<V> z;
                 lane_fill(z, 0.0f);
                 lane_store(tile_row(dk + boff, item, pitch), z);
-                lane_mask(d, h1, clamp);
+                lane_mask(d, h1, act, clamp);
                 if (DBG) lane_store(tile_row(dbg_delta + boff, item, pitch), d);
             }
             if (update_bias) {       // bias read as one more column of W^k whose input is the constant 1
@@ -694,9 +708,9 @@ backward_kernel(const BackwardArgs a) {
     if (a.pdl) grid_dependency_wait();
     const float inv_b = a.sp->inv_b;
     const float step = a.sp->eta * inv_b;
-    if (MIRROR) backward_col_units<G, V, CPS>(a.cols, a.xprev, a.dk, a.dprev, a.n, a.clamp, step, inv_b, first, stride);
+    if (MIRROR) backward_col_units<G, V, CPS>(a.cols, a.xprev, a.dk, a.dprev, a.n, a.clamp, a.act, step, inv_b, first, stride);
     backward_row_units<G, V, CPS, FROM_S, SCATTER, DBG>(a.rows, a.bias, a.xk, a.xprev, a.dk, a.dprev, a.dbg_delta, a.dbg_grad, a.n,
-                                                        a.clamp, step, inv_b, a.update_bias, a.skip_dead, first, stride);
+                                                        a.clamp, a.act, step, inv_b, a.update_bias, a.skip_dead, first, stride);
     if (a.pdl) grid_launch_dependents();
 }
 

@@ -162,8 +162,10 @@ Geometry geometry(int cols) {
 
 int validate_cfg(const sdnn_config* cfg) {
     if (!cfg) return fail(nullptr, SDNN_ERR_INVALID_ARG, "cfg is NULL");
-    if (cfg->activation != 0) return fail(nullptr, SDNN_ERR_UNIMPLEMENTED, "only activation 0 (clamped ReLU) is implemented");
-    if (!(cfg->clamp > 0.0f) || !std::isfinite(cfg->clamp)) return fail(nullptr, SDNN_ERR_INVALID_ARG, "clamp must be finite and > 0");
+    if (cfg->activation != SDNN_ACT_CLAMPED_RELU && cfg->activation != SDNN_ACT_SIGMOID)
+        return fail(nullptr, SDNN_ERR_UNIMPLEMENTED, "activation must be 0 (clamped ReLU) or 1 (sigmoid)");
+    if (cfg->activation == SDNN_ACT_CLAMPED_RELU && (!(cfg->clamp > 0.0f) || !std::isfinite(cfg->clamp)))
+        return fail(nullptr, SDNN_ERR_INVALID_ARG, "clamp must be finite and > 0");
     if (cfg->max_batch < 1) return fail(nullptr, SDNN_ERR_INVALID_ARG, "max_batch must be >= 1");
     if (cfg->train && cfg->max_batch > 128) return fail(nullptr, SDNN_ERR_INVALID_ARG, "training handles support max_batch <= 128");
     if ((cfg->flags & SDNN_FLAG_BWD_ATOMICS) && (cfg->flags & SDNN_FLAG_BWD_CSC))
@@ -311,7 +313,7 @@ void launch_forward_gv(sdnn* h, int layer, const float* xin, float* xout, int ld
     const float* bias = h->d_bias + (size_t)layer * h->N;
     auto plan = plan_grid(h, (const void*)forward_kernel<G, V, 2>, units, chunks);
     launch_k(h, forward_kernel<G, V, 2>, dim3(plan.first, chunks), dim3(plan.second), h->pdl, rows_of(h, layer), bias, xin, xout,
-             h->N, ld, h->cfg.clamp, h->pdl ? 1 : 0, track ? (const int*)h->cs.ncols : (const int*)nullptr,
+             h->N, ld, h->cfg.clamp, h->cfg.activation, h->pdl ? 1 : 0, track ? (const int*)h->cs.ncols : (const int*)nullptr,
              track ? h->cs.flags : (int*)nullptr);
 }
 
@@ -350,6 +352,7 @@ void launch_backward_gvc(sdnn* h, int layer, int ld) {
     a.sp = h->d_sp;
     a.n = h->N;
     a.clamp = h->cfg.clamp;
+    a.act = h->cfg.activation;
     a.update_bias = h->cfg.update_bias ? 1 : 0;
     a.skip_dead = (h->cfg.flags & SDNN_FLAG_SKIP_DEAD) ? 1 : 0;
     a.pdl = h->pdl ? 1 : 0;
@@ -412,7 +415,7 @@ void launch_output_gradient(sdnn* h, int ld) {
     const long long vecs = (long long)h->N * (ld / 4);
     const int grid = (int)std::min<long long>((vecs + 255) / 256, (long long)h->sms * 8);
     output_gradient_kernel<<<grid, 256, 0, h->stream>>>(h->d_acts + (size_t)h->L * tile, h->d_yt, dl, h->N, ld, h->cfg.clamp,
-                                                        h->d_sp, h->d_loss);
+                                                        h->cfg.activation, h->d_sp, h->d_loss);
     count_launch(h);
 }
 
@@ -489,7 +492,7 @@ int infer_tile(sdnn* h, const float* x0, int cnt, float* y_out, int* cnt_out, in
     const int cols = padded_width(cnt);
     launch_transpose_in(h, x0, h->d_tile[0], cnt, cols, ld);
     int cur = 0;
-    bool track = h->compaction;
+    bool track = h->compaction && h->cfg.activation == SDNN_ACT_CLAMPED_RELU;      // sigmoid(b) is never 0: nothing ever dies
     for (int l = 0; l < h->L && track; ++l) track = h->bias_nonpositive[l] != 0;     // the zero vector must be a fixed point
     if (track) {
         const Geometry q = geometry(cols);

@@ -71,7 +71,7 @@ def test_bad_csr_is_rejected_on_the_host(pkg, mutate, needle):
 
 @pytest.mark.parametrize("kw,code", [
     (dict(max_batch=0), -1), (dict(clamp=0.0), -1), (dict(clamp=float("nan")), -1),
-    (dict(activation=1), -6), (dict(max_batch=129, train=True), -1), (dict(flags=0x3), -1),
+    (dict(activation=2), -6), (dict(max_batch=129, train=True), -1), (dict(flags=0x3), -1),
 ])
 def test_bad_config_is_rejected(pkg, kw, code):
     with pytest.raises(pkg.SdnnError) as ei:

@@ -29,7 +29,8 @@ def sdnn():
 
 
 # ----------------------------------------------------------------------------------------------
-def train_parity(torch, arrays, batches, eta, update_bias=False, flags=0, clamp=32.0, expect_live=None, sync=True):
+def train_parity(torch, arrays, batches, eta, update_bias=False, flags=0, clamp=32.0, expect_live=None, sync=True,
+                 activation="clamped_relu"):
     """Runs len(batches) SGD steps on both sides, comparing everything after every step.
 
     sync=True: before every step after the first the oracle rounds its parameters to fp32 (the library's
@@ -42,9 +43,10 @@ def train_parity(torch, arrays, batches, eta, update_bias=False, flags=0, clamp=
     rp, col, val, bias = arrays
     L, n = len(col), len(bias[0])
     B = batches[0][0].shape[0]
+    sigmoid = activation == "sigmoid"
     h = pkg.Sdnn.create(rp, col, val, bias, max_batch=B, train=True, clamp=clamp, update_bias=update_bias,
-                        flags=pkg.FLAG_KEEP_DEBUG | flags)
-    ora = OracleNet(rp, col, val, bias, clamp=clamp, update_bias=update_bias)
+                        flags=pkg.FLAG_KEEP_DEBUG | flags, activation=pkg.ACT_SIGMOID if sigmoid else pkg.ACT_CLAMPED_RELU)
+    ora = OracleNet(rp, col, val, bias, clamp=clamp, update_bias=update_bias, activation=activation)
     stats = dict(ambiguous=0, flipped=0, entries=0, worst=0.0, max_err=0.0, grad_nonzero=False)
     for step, (x0, y) in enumerate(batches):
         if sync and step > 0:
@@ -60,7 +62,7 @@ def train_parity(torch, arrays, batches, eta, update_bias=False, flags=0, clamp=
             return acts[k]
 
         proto = KinkProtocol(gpu_x, clamp=clamp)
-        out = ora.train_step(x0, y, eta, mask_hook=proto)
+        out = ora.train_step(x0, y, eta, mask_hook=None if sigmoid else proto)      # the sigmoid has no kinks
         assert proto.hard_mismatch == 0, f"{proto.hard_mismatch} derivative-mask mismatches outside the ambiguous set " \
                                          f"(worst margin/tau = {proto.worst:.3g})"
         errs = {}
@@ -197,6 +199,46 @@ def test_train_saturating_hits_upper_kink(torch_cuda):
 def test_train_scaled_configs(torch_cuda, spec, B, steps, bwd):
     st = train_parity(torch_cuda, gen.network(spec), batches_for(spec, B, steps), eta=1e-3, flags=BWD_MODES[bwd])
     print(spec.name, st)
+
+
+@pytest.mark.parametrize("bwd", sorted(BWD_MODES))
+@pytest.mark.parametrize("B", [1, 5, 16, 64])
+def test_train_sigmoid_ragged_small(torch_cuda, B, bwd):
+    """Sigmoid activation (the paper's experimental setup), ragged rows, bias update on for odd B."""
+    rng = np.random.default_rng(300 + B)
+    arrays = ragged_net(rng, n=203, layers=4, kmax=12)
+    batches = [(rng.uniform(0, 1.0, size=(B, 203)).astype(np.float32), rng.uniform(0, 1, size=(B, 203)).astype(np.float32))
+               for _ in range(3)]
+    train_parity(torch_cuda, arrays, batches, eta=0.05, update_bias=(B % 2 == 1), flags=BWD_MODES[bwd], expect_live=True,
+                 activation="sigmoid")
+
+
+def test_train_paper_setup_sigmoid_uniform_weights(torch_cuda):
+    """Section 6 of the paper: sigmoid, weights uniform in [-1, 1], eta = 0.01, MSE; 1024 x 120 net, per-sample SGD
+    (B = 1, Algorithm 1 verbatim) and a minibatch of 16 on a shallower net of 4096 neurons."""
+    spec = gen.CFG1_TRAIN.paper_setup()
+    st = train_parity(torch_cuda, gen.network(spec), batches_for(spec, 1, 4), eta=0.01, expect_live=True, activation="sigmoid")
+    print(spec.name, st)
+    spec = gen.CFG3.scaled(4096, 24).paper_setup()
+    st = train_parity(torch_cuda, gen.network(spec), batches_for(spec, 16, 2), eta=0.01, expect_live=True, activation="sigmoid")
+    print(spec.name, st)
+
+
+def test_infer_sigmoid_matches_oracle(torch_cuda):
+    pkg = sdnn()
+    spec = gen.CFG2.scaled(1024, 10).paper_setup()
+    rp, col, val, bias = gen.network(spec)
+    x0 = gen.inputs(spec, 300)
+    h = pkg.Sdnn.create(rp, col, val, bias, max_batch=256, activation=pkg.ACT_SIGMOID, flags=pkg.FLAG_SKIP_DEAD)
+    yd = torch_cuda.empty((300, spec.n), dtype=torch_cuda.float32, device="cuda")
+    cd = torch_cuda.empty(300, dtype=torch_cuda.int32, device="cuda")
+    h.infer_batch(torch_cuda.from_numpy(x0).cuda(), 300, yd, cd, None, 0)
+    xl = OracleNet(rp, col, val, bias, activation="sigmoid").infer(x0)
+    check_close(yd.cpu().numpy(), xl, "sigmoid x^L")
+    assert (cd.cpu().numpy() == spec.n).all()            # a sigmoid output is never zero
+    with pytest.raises(pkg.SdnnError):
+        h.get_liveness()                                 # nothing can die, so the flag has no effect
+    h.destroy()
 
 
 def test_train_cfg3_live_full_size(torch_cuda):

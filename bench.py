@@ -45,7 +45,16 @@ WORKLOADS = {
     "cfg2-live": (gen.CFG2.live(), "infer", 1024, 60000),
     "cfg4": (gen.CFG4, "infer", 1024, 60000),
     "cfg4-live": (gen.CFG4.live(), "infer", 1024, 60000),
+    # the paper's own training setup (Section 6): sigmoid, weights uniform in [-1, 1], eta = 0.01
+    "cfg3-paper": (gen.CFG3.paper_setup(), "train", 64, 64),
+    "cfg5-paper": (gen.CFG5.paper_setup(), "train", 16, 16),
+    "cfg1-paper": (gen.CFG1_TRAIN.paper_setup(), "train", 1, 1),
 }
+
+
+def setup_of(spec):
+    """(activation name, activation code, eta) of a workload: the paper's setup for the '-paper' nets."""
+    return ("sigmoid", 1, 1e-2) if spec.name.endswith("-paper") else ("clamped_relu", 0, ETA)
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
@@ -117,12 +126,13 @@ def oracle_train_sample(spec, B, layers, steps, warmup):
     """Times the float64 oracle's train step on the first `layers` layers of the net (full N, full B)."""
     from oracle import OracleNet
     sl = spec.sliced(layers)
-    ora = OracleNet(*gen.network(sl))
+    act, _, eta = setup_of(spec)
+    ora = OracleNet(*gen.network(sl), activation=act)
     times = []
     for s in range(warmup + steps):
         x0, y = gen.inputs(sl, B, step=s), gen.targets(sl, B, step=s)
         t = time.perf_counter()
-        ora.train_step(x0, y, ETA, keep=())
+        ora.train_step(x0, y, eta, keep=())
         dt = time.perf_counter() - t
         if s >= warmup:
             times.append(dt)
@@ -133,7 +143,7 @@ def oracle_train_sample(spec, B, layers, steps, warmup):
 def oracle_infer_sample(spec, inputs, layers, steps, warmup):
     from oracle import OracleNet
     sl = spec.sliced(layers)
-    ora = OracleNet(*gen.network(sl))
+    ora = OracleNet(*gen.network(sl), activation=setup_of(spec)[0])
     x0 = gen.inputs(sl, inputs)
     times = []
     for s in range(warmup + steps):
@@ -186,7 +196,7 @@ def metric_name(kind):
 def workload_config(wname, spec, kind, batch):
     cfg = {"workload": f"{wname}: {spec.name} {spec.n} neurons x {spec.layers} layers, {spec.k} nnz/row, "
                        + (f"minibatch {batch}, fresh minibatch per step" if kind == "train" else f"batch tile {batch}"),
-           "mode": "dense (no data-dependent skipping)",
+           "mode": "dense (no data-dependent skipping)", "activation": setup_of(spec)[0],
            "l2": "working set per step (weights + activations) is larger than L2; no explicit flush"
            if spec.total_nnz * 8 > 256e6 else "explicit L2 flush (256 MB write) before every timed step"}
     return cfg
@@ -245,8 +255,9 @@ def main():
     t_setup = time.perf_counter()
     L, N = spec.layers, spec.n
     flags = args.flags
+    act_name, act_code, eta = setup_of(spec)
     h = pkg.Sdnn.create_deferred(L, N, [spec.nnz_per_layer] * L, max_batch=batch, train=(kind == "train"),
-                                 flags=flags, stream=stream.cuda_stream, device=local_rank)
+                                 flags=flags, stream=stream.cuda_stream, device=local_rank, activation=act_code)
     for l in range(L):
         h.load_layer(l, *gen.layer(spec, l))
     h.finalize()
@@ -269,10 +280,10 @@ def main():
             hy = [y.cpu().pin_memory() for y in ys]
 
             def step(i):
-                h.train_step(xs[i], ys[i], batch, ETA)
+                h.train_step(xs[i], ys[i], batch, eta)
 
             def step_e2e(i):
-                return h.train_step(hx[i], hy[i], batch, ETA, want_loss=True, host=True)
+                return h.train_step(hx[i], hy[i], batch, eta, want_loss=True, host=True)
 
             h2d, d2h = 2 * batch * N * 4, 4
         else:

@@ -241,6 +241,53 @@ def test_infer_sigmoid_matches_oracle(torch_cuda):
     h.destroy()
 
 
+@pytest.mark.parametrize("bwd", sorted(BWD_MODES))
+@pytest.mark.parametrize("variant", ["dead", "live", "half"])
+def test_train_skipping_dead_rows_gives_dense_results(torch_cuda, bwd, variant):
+    """SDNN_FLAG_SKIP_DEAD in training (units of rows whose delta is zero for every input skip their entries):
+    same parity as dense mode on a net that is dead from layer 3 on, on a live one, and on a net where half of the
+    output neurons have a target equal to their output (so whole units really are skipped while others work)."""
+    pkg = sdnn()
+    spec = gen.CFG3.scaled(1024, 8)
+    if variant != "dead":
+        spec = spec.live()
+    arrays = gen.network(spec)
+    batches = batches_for(spec, 16, 2)
+    if variant == "half":
+        ora = OracleNet(*arrays)
+        fixed = []
+        for x0, y in batches:
+            xl = ora.infer(x0).astype(np.float32)
+            y = y.copy(); y[:, :512] = xl[:, :512]           # zero error, hence zero delta^L, on the first 512 neurons
+            fixed.append((x0, y))
+        batches = fixed[:1]                                   # the oracle's own weights must not have moved: one step
+    train_parity(torch_cuda, arrays, batches, eta=1e-3, flags=BWD_MODES[bwd] | pkg.FLAG_SKIP_DEAD,
+                 expect_live=(variant != "dead"))
+
+
+def test_infer_many_tiles_with_dead_inputs_dropped(torch_cuda):
+    """Several tiles (the last one ragged) with SDNN_FLAG_SKIP_DEAD, host buffers: every tile starts from a fresh
+    column map, and the outputs land at the right inputs."""
+    pkg = sdnn()
+    spec = gen.CFG2.scaled(512, 6).live()
+    rp, col, val, bias = gen.network(spec)
+    cnt = 1500
+    x0 = gen.inputs(spec, cnt)
+    x0[np.arange(cnt) % 3 != 0] = 0.0                         # two thirds of the inputs die at once
+    h = pkg.Sdnn.create(rp, col, val, bias, max_batch=512, flags=pkg.FLAG_SKIP_DEAD)
+    y = np.empty((cnt, spec.n), dtype=np.float32); c = np.empty(cnt, dtype=np.int32)
+    idx = np.empty(cnt * spec.n, dtype=np.int32)
+    total = h.infer_batch(x0, cnt, y, c, idx, cnt * spec.n, want_total=True, host=True)
+    h.destroy()
+    xl = OracleNet(rp, col, val, bias).infer(x0)
+    check_close(y, xl, "x^L over four tiles")
+    assert not y[np.arange(cnt) % 3 != 0].any() and total == int(c.sum()) and total > 0
+    starts = np.concatenate([[0], np.cumsum(c)])
+    for b in (0, 3, 511, 513, 1023, 1026, 1497):
+        ids = idx[starts[b]:starts[b + 1]]
+        assert np.array_equal(ids, np.flatnonzero(y[b] != 0.0))
+
+
 def test_train_cfg3_live_full_size(torch_cuda):
     """Config 3 at full size (16384 x 480, B = 64), live companion, one step."""
     spec = gen.CFG3.live()

@@ -117,22 +117,31 @@ __device__ __forceinline__ void lane_store(float* p, const Lane<8>& v) {
                  :: "l"(p), "f"(v.a.x), "f"(v.a.y), "f"(v.a.z), "f"(v.a.w), "f"(v.b.x), "f"(v.b.y), "f"(v.b.z), "f"(v.b.w) : "memory");
 }
 
-#define SDNN_F4_FMA(W, X, A) A.x = fmaf(W, X.x, A.x); A.y = fmaf(W, X.y, A.y); A.z = fmaf(W, X.z, A.z); A.w = fmaf(W, X.w, A.w);
-__device__ __forceinline__ void lane_fma(float w, const Lane<4>& x, Lane<4>& acc) { SDNN_F4_FMA(w, x.a, acc.a) }
-__device__ __forceinline__ void lane_fma(float w, const Lane<8>& x, Lane<8>& acc) { SDNN_F4_FMA(w, x.a, acc.a) SDNN_F4_FMA(w, x.b, acc.b) }
-
-// Partial dot product of one lane: its batch columns of delta (d) against those of x.  Written with explicit
-// roundings and a fixed order so that the row pass and the column pass, which swap the roles of the gathered
-// and the resident operand, produce the same bits (a*b and fma(a,b,c) are symmetric in a and b).
-__device__ __forceinline__ float dot_f4(const float4& d, const float4& x, float s) {
-    return __fmaf_rn(d.w, x.w, __fmaf_rn(d.z, x.z, __fmaf_rn(d.y, x.y, __fmaf_rn(d.x, x.x, s))));
+// acc += w * x with packed two-wide fp32 FMAs (sm_100): half the issue slots of scalar FMAs
+__device__ __forceinline__ void f4_fma(float w, const float4& x, float4& a) {
+    const float2 ww = make_float2(w, w);
+    const float2 lo = __ffma2_rn(ww, make_float2(x.x, x.y), make_float2(a.x, a.y));
+    const float2 hi = __ffma2_rn(ww, make_float2(x.z, x.w), make_float2(a.z, a.w));
+    a = make_float4(lo.x, lo.y, hi.x, hi.y);
 }
+__device__ __forceinline__ void lane_fma(float w, const Lane<4>& x, Lane<4>& acc) { f4_fma(w, x.a, acc.a); }
+__device__ __forceinline__ void lane_fma(float w, const Lane<8>& x, Lane<8>& acc) { f4_fma(w, x.a, acc.a); f4_fma(w, x.b, acc.b); }
+
+// Partial dot product of one lane: its batch columns of delta (d) against those of x, even and odd columns in
+// the two halves of packed FMAs, added at the end.  Written with explicit roundings and a fixed order so that the
+// row pass and the column pass, which swap the roles of the gathered and the resident operand, produce the same
+// bits (a*b and fma(a,b,c) are symmetric in a and b).
 __device__ __forceinline__ float lane_dot(const Lane<4>& d, const Lane<4>& x) {
-    return __fmaf_rn(d.a.w, x.a.w, __fmaf_rn(d.a.z, x.a.z, __fmaf_rn(d.a.y, x.a.y, __fmul_rn(d.a.x, x.a.x))));
+    float2 p = __fmul2_rn(make_float2(d.a.x, d.a.y), make_float2(x.a.x, x.a.y));
+    p = __ffma2_rn(make_float2(d.a.z, d.a.w), make_float2(x.a.z, x.a.w), p);
+    return __fadd_rn(p.x, p.y);
 }
 __device__ __forceinline__ float lane_dot(const Lane<8>& d, const Lane<8>& x) {
-    const float s = __fmaf_rn(d.a.w, x.a.w, __fmaf_rn(d.a.z, x.a.z, __fmaf_rn(d.a.y, x.a.y, __fmul_rn(d.a.x, x.a.x))));
-    return dot_f4(d.b, x.b, s);
+    float2 p = __fmul2_rn(make_float2(d.a.x, d.a.y), make_float2(x.a.x, x.a.y));
+    p = __ffma2_rn(make_float2(d.a.z, d.a.w), make_float2(x.a.z, x.a.w), p);
+    p = __ffma2_rn(make_float2(d.b.x, d.b.y), make_float2(x.b.x, x.b.y), p);
+    p = __ffma2_rn(make_float2(d.b.z, d.b.w), make_float2(x.b.z, x.b.w), p);
+    return __fadd_rn(p.x, p.y);
 }
 
 // d *= f'(z) with f' taken from the stored output x

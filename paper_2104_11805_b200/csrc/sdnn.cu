@@ -94,6 +94,9 @@ struct sdnn {
     // staging for the *_host entry points (allocated on first use)
     float* d_stage_a = nullptr;
     float* d_stage_b = nullptr;
+    float* d_stage_a2 = nullptr;        // second input stage of sdnn_infer_batch_host: tile t+1 is copied while tile t computes
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t ev_copied[2] = {nullptr, nullptr}, ev_consumed[2] = {nullptr, nullptr};
     int* d_stage_cnt = nullptr;
     int* d_stage_idx = nullptr;
     int64_t stage_idx_cap = 0;
@@ -604,6 +607,9 @@ void sdnn_destroy(sdnn_t* h) {
     if (h->stream || h->own_stream) cudaStreamSynchronize(h->stream);
     if (h->graph) cudaGraphExecDestroy(h->graph);
     for (cudaEvent_t e : h->ev) if (e) cudaEventDestroy(e);
+    for (cudaEvent_t e : h->ev_copied) if (e) cudaEventDestroy(e);
+    for (cudaEvent_t e : h->ev_consumed) if (e) cudaEventDestroy(e);
+    if (h->copy_stream) { cudaStreamSynchronize(h->copy_stream); cudaStreamDestroy(h->copy_stream); }
     for (void* p : h->allocs) cudaFree(p);
     if (h->own_stream) cudaStreamDestroy(h->stream);
     delete h;
@@ -890,15 +896,33 @@ int sdnn_infer_batch_host(sdnn_t* h, const float* x0, int64_t n_inputs, float* y
     const bool want_sets = nz_count_out || nz_index_out || nz_total_out;
     if (want_sets) CU(h, cudaMemsetAsync(h->d_running, 0, sizeof(long long), h->stream));
     const int T = h->cfg.max_batch;
-    for (int64_t t0 = 0; t0 < n_inputs; t0 += T) {
+    // two input stages and a copy stream: the copy of tile t+1 runs under the layers of tile t
+    if (!h->copy_stream) {
+        CU(h, cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking));
+        for (int q = 0; q < 2; ++q) {
+            CU(h, cudaEventCreateWithFlags(&h->ev_copied[q], cudaEventDisableTiming));
+            CU(h, cudaEventCreateWithFlags(&h->ev_consumed[q], cudaEventDisableTiming));
+        }
+        if ((rc = dev_alloc(h, &h->d_stage_a2, (size_t)h->cfg.max_batch * h->N, false))) return rc;
+    }
+    float* stage[2] = {h->d_stage_a, h->d_stage_a2};
+    CU(h, cudaEventRecord(h->ev_consumed[0], h->stream));       // the stages may still be read by earlier work on the stream
+    CU(h, cudaEventRecord(h->ev_consumed[1], h->stream));
+    int64_t tile_no = 0;
+    for (int64_t t0 = 0; t0 < n_inputs; t0 += T, ++tile_no) {
         const int cnt = (int)((n_inputs - t0 < T) ? (n_inputs - t0) : T);
         const size_t bytes = (size_t)cnt * h->N * sizeof(float);
-        CU(h, cudaMemcpyAsync(h->d_stage_a, x0 + (size_t)t0 * h->N, bytes, cudaMemcpyHostToDevice, h->stream));
-        rc = infer_tile(h, h->d_stage_a, cnt, y_out ? h->d_stage_b : nullptr, nz_count_out ? h->d_stage_cnt : nullptr,
+        const int q = (int)(tile_no & 1);
+        CU(h, cudaStreamWaitEvent(h->copy_stream, h->ev_consumed[q], 0));
+        CU(h, cudaMemcpyAsync(stage[q], x0 + (size_t)t0 * h->N, bytes, cudaMemcpyHostToDevice, h->copy_stream));
+        CU(h, cudaEventRecord(h->ev_copied[q], h->copy_stream));
+        CU(h, cudaStreamWaitEvent(h->stream, h->ev_copied[q], 0));
+        rc = infer_tile(h, stage[q], cnt, y_out ? h->d_stage_b : nullptr, nz_count_out ? h->d_stage_cnt : nullptr,
                         nz_index_out ? h->d_stage_idx : nullptr, nz_index_capacity, want_sets);
         if (rc) return rc;
         if (y_out) CU(h, cudaMemcpyAsync(y_out + (size_t)t0 * h->N, h->d_stage_b, bytes, cudaMemcpyDeviceToHost, h->stream));
         if (nz_count_out) CU(h, cudaMemcpyAsync(nz_count_out + t0, h->d_stage_cnt, (size_t)cnt * sizeof(int), cudaMemcpyDeviceToHost, h->stream));
+        CU(h, cudaEventRecord(h->ev_consumed[q], h->stream));
     }
     long long total = 0;
     if (want_sets) CU(h, cudaMemcpyAsync(&total, h->d_running, sizeof total, cudaMemcpyDeviceToHost, h->stream));

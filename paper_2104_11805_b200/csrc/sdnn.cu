@@ -626,6 +626,9 @@ int sdnn_create_deferred(sdnn_t** out, int32_t n_layers, int32_t n_neurons, cons
     for (int l = 0; l < n_layers; ++l)
         if (nnz_per_layer[l] < 0 || nnz_per_layer[l] > INT32_MAX)
             return fail(nullptr, SDNN_ERR_INVALID_ARG, "layer %d: stored-entry count outside [0, 2^31)", l);
+    // the kernels address a tile row with a 32-bit multiply-add: one tile must stay below 4 GiB
+    if ((int64_t)n_neurons * padded_width(cfg->max_batch) * (int64_t)sizeof(float) >= (1LL << 32))
+        return fail(nullptr, SDNN_ERR_INVALID_ARG, "n_neurons * padded(max_batch) * 4 bytes must stay below 4 GiB: lower max_batch (inference works in tiles of max_batch inputs)");
 
     int ndev = 0;
     cudaError_t e = cudaGetDeviceCount(&ndev);

@@ -96,3 +96,11 @@ def test_null_handle_calls_do_not_crash(pkg):
     assert lib.sdnn_get_weights(None, 0, None, None) == -1
     assert lib.sdnn_kernel_launches(None) == 0
     lib.sdnn_destroy(None)
+
+
+def test_tile_beyond_4_gib_is_rejected_before_any_device_work(pkg):
+    """One activation tile (n_neurons x padded max_batch floats) must stay below 4 GiB; checked on the host."""
+    nnz = np.zeros(1, dtype=np.int64)
+    with pytest.raises(pkg.SdnnError) as ei:
+        pkg.Sdnn.create_deferred(1, 1 << 20, nnz, max_batch=1024)
+    assert ei.value.code == -1 and "4 GiB" in ei.value.message

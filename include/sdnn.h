@@ -80,7 +80,9 @@ typedef struct {
     int32_t  activation;   /* SDNN_ACT_CLAMPED_RELU or SDNN_ACT_SIGMOID */
     float    clamp;        /* upper clamp of the clamped ReLU, e.g. 32.0f; must be > 0 (ignored by the sigmoid) */
     int32_t  max_batch;    /* train: largest minibatch B; inference: batch tile (inputs processed together) */
-    int32_t  train;        /* 0: inference only (no stored activations); 1: sdnn_train_step allowed */
+    int32_t  train;        /* 0: inference only (no stored activations); 1: sdnn_train_step allowed.  A training
+                              handle stores x^0..x^L of one minibatch and, unless SDNN_FLAG_BWD_ATOMICS is set, a second
+                              (transposed) copy of the indices and values of every layer but the first */
     int32_t  update_bias;  /* 1: b^k <- b^k - eta * mean_b delta^k_b (bias read as a column of W^k); 0: bias frozen */
     uint32_t flags;        /* SDNN_FLAG_* */
     void*    cuda_stream;  /* cudaStream_t to issue work on; NULL = a stream the handle creates, which orders

@@ -374,6 +374,33 @@ def test_infer_dropping_dead_inputs_gives_dense_results(torch_cuda, variant):
         assert want[-1] == 0 and t0 == 0
 
 
+@pytest.mark.parametrize("variant", ["base", "live"])
+def test_infer_cfg4_in_the_benchmark_launch_shape_sampled(torch_cuda, variant):
+    """Config 4 at full size in the launch shape bench.py times (tiles of 1024 inputs; one full tile and a ragged
+    one).  Inputs are independent of one another, so the oracle checks a sample of them one by one."""
+    pkg = sdnn()
+    spec = gen.CFG4 if variant == "base" else gen.CFG4.live()
+    rp, col, val, bias = gen.network(spec)
+    cnt = 1100
+    x0 = gen.inputs(spec, cnt, start=30000)
+    h = pkg.Sdnn.create(rp, col, val, bias, max_batch=1024)
+    yd = torch_cuda.empty((cnt, spec.n), dtype=torch_cuda.float32, device="cuda")
+    cd = torch_cuda.empty(cnt, dtype=torch_cuda.int32, device="cuda")
+    h.infer_batch(torch_cuda.from_numpy(x0).cuda(), cnt, yd, cd, None, 0)
+    h.destroy()
+    sample = np.unique(np.concatenate([[0, 1, 255, 256, 511, 1023, 1024, 1099],
+                                       np.random.default_rng(9).integers(0, cnt, size=24)]))
+    xl = OracleNet(rp, col, val, bias).infer(x0[sample])
+    y = yd[torch_cuda.from_numpy(sample).cuda()].cpu().numpy()
+    check_close(y, xl, "sampled x^L")
+    counts = cd.cpu().numpy()
+    assert np.array_equal(counts[sample], (y != 0.0).sum(axis=1))
+    if variant == "base":
+        assert not xl.any() and not counts.any()
+    else:
+        assert xl.any()
+
+
 # ---------------------------------------------------------------------------------------------- API behaviour on a device
 def test_capacity_too_small_reports_needed(torch_cuda):
     pkg = sdnn()

@@ -211,6 +211,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=None, help="use only the first LAYERS layers (profiling captures)")
     ap.add_argument("--inputs", type=int, default=None, help="inference: number of inputs per call")
+    ap.add_argument("--tile", type=int, default=None, help="inference: batch tile (max_batch of the handle)")
+    ap.add_argument("--net", default=None, metavar="N,L",
+                    help="same recipe at another size, e.g. 65536,1920 for the deeper grids of the paper's Table 2")
     ap.add_argument("--flags", type=lambda s: int(s, 0), default=0, help="extra SDNN_FLAG_* bits")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -219,6 +222,11 @@ def main():
     if args.warmup < 3 and args.layers is None:
         args.warmup = 3
     spec, kind, batch, n_inputs = WORKLOADS[args.workload]
+    if args.tile and kind == "infer":
+        batch = args.tile
+    if args.net:
+        n_, l_ = (int(v) for v in args.net.split(","))
+        spec = spec.scaled(n_, l_)
     if args.layers:
         spec = spec.sliced(args.layers)
     if args.inputs and kind == "infer":
@@ -415,24 +423,27 @@ def main():
                  "step_bytes": (fwd_bytes + bwd_bytes) * L,
                  "step_GBps": (fwd_bytes + bwd_bytes) * L / (ms_per_step * 1e-3) / 1e9}
     else:
+        batch = h.infer_tile_width()           # the library narrows the tile when two of them would not fit in L2
         tiles = (n_inputs + batch - 1) // batch
         dom = "forward_kernel"
         per_launch_ms = ms_per_step / (tiles * L)      # includes the (small) transpose and count kernels of each tile
         # per launch: the layer's indices and values once, the activation tile read and written once
         alg = 8 * nnz_l + 2 * N * min(batch, n_inputs) * 4
-        extra = {"tiles": tiles, "note": "launch time = call time / forward launches (upper bound)"}
+        extra = {"tiles": tiles, "tile_inputs": batch, "note": "launch time = call time / forward launches (upper bound)"}
     # what bounds these launches instead of HBM: random gathers of tile rows out of L2 (measured now, on this device)
     if kind == "train":
         row_bytes, gathers = 4 * ld, (2 if dom == "backward_kernel" else 1) * nnz_l
         table_rows = 1 << (N - 1).bit_length()
     else:
-        row_bytes, gathers = 512, nnz_l * (min(batch, n_inputs) * 4 + 511) // 512
-        table_rows = 1 << max(0, (N * min(batch, n_inputs) * 4 // 512 - 1).bit_length())
+        row_bytes = min(1024, 4 * (1 << (min(batch, n_inputs) - 1).bit_length()))      # one chunk of a tile row
+        gathers = nnz_l * ((min(batch, n_inputs) * 4 + row_bytes - 1) // row_bytes)
+        table_rows = 1 << max(0, (N * min(batch, n_inputs) * 4 // row_bytes - 1).bit_length())
     table_rows = min(table_rows, (1 << 30) // row_bytes)
     try:
-        gather_rate = pkg.probe_gather_rate(min(row_bytes, 512), table_rows)
+        gather_rate = pkg.probe_gather_rate(row_bytes, table_rows)
         floor_ms = gathers / gather_rate * 1e3
-        extra["gather_bound"] = {"probe_rows_per_s": gather_rate, "row_bytes": min(row_bytes, 512), "table_rows": table_rows,
+        extra["gather_bound"] = {"probe_rows_per_s": gather_rate, "row_bytes": row_bytes, "table_rows": table_rows,
+                                 "note": "uniformly random rows: a layer whose pattern is local can beat this floor",
                                  "gathers_per_launch": gathers, "floor_ms_per_launch": floor_ms,
                                  "frac_of_gather_floor": floor_ms / per_launch_ms if per_launch_ms else None}
     except Exception as exc:      # the probe is a diagnostic; the line stands without it

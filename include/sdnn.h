@@ -125,7 +125,9 @@ int sdnn_finalize(sdnn_t* h);
  *   nz_index_out  device int32[nz_index_capacity]: for input 0, 1, ... in turn, the ascending
  *                 neuron ids i with x^L(i) != 0, concatenated; or NULL
  *   nz_total_out  host int64*: total number of ids (sum of counts), or NULL
- * The batch is processed in tiles of cfg.max_batch inputs.  If nz_index_out is given and the
+ * The batch is processed in tiles of at most cfg.max_batch inputs (narrower ones, a power of two >= 128, when two
+ * activation tiles of max_batch inputs would not fit in the L2 cache and the sparsity pattern is not local: the
+ * gathers of a layer then come out of L2 instead of HBM).  If nz_index_out is given and the
  * capacity is too small, only the ids at positions below the capacity are written, *nz_total_out
  * (if given) holds the needed capacity and the call returns SDNN_ERR_INVALID_ARG; y_out and
  * nz_count_out are still valid.  n_inputs == 0 is a valid no-op.
@@ -133,6 +135,9 @@ int sdnn_finalize(sdnn_t* h);
 int sdnn_infer_batch(sdnn_t* h, const float* x0, int64_t n_inputs, float* y_out,
                      int32_t* nz_count_out, int32_t* nz_index_out, int64_t nz_index_capacity,
                      int64_t* nz_total_out);
+
+/* Inputs per tile that sdnn_infer_batch uses on this handle (see above); 0 before sdnn_finalize. */
+int32_t sdnn_infer_tile_width(const sdnn_t* h);
 
 /* Same call with every array in HOST memory (pinned or pageable); the library stages the
  * copies itself, tile by tile, and returns when the outputs are in place. */
@@ -198,7 +203,8 @@ int sdnn_mirror_mismatches(sdnn_t* h, int32_t layer, int64_t* count_out);
 
 /*
  * Measures what bounds the layer kernels on the current device (diagnostic; the paper has no counterpart): the
- * rate at which an SM array can gather random rows of `row_bytes` bytes (16 .. 512, a power of two) out of a table
+ * rate at which an SM array can gather random rows of `row_bytes` bytes (16 .. 1024, a power of two; read with the
+ * layer kernels' own 256-bit accesses) out of a table
  * of `table_rows` rows (a power of two; at most 1 GiB in all) that sits in L2 or, if larger, in HBM, with nothing
  * else competing for the load pipe.  A layer with nnz stored entries and a padded batch of ld inputs gathers
  * nnz rows of 4*ld bytes in the forward product and 2*nnz in the backward launch (transposed realisation), so

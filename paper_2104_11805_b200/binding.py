@@ -54,6 +54,7 @@ _PROTOS = {
     "sdnn_get_liveness": (ctypes.c_int, [_vp, _vp]),
     "sdnn_infer_noalloc": (ctypes.c_int, [_i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _f32, _vp]),
     "sdnn_kernel_launches": (_i64, [_vp]),
+    "sdnn_infer_tile_width": (_i32, [_vp]),
     "sdnn_device_bytes": (_i64, [_vp]),
     "sdnn_destroy": (None, [_vp]),
     "sdnn_last_error": (ctypes.c_char_p, [_vp]),
@@ -247,6 +248,10 @@ class Sdnn:
         out = np.empty(self.n_layers, dtype=np.int32)
         self._check(self._lib.sdnn_get_liveness(self._h, out.ctypes.data))
         return out
+
+    def infer_tile_width(self):
+        """Inputs per tile that infer_batch uses on this handle."""
+        return int(self._lib.sdnn_infer_tile_width(self._h))
 
     def kernel_launches(self):
         return int(self._lib.sdnn_kernel_launches(self._h))

@@ -875,25 +875,26 @@ __global__ void __launch_bounds__(256) expand_kernel(ColState s, const float* __
 // ---------------------------------------------------------------------------------------------
 // Probe of the bound of the layer kernels: nothing but random row gathers out of a table, with the indices made
 // in registers (a linear congruential sequence per lane group, masked to the table), so that only the gathers
-// use the load pipe.  G lanes of 16 bytes per row, eight gathers in flight per lane.
-template <int G>
+// use the load pipe.  G lanes of V floats per row (the layer kernels' own access width), eight gathers in flight
+// per lane.
+template <int G, int V>
 __global__ void __launch_bounds__(256)
 gather_probe_kernel(const float* __restrict__ table, float* __restrict__ sink, unsigned row_mask, int per_group, unsigned seed) {
     const int tid = blockIdx.x * blockDim.x + threadIdx.x;
     const int sub = threadIdx.x % G;
     unsigned st = (unsigned)(tid / G) * 2654435761u + seed;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float acc = 0.f;
     for (int q = 0; q < per_group; q += 8) {
         unsigned c[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) { st = st * 1664525u + 1013904223u; c[u] = (st >> 8) & row_mask; }
-        float4 v[8];
+        Lane<V> v[8];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) v[u] = gather_f4(table + (size_t)c[u] * (4 * G) + sub * 4);
+        for (int u = 0; u < 8; ++u) lane_gather(v[u], table + (size_t)c[u] * (V * G) + sub * V);
 #pragma unroll
-        for (int u = 0; u < 8; ++u) { acc.x += v[u].x; acc.y += v[u].y; acc.z += v[u].z; acc.w += v[u].w; }
+        for (int u = 0; u < 8; ++u) acc += lane_sum(v[u]);
     }
-    if (acc.x + acc.y + acc.z + acc.w == 123.456f) sink[0] = acc.x;      // the table is all zero: never taken, keeps the loads alive
+    if (acc == 123.456f) sink[0] = acc;      // the table is all zero: never taken, keeps the loads alive
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -85,6 +85,8 @@ struct sdnn {
     int* d_tile_cnt = nullptr;
     long long* d_offs = nullptr;
     long long* d_running = nullptr;
+    int l2_bytes = 0;
+    std::vector<char> local_pattern;    // per layer: blocks of 1024 rows touch few distinct columns (see infer_tile_width)
     bool compaction = false;            // SDNN_FLAG_SKIP_DEAD asked for; effective while no bias is positive
     std::vector<char> bias_nonpositive; // per layer
     ColState cs{};                      // device state of the live-column bookkeeping
@@ -542,6 +544,24 @@ int infer_tile(sdnn* h, const float* x0, int cnt, float* y_out, int* cnt_out, in
     return SDNN_OK;
 }
 
+// Inputs per inference tile.  The gathers of a layer read the whole activation tile at random, so the two
+// ping-pong tiles should sit in L2: unless every layer's pattern is local (each block of rows reads few tile rows,
+// which the cache then holds whatever the tile's size), the tile is narrowed to the widest power of two >= 128
+// for which both tiles take at most 55 % of the L2.
+int infer_tile_width(const sdnn* h) {
+    int T = h->cfg.max_batch;
+    bool local = true;
+    for (char c : h->local_pattern) local = local && c;
+    if (local || h->l2_bytes <= 0) return T;
+    const double budget = 0.55 * (double)h->l2_bytes;
+    while (T > 128 && 2.0 * h->N * padded_width(T) * sizeof(float) > budget) {
+        int p = 128;
+        while (p * 2 < T) p *= 2;      // largest power of two below T (at least 128)
+        T = p;
+    }
+    return T;
+}
+
 int check_infer_args(sdnn* h, const float* x0, int64_t n_inputs, int32_t* idx, int64_t cap) {
     if (!h) return SDNN_ERR_INVALID_ARG;
     if (!h->finalized) return fail(h, SDNN_ERR_STATE, "handle is not finalized");
@@ -599,6 +619,7 @@ const char* sdnn_version(void) { return "sdnn 0.2 (sm_100a)"; }
 const char* sdnn_last_error(const sdnn_t* h) { return h ? h->err.c_str() : g_create_error.c_str(); }
 
 int64_t sdnn_kernel_launches(const sdnn_t* h) { return h ? h->launches : 0; }
+int32_t sdnn_infer_tile_width(const sdnn_t* h) { return (h && h->finalized) ? infer_tile_width(h) : 0; }
 int64_t sdnn_device_bytes(const sdnn_t* h) { return h ? h->dev_bytes : 0; }
 
 void sdnn_destroy(sdnn_t* h) {
@@ -648,6 +669,7 @@ int sdnn_create_deferred(sdnn_t** out, int32_t n_layers, int32_t n_neurons, cons
     }
     if ((e = cudaDeviceGetAttribute(&h->sms, cudaDevAttrMultiProcessorCount, h->device)) != cudaSuccess || h->sms < 1)
         return bail(cuda_fail(h, e, "cudaDeviceGetAttribute(multiprocessor count)"));
+    if (cudaDeviceGetAttribute(&h->l2_bytes, cudaDevAttrL2CacheSize, h->device) != cudaSuccess) { cudaGetLastError(); h->l2_bytes = 0; }
     if (!h->stream) {   // the legacy default stream cannot be captured into a graph: use a blocking stream of our own,
                         // which still orders itself against work on the legacy default stream
         if ((e = cudaStreamCreate(&h->stream)) != cudaSuccess) { h->stream = nullptr; return bail(cuda_fail(h, e, "cudaStreamCreate")); }
@@ -693,6 +715,7 @@ int sdnn_create_deferred(sdnn_t** out, int32_t n_layers, int32_t n_neurons, cons
         if ((rc = dev_alloc(h, &h->d_running, 1, true))) return bail(rc);
         h->compaction = (cfg->flags & SDNN_FLAG_SKIP_DEAD) != 0;
         h->bias_nonpositive.assign(n_layers, 0);
+        h->local_pattern.assign(n_layers, 0);
         if (h->compaction) {
             int* blk = nullptr;
             if ((rc = dev_alloc(h, &blk, 3 * (size_t)h->ld_max + 4, true))) return bail(rc);
@@ -798,6 +821,16 @@ int sdnn_load_layer(sdnn_t* h, int32_t layer, const int32_t* row_ptr, const int3
         for (int i = 0; i < N && nonpos; ++i) nonpos = !(bias[i] > 0.0f);
         h->bias_nonpositive[layer] = nonpos ? 1 : 0;
     }
+    {   // locality of the pattern: distinct columns touched by each block of 1024 consecutive rows, summed over the blocks
+        std::vector<int> stamp(N, -1);
+        int64_t distinct = 0;
+        for (int i = 0; i < N; ++i) {
+            const int blk = i >> 10;
+            for (int p = row_ptr[i]; p < row_ptr[i + 1]; ++p)
+                if (stamp[col_idx[p]] != blk) { stamp[col_idx[p]] = blk; ++distinct; }
+        }
+        h->local_pattern[layer] = distinct <= 2 * (int64_t)N ? 1 : 0;
+    }
     h->loaded[layer] = 1;
     return SDNN_OK;
 }
@@ -868,7 +901,7 @@ int sdnn_infer_batch(sdnn_t* h, const float* x0, int64_t n_inputs, float* y_out,
     CU(h, cudaSetDevice(h->device));
     const bool want_sets = nz_count_out || nz_index_out || nz_total_out;
     if (want_sets) CU(h, cudaMemsetAsync(h->d_running, 0, sizeof(long long), h->stream));
-    const int T = h->cfg.max_batch;
+    const int T = infer_tile_width(h);
     for (int64_t t0 = 0; t0 < n_inputs; t0 += T) {
         const int cnt = (int)((n_inputs - t0 < T) ? (n_inputs - t0) : T);
         rc = infer_tile(h, x0 + (size_t)t0 * h->N, cnt, y_out ? y_out + (size_t)t0 * h->N : nullptr,
@@ -898,7 +931,7 @@ int sdnn_infer_batch_host(sdnn_t* h, const float* x0, int64_t n_inputs, float* y
     }
     const bool want_sets = nz_count_out || nz_index_out || nz_total_out;
     if (want_sets) CU(h, cudaMemsetAsync(h->d_running, 0, sizeof(long long), h->stream));
-    const int T = h->cfg.max_batch;
+    const int T = infer_tile_width(h);
     // two input stages and a copy stream: the copy of tile t+1 runs under the layers of tile t
     if (!h->copy_stream) {
         CU(h, cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking));
@@ -1074,12 +1107,12 @@ int sdnn_get_liveness(sdnn_t* h, int32_t* live_inputs_out) {
 // Gather-rate probe (see sdnn_probe_gather_rate in the header).
 namespace {
 
-template <int G>
+template <int G, int V>
 float run_gather_probe(const float* table, float* sink, unsigned mask, int per_group, int grid, cudaStream_t st, int reps,
                        cudaEvent_t a, cudaEvent_t b) {
-    for (int i = 0; i < 2; ++i) gather_probe_kernel<G><<<grid, 256, 0, st>>>(table, sink, mask, per_group, 17u + i);
+    for (int i = 0; i < 2; ++i) gather_probe_kernel<G, V><<<grid, 256, 0, st>>>(table, sink, mask, per_group, 17u + i);
     cudaEventRecord(a, st);
-    for (int i = 0; i < reps; ++i) gather_probe_kernel<G><<<grid, 256, 0, st>>>(table, sink, mask, per_group, 101u + i);
+    for (int i = 0; i < reps; ++i) gather_probe_kernel<G, V><<<grid, 256, 0, st>>>(table, sink, mask, per_group, 101u + i);
     cudaEventRecord(b, st);
     cudaEventSynchronize(b);
     float ms = 0.f;
@@ -1092,8 +1125,9 @@ float run_gather_probe(const float* table, float* sink, unsigned mask, int per_g
 extern "C" int sdnn_probe_gather_rate(int32_t row_bytes, int64_t table_rows, double* rows_per_second) {
     if (!rows_per_second) return fail(nullptr, SDNN_ERR_INVALID_ARG, "rows_per_second is NULL");
     *rows_per_second = 0.0;
-    if (row_bytes != 16 && row_bytes != 32 && row_bytes != 64 && row_bytes != 128 && row_bytes != 256 && row_bytes != 512)
-        return fail(nullptr, SDNN_ERR_INVALID_ARG, "row_bytes must be 16, 32, 64, 128, 256 or 512");
+    if (row_bytes != 16 && row_bytes != 32 && row_bytes != 64 && row_bytes != 128 && row_bytes != 256 && row_bytes != 512 &&
+        row_bytes != 1024)
+        return fail(nullptr, SDNN_ERR_INVALID_ARG, "row_bytes must be 16, 32, 64, 128, 256, 512 or 1024");
     if (table_rows < 1 || (table_rows & (table_rows - 1)) || table_rows * row_bytes > (1LL << 30))
         return fail(nullptr, SDNN_ERR_INVALID_ARG, "table_rows must be a power of two with table_rows * row_bytes <= 1 GiB");
     int dev = 0, sms = 0;
@@ -1111,18 +1145,20 @@ extern "C" int sdnn_probe_gather_rate(int32_t row_bytes, int64_t table_rows, dou
         rc = fail(nullptr, SDNN_ERR_OOM, "could not allocate the probe's table");
     } else {
         cudaMemsetAsync(table, 0, bytes, st);
-        const int g = row_bytes / 16, grid = sms * 4;                 // 1024 threads per SM: the rate no longer grows beyond that
+        // threads per SM at which the rate stops growing: 1024 for rows of up to 64 bytes, 2048 for wider ones
+        const int g = row_bytes == 16 ? 1 : row_bytes / 32, grid = sms * (row_bytes >= 128 ? 8 : 4);      // 256-bit lanes
         const int64_t groups = (int64_t)grid * 256 / g;
         const int per_group = (int)std::max<int64_t>(8, ((int64_t)1 << 22) / groups / 8 * 8);
         const unsigned mask = (unsigned)(table_rows - 1);
         float ms = 0.f;
-        switch (g) {
-            case 1: ms = run_gather_probe<1>(table, sink, mask, per_group, grid, st, 20, a, b); break;
-            case 2: ms = run_gather_probe<2>(table, sink, mask, per_group, grid, st, 20, a, b); break;
-            case 4: ms = run_gather_probe<4>(table, sink, mask, per_group, grid, st, 20, a, b); break;
-            case 8: ms = run_gather_probe<8>(table, sink, mask, per_group, grid, st, 20, a, b); break;
-            case 16: ms = run_gather_probe<16>(table, sink, mask, per_group, grid, st, 20, a, b); break;
-            default: ms = run_gather_probe<32>(table, sink, mask, per_group, grid, st, 20, a, b); break;
+        switch (row_bytes) {
+            case 16: ms = run_gather_probe<1, 4>(table, sink, mask, per_group, grid, st, 20, a, b); break;
+            case 32: ms = run_gather_probe<1, 8>(table, sink, mask, per_group, grid, st, 20, a, b); break;
+            case 64: ms = run_gather_probe<2, 8>(table, sink, mask, per_group, grid, st, 20, a, b); break;
+            case 128: ms = run_gather_probe<4, 8>(table, sink, mask, per_group, grid, st, 20, a, b); break;
+            case 256: ms = run_gather_probe<8, 8>(table, sink, mask, per_group, grid, st, 20, a, b); break;
+            case 512: ms = run_gather_probe<16, 8>(table, sink, mask, per_group, grid, st, 20, a, b); break;
+            default: ms = run_gather_probe<32, 8>(table, sink, mask, per_group, grid, st, 20, a, b); break;
         }
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess || !(ms > 0.f)) rc = cuda_fail(nullptr, e, "gather probe");

@@ -417,7 +417,10 @@ def main():
         dom = "backward_kernel" if bwd_ms >= fwd_ms else "forward_kernel"
         per_launch_ms = (bwd_ms if dom == "backward_kernel" else fwd_ms) / L
         alg = bwd_bytes if dom == "backward_kernel" else fwd_bytes
-        extra = {"fwd_ms_per_step": fwd_ms, "bwd_ms_per_step": bwd_ms,
+        extra = {"backward_launches": "per layer one column-unit launch (backward_kernel<..,1,..>) on the main stream and one "
+                                      "row-unit launch (backward_kernel<..,0,..>) on a side stream, running beside each other; "
+                                      "launch_ms is the backward chain's time per layer, bytes and gathers are those of both",
+                 "fwd_ms_per_step": fwd_ms, "bwd_ms_per_step": bwd_ms,
                  "fwd_GBps": fwd_bytes * L / (fwd_ms * 1e-3) / 1e9 if fwd_ms else None,
                  "bwd_GBps": bwd_bytes * L / (bwd_ms * 1e-3) / 1e9 if bwd_ms else None,
                  "step_bytes": (fwd_bytes + bwd_bytes) * L,

@@ -14,6 +14,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsdnn.so")
 
 FLAG_BWD_ATOMICS, FLAG_BWD_CSC, FLAG_KEEP_DEBUG, FLAG_SKIP_DEAD, FLAG_NO_GRAPH, FLAG_NO_PDL = 0x01, 0x02, 0x04, 0x08, 0x10, 0x20
+FLAG_BWD_ONE_LAUNCH = 0x80
 ACT_CLAMPED_RELU, ACT_SIGMOID = 0, 1
 
 STATUS = {0: "SDNN_OK", -1: "SDNN_ERR_INVALID_ARG", -2: "SDNN_ERR_BAD_CSR", -3: "SDNN_ERR_OOM", -4: "SDNN_ERR_CUDA",

@@ -530,6 +530,7 @@ struct BackwardArgs {
     float clamp;
     int act;                  // activation (ACT_*)
     int update_bias, skip_dead, pdl;
+    int cols_only;            // MIRROR: leave the row units to a separate launch (which may run beside the next layer's column units)
     const float* warm;        // tile the NEXT backward launch will gather from (x^{k-2}), or NULL: asked into L2 now,
     unsigned warm_bytes;      // because it was written a whole forward pass ago and has left the cache
 };
@@ -718,6 +719,7 @@ backward_kernel(const BackwardArgs a) {
     const float inv_b = a.sp->inv_b;
     const float step = a.sp->eta * inv_b;
     if (MIRROR) backward_col_units<G, V, CPS>(a.cols, a.xprev, a.dk, a.dprev, a.n, a.clamp, a.act, step, inv_b, first, stride);
+    if (MIRROR && a.cols_only) { if (a.pdl) grid_launch_dependents(); return; }
     backward_row_units<G, V, CPS, FROM_S, SCATTER, DBG>(a.rows, a.bias, a.xk, a.xprev, a.dk, a.dprev, a.dbg_delta, a.dbg_grad, a.n,
                                                         a.clamp, a.act, step, inv_b, a.update_bias, a.skip_dead, first, stride);
     if (a.pdl) grid_launch_dependents();

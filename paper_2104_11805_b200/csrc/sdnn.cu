@@ -69,6 +69,11 @@ struct sdnn {
     float* d_acts = nullptr;            // [(L+1)][N][ld]: x^0 .. x^L of the current step
     float* d_s[2] = {nullptr, nullptr}; // atomics: alternating S = W^T delta tiles (all-zero between steps); mirror: delta tiles
     float* d_dl = nullptr;              // delta^L tile (atomics realisation)
+    float* d_delta_all = nullptr;       // split backward: [L][N][ld], every delta^k of the step
+    bool split = false;                 // transposed realisation with the row units as launches of their own on side_stream
+    cudaStream_t side_stream = nullptr, launch_stream = nullptr;     // launch_stream: where launch_k currently enqueues (NULL = stream)
+    std::vector<cudaEvent_t> ev_delta;  // [L] delta^k (0-based layer) complete
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     float* d_yt = nullptr;              // target tile
     StepParams* d_sp = nullptr;
     double* d_loss = nullptr;
@@ -77,6 +82,7 @@ struct sdnn {
     int last_b = 0, last_ld = 0;
     cudaGraphExec_t graph = nullptr;
     int graph_ld = 0;
+    int64_t graph_launches = 0;         // kernel nodes of the captured step
     cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};   // before forward chain, between, after backward chain
 
     // inference
@@ -303,7 +309,7 @@ Sliced cols_of(sdnn* h, int layer) {
 template <typename... KArgs, typename... Args>
 cudaError_t launch_k(sdnn* h, void (*kernel)(KArgs...), dim3 grid, dim3 block, bool pdl, Args... args) {
     cudaLaunchConfig_t lc = {};
-    lc.gridDim = grid; lc.blockDim = block; lc.dynamicSmemBytes = 0; lc.stream = h->stream;
+    lc.gridDim = grid; lc.blockDim = block; lc.dynamicSmemBytes = 0; lc.stream = h->launch_stream ? h->launch_stream : h->stream;
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[0].val.programmaticStreamSerializationAllowed = 1;
@@ -339,11 +345,14 @@ void launch_forward(sdnn* h, int layer, const float* xin, float* xout, int ld, i
 
 // delta tile of layer `layer` (0-based; the paper's delta^{layer+1}) in the transposed realisation
 float* delta_tile(sdnn* h, int layer, size_t tile) {
-    return h->d_dbg_delta ? h->d_dbg_delta + (size_t)layer * tile : h->d_s[layer & 1];
+    if (h->d_dbg_delta) return h->d_dbg_delta + (size_t)layer * tile;
+    if (h->d_delta_all) return h->d_delta_all + (size_t)layer * tile;
+    return h->d_s[layer & 1];
 }
 
+// part: 0 = the whole layer in one launch; 1 = column units only; 2 = row units only (transposed realisation)
 template <int G, int V, int CPS>
-void launch_backward_gvc(sdnn* h, int layer, int ld) {
+void launch_backward_gvc(sdnn* h, int layer, int ld, int part) {
     constexpr int RPW = 32 / G;
     const size_t tile = (size_t)h->N * ld;
     const bool last = layer == h->L - 1, prop = layer > 0;
@@ -375,11 +384,13 @@ void launch_backward_gvc(sdnn* h, int layer, int ld) {
     } while (0)
     if (h->mirror) {
         a.dk = delta_tile(h, layer, tile);
-        if (prop) {
+        if (prop && part != 2) {
             a.cols = cols_of(h, layer);
             a.dprev = delta_tile(h, layer - 1, tile);
+            a.cols_only = part == 1 ? 1 : 0;
             SDNN_BWD(false, false, true);
-        } else {
+        } else if (part != 1) {
+            if (part == 2) { a.pdl = 0; a.warm = nullptr; }
             SDNN_BWD(false, false, false);
         }
     } else {
@@ -396,19 +407,19 @@ void launch_backward_gvc(sdnn* h, int layer, int ld) {
 }
 
 template <int G, int V>
-void launch_backward_gv(sdnn* h, int layer, int ld) {
-    launch_backward_gvc<G, V, 2>(h, layer, ld);
+void launch_backward_gv(sdnn* h, int layer, int ld, int part) {
+    launch_backward_gvc<G, V, 2>(h, layer, ld, part);
 }
 
-void launch_backward(sdnn* h, int layer, int ld) {
+void launch_backward(sdnn* h, int layer, int ld, int part = 0) {
     const Geometry q = geometry(ld);
-    if (q.v == 4) launch_backward_gv<1, 4>(h, layer, ld);
+    if (q.v == 4) launch_backward_gv<1, 4>(h, layer, ld, part);
     else switch (q.g) {
-        case 1: launch_backward_gv<1, 8>(h, layer, ld); break;
-        case 2: launch_backward_gv<2, 8>(h, layer, ld); break;
-        case 4: launch_backward_gv<4, 8>(h, layer, ld); break;
-        case 8: launch_backward_gv<8, 8>(h, layer, ld); break;
-        default: launch_backward_gv<16, 8>(h, layer, ld); break;
+        case 1: launch_backward_gv<1, 8>(h, layer, ld, part); break;
+        case 2: launch_backward_gv<2, 8>(h, layer, ld, part); break;
+        case 4: launch_backward_gv<4, 8>(h, layer, ld, part); break;
+        case 8: launch_backward_gv<8, 8>(h, layer, ld, part); break;
+        default: launch_backward_gv<16, 8>(h, layer, ld, part); break;
     }
     count_launch(h);
 }
@@ -439,7 +450,27 @@ void enqueue_step_body(sdnn* h, int ld, unsigned flags) {
         launch_forward(h, k, h->d_acts + (size_t)k * tile, h->d_acts + (size_t)(k + 1) * tile, ld, ld);
     cudaEventRecordWithFlags(h->ev[1], h->stream, flags);
     launch_output_gradient(h, ld);
-    for (int k = h->L - 1; k >= 0; --k) launch_backward(h, k, ld);
+    if (h->split) {
+        // column units chain on the main stream; the row units of layer k only need delta^k and x^{k-1}, so they run on
+        // the side stream beside the column units of the layers below
+        cudaEventRecord(h->ev_fork, h->stream);
+        cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0);
+        cudaEventRecord(h->ev_delta[h->L - 1], h->stream);
+        for (int k = h->L - 1; k >= 0; --k) {
+            cudaStreamWaitEvent(h->side_stream, h->ev_delta[k], 0);
+            h->launch_stream = h->side_stream;
+            launch_backward(h, k, ld, 2);
+            h->launch_stream = nullptr;
+            if (k > 0) {
+                launch_backward(h, k, ld, 1);
+                cudaEventRecord(h->ev_delta[k - 1], h->stream);
+            }
+        }
+        cudaEventRecord(h->ev_join, h->side_stream);
+        cudaStreamWaitEvent(h->stream, h->ev_join, 0);
+    } else {
+        for (int k = h->L - 1; k >= 0; --k) launch_backward(h, k, ld);
+    }
     cudaEventRecordWithFlags(h->ev[2], h->stream, flags);
 }
 
@@ -459,6 +490,7 @@ int train_step_device(sdnn* h, const float* x0, const float* target, int B, floa
             CU(h, cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal));
             enqueue_step_body(h, ld, cudaEventRecordExternal);
             cudaError_t e = cudaStreamEndCapture(h->stream, &g);
+            h->graph_launches = h->launches - before;
             h->launches = before;
             if (e != cudaSuccess) return cuda_fail(h, e, "cudaStreamEndCapture");
             e = cudaGraphInstantiate(&h->graph, g, 0);
@@ -467,7 +499,7 @@ int train_step_device(sdnn* h, const float* x0, const float* target, int B, floa
             h->graph_ld = ld;
         }
         CU(h, cudaGraphLaunch(h->graph, h->stream));
-        count_launch(h, 2 * h->L + 1);
+        count_launch(h, (int)h->graph_launches);
     }
     CU(h, cudaGetLastError());
     h->stepped = true; h->last_b = B; h->last_ld = ld;
@@ -628,6 +660,10 @@ void sdnn_destroy(sdnn_t* h) {
     if (h->stream || h->own_stream) cudaStreamSynchronize(h->stream);
     if (h->graph) cudaGraphExecDestroy(h->graph);
     for (cudaEvent_t e : h->ev) if (e) cudaEventDestroy(e);
+    for (cudaEvent_t e : h->ev_delta) if (e) cudaEventDestroy(e);
+    if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+    if (h->ev_join) cudaEventDestroy(h->ev_join);
+    if (h->side_stream) { cudaStreamSynchronize(h->side_stream); cudaStreamDestroy(h->side_stream); }
     for (cudaEvent_t e : h->ev_copied) if (e) cudaEventDestroy(e);
     for (cudaEvent_t e : h->ev_consumed) if (e) cudaEventDestroy(e);
     if (h->copy_stream) { cudaStreamSynchronize(h->copy_stream); cudaStreamDestroy(h->copy_stream); }
@@ -696,6 +732,16 @@ int sdnn_create_deferred(sdnn_t** out, int32_t n_layers, int32_t n_neurons, cons
         for (cudaEvent_t& ev : h->ev)
             if ((e = cudaEventCreate(&ev)) != cudaSuccess) { ev = nullptr; return bail(cuda_fail(h, e, "cudaEventCreate")); }
         if ((rc = dev_alloc(h, &h->d_acts, (L + 1) * tile, false))) return bail(rc);
+        h->split = h->mirror && !(cfg->flags & SDNN_FLAG_BWD_ONE_LAUNCH);
+        if (h->split) {
+            if (!(cfg->flags & SDNN_FLAG_KEEP_DEBUG) && (rc = dev_alloc(h, &h->d_delta_all, L * tile, true))) return bail(rc);
+            if ((e = cudaStreamCreateWithFlags(&h->side_stream, cudaStreamNonBlocking)) != cudaSuccess) return bail(cuda_fail(h, e, "cudaStreamCreate"));
+            h->ev_delta.assign(n_layers, nullptr);
+            for (cudaEvent_t& ev : h->ev_delta)
+                if ((e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming)) != cudaSuccess) { ev = nullptr; return bail(cuda_fail(h, e, "cudaEventCreate")); }
+            if ((e = cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming)) != cudaSuccess) return bail(cuda_fail(h, e, "cudaEventCreate"));
+            if ((e = cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming)) != cudaSuccess) return bail(cuda_fail(h, e, "cudaEventCreate"));
+        }
         if ((rc = dev_alloc(h, &h->d_s[0], tile, true))) return bail(rc);
         if ((rc = dev_alloc(h, &h->d_s[1], tile, true))) return bail(rc);
         if (!h->mirror && (rc = dev_alloc(h, &h->d_dl, tile, true))) return bail(rc);

@@ -137,7 +137,7 @@ def batches_for(spec, B, steps):
 
 
 # ---------------------------------------------------------------------------------------------- train
-BWD_MODES = {"transposed": 0x02, "atomics": 0x01}
+BWD_MODES = {"transposed": 0x02, "transposed_one_launch": 0x82, "atomics": 0x01}
 
 
 @pytest.mark.parametrize("B", [1, 3, 4, 7, 16, 33, 64, 100, 128])
@@ -164,11 +164,12 @@ def test_train_free_running_trajectories_stay_close(torch_cuda, bwd):
     train_parity(torch_cuda, arrays, batches, eta=0.005, sync=False, flags=BWD_MODES[bwd], expect_live=True)
 
 
-@pytest.mark.parametrize("extra", ["no_graph", "no_pdl", "no_graph_no_pdl"])
+@pytest.mark.parametrize("extra", ["no_graph", "no_pdl", "no_graph_no_pdl", "one_launch", "one_launch_no_graph"])
 def test_train_launch_variants_match(torch_cuda, extra):
     """Kernel-by-kernel launches and launches without programmatic dependent launch give the same results."""
     pkg = sdnn()
-    flags = {"no_graph": pkg.FLAG_NO_GRAPH, "no_pdl": pkg.FLAG_NO_PDL, "no_graph_no_pdl": pkg.FLAG_NO_GRAPH | pkg.FLAG_NO_PDL}[extra]
+    flags = {"no_graph": pkg.FLAG_NO_GRAPH, "no_pdl": pkg.FLAG_NO_PDL, "no_graph_no_pdl": pkg.FLAG_NO_GRAPH | pkg.FLAG_NO_PDL,
+             "one_launch": pkg.FLAG_BWD_ONE_LAUNCH, "one_launch_no_graph": pkg.FLAG_BWD_ONE_LAUNCH | pkg.FLAG_NO_GRAPH}[extra]
     rng = np.random.default_rng(5)
     arrays = ragged_net(rng, n=130, layers=4, kmax=8)
     batches = [(rng.uniform(0, 1.5, size=(16, 130)).astype(np.float32), rng.uniform(0, 1, size=(16, 130)).astype(np.float32))

@@ -432,7 +432,11 @@ def main():
         per_launch_ms = ms_per_step / (tiles * L)      # includes the (small) transpose and count kernels of each tile
         # per launch: the layer's indices and values once, the activation tile read and written once
         alg = 8 * nnz_l + 2 * N * min(batch, n_inputs) * 4
-        extra = {"tiles": tiles, "tile_inputs": batch, "note": "launch time = call time / forward launches (upper bound)"}
+        in_flight = h.infer_tiles_in_flight() if tiles > 1 else 1
+        extra = {"tiles": tiles, "tile_inputs": batch, "tiles_in_flight": in_flight,
+                 "note": "launch time = call time / forward launches (upper bound)" +
+                         ("; two tiles run beside each other on two streams, so this is the time the device spends per "
+                          "launch, not one launch's start-to-end duration" if in_flight > 1 else "")}
     # what bounds these launches instead of HBM: random gathers of tile rows out of L2 (measured now, on this device)
     if kind == "train":
         row_bytes, gathers = 4 * ld, (2 if dom == "backward_kernel" else 1) * nnz_l

@@ -76,6 +76,7 @@ typedef enum {
                                     /* own on a second stream, beside the column units of the layers below; that keeps   */
                                     /* every delta^k of a step (N * padded(B) * 4 bytes per layer more) and is faster    */
 #define SDNN_FLAG_NO_PDL      0x20u /* do not let a layer's kernel start its prologue under the previous layer's tail */
+#define SDNN_FLAG_ONE_TILE    0x40u /* inference: one tile in flight at a time (see sdnn_infer_batch)               */
 
 #define SDNN_ACT_CLAMPED_RELU 0
 #define SDNN_ACT_SIGMOID      1
@@ -131,7 +132,12 @@ int sdnn_finalize(sdnn_t* h);
  *   nz_total_out  host int64*: total number of ids (sum of counts), or NULL
  * The batch is processed in tiles of at most cfg.max_batch inputs (narrower ones, a power of two >= 128, when two
  * activation tiles of max_batch inputs would not fit in the L2 cache and the sparsity pattern is not local: the
- * gathers of a layer then come out of L2 instead of HBM).  If nz_index_out is given and the
+ * gathers of a layer then come out of L2 instead of HBM).  Tiles are independent; a batch of more than one tile
+ * keeps two in flight, each on a stream of its own (the second stream and its two activation tiles are created at
+ * the first such call), so that the start and tail of one tile's launches are filled by the other's;
+ * SDNN_FLAG_ONE_TILE turns that off.  The call is ordered on the handle's stream either way:
+ * work enqueued there before it is seen, and everything the call launched is complete once that stream has caught
+ * up.  If nz_index_out is given and the
  * capacity is too small, only the ids at positions below the capacity are written, *nz_total_out
  * (if given) holds the needed capacity and the call returns SDNN_ERR_INVALID_ARG; y_out and
  * nz_count_out are still valid.  n_inputs == 0 is a valid no-op.
@@ -142,6 +148,10 @@ int sdnn_infer_batch(sdnn_t* h, const float* x0, int64_t n_inputs, float* y_out,
 
 /* Inputs per tile that sdnn_infer_batch uses on this handle (see above); 0 before sdnn_finalize. */
 int32_t sdnn_infer_tile_width(const sdnn_t* h);
+
+/* Tiles that sdnn_infer_batch keeps in flight on this handle when a batch has more than one (1 or 2; see above);
+ * 0 before sdnn_finalize. */
+int32_t sdnn_infer_tiles_in_flight(const sdnn_t* h);
 
 /* Same call with every array in HOST memory (pinned or pageable); the library stages the
  * copies itself, tile by tile, and returns when the outputs are in place. */

@@ -15,6 +15,7 @@ LIB_PATH = os.path.join(_HERE, "libsdnn.so")
 
 FLAG_BWD_ATOMICS, FLAG_BWD_CSC, FLAG_KEEP_DEBUG, FLAG_SKIP_DEAD, FLAG_NO_GRAPH, FLAG_NO_PDL = 0x01, 0x02, 0x04, 0x08, 0x10, 0x20
 FLAG_BWD_ONE_LAUNCH = 0x80
+FLAG_ONE_TILE = 0x40
 ACT_CLAMPED_RELU, ACT_SIGMOID = 0, 1
 
 STATUS = {0: "SDNN_OK", -1: "SDNN_ERR_INVALID_ARG", -2: "SDNN_ERR_BAD_CSR", -3: "SDNN_ERR_OOM", -4: "SDNN_ERR_CUDA",
@@ -56,6 +57,7 @@ _PROTOS = {
     "sdnn_infer_noalloc": (ctypes.c_int, [_i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _f32, _vp]),
     "sdnn_kernel_launches": (_i64, [_vp]),
     "sdnn_infer_tile_width": (_i32, [_vp]),
+    "sdnn_infer_tiles_in_flight": (_i32, [_vp]),
     "sdnn_device_bytes": (_i64, [_vp]),
     "sdnn_destroy": (None, [_vp]),
     "sdnn_last_error": (ctypes.c_char_p, [_vp]),
@@ -253,6 +255,10 @@ class Sdnn:
     def infer_tile_width(self):
         """Inputs per tile that infer_batch uses on this handle."""
         return int(self._lib.sdnn_infer_tile_width(self._h))
+
+    def infer_tiles_in_flight(self):
+        """Tiles infer_batch keeps in flight on this handle when a batch has several (1 or 2)."""
+        return int(self._lib.sdnn_infer_tiles_in_flight(self._h))
 
     def kernel_launches(self):
         return int(self._lib.sdnn_kernel_launches(self._h))

@@ -34,6 +34,24 @@ struct RowShape {
     int64_t start(int i) const { return uniform_k >= 0 ? (int64_t)i * uniform_k : row_ptr[i]; }
 };
 
+// Buffers of one inference tile in flight.  Tiles are independent of one another (so are the inputs), and a
+// handle may work on two at a time, each on its own stream, so that the ramp and tail of one tile's launches are
+// filled by the other's.
+struct InferLane {
+    cudaStream_t stream = nullptr;         // lane 0: the handle's stream
+    float* tile[2] = {nullptr, nullptr};   // ping-pong activation tiles
+    int* seg_cnt = nullptr;
+    int* tile_cnt = nullptr;
+    long long* offs = nullptr;
+    ColState cs{};                         // live-column bookkeeping (SDNN_FLAG_SKIP_DEAD)
+    int* live_hist = nullptr;              // [L] live inputs after each layer of this lane's most recent tile
+    float* stage_out = nullptr;            // host entry point: staged x^L and counts of this lane's tile
+    int* stage_cnt = nullptr;
+    cudaEvent_t ev_scan = nullptr;         // this lane's last scan of the running id total is done
+    cudaEvent_t ev_done = nullptr;         // everything this lane was given in the current call is done
+    bool ready = false;
+};
+
 struct LayerMem {
     int64_t r_elems = 0, c_elems = 0;      // padded lengths of the two sliced copies
     int* r_idx = nullptr; float* r_val = nullptr; float* r_grad = nullptr;
@@ -86,17 +104,15 @@ struct sdnn {
     cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};   // before forward chain, between, after backward chain
 
     // inference
-    float* d_tile[2] = {nullptr, nullptr};
-    int* d_seg_cnt = nullptr;
-    int* d_tile_cnt = nullptr;
-    long long* d_offs = nullptr;
+    InferLane lane[2];
+    InferLane* cur = nullptr;           // lane the launch helpers currently work for
+    cudaEvent_t last_scan_ev = nullptr, ev_lane_start = nullptr;
+    int live_lane = 0;
     long long* d_running = nullptr;
     int l2_bytes = 0;
     std::vector<char> local_pattern;    // per layer: blocks of 1024 rows touch few distinct columns (see infer_tile_width)
     bool compaction = false;            // SDNN_FLAG_SKIP_DEAD asked for; effective while no bias is positive
     std::vector<char> bias_nonpositive; // per layer
-    ColState cs{};                      // device state of the live-column bookkeeping
-    int* d_live_hist = nullptr;         // [L] live inputs after each layer of the most recent tile
     bool live_valid = false;
 
     // staging for the *_host entry points (allocated on first use)
@@ -324,8 +340,8 @@ void launch_forward_gv(sdnn* h, int layer, const float* xin, float* xout, int ld
     const float* bias = h->d_bias + (size_t)layer * h->N;
     auto plan = plan_grid(h, (const void*)forward_kernel<G, V, 2>, units, chunks);
     launch_k(h, forward_kernel<G, V, 2>, dim3(plan.first, chunks), dim3(plan.second), h->pdl, rows_of(h, layer), bias, xin, xout,
-             h->N, ld, h->cfg.clamp, h->cfg.activation, h->pdl ? 1 : 0, track ? (const int*)h->cs.ncols : (const int*)nullptr,
-             track ? h->cs.flags : (int*)nullptr);
+             h->N, ld, h->cfg.clamp, h->cfg.activation, h->pdl ? 1 : 0, track ? (const int*)h->cur->cs.ncols : (const int*)nullptr,
+             track ? h->cur->cs.flags : (int*)nullptr);
 }
 
 // track: compaction mode (process only the live columns, mark the columns that stay live)
@@ -437,7 +453,7 @@ void launch_output_gradient(sdnn* h, int ld) {
 
 void launch_transpose_in(sdnn* h, const float* src, float* dst, int cnt, int cols, int ld) {
     dim3 grid((h->N + 31) / 32, (cols + 31) / 32), block(32, 8);
-    transpose_in_kernel<<<grid, block, 0, h->stream>>>(src, dst, h->N, cnt, cols, ld);
+    transpose_in_kernel<<<grid, block, 0, h->launch_stream ? h->launch_stream : h->stream>>>(src, dst, h->N, cnt, cols, ld);
     count_launch(h);
 }
 
@@ -522,12 +538,39 @@ int check_train_args(sdnn* h, const float* x0, const float* target, int B, float
     return SDNN_OK;
 }
 
-// One tile of inference on device buffers: x0 [cnt][N] -> outputs for these cnt inputs.
-int infer_tile(sdnn* h, const float* x0, int cnt, float* y_out, int* cnt_out, int* idx_out, long long capacity,
+int alloc_lane(sdnn* h, InferLane& ln, bool own_stream) {
+    if (ln.ready) return SDNN_OK;
+    const size_t N = (size_t)h->N, tile = N * (size_t)h->ld_max, nseg = (N + NZ_SEG - 1) / NZ_SEG;
+    int rc;
+    if (own_stream) CU(h, cudaStreamCreateWithFlags(&ln.stream, cudaStreamNonBlocking));
+    else ln.stream = h->stream;
+    CU(h, cudaEventCreateWithFlags(&ln.ev_scan, cudaEventDisableTiming));
+    CU(h, cudaEventCreateWithFlags(&ln.ev_done, cudaEventDisableTiming));
+    if ((rc = dev_alloc(h, &ln.tile[0], tile, false))) return rc;
+    if ((rc = dev_alloc(h, &ln.tile[1], tile, false))) return rc;
+    if ((rc = dev_alloc(h, &ln.seg_cnt, nseg * (size_t)h->ld_max, false))) return rc;
+    if ((rc = dev_alloc(h, &ln.tile_cnt, (size_t)h->ld_max, false))) return rc;
+    if ((rc = dev_alloc(h, &ln.offs, (size_t)h->ld_max, false))) return rc;
+    if (h->compaction) {
+        int* blk = nullptr;
+        if ((rc = dev_alloc(h, &blk, 3 * (size_t)h->ld_max + 4, true))) return rc;
+        ln.cs.colmap = blk; ln.cs.perm = blk + h->ld_max; ln.cs.flags = blk + 2 * (size_t)h->ld_max;
+        ln.cs.ncols = blk + 3 * (size_t)h->ld_max; ln.cs.old_ncols = ln.cs.ncols + 1; ln.cs.do_compact = ln.cs.ncols + 2;
+        if ((rc = dev_alloc(h, &ln.live_hist, (size_t)h->L, true))) return rc;
+    }
+    ln.ready = true;
+    return SDNN_OK;
+}
+
+// One tile of inference on device buffers, on lane `ln`: x0 [cnt][N] -> outputs for these cnt inputs.
+int infer_tile(sdnn* h, InferLane& ln, const float* x0, int cnt, float* y_out, int* cnt_out, int* idx_out, long long capacity,
                bool want_sets) {
     const int ld = h->ld_max;
     const int cols = padded_width(cnt);
-    launch_transpose_in(h, x0, h->d_tile[0], cnt, cols, ld);
+    cudaStream_t st = ln.stream;
+    h->cur = &ln;
+    h->launch_stream = st;
+    launch_transpose_in(h, x0, ln.tile[0], cnt, cols, ld);
     int cur = 0;
     bool track = h->compaction && h->cfg.activation == SDNN_ACT_CLAMPED_RELU;      // sigmoid(b) is never 0: nothing ever dies
     for (int l = 0; l < h->L && track; ++l) track = h->bias_nonpositive[l] != 0;     // the zero vector must be a fixed point
@@ -535,40 +578,47 @@ int infer_tile(sdnn* h, const float* x0, int cnt, float* y_out, int* cnt_out, in
         const Geometry q = geometry(cols);
         const int chunk = q.g * q.v;
         const int rows_grid = std::min((h->N + 7) / 8, h->sms * 8);
-        cols_init_kernel<<<(ld + 255) / 256, 256, 0, h->stream>>>(h->cs, cnt, ld);
+        cols_init_kernel<<<(ld + 255) / 256, 256, 0, st>>>(ln.cs, cnt, ld);
         count_launch(h);
         for (int k = 0; k < h->L; ++k) {
-            launch_forward(h, k, h->d_tile[cur], h->d_tile[cur ^ 1], ld, cols, true);
+            launch_forward(h, k, ln.tile[cur], ln.tile[cur ^ 1], ld, cols, true);
             cur ^= 1;
-            live_kernel<<<1, 1024, 0, h->stream>>>(h->cs, h->d_live_hist + k, chunk);
-            compact_kernel<<<rows_grid, 256, 0, h->stream>>>(h->cs, h->d_tile[cur], h->N, ld, chunk);
+            live_kernel<<<1, 1024, 0, st>>>(ln.cs, ln.live_hist + k, chunk);
+            compact_kernel<<<rows_grid, 256, 0, st>>>(ln.cs, ln.tile[cur], h->N, ld, chunk);
             count_launch(h, 2);
         }
-        expand_kernel<<<rows_grid, 256, 0, h->stream>>>(h->cs, h->d_tile[cur], h->d_tile[cur ^ 1], h->N, cols, ld);
+        expand_kernel<<<rows_grid, 256, 0, st>>>(ln.cs, ln.tile[cur], ln.tile[cur ^ 1], h->N, cols, ld);
         count_launch(h);
         cur ^= 1;
         h->live_valid = true;
+        h->live_lane = (int)(&ln - h->lane);
     } else {
         for (int k = 0; k < h->L; ++k) {
-            launch_forward(h, k, h->d_tile[cur], h->d_tile[cur ^ 1], ld, cols);
+            launch_forward(h, k, ln.tile[cur], ln.tile[cur ^ 1], ld, cols);
             cur ^= 1;
         }
     }
-    const float* xl = h->d_tile[cur];
+    h->launch_stream = nullptr;
+    h->cur = &h->lane[0];
+    const float* xl = ln.tile[cur];
     if (y_out) {
         dim3 grid((h->N + 31) / 32, (cnt + 31) / 32), block(32, 8);
-        transpose_out_kernel<<<grid, block, 0, h->stream>>>(xl, y_out, h->N, cnt, ld);
+        transpose_out_kernel<<<grid, block, 0, st>>>(xl, y_out, h->N, cnt, ld);
         count_launch(h);
     }
     if (want_sets) {
         const int nseg = (h->N + NZ_SEG - 1) / NZ_SEG;
         dim3 grid(nseg, (cnt + 127) / 128);
-        nz_count_kernel<<<grid, 128, 0, h->stream>>>(xl, h->d_seg_cnt, h->N, cnt, ld);
-        nz_scan_segments_kernel<<<(cnt + 127) / 128, 128, 0, h->stream>>>(h->d_seg_cnt, h->d_tile_cnt, nseg, cnt, ld);
-        nz_scan_inputs_kernel<<<1, 1024, 0, h->stream>>>(h->d_tile_cnt, h->d_offs, h->d_running, cnt_out, cnt);
+        nz_count_kernel<<<grid, 128, 0, st>>>(xl, ln.seg_cnt, h->N, cnt, ld);
+        nz_scan_segments_kernel<<<(cnt + 127) / 128, 128, 0, st>>>(ln.seg_cnt, ln.tile_cnt, nseg, cnt, ld);
+        // the running total of ids is carried from tile to tile: the scans of successive tiles run in order
+        if (h->last_scan_ev && h->last_scan_ev != ln.ev_scan) CU(h, cudaStreamWaitEvent(st, h->last_scan_ev, 0));
+        nz_scan_inputs_kernel<<<1, 1024, 0, st>>>(ln.tile_cnt, ln.offs, h->d_running, cnt_out, cnt);
+        CU(h, cudaEventRecord(ln.ev_scan, st));
+        h->last_scan_ev = ln.ev_scan;
         count_launch(h, 3);
         if (idx_out) {
-            nz_fill_kernel<<<grid, 128, 0, h->stream>>>(xl, h->d_seg_cnt, h->d_offs, idx_out, capacity, h->N, cnt, ld);
+            nz_fill_kernel<<<grid, 128, 0, st>>>(xl, ln.seg_cnt, ln.offs, idx_out, capacity, h->N, cnt, ld);
             count_launch(h);
         }
     }
@@ -592,6 +642,36 @@ int infer_tile_width(const sdnn* h) {
         T = p;
     }
     return T;
+}
+
+// Tiles in flight, each on a stream of its own.  Two: a third adds a percent or two at most and costs two more
+// activation tiles.  The gathers of a layer touch its input tile only, so the second lane doubles what should stay
+// in L2 from one tile to two, which the tile width already allows for.
+int infer_lanes(const sdnn* h, int /*T*/) {
+    return (h->cfg.flags & SDNN_FLAG_ONE_TILE) ? 1 : 2;
+}
+
+// start / end of a batch that may use the second lane: lane 1 sees what the handle's stream has done so far, and the
+// handle's stream ends up behind everything lane 1 did
+int lanes_begin(sdnn* h, int lanes) {
+    h->last_scan_ev = nullptr;
+    if (lanes < 2) return SDNN_OK;
+    if (!h->ev_lane_start) CU(h, cudaEventCreateWithFlags(&h->ev_lane_start, cudaEventDisableTiming));
+    CU(h, cudaEventRecord(h->ev_lane_start, h->stream));
+    for (int i = 1; i < lanes; ++i) {
+        int rc = alloc_lane(h, h->lane[i], true);
+        if (rc) return rc;
+        CU(h, cudaStreamWaitEvent(h->lane[i].stream, h->ev_lane_start, 0));
+    }
+    return SDNN_OK;
+}
+int lanes_end(sdnn* h, int lanes) {
+    for (int i = 1; i < lanes; ++i) {
+        if (!h->lane[i].ready) continue;
+        CU(h, cudaEventRecord(h->lane[i].ev_done, h->lane[i].stream));
+        CU(h, cudaStreamWaitEvent(h->stream, h->lane[i].ev_done, 0));
+    }
+    return SDNN_OK;
 }
 
 int check_infer_args(sdnn* h, const float* x0, int64_t n_inputs, int32_t* idx, int64_t cap) {
@@ -652,6 +732,7 @@ const char* sdnn_last_error(const sdnn_t* h) { return h ? h->err.c_str() : g_cre
 
 int64_t sdnn_kernel_launches(const sdnn_t* h) { return h ? h->launches : 0; }
 int32_t sdnn_infer_tile_width(const sdnn_t* h) { return (h && h->finalized) ? infer_tile_width(h) : 0; }
+int32_t sdnn_infer_tiles_in_flight(const sdnn_t* h) { return (h && h->finalized) ? infer_lanes(h, infer_tile_width(h)) : 0; }
 int64_t sdnn_device_bytes(const sdnn_t* h) { return h ? h->dev_bytes : 0; }
 
 void sdnn_destroy(sdnn_t* h) {
@@ -660,6 +741,12 @@ void sdnn_destroy(sdnn_t* h) {
     if (h->stream || h->own_stream) cudaStreamSynchronize(h->stream);
     if (h->graph) cudaGraphExecDestroy(h->graph);
     for (cudaEvent_t e : h->ev) if (e) cudaEventDestroy(e);
+    for (InferLane& ln : h->lane) {
+        if (ln.ev_scan) cudaEventDestroy(ln.ev_scan);
+        if (ln.ev_done) cudaEventDestroy(ln.ev_done);
+        if (ln.stream && ln.stream != h->stream) { cudaStreamSynchronize(ln.stream); cudaStreamDestroy(ln.stream); }
+    }
+    if (h->ev_lane_start) cudaEventDestroy(h->ev_lane_start);
     for (cudaEvent_t e : h->ev_delta) if (e) cudaEventDestroy(e);
     if (h->ev_fork) cudaEventDestroy(h->ev_fork);
     if (h->ev_join) cudaEventDestroy(h->ev_join);
@@ -753,22 +840,13 @@ int sdnn_create_deferred(sdnn_t** out, int32_t n_layers, int32_t n_neurons, cons
     }
     {   // inference buffers (a training handle can also infer)
         const size_t nseg = (N + NZ_SEG - 1) / NZ_SEG;
-        if ((rc = dev_alloc(h, &h->d_tile[0], tile, false))) return bail(rc);
-        if ((rc = dev_alloc(h, &h->d_tile[1], tile, false))) return bail(rc);
-        if ((rc = dev_alloc(h, &h->d_seg_cnt, nseg * (size_t)h->ld_max, false))) return bail(rc);
-        if ((rc = dev_alloc(h, &h->d_tile_cnt, (size_t)h->ld_max, false))) return bail(rc);
-        if ((rc = dev_alloc(h, &h->d_offs, (size_t)h->ld_max, false))) return bail(rc);
-        if ((rc = dev_alloc(h, &h->d_running, 1, true))) return bail(rc);
+        (void)nseg;
         h->compaction = (cfg->flags & SDNN_FLAG_SKIP_DEAD) != 0;
         h->bias_nonpositive.assign(n_layers, 0);
         h->local_pattern.assign(n_layers, 0);
-        if (h->compaction) {
-            int* blk = nullptr;
-            if ((rc = dev_alloc(h, &blk, 3 * (size_t)h->ld_max + 4, true))) return bail(rc);
-            h->cs.colmap = blk; h->cs.perm = blk + h->ld_max; h->cs.flags = blk + 2 * (size_t)h->ld_max;
-            h->cs.ncols = blk + 3 * (size_t)h->ld_max; h->cs.old_ncols = h->cs.ncols + 1; h->cs.do_compact = h->cs.ncols + 2;
-            if ((rc = dev_alloc(h, &h->d_live_hist, L, true))) return bail(rc);
-        }
+        if ((rc = dev_alloc(h, &h->d_running, 1, true))) return bail(rc);
+        if ((rc = alloc_lane(h, h->lane[0], false))) return bail(rc);
+        h->cur = &h->lane[0];
     }
     *out = h;
     return SDNN_OK;
@@ -948,12 +1026,17 @@ int sdnn_infer_batch(sdnn_t* h, const float* x0, int64_t n_inputs, float* y_out,
     const bool want_sets = nz_count_out || nz_index_out || nz_total_out;
     if (want_sets) CU(h, cudaMemsetAsync(h->d_running, 0, sizeof(long long), h->stream));
     const int T = infer_tile_width(h);
-    for (int64_t t0 = 0; t0 < n_inputs; t0 += T) {
+    const int lanes = n_inputs > T ? infer_lanes(h, T) : 1;
+    if ((rc = lanes_begin(h, lanes))) return rc;
+    int64_t tile_no = 0;
+    for (int64_t t0 = 0; t0 < n_inputs; t0 += T, ++tile_no) {
         const int cnt = (int)((n_inputs - t0 < T) ? (n_inputs - t0) : T);
-        rc = infer_tile(h, x0 + (size_t)t0 * h->N, cnt, y_out ? y_out + (size_t)t0 * h->N : nullptr,
+        rc = infer_tile(h, h->lane[tile_no % lanes], x0 + (size_t)t0 * h->N, cnt, y_out ? y_out + (size_t)t0 * h->N : nullptr,
                         nz_count_out ? nz_count_out + t0 : nullptr, nz_index_out, nz_index_capacity, want_sets);
-        if (rc) return rc;
+        if (rc) break;
     }
+    const int rc_end = lanes_end(h, lanes);
+    if (rc || rc_end) return rc ? rc : rc_end;
     if (nz_total_out || nz_index_out) {
         long long total = 0;
         CU(h, cudaMemcpyAsync(&total, h->d_running, sizeof total, cudaMemcpyDeviceToHost, h->stream));
@@ -990,22 +1073,33 @@ int sdnn_infer_batch_host(sdnn_t* h, const float* x0, int64_t n_inputs, float* y
     float* stage[2] = {h->d_stage_a, h->d_stage_a2};
     CU(h, cudaEventRecord(h->ev_consumed[0], h->stream));       // the stages may still be read by earlier work on the stream
     CU(h, cudaEventRecord(h->ev_consumed[1], h->stream));
+    const int lanes = n_inputs > T ? infer_lanes(h, T) : 1;
+    if ((rc = lanes_begin(h, lanes))) return rc;
+    h->lane[0].stage_out = h->d_stage_b;
+    h->lane[0].stage_cnt = h->d_stage_cnt;
+    if (lanes == 2 && !h->lane[1].stage_out) {
+        if ((rc = dev_alloc(h, &h->lane[1].stage_out, (size_t)h->cfg.max_batch * h->N, false))) return rc;
+        if ((rc = dev_alloc(h, &h->lane[1].stage_cnt, (size_t)h->cfg.max_batch, false))) return rc;
+    }
     int64_t tile_no = 0;
     for (int64_t t0 = 0; t0 < n_inputs; t0 += T, ++tile_no) {
         const int cnt = (int)((n_inputs - t0 < T) ? (n_inputs - t0) : T);
         const size_t bytes = (size_t)cnt * h->N * sizeof(float);
         const int q = (int)(tile_no & 1);
+        InferLane& ln = h->lane[tile_no % lanes];
         CU(h, cudaStreamWaitEvent(h->copy_stream, h->ev_consumed[q], 0));
         CU(h, cudaMemcpyAsync(stage[q], x0 + (size_t)t0 * h->N, bytes, cudaMemcpyHostToDevice, h->copy_stream));
         CU(h, cudaEventRecord(h->ev_copied[q], h->copy_stream));
-        CU(h, cudaStreamWaitEvent(h->stream, h->ev_copied[q], 0));
-        rc = infer_tile(h, stage[q], cnt, y_out ? h->d_stage_b : nullptr, nz_count_out ? h->d_stage_cnt : nullptr,
+        CU(h, cudaStreamWaitEvent(ln.stream, h->ev_copied[q], 0));
+        rc = infer_tile(h, ln, stage[q], cnt, y_out ? ln.stage_out : nullptr, nz_count_out ? ln.stage_cnt : nullptr,
                         nz_index_out ? h->d_stage_idx : nullptr, nz_index_capacity, want_sets);
-        if (rc) return rc;
-        if (y_out) CU(h, cudaMemcpyAsync(y_out + (size_t)t0 * h->N, h->d_stage_b, bytes, cudaMemcpyDeviceToHost, h->stream));
-        if (nz_count_out) CU(h, cudaMemcpyAsync(nz_count_out + t0, h->d_stage_cnt, (size_t)cnt * sizeof(int), cudaMemcpyDeviceToHost, h->stream));
-        CU(h, cudaEventRecord(h->ev_consumed[q], h->stream));
+        if (rc) break;
+        if (y_out) CU(h, cudaMemcpyAsync(y_out + (size_t)t0 * h->N, ln.stage_out, bytes, cudaMemcpyDeviceToHost, ln.stream));
+        if (nz_count_out) CU(h, cudaMemcpyAsync(nz_count_out + t0, ln.stage_cnt, (size_t)cnt * sizeof(int), cudaMemcpyDeviceToHost, ln.stream));
+        CU(h, cudaEventRecord(h->ev_consumed[q], ln.stream));
     }
+    const int rc_end = lanes_end(h, lanes);
+    if (rc || rc_end) return rc ? rc : rc_end;
     long long total = 0;
     if (want_sets) CU(h, cudaMemcpyAsync(&total, h->d_running, sizeof total, cudaMemcpyDeviceToHost, h->stream));
     CU(h, cudaStreamSynchronize(h->stream));
@@ -1143,7 +1237,7 @@ int sdnn_get_liveness(sdnn_t* h, int32_t* live_inputs_out) {
     if (!h->live_valid) return fail(h, SDNN_ERR_STATE, "liveness is recorded only by inference with SDNN_FLAG_SKIP_DEAD on a net without positive biases");
     CU(h, cudaSetDevice(h->device));
     CU(h, cudaStreamSynchronize(h->stream));
-    CU(h, cudaMemcpy(live_inputs_out, h->d_live_hist, (size_t)h->L * sizeof(int), cudaMemcpyDeviceToHost));
+    CU(h, cudaMemcpy(live_inputs_out, h->lane[h->live_lane].live_hist, (size_t)h->L * sizeof(int), cudaMemcpyDeviceToHost));
     return SDNN_OK;
 }
 

@@ -289,6 +289,51 @@ def test_infer_many_tiles_with_dead_inputs_dropped(torch_cuda):
         assert np.array_equal(ids, np.flatnonzero(y[b] != 0.0))
 
 
+@pytest.mark.parametrize("host", [False, True])
+@pytest.mark.parametrize("skip_dead", [False, True])
+def test_infer_two_tiles_in_flight_equals_one_at_a_time(torch_cuda, host, skip_dead):
+    """Seven tiles (the last ragged) alternate between two streams by default; with SDNN_FLAG_ONE_TILE they run one
+    after the other.  Outputs, counts, the concatenated id list and its total must be the same bit for bit, and
+    equal to the oracle's: the id list is where the tiles are not independent (a running total is carried over)."""
+    torch = torch_cuda
+    pkg = sdnn()
+    spec = gen.CFG2.scaled(512, 5).live()
+    rp, col, val, bias = gen.network(spec)
+    cnt = 128 * 6 + 37
+    x0 = gen.inputs(spec, cnt)
+    x0[np.arange(cnt) % 5 == 1] = 0.0
+    got = {}
+    for name, extra in (("two", 0), ("one", pkg.FLAG_ONE_TILE)):
+        h = pkg.Sdnn.create(rp, col, val, bias, max_batch=128, flags=extra | (pkg.FLAG_SKIP_DEAD if skip_dead else 0))
+        assert h.infer_tile_width() == 128
+        if host:
+            y = np.empty((cnt, spec.n), dtype=np.float32); c = np.empty(cnt, dtype=np.int32)
+            idx = np.full(cnt * spec.n, -1, dtype=np.int32)
+            total = h.infer_batch(x0, cnt, y, c, idx, idx.size, want_total=True, host=True)
+        else:
+            dx = torch.from_numpy(x0).cuda()
+            dy = torch.empty((cnt, spec.n), dtype=torch.float32, device="cuda")
+            dc = torch.empty(cnt, dtype=torch.int32, device="cuda")
+            di = torch.full((cnt * spec.n,), -1, dtype=torch.int32, device="cuda")
+            for _ in range(2):                                   # the second call reuses the second stream's buffers
+                total = h.infer_batch(dx.data_ptr(), cnt, dy.data_ptr(), dc.data_ptr(), di.data_ptr(), di.numel(), want_total=True)
+            torch.cuda.synchronize()
+            y, c, idx = dy.cpu().numpy(), dc.cpu().numpy(), di.cpu().numpy()
+        if skip_dead:
+            live = h.get_liveness()
+            assert live[-1] == int((c[128 * 6:] > 0).sum()), "liveness is that of the last tile"
+        h.destroy()
+        got[name] = (y, c, idx, total)
+    for a, b in zip(got["two"], got["one"]):
+        assert np.array_equal(a, b)
+    y, c, idx, total = got["two"]
+    xl = OracleNet(rp, col, val, bias).infer(x0)
+    check_close(y, xl, "x^L over seven tiles")
+    assert np.array_equal(c, (y != 0).sum(axis=1)) and total == int(c.sum()) and total > 0
+    assert np.array_equal(idx[:total], np.nonzero(y)[1])
+    assert (idx[total:] == -1).all()
+
+
 def test_train_cfg3_live_full_size(torch_cuda):
     """Config 3 at full size (16384 x 480, B = 64), live companion, one step."""
     spec = gen.CFG3.live()

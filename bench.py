@@ -214,6 +214,9 @@ def main():
     ap.add_argument("--tile", type=int, default=None, help="inference: batch tile (max_batch of the handle)")
     ap.add_argument("--net", default=None, metavar="N,L",
                     help="same recipe at another size, e.g. 65536,1920 for the deeper grids of the paper's Table 2")
+    ap.add_argument("--pattern", default=None, choices=["uniform", "windowed"],
+                    help="same recipe with the other pattern family: columns uniform over [0, N), or over the 1024 columns "
+                         "that a block of 1024 rows shares (the locality a good neuron order gives)")
     ap.add_argument("--flags", type=lambda s: int(s, 0), default=0, help="extra SDNN_FLAG_* bits")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -227,6 +230,9 @@ def main():
     if args.net:
         n_, l_ = (int(v) for v in args.net.split(","))
         spec = spec.scaled(n_, l_)
+    if args.pattern and args.pattern != spec.pattern:
+        import dataclasses
+        spec = dataclasses.replace(spec, name=f"{spec.name}-{args.pattern}", pattern=args.pattern, window=min(1024, spec.n))
     if args.layers:
         spec = spec.sliced(args.layers)
     if args.inputs and kind == "infer":
@@ -456,7 +462,7 @@ def main():
     except Exception as exc:      # the probe is a diagnostic; the line stands without it
         extra["gather_bound"] = {"error": str(exc)}
     achieved = alg / (per_launch_ms * 1e-3) / 1e9 if per_launch_ms else None
-    traffic = NCU_TRAFFIC.get((args.workload.replace("-live", ""), dom)) if not args.layers or kind == "train" else None
+    traffic = NCU_TRAFFIC.get((args.workload.replace("-live", ""), dom)) if (not args.layers or kind == "train") and not args.pattern and not args.net else None
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
                 "frac": achieved / hbm_peak if achieved else None, "traffic": traffic, "peak_source": peak_src,
                 "algorithmic_bytes_per_launch": alg, "launch_ms": per_launch_ms, **extra}

@@ -657,12 +657,12 @@ int lanes_begin(sdnn* h, int lanes) {
     h->last_scan_ev = nullptr;
     if (lanes < 2) return SDNN_OK;
     if (!h->ev_lane_start) CU(h, cudaEventCreateWithFlags(&h->ev_lane_start, cudaEventDisableTiming));
-    CU(h, cudaEventRecord(h->ev_lane_start, h->stream));
-    for (int i = 1; i < lanes; ++i) {
+    for (int i = 1; i < lanes; ++i) {      // before the event: new buffers are zeroed on the handle's stream
         int rc = alloc_lane(h, h->lane[i], true);
         if (rc) return rc;
-        CU(h, cudaStreamWaitEvent(h->lane[i].stream, h->ev_lane_start, 0));
     }
+    CU(h, cudaEventRecord(h->ev_lane_start, h->stream));
+    for (int i = 1; i < lanes; ++i) CU(h, cudaStreamWaitEvent(h->lane[i].stream, h->ev_lane_start, 0));
     return SDNN_OK;
 }
 int lanes_end(sdnn* h, int lanes) {
@@ -839,8 +839,6 @@ int sdnn_create_deferred(sdnn_t** out, int32_t n_layers, int32_t n_neurons, cons
             if ((rc = dev_alloc(h, &h->d_dbg_delta, L * tile, true))) return bail(rc);
     }
     {   // inference buffers (a training handle can also infer)
-        const size_t nseg = (N + NZ_SEG - 1) / NZ_SEG;
-        (void)nseg;
         h->compaction = (cfg->flags & SDNN_FLAG_SKIP_DEAD) != 0;
         h->bias_nonpositive.assign(n_layers, 0);
         h->local_pattern.assign(n_layers, 0);

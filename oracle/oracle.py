@@ -24,6 +24,13 @@ verbatim); delta^0 is never formed (x^0 is data, no z^0 exists); the bias is
 frozen unless update_bias is set, in which case b^k <- b^k - eta * mean_b delta^k_b
 (the bias read as one more column of W^k whose input is the constant 1).
 
+train_step_averaged is the other reading of the same remark ("the gradient vector delta^L ... is computed as the
+averages of gradients over the batch ... a single gradient vector is backpropagated"): delta^L = mean_b delta^L_b,
+then the backward loop above for ONE vector, paired with the batch means xbar^{k-1} = mean_b x^{k-1}_b, f' being
+evaluated from xbar^{k-1} as it is from a single input's x^{k-1}.  The remark does not fix that pairing:
+PARITY UNPINNED for this function as far as the paper goes; the pins only hold it to Algorithm 1 where the two
+must agree (B = 1, a batch of identical inputs) and to a dense restatement.
+
 All inputs are the fp32 numbers the GPU sees, widened to float64; all arithmetic
 is float64.  Heavy loops live in sdnn_oracle.c; this file only sequences them.
 """
@@ -206,3 +213,41 @@ class OracleNet:
             out["bias_grad"] = bgrads
         out["masks"] = masks
         return out
+
+    def derivative_from_activation(self, x: np.ndarray) -> np.ndarray:
+        """f' written in terms of x = f(z): clamped ReLU: 1 strictly inside (0, c); sigmoid: x (1 - x)."""
+        if self.activation == "sigmoid":
+            return x * (1.0 - x)
+        return ((x > 0.0) & (x < self.clamp)).astype(np.float64)
+
+    def train_step_averaged(self, x0, y, eta: float):
+        """Minibatch step in the averaged form (Discussion of Section 5): forward on the whole batch, delta^L averaged
+        over the batch, one vector backpropagated as in Algorithm 1 with the batch means of the activations.
+        Mutates the weights.  Returns dict(loss, x=[x^0..x^L] per input, xbar=[...], delta=[None, d^1..d^L] (each [1, n]),
+        grad=[G^1..G^L] with G^k = delta^k (x) xbar^{k-1} on the stored entries)."""
+        x = _f64(x0)
+        y = _f64(y, x.shape)
+        nb = x.shape[0]
+        eta = float(np.float32(eta))
+        xs = [x]
+        z = None
+        for k in range(self.layers):
+            z, x, _ = self.forward_layer(k, x)
+            xs.append(x)
+        xbar = [v.mean(axis=0, keepdims=True) for v in xs]
+        diff = xs[-1] - y
+        loss = float((diff * diff).sum() / (2.0 * nb))
+        delta = (diff * self.derivative_mask(z)).mean(axis=0, keepdims=True)     # average of the per-input output gradients
+        deltas = [None] * (self.layers + 1)
+        grads = [None] * self.layers
+        for k in range(self.layers - 1, -1, -1):
+            deltas[k + 1] = delta
+            s = self.transposed_product(k, delta) if k > 0 else None      # uses W before its update
+            g = self.masked_gradient(k, delta, xbar[k])
+            self.w[k] -= eta * g
+            grads[k] = g
+            if self.update_bias:
+                self.bias[k] -= eta * delta[0]
+            if k > 0:
+                delta = s * self.derivative_from_activation(xbar[k])
+        return {"loss": loss, "x": xs, "xbar": xbar, "delta": deltas, "grad": grads}

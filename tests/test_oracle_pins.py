@@ -450,3 +450,93 @@ def test_sigmoid_scalar_recurrence_and_mask_hook_refusal():
         net.train_step(np.zeros((1, n), np.float32), np.zeros((1, n), np.float32), 0.1, mask_hook=lambda *a: a[-1])
     with pytest.raises(ValueError):
         OracleNet([rp], [col], [val], [bias], activation="tanh")
+
+
+# ------------------------------------------------------------------ averaged form of the minibatch step (Discussion of Section 5)
+def _dense_averaged_step(Ws, Ms, bs, x0, y, eta, activation, clamp=32.0):
+    """The averaged step on dense masked matrices, one neuron at a time (loops, no shared code with the oracle)."""
+    f = _sig if activation == "sigmoid" else (lambda z: np.clip(z, 0.0, clamp))
+    dx = (lambda x: x * (1.0 - x)) if activation == "sigmoid" else (lambda x: ((x > 0) & (x < clamp)).astype(float))
+    B, n, L = x0.shape[0], x0.shape[1], len(Ws)
+    xs = [x0]
+    for W, b in zip(Ws, bs):
+        xs.append(f(xs[-1] @ W.T + b))
+    xbar = [v.sum(axis=0) / B for v in xs]
+    d = np.zeros(n)
+    for bb in range(B):                                   # average of the per-input output gradients
+        d += (xs[L][bb] - y[bb]) * dx(xs[L][bb]) / B
+    newW, deltas = [None] * L, [None] * (L + 1)
+    for k in range(L, 0, -1):
+        deltas[k] = d
+        W, M = Ws[k - 1], Ms[k - 1]
+        back = np.zeros(n)
+        upd = W.copy()
+        for i in range(n):
+            for j in range(n):
+                if M[i, j]:
+                    back[j] += W[i, j] * d[i]                       # old weight
+                    upd[i, j] = W[i, j] - eta * d[i] * xbar[k - 1][j]
+        newW[k - 1] = upd
+        d = back * dx(xbar[k - 1])
+    return newW, deltas, ((xs[L] - y) ** 2).sum() / (2 * B)
+
+
+@pytest.mark.parametrize("activation,seed", [("clamped_relu", 11), ("sigmoid", 12)])
+def test_averaged_step_matches_a_dense_restatement(activation, seed):
+    if activation == "sigmoid":
+        rp, c, v, b, x0, y = _sig_case(seed, n=9, layers=3, k=4, B=4)
+    else:
+        rp, c, v, b, x0, y, _, _ = live_case(seed, n=9, layers=3, k=4, B=4)
+    n, L, eta = len(b[0]), len(c), float(np.float32(0.05))
+    dn = [dense_of(rp[l], c[l], v[l].astype(float), n) for l in range(L)]
+    newW, deltas, loss = _dense_averaged_step([d[0] for d in dn], [d[1] for d in dn], [bb.astype(float) for bb in b],
+                                              x0.astype(float), y.astype(float), eta, activation)
+    net = OracleNet(rp, c, v, b, activation=activation)
+    out = net.train_step_averaged(x0, y, eta)
+    assert abs(out["loss"] - loss) <= 1e-13 * max(1.0, loss)
+    for k in range(L):
+        np.testing.assert_allclose(out["delta"][k + 1][0], deltas[k + 1], rtol=1e-12, atol=1e-15)
+        np.testing.assert_allclose(net.w[k], csr_gather(newW[k], rp[k], c[k], n), rtol=1e-12, atol=1e-15)
+        assert np.abs(out["delta"][k + 1]).max() > 1e-6                 # the comparison is not vacuous
+
+
+@pytest.mark.parametrize("activation", ["clamped_relu", "sigmoid"])
+def test_averaged_step_is_algorithm_1_where_the_two_must_agree(activation):
+    """B = 1: the averaged step is the plain step.  A batch of B copies of one input: every mean is that input's
+    vector, so the averaged step is the single-input step too (and so is the exact minibatch step)."""
+    if activation == "sigmoid":
+        rp, c, v, b, x0, y = _sig_case(21, n=11, layers=4, k=4, B=1)
+    else:
+        rp, c, v, b, x0, y, _, _ = live_case(21, n=11, layers=4, k=4, B=1)
+    eta = 0.03
+    one = OracleNet(rp, c, v, b, activation=activation)
+    ref = one.train_step(x0, y, eta)
+    avg = OracleNet(rp, c, v, b, activation=activation)
+    out = avg.train_step_averaged(x0, y, eta)
+    assert out["loss"] == ref["loss"]
+    for k in range(len(c)):
+        assert np.array_equal(avg.w[k], one.w[k])
+        assert np.array_equal(out["delta"][k + 1], ref["delta"][k + 1])
+    rep = OracleNet(rp, c, v, b, activation=activation)
+    out5 = rep.train_step_averaged(np.repeat(x0, 5, axis=0), np.repeat(y, 5, axis=0), eta)
+    assert abs(out5["loss"] - ref["loss"]) <= 1e-14 * max(1.0, ref["loss"])
+    for k in range(len(c)):
+        np.testing.assert_allclose(rep.w[k], one.w[k], rtol=1e-13, atol=1e-16)
+
+
+def test_averaged_step_differs_from_the_exact_minibatch_step_and_keeps_the_pattern():
+    """It is an approximation: on a batch of different inputs its update is not the mean of the per-input gradients
+    (the product of the means is not the mean of the products).  Like the exact step it only touches stored entries,
+    and with update_bias the bias moves by -eta * delta^k."""
+    rp, c, v, b, x0, y = _sig_case(31, n=10, layers=3, k=4, B=4)
+    eta = 0.1
+    exact = OracleNet(rp, c, v, b, activation="sigmoid")
+    exact.train_step(x0, y, eta)
+    avg = OracleNet(rp, c, v, b, activation="sigmoid", update_bias=True)
+    out = avg.train_step_averaged(x0, y, eta)
+    assert max(np.abs(avg.w[k] - exact.w[k]).max() for k in range(3)) > 1e-6
+    for k in range(3):
+        assert avg.w[k].shape == v[k].shape
+        np.testing.assert_allclose(avg.bias[k], b[k].astype(float) - float(np.float32(eta)) * out["delta"][k + 1][0], rtol=1e-13)
+        np.testing.assert_allclose(out["grad"][k], (np.asarray(v[k], dtype=float) - avg.w[k]) / float(np.float32(eta)),
+                                   rtol=1e-9, atol=1e-12)

@@ -122,7 +122,7 @@ class ClockSampler:
                 "samples": len(self.samples)}
 
 
-def oracle_train_sample(spec, B, layers, steps, warmup):
+def oracle_train_sample(spec, B, layers, steps, warmup, averaged=False):
     """Times the float64 oracle's train step on the first `layers` layers of the net (full N, full B)."""
     from oracle import OracleNet
     sl = spec.sliced(layers)
@@ -132,7 +132,10 @@ def oracle_train_sample(spec, B, layers, steps, warmup):
     for s in range(warmup + steps):
         x0, y = gen.inputs(sl, B, step=s), gen.targets(sl, B, step=s)
         t = time.perf_counter()
-        ora.train_step(x0, y, eta, keep=())
+        if averaged:
+            ora.train_step_averaged(x0, y, eta)
+        else:
+            ora.train_step(x0, y, eta, keep=())
         dt = time.perf_counter() - t
         if s >= warmup:
             times.append(dt)
@@ -170,7 +173,7 @@ def run_reference(args, spec, kind, batch, wname):
     cores = os.cpu_count()
     layers, inputs = oracle_sample_shape(spec, kind, batch, budget_edges=1.0e9)
     if kind == "train":
-        edges, times = oracle_train_sample(spec, inputs, layers, args.steps, args.warmup)
+        edges, times = oracle_train_sample(spec, inputs, layers, args.steps, args.warmup, args.averaged)
         sample = f"train step on layers 1..{layers} of {spec.layers} at full width N={spec.n}, B={inputs}"
     else:
         edges, times = oracle_infer_sample(spec, inputs, layers, args.steps, args.warmup)
@@ -181,7 +184,7 @@ def run_reference(args, spec, kind, batch, wname):
         "impl": "reference", "metric": metric_name(kind), "value": value, "unit": "edges/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": workload_config(wname, spec, kind, batch),
+        "config": workload_config(wname, spec, kind, batch, args.averaged),
         "cpu_baseline": {"value": value, "unit": "edges/s", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "edges/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -193,9 +196,10 @@ def metric_name(kind):
     return "edges_per_sec_train_step" if kind == "train" else "edges_per_sec_inference"
 
 
-def workload_config(wname, spec, kind, batch):
+def workload_config(wname, spec, kind, batch, averaged=False):
     cfg = {"workload": f"{wname}: {spec.name} {spec.n} neurons x {spec.layers} layers, {spec.k} nnz/row, "
-                       + (f"minibatch {batch}, fresh minibatch per step" if kind == "train" else f"batch tile {batch}"),
+                       + (f"minibatch {batch}, fresh minibatch per step" if kind == "train" else f"batch tile {batch}")
+                       + (", averaged form of the step (one batch-averaged vector backpropagated)" if averaged and kind == "train" else ""),
            "mode": "dense (no data-dependent skipping)", "activation": setup_of(spec)[0],
            "l2": "working set per step (weights + activations) is larger than L2; no explicit flush"
            if spec.total_nnz * 8 > 256e6 else "explicit L2 flush (256 MB write) before every timed step"}
@@ -217,6 +221,9 @@ def main():
     ap.add_argument("--pattern", default=None, choices=["uniform", "windowed"],
                     help="same recipe with the other pattern family: columns uniform over [0, N), or over the 1024 columns "
                          "that a block of 1024 rows shares (the locality a good neuron order gives)")
+    ap.add_argument("--averaged", action="store_true",
+                    help="train workloads: the averaged form of the minibatch step (one batch-averaged gradient vector is "
+                         "backpropagated; sdnn_train_step_averaged) instead of the exact minibatch step")
     ap.add_argument("--flags", type=lambda s: int(s, 0), default=0, help="extra SDNN_FLAG_* bits")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -294,10 +301,17 @@ def main():
             hy = [y.cpu().pin_memory() for y in ys]
 
             def step(i):
-                h.train_step(xs[i], ys[i], batch, eta)
+                h.train_step(xs[i], ys[i], batch, eta, averaged=args.averaged)
 
-            def step_e2e(i):
-                return h.train_step(hx[i], hy[i], batch, eta, want_loss=True, host=True)
+            if args.averaged:       # device pointers only: the copies from the pinned buffers are made here, on the same stream
+                dx, dy = torch.empty_like(xs[0]), torch.empty_like(ys[0])
+
+                def step_e2e(i):
+                    dx.copy_(hx[i], non_blocking=True); dy.copy_(hy[i], non_blocking=True)
+                    return h.train_step(dx, dy, batch, eta, want_loss=True, averaged=True)
+            else:
+                def step_e2e(i):
+                    return h.train_step(hx[i], hy[i], batch, eta, want_loss=True, host=True)
 
             h2d, d2h = 2 * batch * N * 4, 4
         else:
@@ -385,7 +399,7 @@ def main():
             e2e_value, per = shard.job_throughput(e2e_edges, max(wall_ms, dev_ms) / k_e2e, world, device="cuda")
             e2e = {"value": e2e_value, "unit": "edges/s", "h2d_bytes_per_step": h2d,
                    "d2h_bytes_per_step": d2h, "ms_per_step": per,
-                   "api": "sdnn_train_step_host" if kind == "train" else f"sdnn_infer_batch_host on {n_e2e} inputs"}
+                   "api": ("pinned-to-device copies + sdnn_train_step_averaged" if args.averaged else "sdnn_train_step_host") if kind == "train" else f"sdnn_infer_batch_host on {n_e2e} inputs"}
 
     # -------------------------------------------------------------------- inference: the same call with dead inputs dropped
     compaction = None
@@ -417,8 +431,9 @@ def main():
     nnz_l = spec.nnz_per_layer
     if kind == "train":
         ld = max(4, 1 << (batch - 1).bit_length())
+        ld_bwd = 4 if args.averaged else ld       # the averaged form backpropagates one vector
         # backward+update launch: index read + value read + value write per stored entry, x^{k-1} tile read once
-        bwd_bytes = 12 * nnz_l + N * ld * 4
+        bwd_bytes = 12 * nnz_l + N * ld_bwd * 4
         fwd_bytes = 8 * nnz_l + N * ld * 4
         dom = "backward_kernel" if bwd_ms >= fwd_ms else "forward_kernel"
         per_launch_ms = (bwd_ms if dom == "backward_kernel" else fwd_ms) / L
@@ -445,7 +460,7 @@ def main():
                           "launch, not one launch's start-to-end duration" if in_flight > 1 else "")}
     # what bounds these launches instead of HBM: random gathers of tile rows out of L2 (measured now, on this device)
     if kind == "train":
-        row_bytes, gathers = 4 * ld, (2 if dom == "backward_kernel" else 1) * nnz_l
+        row_bytes, gathers = 4 * (ld_bwd if dom == "backward_kernel" else ld), (2 if dom == "backward_kernel" else 1) * nnz_l
         table_rows = 1 << (N - 1).bit_length()
     else:
         row_bytes = min(1024, 4 * (1 << (min(batch, n_inputs) - 1).bit_length()))      # one chunk of a tile row
@@ -472,7 +487,7 @@ def main():
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         layers_s, inputs_s = oracle_sample_shape(spec, kind, batch, budget_edges=1.5e9)
         if kind == "train":
-            edges, times = oracle_train_sample(spec, inputs_s, layers_s, 2, 1)
+            edges, times = oracle_train_sample(spec, inputs_s, layers_s, 2, 1, args.averaged)
             sample = f"2 train steps on layers 1..{layers_s} of {L} at full width N={N}, B={inputs_s}"
         else:
             edges, times = oracle_infer_sample(spec, inputs_s, layers_s, 2, 1)
@@ -485,7 +500,7 @@ def main():
             "metric": metric_name(kind), "value": value, "unit": "edges/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {**workload_config(args.workload, spec, kind, batch),
+            "config": {**workload_config(args.workload, spec, kind, batch, args.averaged),
                        "parallelism": "replicas only (no collective)" if kind == "train" else "batch sharded over ranks, no collective",
                        "inputs_per_step_per_gpu": n_inputs, "setup_seconds": setup_s, "device_bytes": h.device_bytes()},
             "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,

@@ -176,6 +176,21 @@ int sdnn_train_step_host(sdnn_t* h, const float* x0, const float* target, int32_
                          float* loss_out);
 
 /*
+ * The minibatch step in the averaged form that the Discussion of Section 5 describes: the forward pass runs
+ * on all B inputs (X^k = f(W^k X^{k-1})), the final-layer gradient is the average over the batch,
+ *     delta^L = (1/B) sum_b (x^L_b - y_b) (.) f'(x^L_b),
+ * and that ONE vector is backpropagated, SpBP (Algorithm 3) running as for a single input with step eta.  The passage
+ * does not say which x^{k-1} and f'(z^{k-1}) the single vector is paired with; this library takes the batch mean
+ * xbar^{k-1} = (1/B) sum_b x^{k-1}_b for both (f' evaluated from xbar^{k-1} exactly as a single input's is from
+ * x^{k-1}): W^k(i,j) -= eta * delta^k(i) * xbar^{k-1}(j) on the stored entries, delta^{k-1} = (W^k)^T delta^k (.) f'(xbar^{k-1}).
+ * An approximation of sdnn_train_step (which averages the per-input gradients instead); identical to it at B = 1.
+ * Arguments, return values and state as sdnn_train_step (device pointers; J is the same loss).  Afterwards
+ * sdnn_get_delta returns the single backpropagated vector (float[1][N]) and sdnn_get_gradient delta^k (x) xbar^{k-1}.
+ */
+int sdnn_train_step_averaged(sdnn_t* h, const float* x0, const float* target, int32_t B, float eta,
+                             float* loss_out);
+
+/*
  * Current parameters of one layer (0-based), in the caller's original CSR order.
  *   values_out  host float[nnz_l], or NULL;   bias_out  host float[N], or NULL
  * Synchronises the stream.  Creating a new handle from these arrays resumes training.

@@ -45,6 +45,7 @@ _PROTOS = {
     "sdnn_infer_batch_host": (ctypes.c_int, [_vp, _vp, _i64, _vp, _vp, _vp, _i64, ctypes.POINTER(_i64)]),
     "sdnn_train_step": (ctypes.c_int, [_vp, _vp, _vp, _i32, _f32, ctypes.POINTER(_f32)]),
     "sdnn_train_step_host": (ctypes.c_int, [_vp, _vp, _vp, _i32, _f32, ctypes.POINTER(_f32)]),
+    "sdnn_train_step_averaged": (ctypes.c_int, [_vp, _vp, _vp, _i32, _f32, ctypes.POINTER(_f32)]),
     "sdnn_get_weights": (ctypes.c_int, [_vp, _i32, _vp, _vp]),
     "sdnn_set_weights": (ctypes.c_int, [_vp, _i32, _vp, _vp]),
     "sdnn_get_activations": (ctypes.c_int, [_vp, _i32, _vp]),
@@ -202,9 +203,13 @@ class Sdnn:
         self._check(rc)
         return total.value if want_total else None
 
-    def train_step(self, x0, target, B, eta, want_loss=False, host=False):
+    def train_step(self, x0, target, B, eta, want_loss=False, host=False, averaged=False):
+        """One minibatch step.  averaged=True: the averaged form (one backpropagated vector; device pointers only)."""
         loss = ctypes.c_float(0.0)
-        fn = self._lib.sdnn_train_step_host if host else self._lib.sdnn_train_step
+        if averaged and host:
+            raise ValueError("the averaged step takes device pointers")
+        fn = (self._lib.sdnn_train_step_averaged if averaged else
+              self._lib.sdnn_train_step_host if host else self._lib.sdnn_train_step)
         self._check(fn(self._h, _addr(x0), _addr(target), B, eta, ctypes.byref(loss) if want_loss else None))
         return loss.value if want_loss else None
 

@@ -495,6 +495,55 @@ output_gradient_kernel(const float* __restrict__ xl, const float* __restrict__ y
 }
 
 // ---------------------------------------------------------------------------------------------
+// Minibatch step in the averaged form (Discussion of Section 5: the output gradients of the batch are averaged and ONE vector is
+// backpropagated, SpBP running as for a single input).  The single input SpBP then works with is the batch mean of
+// each x^k; the two kernels below form those means and the averaged delta^L as tiles of padded width 4 (value in
+// column 0, zeros in columns 1..3), which the backward kernels process like a step with B = 1.
+//   spb: the real batch (batch = B, inv_b = 1/B); sums run over b = 0..B-1 in that order.
+__global__ void __launch_bounds__(256)
+batch_mean_kernel(const float* __restrict__ acts, float* __restrict__ mean, long long rows, int ld,
+                  const StepParams* __restrict__ spb) {
+    const int nb = spb->batch;
+    const float inv = spb->inv_b;
+    for (long long r = (long long)blockIdx.x * blockDim.x + threadIdx.x; r < rows; r += (long long)gridDim.x * blockDim.x) {
+        const float* a = acts + r * ld;
+        float s = 0.0f;
+        for (int b = 0; b < nb; ++b) s += a[b];
+        st_f4(mean + r * 4, make_float4(s * inv, 0.0f, 0.0f, 0.0f));
+    }
+}
+
+// delta^L = (1/B) sum_b (x^L_b - y_b) (.) f'(x^L_b); J = 1/(2B) sum_b |x^L_b - y_b|^2 as in output_gradient_kernel.
+__global__ void __launch_bounds__(256)
+output_gradient_averaged_kernel(const float* __restrict__ xl, const float* __restrict__ y, float* __restrict__ delta,
+                                int n, int ld, float clamp, int act, const StepParams* __restrict__ spb,
+                                double* __restrict__ loss) {
+    const int nb = spb->batch;
+    float sq = 0.0f;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+        const float* x = xl + (size_t)i * ld;
+        const float* t = y + (size_t)i * ld;
+        float acc = 0.0f;
+        for (int b = 0; b < nb; ++b) {
+            const float e = x[b] - t[b];
+            sq = fmaf(e, e, sq);
+            acc = fmaf(e, derivative(x[b], act, clamp), acc);
+        }
+        st_f4(delta + (size_t)i * 4, make_float4(acc * spb->inv_b, 0.0f, 0.0f, 0.0f));
+    }
+    __shared__ float part[8];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = sq;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double tot = 0.0;
+        for (int q = 0; q < (int)(blockDim.x >> 5); ++q) tot += (double)part[q];
+        if (tot != 0.0) atomicAdd(loss, 0.5 * tot * (double)spb->inv_b);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // Backward + update of one layer k (Algorithm 1, loop body), two realisations.
 //
 // Row units (always): for row i of W^k with delta^k[i,:] in registers, for each stored (i,j):

@@ -97,10 +97,15 @@ struct sdnn {
     double* d_loss = nullptr;
     float* d_dbg_delta = nullptr;       // [L][N][ld]   (KEEP_DEBUG)
     unsigned long long* d_mismatch = nullptr;
-    int last_b = 0, last_ld = 0;
-    cudaGraphExec_t graph = nullptr;
-    int graph_ld = 0;
-    int64_t graph_launches = 0;         // kernel nodes of the captured step
+    int last_b = 0, last_ld = 0;        // batch and padded width of the last step's activations
+    int last_delta_b = 0, last_delta_ld = 0;   // ... of its deltas (1 and 4 after a step in the averaged form)
+    // averaged form of the minibatch step (allocated at its first use)
+    float* d_mean = nullptr;            // [(L+1)][N][4]: batch means of x^0 .. x^L
+    StepParams* d_sp_batch = nullptr;   // the real batch, while d_sp describes the single backpropagated vector
+    const float* bwd_acts = nullptr;    // activations the backward launches read (NULL: d_acts)
+    cudaGraphExec_t graph = nullptr, graph_avg = nullptr;
+    int graph_ld = 0, graph_avg_ld = 0;
+    int64_t graph_launches = 0, graph_avg_launches = 0;   // kernel nodes of the captured steps
     cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};   // before forward chain, between, after backward chain
 
     // inference
@@ -376,8 +381,9 @@ void launch_backward_gvc(sdnn* h, int layer, int ld, int part) {
     BackwardArgs a{};
     a.rows = rows_of(h, layer);
     a.bias = h->d_bias + (size_t)layer * h->N;
-    a.xk = h->d_acts + (size_t)(layer + 1) * tile;
-    a.xprev = h->d_acts + (size_t)layer * tile;
+    const float* acts = h->bwd_acts ? h->bwd_acts : h->d_acts;
+    a.xk = acts + (size_t)(layer + 1) * tile;
+    a.xprev = acts + (size_t)layer * tile;
     a.dbg_grad = h->lay[layer].r_grad;
     a.sp = h->d_sp;
     a.n = h->N;
@@ -386,7 +392,7 @@ void launch_backward_gvc(sdnn* h, int layer, int ld, int part) {
     a.update_bias = h->cfg.update_bias ? 1 : 0;
     a.skip_dead = (h->cfg.flags & SDNN_FLAG_SKIP_DEAD) ? 1 : 0;
     a.pdl = h->pdl ? 1 : 0;
-    a.warm = (layer >= 1) ? h->d_acts + (size_t)(layer - 1) * tile : nullptr;
+    a.warm = (layer >= 1) ? acts + (size_t)(layer - 1) * tile : nullptr;
     a.warm_bytes = (unsigned)(tile * sizeof(float));
 #define SDNN_BWD(FROM_S, SCAT, MIR)                                                            \
     do {                                                                                       \
@@ -457,15 +463,8 @@ void launch_transpose_in(sdnn* h, const float* src, float* dst, int cnt, int col
     count_launch(h);
 }
 
-// forward + backward chain of one train step on the internal buffers; `flags` selects how the three
-// timing events are recorded (as external event-record nodes while capturing a graph)
-void enqueue_step_body(sdnn* h, int ld, unsigned flags) {
-    const size_t tile = (size_t)h->N * ld;
-    cudaEventRecordWithFlags(h->ev[0], h->stream, flags);
-    for (int k = 0; k < h->L; ++k)
-        launch_forward(h, k, h->d_acts + (size_t)k * tile, h->d_acts + (size_t)(k + 1) * tile, ld, ld);
-    cudaEventRecordWithFlags(h->ev[1], h->stream, flags);
-    launch_output_gradient(h, ld);
+// backward chain of one train step over tiles of padded width ld
+void enqueue_backward_chain(sdnn* h, int ld) {
     if (h->split) {
         // column units chain on the main stream; the row units of layer k only need delta^k and x^{k-1}, so they run on
         // the side stream beside the column units of the layers below
@@ -487,38 +486,83 @@ void enqueue_step_body(sdnn* h, int ld, unsigned flags) {
     } else {
         for (int k = h->L - 1; k >= 0; --k) launch_backward(h, k, ld);
     }
+}
+
+// forward + backward chain of one train step on the internal buffers; `flags` selects how the three
+// timing events are recorded (as external event-record nodes while capturing a graph).
+// averaged: the forward chain runs on the whole batch, then the batch means of x^0..x^L and the averaged delta^L are
+// formed and the backward chain runs on those single vectors (tiles of padded width 4).
+void enqueue_step_body(sdnn* h, int ld, unsigned flags, bool averaged) {
+    const size_t tile = (size_t)h->N * ld;
+    cudaEventRecordWithFlags(h->ev[0], h->stream, flags);
+    for (int k = 0; k < h->L; ++k)
+        launch_forward(h, k, h->d_acts + (size_t)k * tile, h->d_acts + (size_t)(k + 1) * tile, ld, ld);
+    cudaEventRecordWithFlags(h->ev[1], h->stream, flags);
+    if (!averaged) {
+        launch_output_gradient(h, ld);
+        enqueue_backward_chain(h, ld);
+    } else {
+        const long long rows = (long long)(h->L + 1) * h->N;
+        const int grid_m = (int)std::min<long long>((rows + 255) / 256, (long long)h->sms * 16);
+        batch_mean_kernel<<<grid_m, 256, 0, h->stream>>>(h->d_acts, h->d_mean, rows, ld, h->d_sp_batch);
+        const size_t tile1 = (size_t)h->N * 4;
+        float* dl = h->mirror ? delta_tile(h, h->L - 1, tile1)
+                              : (h->d_dbg_delta ? h->d_dbg_delta + (size_t)(h->L - 1) * tile1 : h->d_dl);
+        const int grid_g = std::min((h->N + 255) / 256, h->sms * 8);
+        output_gradient_averaged_kernel<<<grid_g, 256, 0, h->stream>>>(h->d_acts + (size_t)h->L * tile, h->d_yt, dl, h->N, ld,
+                                                                     h->cfg.clamp, h->cfg.activation, h->d_sp_batch, h->d_loss);
+        count_launch(h, 2);
+        h->bwd_acts = h->d_mean;
+        enqueue_backward_chain(h, 4);
+        h->bwd_acts = nullptr;
+    }
     cudaEventRecordWithFlags(h->ev[2], h->stream, flags);
 }
 
-int train_step_device(sdnn* h, const float* x0, const float* target, int B, float eta, float* loss_out) {
+int train_step_device(sdnn* h, const float* x0, const float* target, int B, float eta, float* loss_out, bool averaged = false) {
     const int ld = padded_width(B);
-    set_step_params_kernel<<<1, 1, 0, h->stream>>>(h->d_sp, eta, B, h->d_loss);
-    count_launch(h);
+    if (averaged) {
+        if (!h->d_mean) {
+            int rc;
+            if ((rc = dev_alloc(h, &h->d_mean, (size_t)(h->L + 1) * h->N * 4, true))) return rc;
+            if ((rc = dev_alloc(h, &h->d_sp_batch, 1, true))) return rc;
+        }
+        set_step_params_kernel<<<1, 1, 0, h->stream>>>(h->d_sp_batch, eta, B, h->d_loss);
+        set_step_params_kernel<<<1, 1, 0, h->stream>>>(h->d_sp, eta, 1, h->d_loss);
+        count_launch(h, 2);
+    } else {
+        set_step_params_kernel<<<1, 1, 0, h->stream>>>(h->d_sp, eta, B, h->d_loss);
+        count_launch(h);
+    }
     launch_transpose_in(h, x0, h->d_acts, B, ld, ld);
     launch_transpose_in(h, target, h->d_yt, B, ld, ld);
     if (h->cfg.flags & SDNN_FLAG_NO_GRAPH) {
-        enqueue_step_body(h, ld, cudaEventRecordDefault);
+        enqueue_step_body(h, ld, cudaEventRecordDefault, averaged);
     } else {
-        if (!h->graph || h->graph_ld != ld) {
-            if (h->graph) { cudaGraphExecDestroy(h->graph); h->graph = nullptr; }
+        cudaGraphExec_t& graph = averaged ? h->graph_avg : h->graph;
+        int& graph_ld = averaged ? h->graph_avg_ld : h->graph_ld;
+        int64_t& graph_launches = averaged ? h->graph_avg_launches : h->graph_launches;
+        if (!graph || graph_ld != ld) {
+            if (graph) { cudaGraphExecDestroy(graph); graph = nullptr; }
             cudaGraph_t g = nullptr;
             const int64_t before = h->launches;
             CU(h, cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal));
-            enqueue_step_body(h, ld, cudaEventRecordExternal);
+            enqueue_step_body(h, ld, cudaEventRecordExternal, averaged);
             cudaError_t e = cudaStreamEndCapture(h->stream, &g);
-            h->graph_launches = h->launches - before;
+            graph_launches = h->launches - before;
             h->launches = before;
             if (e != cudaSuccess) return cuda_fail(h, e, "cudaStreamEndCapture");
-            e = cudaGraphInstantiate(&h->graph, g, 0);
+            e = cudaGraphInstantiate(&graph, g, 0);
             cudaGraphDestroy(g);
-            if (e != cudaSuccess) { h->graph = nullptr; return cuda_fail(h, e, "cudaGraphInstantiate"); }
-            h->graph_ld = ld;
+            if (e != cudaSuccess) { graph = nullptr; return cuda_fail(h, e, "cudaGraphInstantiate"); }
+            graph_ld = ld;
         }
-        CU(h, cudaGraphLaunch(h->graph, h->stream));
-        count_launch(h, (int)h->graph_launches);
+        CU(h, cudaGraphLaunch(graph, h->stream));
+        count_launch(h, (int)graph_launches);
     }
     CU(h, cudaGetLastError());
     h->stepped = true; h->last_b = B; h->last_ld = ld;
+    h->last_delta_b = averaged ? 1 : B; h->last_delta_ld = averaged ? 4 : ld;
     if (loss_out) {
         double j = 0.0;
         CU(h, cudaMemcpyAsync(&j, h->d_loss, sizeof(double), cudaMemcpyDeviceToHost, h->stream));
@@ -740,6 +784,7 @@ void sdnn_destroy(sdnn_t* h) {
     cudaSetDevice(h->device);
     if (h->stream || h->own_stream) cudaStreamSynchronize(h->stream);
     if (h->graph) cudaGraphExecDestroy(h->graph);
+    if (h->graph_avg) cudaGraphExecDestroy(h->graph_avg);
     for (cudaEvent_t e : h->ev) if (e) cudaEventDestroy(e);
     for (InferLane& ln : h->lane) {
         if (ln.ev_scan) cudaEventDestroy(ln.ev_scan);
@@ -1002,6 +1047,13 @@ int sdnn_train_step(sdnn_t* h, const float* x0, const float* target, int32_t B, 
     return train_step_device(h, x0, target, B, eta, loss_out);
 }
 
+int sdnn_train_step_averaged(sdnn_t* h, const float* x0, const float* target, int32_t B, float eta, float* loss_out) {
+    int rc = check_train_args(h, x0, target, B, eta);
+    if (rc) return rc;
+    CU(h, cudaSetDevice(h->device));
+    return train_step_device(h, x0, target, B, eta, loss_out, true);
+}
+
 int sdnn_train_step_host(sdnn_t* h, const float* x0, const float* target, int32_t B, float eta, float* loss_out) {
     int rc = check_train_args(h, x0, target, B, eta);
     if (rc) return rc;
@@ -1176,9 +1228,9 @@ int sdnn_mirror_mismatches(sdnn_t* h, int32_t layer, int64_t* count_out) {
     return SDNN_OK;
 }
 
-static int fetch_tile(sdnn_t* h, const float* tile, float* out) {
+static int fetch_tile(sdnn_t* h, const float* tile, float* out, int B, int ld) {
     // tile [N][ld] on the device -> out [B][N] on the host
-    const int B = h->last_b, ld = h->last_ld, N = h->N;
+    const int N = h->N;
     std::vector<float> tmp((size_t)N * ld);
     CU(h, cudaSetDevice(h->device));
     CU(h, cudaStreamSynchronize(h->stream));
@@ -1192,14 +1244,14 @@ int sdnn_get_activations(sdnn_t* h, int32_t layer, float* out) {
     if (!h || !out) return SDNN_ERR_INVALID_ARG;
     if (!h->stepped) return fail(h, SDNN_ERR_STATE, "no train step has run");
     if (layer < 0 || layer > h->L) return fail(h, SDNN_ERR_INVALID_ARG, "layer %d outside [0, %d]", layer, h->L);
-    return fetch_tile(h, h->d_acts + (size_t)layer * h->N * h->last_ld, out);
+    return fetch_tile(h, h->d_acts + (size_t)layer * h->N * h->last_ld, out, h->last_b, h->last_ld);
 }
 
 int sdnn_get_delta(sdnn_t* h, int32_t layer, float* out) {
     if (!h || !out) return SDNN_ERR_INVALID_ARG;
     if (!h->stepped || !h->d_dbg_delta) return fail(h, SDNN_ERR_STATE, "needs SDNN_FLAG_KEEP_DEBUG and a train step");
     if (layer < 1 || layer > h->L) return fail(h, SDNN_ERR_INVALID_ARG, "layer %d outside [1, %d]", layer, h->L);
-    return fetch_tile(h, h->d_dbg_delta + (size_t)(layer - 1) * h->N * h->last_ld, out);
+    return fetch_tile(h, h->d_dbg_delta + (size_t)(layer - 1) * h->N * h->last_delta_ld, out, h->last_delta_b, h->last_delta_ld);
 }
 
 int sdnn_get_gradient(sdnn_t* h, int32_t layer, float* out) {

@@ -225,6 +225,101 @@ def test_train_paper_setup_sigmoid_uniform_weights(torch_cuda):
     print(spec.name, st)
 
 
+def averaged_parity(torch, arrays, batches, eta, flags=0, update_bias=False, activation="sigmoid"):
+    """The averaged form of the minibatch step on both sides, everything compared after every step (parameters
+    re-synchronised before each step as in train_parity)."""
+    pkg = sdnn()
+    rp, col, val, bias = arrays
+    L, n = len(col), len(bias[0])
+    B = batches[0][0].shape[0]
+    h = pkg.Sdnn.create(rp, col, val, bias, max_batch=B, train=True, update_bias=update_bias, flags=pkg.FLAG_KEEP_DEBUG | flags,
+                        activation=pkg.ACT_SIGMOID if activation == "sigmoid" else pkg.ACT_CLAMPED_RELU)
+    ora = OracleNet(rp, col, val, bias, update_bias=update_bias, activation=activation)
+    worst = 0.0
+    for step, (x0, y) in enumerate(batches):
+        if step > 0:
+            ora.quantize_state()
+            for l in range(L):
+                h.set_weights(l, ora.w[l], ora.bias[l])
+        loss_g = h.train_step(torch.from_numpy(x0).cuda(), torch.from_numpy(y).cuda(), B, eta, want_loss=True, averaged=True)
+        out = ora.train_step_averaged(x0, y, eta)
+        errs = {"loss": abs(loss_g - out["loss"]) / max(abs(out["loss"]), 1e-30)}
+        for k in range(1, L + 1):
+            errs[f"x{k}"] = check_close(h.get_activations(k, B), out["x"][k], f"step {step} x^{k}")
+            errs[f"d{k}"] = check_close(h.get_delta(k, 1), out["delta"][k], f"step {step} delta^{k}")
+            errs[f"g{k}"] = check_close(h.get_gradient(k), out["grad"][k - 1], f"step {step} G^{k}")
+            w, b = h.get_weights(k - 1)
+            errs[f"w{k}"] = check_close(w, ora.w[k - 1], f"step {step} W^{k}")
+            errs[f"b{k}"] = check_close(b, ora.bias[k - 1], f"step {step} b^{k}")
+            assert np.any(out["grad"][k - 1] != 0.0), "vacuous: the gradient is zero"
+            assert h.mirror_mismatches(k - 1) == 0
+        key = max(errs, key=errs.get)
+        assert errs[key] <= TOL, f"{key}: rel err {errs[key]:.3g} > {TOL}"
+        worst = max(worst, errs[key])
+    h.destroy()
+    return worst
+
+
+@pytest.mark.parametrize("bwd", sorted(BWD_MODES))
+@pytest.mark.parametrize("B", [1, 5, 16, 64])
+def test_train_averaged_form_sigmoid_ragged_small(torch_cuda, B, bwd):
+    """Averaged minibatch step (batch-averaged delta^L, one vector backpropagated with the batch means), sigmoid."""
+    rng = np.random.default_rng(500 + B)
+    arrays = ragged_net(rng, n=203, layers=4, kmax=12)
+    batches = [(rng.uniform(0, 1.0, size=(B, 203)).astype(np.float32), rng.uniform(0, 1, size=(B, 203)).astype(np.float32))
+               for _ in range(3)]
+    averaged_parity(torch_cuda, arrays, batches, eta=0.05, flags=BWD_MODES[bwd], update_bias=(B % 2 == 1))
+
+
+@pytest.mark.parametrize("bwd", sorted(BWD_MODES))
+def test_train_averaged_form_clamped_relu(torch_cuda, bwd):
+    rng = np.random.default_rng(77)
+    arrays = ragged_net(rng, n=301, layers=4, kmax=10, scale=0.5)
+    batches = [(rng.uniform(0, 1.0, size=(16, 301)).astype(np.float32), rng.uniform(0, 1, size=(16, 301)).astype(np.float32))
+               for _ in range(2)]
+    averaged_parity(torch_cuda, arrays, batches, eta=0.01, flags=BWD_MODES[bwd], activation="clamped_relu")
+
+
+def test_train_averaged_form_on_the_paper_setup_and_graph_reuse(torch_cuda):
+    """4096 x 24 net with the paper's setup, B = 16; then averaged and exact steps alternate on one handle (each has a
+    captured launch sequence of its own) and match two oracles run the same way."""
+    spec = gen.CFG3.scaled(4096, 24).paper_setup()
+    print("worst", averaged_parity(torch_cuda, gen.network(spec), batches_for(spec, 16, 2), eta=0.01))
+    pkg = sdnn()
+    torch = torch_cuda
+    spec = gen.CFG3.scaled(1024, 6).paper_setup()
+    rp, col, val, bias = gen.network(spec)
+    h = pkg.Sdnn.create(rp, col, val, bias, max_batch=8, train=True, activation=pkg.ACT_SIGMOID)
+    ora = OracleNet(rp, col, val, bias, activation="sigmoid")
+    for step, (x0, y) in enumerate(batches_for(spec, 8, 4)):
+        avg = step % 2 == 0
+        loss_g = h.train_step(torch.from_numpy(x0).cuda(), torch.from_numpy(y).cuda(), 8, 0.01, want_loss=True, averaged=avg)
+        out = ora.train_step_averaged(x0, y, 0.01) if avg else ora.train_step(x0, y, 0.01)
+        assert abs(loss_g - out["loss"]) <= TOL * abs(out["loss"])
+        for l in range(spec.layers):
+            check_close(h.get_weights(l, want_bias=False), ora.w[l], f"step {step} W^{l + 1}")
+    h.destroy()
+
+
+def test_train_averaged_form_is_the_plain_step_for_one_input(torch_cuda):
+    """B = 1: the mean of one vector is the vector; both entry points must leave the same bits."""
+    pkg = sdnn()
+    torch = torch_cuda
+    rng = np.random.default_rng(9)
+    rp, col, val, bias = ragged_net(rng, n=203, layers=5, kmax=12)
+    x0 = rng.uniform(0, 1, size=(1, 203)).astype(np.float32); y = rng.uniform(0, 1, size=(1, 203)).astype(np.float32)
+    got = []
+    for avg in (False, True):
+        h = pkg.Sdnn.create(rp, col, val, bias, max_batch=4, train=True, update_bias=True)
+        for _ in range(3):
+            loss = h.train_step(torch.from_numpy(x0).cuda(), torch.from_numpy(y).cuda(), 1, 0.02, want_loss=True, averaged=avg)
+        got.append((loss, [h.get_weights(l) for l in range(5)]))
+        h.destroy()
+    assert got[0][0] == got[1][0]
+    for (w0, b0), (w1, b1) in zip(got[0][1], got[1][1]):
+        assert np.array_equal(w0, w1) and np.array_equal(b0, b1)
+
+
 def test_infer_sigmoid_matches_oracle(torch_cuda):
     pkg = sdnn()
     spec = gen.CFG2.scaled(1024, 10).paper_setup()

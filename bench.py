@@ -438,9 +438,14 @@ def main():
         dom = "backward_kernel" if bwd_ms >= fwd_ms else "forward_kernel"
         per_launch_ms = (bwd_ms if dom == "backward_kernel" else fwd_ms) / L
         alg = bwd_bytes if dom == "backward_kernel" else fwd_bytes
-        extra = {"backward_launches": "per layer one column-unit launch (backward_kernel<..,1,..>) on the main stream and one "
-                                      "row-unit launch (backward_kernel<..,0,..>) on a side stream, running beside each other; "
+        # tiles of padded width 4 (B <= 4, or the averaged form's backward chain) run the entry-parallel kernels
+        ep = not (args.flags & 0x81)
+        names = ("backward_col_ep_kernel", "backward_row_ep_kernel") if ep and ld_bwd == 4 else \
+                ("backward_kernel<..,1,..>", "backward_kernel<..,0,..>")
+        extra = {"backward_launches": f"per layer one column-unit launch ({names[0]}) on the main stream and one "
+                                      f"row-unit launch ({names[1]}) on a side stream, running beside each other; "
                                       "launch_ms is the backward chain's time per layer, bytes and gathers are those of both",
+                 "kernel_names": {"forward": "forward_ep_kernel" if ep and ld == 4 else "forward_kernel", "backward": list(names)},
                  "fwd_ms_per_step": fwd_ms, "bwd_ms_per_step": bwd_ms,
                  "fwd_GBps": fwd_bytes * L / (fwd_ms * 1e-3) / 1e9 if fwd_ms else None,
                  "bwd_GBps": bwd_bytes * L / (bwd_ms * 1e-3) / 1e9 if bwd_ms else None,

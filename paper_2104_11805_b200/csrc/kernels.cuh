@@ -775,6 +775,175 @@ backward_kernel(const BackwardArgs a) {
 }
 
 // ---------------------------------------------------------------------------------------------
+// Layer kernels for tiles of padded width 4 (B <= 4: per-input SGD as in Algorithm 1, single vectors).
+// With so few batch entries a row's work is its entries, not its batch: a lane per row (the mapping above) leaves a
+// 1024-neuron layer to 32 warps that each walk 32 entries in four dependent steps.  Here a warp takes one SLICE of 16
+// rows and a lane takes (row r = lane & 15, every second chunk starting at lane >> 4): the 32 lanes of one iteration
+// read 512 contiguous bytes of indices and of values, up to EP_IT iterations (8 chunks, 32 entries per row) are in
+// flight together, so a row of up to 32 entries costs one memory round trip for its entries and one for its
+// gathers; the two lanes of a row add their partial sums with one shuffle.  Arithmetic per entry is the same as in
+// the kernels above (lane_dot, fma(-step, g, w)), so the two copies of a layer stay bit-identical here too.
+constexpr int EP_IT = 4;
+
+struct EpShape { int lane, r, h, so, nch, item; };
+__device__ __forceinline__ EpShape ep_shape(const Sliced& m, int n) {
+    EpShape e;
+    e.lane = threadIdx.x & 31; e.r = e.lane & 15; e.h = e.lane >> 4;
+    const int s = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int ns = (n + SLICE - 1) / SLICE;
+    e.so = 0; e.nch = 0; e.item = n;
+    if (s < ns) {
+        e.so = m.slice_off[s];
+        e.nch = (m.slice_off[s + 1] - e.so) / CHUNK_ROW;
+        e.item = min(n, s * SLICE + e.r);
+    }
+    return e;
+}
+
+#define SDNN_EP_LOAD_IDX(C, T0)                                                                         \
+    _Pragma("unroll") for (int i = 0; i < EP_IT; ++i) {                                                  \
+        const int t = (T0) + 2 * i + e.h;                                                                \
+        C[i] = (t < e.nch) ? __ldcs(reinterpret_cast<const int4*>(m.idx + e.so + t * CHUNK_ROW + e.r * 4)) : make_int4(0, 0, 0, 0); \
+    }
+
+__global__ void __launch_bounds__(128)
+forward_ep_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict__ xin, float* __restrict__ xout,
+                  int n, float clamp, int act, int pdl) {
+    const EpShape e = ep_shape(m, n);
+    int4 c[EP_IT];
+    SDNN_EP_LOAD_IDX(c, 0)
+    const float b = (e.item < n) ? bias[e.item] : 0.0f;
+    if (pdl) grid_dependency_wait();
+    Lane<4> acc;
+    lane_fill(acc, 0.0f);
+    for (int t0 = 0; t0 < e.nch; t0 += 2 * EP_IT) {
+        float4 w[EP_IT];
+        Lane<4> x[4 * EP_IT];
+#pragma unroll
+        for (int i = 0; i < EP_IT; ++i) {
+            const int t = t0 + 2 * i + e.h;
+            w[i] = (t < e.nch) ? __ldcs(reinterpret_cast<const float4*>(m.val + e.so + t * CHUNK_ROW + e.r * 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int i = 0; i < EP_IT; ++i) { SDNN_GATHER_CHUNK(x, i, c[i], xin, 16u) }
+        if (t0 + 2 * EP_IT < e.nch) { SDNN_EP_LOAD_IDX(c, t0 + 2 * EP_IT) }
+#pragma unroll
+        for (int i = 0; i < EP_IT; ++i) {
+            lane_fma(w[i].x, x[4 * i + 0], acc); lane_fma(w[i].y, x[4 * i + 1], acc);
+            lane_fma(w[i].z, x[4 * i + 2], acc); lane_fma(w[i].w, x[4 * i + 3], acc);
+        }
+    }
+    acc.a.x += __shfl_xor_sync(0xffffffffu, acc.a.x, 16); acc.a.y += __shfl_xor_sync(0xffffffffu, acc.a.y, 16);
+    acc.a.z += __shfl_xor_sync(0xffffffffu, acc.a.z, 16); acc.a.w += __shfl_xor_sync(0xffffffffu, acc.a.w, 16);
+    if (e.h == 0 && e.item < n) {
+        acc.a.x += b; acc.a.y += b; acc.a.z += b; acc.a.w += b;
+        lane_activate(acc, act, clamp);
+        lane_store(xout + (size_t)e.item * 4, acc);
+    }
+    if (pdl) grid_launch_dependents();
+}
+
+// new values of the four entries of chunk t (positions 4t .. 4t+3 of a unit with `len` stored entries; padding keeps its 0)
+__device__ __forceinline__ float4 ep_update(const float4& w, float p0, float p1, float p2, float p3, int t, int len, float step) {
+    const int q = 4 * t;
+    return make_float4(q + 0 < len ? __fmaf_rn(-step, p0, w.x) : w.x, q + 1 < len ? __fmaf_rn(-step, p1, w.y) : w.y,
+                       q + 2 < len ? __fmaf_rn(-step, p2, w.z) : w.z, q + 3 < len ? __fmaf_rn(-step, p3, w.w) : w.w);
+}
+
+// Column units (transposed copy m): delta^{k-1}[j] = (sum_i w(i,j) delta^k[i]) (.) f'(x^{k-1}[j]) with the values before
+// their update, and the update of the transposed copy's values.
+__global__ void __launch_bounds__(128)
+backward_col_ep_kernel(Sliced m, const float* __restrict__ xprev, const float* __restrict__ dk, float* __restrict__ dprev,
+                       int n, float clamp, int act, const StepParams* __restrict__ sp, int pdl) {
+    const EpShape e = ep_shape(m, n);
+    int4 c[EP_IT];
+    SDNN_EP_LOAD_IDX(c, 0)
+    int len = 0, j = 0;
+    if (e.item < n) { len = m.len[e.item]; j = m.order[e.item]; }
+    if (pdl) grid_dependency_wait();
+    const float step = sp->eta * sp->inv_b;
+    Lane<4> xj, acc;
+    lane_fill(xj, 0.0f); lane_fill(acc, 0.0f);
+    if (e.item < n) lane_load(xj, xprev + (size_t)j * 4);
+    for (int t0 = 0; t0 < e.nch; t0 += 2 * EP_IT) {
+        float4 w[EP_IT];
+        Lane<4> d[4 * EP_IT];
+#pragma unroll
+        for (int i = 0; i < EP_IT; ++i) {
+            const int t = t0 + 2 * i + e.h;
+            w[i] = (t < e.nch) ? ld_f4(m.val + e.so + t * CHUNK_ROW + e.r * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int i = 0; i < EP_IT; ++i) { SDNN_GATHER_CHUNK(d, i, c[i], dk, 16u) }
+        if (t0 + 2 * EP_IT < e.nch) { SDNN_EP_LOAD_IDX(c, t0 + 2 * EP_IT) }
+#pragma unroll
+        for (int i = 0; i < EP_IT; ++i) {
+            const int t = t0 + 2 * i + e.h;
+            lane_fma(w[i].x, d[4 * i + 0], acc); lane_fma(w[i].y, d[4 * i + 1], acc);
+            lane_fma(w[i].z, d[4 * i + 2], acc); lane_fma(w[i].w, d[4 * i + 3], acc);
+            if (t < e.nch)
+                st_f4(m.val + e.so + t * CHUNK_ROW + e.r * 4,
+                      ep_update(w[i], lane_dot(d[4 * i + 0], xj), lane_dot(d[4 * i + 1], xj), lane_dot(d[4 * i + 2], xj),
+                                lane_dot(d[4 * i + 3], xj), t, len, step));
+        }
+    }
+    acc.a.x += __shfl_xor_sync(0xffffffffu, acc.a.x, 16); acc.a.y += __shfl_xor_sync(0xffffffffu, acc.a.y, 16);
+    acc.a.z += __shfl_xor_sync(0xffffffffu, acc.a.z, 16); acc.a.w += __shfl_xor_sync(0xffffffffu, acc.a.w, 16);
+    if (e.h == 0 && e.item < n) {
+        lane_mask(acc, xj, act, clamp);
+        lane_store(dprev + (size_t)j * 4, acc);
+    }
+    if (pdl) grid_launch_dependents();
+}
+
+// Row units (row-major copy m): update of its values (and of the bias) from delta^k[i] and the gathered x^{k-1}[j].
+template <bool DBG>
+__global__ void __launch_bounds__(128)
+backward_row_ep_kernel(Sliced m, float* __restrict__ bias, const float* __restrict__ xprev, const float* __restrict__ dk,
+                       float* __restrict__ dbg_grad, int n, const StepParams* __restrict__ sp, int update_bias, int pdl) {
+    const EpShape e = ep_shape(m, n);
+    int4 c[EP_IT];
+    SDNN_EP_LOAD_IDX(c, 0)
+    const int len = (e.item < n) ? m.len[e.item] : 0;
+    if (pdl) grid_dependency_wait();
+    const float inv_b = sp->inv_b;
+    const float step = sp->eta * inv_b;
+    Lane<4> d;
+    lane_fill(d, 0.0f);
+    if (e.item < n) lane_load(d, dk + (size_t)e.item * 4);
+    if (update_bias && e.h == 0 && e.item < n) bias[e.item] -= step * lane_sum(d);
+    for (int t0 = 0; t0 < e.nch; t0 += 2 * EP_IT) {
+        float4 w[EP_IT];
+        Lane<4> x[4 * EP_IT];
+#pragma unroll
+        for (int i = 0; i < EP_IT; ++i) {
+            const int t = t0 + 2 * i + e.h;
+            w[i] = (t < e.nch) ? ld_f4(m.val + e.so + t * CHUNK_ROW + e.r * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int i = 0; i < EP_IT; ++i) { SDNN_GATHER_CHUNK(x, i, c[i], xprev, 16u) }
+        if (t0 + 2 * EP_IT < e.nch) { SDNN_EP_LOAD_IDX(c, t0 + 2 * EP_IT) }
+#pragma unroll
+        for (int i = 0; i < EP_IT; ++i) {
+            const int t = t0 + 2 * i + e.h;
+            if (t < e.nch) {
+                const float p0 = lane_dot(d, x[4 * i + 0]), p1 = lane_dot(d, x[4 * i + 1]), p2 = lane_dot(d, x[4 * i + 2]),
+                            p3 = lane_dot(d, x[4 * i + 3]);
+                const int at = e.so + t * CHUNK_ROW + e.r * 4;
+                st_f4(m.val + at, ep_update(w[i], p0, p1, p2, p3, t, len, step));
+                if (DBG) {
+                    const int q = 4 * t;
+                    st_f4(dbg_grad + at, make_float4(q + 0 < len ? p0 * inv_b : 0.f, q + 1 < len ? p1 * inv_b : 0.f,
+                                                     q + 2 < len ? p2 * inv_b : 0.f, q + 3 < len ? p3 * inv_b : 0.f));
+                }
+            }
+        }
+    }
+    if (pdl) grid_launch_dependents();
+}
+#undef SDNN_EP_LOAD_IDX
+
+// ---------------------------------------------------------------------------------------------
 // Fills the transposed copy's values from the row-major copy: entry (column j, row i) of the transposed
 // copy is looked up by binary search in row i (ascending columns).  One warp per transposed unit.
 // With `mismatch` non-NULL nothing is written; entries whose bits differ from the row-major copy are counted.

@@ -278,7 +278,7 @@ int resident_ctas(sdnn* h, const void* kernel, int block) {
     return occ;
 }
 
-std::pair<int, int> plan_grid(sdnn* h, const void* kernel, int units, int chunks) {
+std::pair<int, int> plan_grid(sdnn* h, const void* kernel, int units, int chunks, int oneshot_wpb = 0) {
     auto key = std::make_tuple(kernel, units, chunks);
     auto it = h->plans.find(key);
     if (it != h->plans.end()) return it->second;
@@ -303,6 +303,7 @@ std::pair<int, int> plan_grid(sdnn* h, const void* kernel, int units, int chunks
             if (eff > best) { best = eff; pick = {gx, block}; }
         }
     }
+    if (oneshot_wpb > 0) pick = {(units + oneshot_wpb - 1) / oneshot_wpb, oneshot_wpb * 32};
     h->plans[key] = pick;
     return pick;
 }
@@ -350,9 +351,18 @@ void launch_forward_gv(sdnn* h, int layer, const float* xin, float* xout, int ld
 }
 
 // track: compaction mode (process only the live columns, mark the columns that stay live)
+// Tiles of padded width 4 take the kernels that give a lane a row's chunk instead of a row (see kernels.cuh), unless
+// the handle asked for one of the other backward realisations: those keep the common kernels at every width.
+bool entry_parallel(const sdnn* h, int ld) {
+    return ld == 4 && !(h->cfg.flags & (SDNN_FLAG_BWD_ATOMICS | SDNN_FLAG_BWD_ONE_LAUNCH));
+}
+
 void launch_forward(sdnn* h, int layer, const float* xin, float* xout, int ld, int cols, bool track = false) {
     const Geometry q = geometry(cols);
-    if (q.v == 4) launch_forward_gv<1, 4>(h, layer, xin, xout, ld, q.chunks, track);
+    if (q.v == 4 && !track && entry_parallel(h, ld)) {
+        launch_k(h, forward_ep_kernel, dim3((h->NS + 3) / 4), dim3(128), h->pdl, rows_of(h, layer),
+                 (const float*)(h->d_bias + (size_t)layer * h->N), xin, xout, h->N, h->cfg.clamp, h->cfg.activation, h->pdl ? 1 : 0);
+    } else if (q.v == 4) launch_forward_gv<1, 4>(h, layer, xin, xout, ld, q.chunks, track);
     else switch (q.g) {
         case 1: launch_forward_gv<1, 8>(h, layer, xin, xout, ld, q.chunks, track); break;
         case 2: launch_forward_gv<2, 8>(h, layer, xin, xout, ld, q.chunks, track); break;
@@ -394,13 +404,18 @@ void launch_backward_gvc(sdnn* h, int layer, int ld, int part) {
     a.pdl = h->pdl ? 1 : 0;
     a.warm = (layer >= 1) ? acts + (size_t)(layer - 1) * tile : nullptr;
     a.warm_bytes = (unsigned)(tile * sizeof(float));
+    // The two launches of a layer in the split realisation run beside each other (and beside those of the next layer):
+    // one warp per CTA and one unit per warp lets the hardware interleave them unit by unit, which measured 6 % (config 5)
+    // and 9 % (config 3) faster than two persistent grids sharing the SMs.  Alone on the device (forward, one launch per
+    // layer) the persistent grid is the faster one.
+    const int os_ = (h->split && part != 0) ? 1 : 0;
 #define SDNN_BWD(FROM_S, SCAT, MIR)                                                            \
     do {                                                                                       \
         if (a.dbg_grad) {                                                                      \
-            auto plan = plan_grid(h, (const void*)backward_kernel<G, V, CPS, FROM_S, SCAT, MIR, true>, units, 1);   \
+            auto plan = plan_grid(h, (const void*)backward_kernel<G, V, CPS, FROM_S, SCAT, MIR, true>, units, 1, os_);   \
             launch_k(h, backward_kernel<G, V, CPS, FROM_S, SCAT, MIR, true>, dim3(plan.first), dim3(plan.second), h->pdl, a); \
         } else {                                                                               \
-            auto plan = plan_grid(h, (const void*)backward_kernel<G, V, CPS, FROM_S, SCAT, MIR, false>, units, 1);  \
+            auto plan = plan_grid(h, (const void*)backward_kernel<G, V, CPS, FROM_S, SCAT, MIR, false>, units, 1, os_);  \
             launch_k(h, backward_kernel<G, V, CPS, FROM_S, SCAT, MIR, false>, dim3(plan.first), dim3(plan.second), h->pdl, a); \
         }                                                                                      \
     } while (0)
@@ -433,9 +448,30 @@ void launch_backward_gv(sdnn* h, int layer, int ld, int part) {
     launch_backward_gvc<G, V, 2>(h, layer, ld, part);
 }
 
+// the two launches of a layer in the split transposed realisation, for tiles of padded width 4
+void launch_backward_ep(sdnn* h, int layer, int part) {
+    const size_t tile = (size_t)h->N * 4;
+    const float* acts = h->bwd_acts ? h->bwd_acts : h->d_acts;
+    const float* xprev = acts + (size_t)layer * tile;
+    const float* dk = delta_tile(h, layer, tile);
+    const dim3 grid((h->NS + 3) / 4), block(128);
+    if (part == 1) {
+        launch_k(h, backward_col_ep_kernel, grid, block, h->pdl, cols_of(h, layer), xprev, dk, delta_tile(h, layer - 1, tile), h->N,
+                 h->cfg.clamp, h->cfg.activation, (const StepParams*)h->d_sp, h->pdl ? 1 : 0);
+    } else {
+        float* bias = h->d_bias + (size_t)layer * h->N;
+        float* grad = h->lay[layer].r_grad;
+        if (grad) launch_k(h, backward_row_ep_kernel<true>, grid, block, false, rows_of(h, layer), bias, xprev, dk, grad, h->N,
+                           (const StepParams*)h->d_sp, h->cfg.update_bias ? 1 : 0, 0);
+        else launch_k(h, backward_row_ep_kernel<false>, grid, block, false, rows_of(h, layer), bias, xprev, dk, grad, h->N,
+                      (const StepParams*)h->d_sp, h->cfg.update_bias ? 1 : 0, 0);
+    }
+}
+
 void launch_backward(sdnn* h, int layer, int ld, int part = 0) {
     const Geometry q = geometry(ld);
-    if (q.v == 4) launch_backward_gv<1, 4>(h, layer, ld, part);
+    if (q.v == 4 && h->split && part != 0 && entry_parallel(h, ld)) launch_backward_ep(h, layer, part);
+    else if (q.v == 4) launch_backward_gv<1, 4>(h, layer, ld, part);
     else switch (q.g) {
         case 1: launch_backward_gv<1, 8>(h, layer, ld, part); break;
         case 2: launch_backward_gv<2, 8>(h, layer, ld, part); break;

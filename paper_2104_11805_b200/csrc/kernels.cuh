@@ -415,6 +415,7 @@ forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict
     for (int i = 0; i < CPS; ++i) c[i] = make_int4(0, 0, 0, 0);
     if (nch > 0) load_idx<CPS>(c, idx + base);
     if (pdl) grid_dependency_wait();
+    if (pdl == 2) grid_launch_dependents();
     // compaction mode: only the first *ncols_dev columns of the tile still hold live inputs
     if (ncols_dev && blockIdx.y * (V * G) >= *ncols_dev) return;
     unsigned live = 0u;       // bit e: column boff + e of some row this lane produced is nonzero
@@ -459,7 +460,7 @@ forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict
         for (int e = 0; e < V; ++e)
             if ((live >> e) & 1u) live_flags[boff + e] = 1;      // many lanes may store the same 1
     }
-    if (pdl) grid_launch_dependents();
+    if (pdl == 1) grid_launch_dependents();
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -765,13 +766,14 @@ backward_kernel(const BackwardArgs a) {
         }
     }
     if (a.pdl) grid_dependency_wait();
+    if (a.pdl == 2) grid_launch_dependents();
     const float inv_b = a.sp->inv_b;
     const float step = a.sp->eta * inv_b;
     if (MIRROR) backward_col_units<G, V, CPS>(a.cols, a.xprev, a.dk, a.dprev, a.n, a.clamp, a.act, step, inv_b, first, stride);
-    if (MIRROR && a.cols_only) { if (a.pdl) grid_launch_dependents(); return; }
+    if (MIRROR && a.cols_only) { if (a.pdl == 1) grid_launch_dependents(); return; }
     backward_row_units<G, V, CPS, FROM_S, SCATTER, DBG>(a.rows, a.bias, a.xk, a.xprev, a.dk, a.dprev, a.dbg_delta, a.dbg_grad, a.n,
                                                         a.clamp, a.act, step, inv_b, a.update_bias, a.skip_dead, first, stride);
-    if (a.pdl) grid_launch_dependents();
+    if (a.pdl == 1) grid_launch_dependents();
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -814,6 +816,7 @@ forward_ep_kernel(Sliced m, const float* __restrict__ bias, const float* __restr
     SDNN_EP_LOAD_IDX(c, 0)
     const float b = (e.item < n) ? bias[e.item] : 0.0f;
     if (pdl) grid_dependency_wait();
+    if (pdl == 2) grid_launch_dependents();
     Lane<4> acc;
     lane_fill(acc, 0.0f);
     for (int t0 = 0; t0 < e.nch; t0 += 2 * EP_IT) {
@@ -840,7 +843,7 @@ forward_ep_kernel(Sliced m, const float* __restrict__ bias, const float* __restr
         lane_activate(acc, act, clamp);
         lane_store(xout + (size_t)e.item * 4, acc);
     }
-    if (pdl) grid_launch_dependents();
+    if (pdl == 1) grid_launch_dependents();
 }
 
 // new values of the four entries of chunk t (positions 4t .. 4t+3 of a unit with `len` stored entries; padding keeps its 0)
@@ -861,6 +864,7 @@ backward_col_ep_kernel(Sliced m, const float* __restrict__ xprev, const float* _
     int len = 0, j = 0;
     if (e.item < n) { len = m.len[e.item]; j = m.order[e.item]; }
     if (pdl) grid_dependency_wait();
+    if (pdl == 2) grid_launch_dependents();
     const float step = sp->eta * sp->inv_b;
     Lane<4> xj, acc;
     lane_fill(xj, 0.0f); lane_fill(acc, 0.0f);
@@ -893,7 +897,7 @@ backward_col_ep_kernel(Sliced m, const float* __restrict__ xprev, const float* _
         lane_mask(acc, xj, act, clamp);
         lane_store(dprev + (size_t)j * 4, acc);
     }
-    if (pdl) grid_launch_dependents();
+    if (pdl == 1) grid_launch_dependents();
 }
 
 // Row units (row-major copy m): update of its values (and of the bias) from delta^k[i] and the gathered x^{k-1}[j].
@@ -906,6 +910,7 @@ backward_row_ep_kernel(Sliced m, float* __restrict__ bias, const float* __restri
     SDNN_EP_LOAD_IDX(c, 0)
     const int len = (e.item < n) ? m.len[e.item] : 0;
     if (pdl) grid_dependency_wait();
+    if (pdl == 2) grid_launch_dependents();
     const float inv_b = sp->inv_b;
     const float step = sp->eta * inv_b;
     Lane<4> d;
@@ -939,7 +944,7 @@ backward_row_ep_kernel(Sliced m, float* __restrict__ bias, const float* __restri
             }
         }
     }
-    if (pdl) grid_launch_dependents();
+    if (pdl == 1) grid_launch_dependents();
 }
 #undef SDNN_EP_LOAD_IDX
 

@@ -177,6 +177,15 @@ int dev_alloc(sdnn* h, T** out, size_t count, bool zero) {
     return SDNN_OK;
 }
 
+// Programmatic dependent launch, the kernels' `pdl` argument: 0 = off; 1 = a CTA lets the next launch go when it is
+// done; 2 = as soon as its own wait for the previous launch has returned, so that CTAs of the next launch move into SM
+// slots as they fall free and run their prologue (shapes, first indices) under this launch's tail.  2 is used where
+// the launch has the device to itself (the forward chains: config 5 13.5 -> 13.1 us per layer, config 3 9.3 -> 8.9 us,
+// a 1024-neuron layer 2.7 -> 1.9 us) and for backward launches of at most one CTA per SM; a larger backward launch
+// shares the SMs with the row-unit launches of the side stream, and early CTAs of the next layer, which only wait,
+// then stand in their way (N = 16384, B = 1: 6 % slower).
+constexpr int PDL_AT_END = 1, PDL_EARLY = 2;
+
 // padded batch width: 4, 8, .., 256, then multiples of 256
 int padded_width(int b) {
     if (b <= 4) return 4;
@@ -346,7 +355,7 @@ void launch_forward_gv(sdnn* h, int layer, const float* xin, float* xout, int ld
     const float* bias = h->d_bias + (size_t)layer * h->N;
     auto plan = plan_grid(h, (const void*)forward_kernel<G, V, 2>, units, chunks);
     launch_k(h, forward_kernel<G, V, 2>, dim3(plan.first, chunks), dim3(plan.second), h->pdl, rows_of(h, layer), bias, xin, xout,
-             h->N, ld, h->cfg.clamp, h->cfg.activation, h->pdl ? 1 : 0, track ? (const int*)h->cur->cs.ncols : (const int*)nullptr,
+             h->N, ld, h->cfg.clamp, h->cfg.activation, h->pdl ? PDL_EARLY : 0, track ? (const int*)h->cur->cs.ncols : (const int*)nullptr,
              track ? h->cur->cs.flags : (int*)nullptr);
 }
 
@@ -361,7 +370,7 @@ void launch_forward(sdnn* h, int layer, const float* xin, float* xout, int ld, i
     const Geometry q = geometry(cols);
     if (q.v == 4 && !track && entry_parallel(h, ld)) {
         launch_k(h, forward_ep_kernel, dim3((h->NS + 3) / 4), dim3(128), h->pdl, rows_of(h, layer),
-                 (const float*)(h->d_bias + (size_t)layer * h->N), xin, xout, h->N, h->cfg.clamp, h->cfg.activation, h->pdl ? 1 : 0);
+                 (const float*)(h->d_bias + (size_t)layer * h->N), xin, xout, h->N, h->cfg.clamp, h->cfg.activation, h->pdl ? PDL_EARLY : 0);
     } else if (q.v == 4) launch_forward_gv<1, 4>(h, layer, xin, xout, ld, q.chunks, track);
     else switch (q.g) {
         case 1: launch_forward_gv<1, 8>(h, layer, xin, xout, ld, q.chunks, track); break;
@@ -401,7 +410,7 @@ void launch_backward_gvc(sdnn* h, int layer, int ld, int part) {
     a.act = h->cfg.activation;
     a.update_bias = h->cfg.update_bias ? 1 : 0;
     a.skip_dead = (h->cfg.flags & SDNN_FLAG_SKIP_DEAD) ? 1 : 0;
-    a.pdl = h->pdl ? 1 : 0;
+    a.pdl = h->pdl ? PDL_AT_END : 0;
     a.warm = (layer >= 1) ? acts + (size_t)(layer - 1) * tile : nullptr;
     a.warm_bytes = (unsigned)(tile * sizeof(float));
     // The two launches of a layer in the split realisation run beside each other (and beside those of the next layer):
@@ -413,9 +422,11 @@ void launch_backward_gvc(sdnn* h, int layer, int ld, int part) {
     do {                                                                                       \
         if (a.dbg_grad) {                                                                      \
             auto plan = plan_grid(h, (const void*)backward_kernel<G, V, CPS, FROM_S, SCAT, MIR, true>, units, 1, os_);   \
+            if (a.pdl && plan.first <= h->sms) a.pdl = PDL_EARLY;                              \
             launch_k(h, backward_kernel<G, V, CPS, FROM_S, SCAT, MIR, true>, dim3(plan.first), dim3(plan.second), h->pdl, a); \
         } else {                                                                               \
             auto plan = plan_grid(h, (const void*)backward_kernel<G, V, CPS, FROM_S, SCAT, MIR, false>, units, 1, os_);  \
+            if (a.pdl && plan.first <= h->sms) a.pdl = PDL_EARLY;                              \
             launch_k(h, backward_kernel<G, V, CPS, FROM_S, SCAT, MIR, false>, dim3(plan.first), dim3(plan.second), h->pdl, a); \
         }                                                                                      \
     } while (0)
@@ -457,7 +468,7 @@ void launch_backward_ep(sdnn* h, int layer, int part) {
     const dim3 grid((h->NS + 3) / 4), block(128);
     if (part == 1) {
         launch_k(h, backward_col_ep_kernel, grid, block, h->pdl, cols_of(h, layer), xprev, dk, delta_tile(h, layer - 1, tile), h->N,
-                 h->cfg.clamp, h->cfg.activation, (const StepParams*)h->d_sp, h->pdl ? 1 : 0);
+                 h->cfg.clamp, h->cfg.activation, (const StepParams*)h->d_sp, !h->pdl ? 0 : (int)grid.x <= h->sms ? PDL_EARLY : PDL_AT_END);
     } else {
         float* bias = h->d_bias + (size_t)layer * h->N;
         float* grad = h->lay[layer].r_grad;

@@ -88,10 +88,14 @@ struct sdnn {
     float* d_s[2] = {nullptr, nullptr}; // atomics: alternating S = W^T delta tiles (all-zero between steps); mirror: delta tiles
     float* d_dl = nullptr;              // delta^L tile (atomics realisation)
     float* d_delta_all = nullptr;       // split backward: [L][N][ld], every delta^k of the step
-    bool split = false;                 // transposed realisation with the row units as launches of their own on side_stream
-    cudaStream_t side_stream = nullptr, launch_stream = nullptr;     // launch_stream: where launch_k currently enqueues (NULL = stream)
+    bool split = false;                 // transposed realisation with the row units as launches of their own on side streams
+    static constexpr int MAX_SIDE = 2;
+    cudaStream_t side_streams[MAX_SIDE] = {nullptr, nullptr};   // the row-unit launches alternate between these
+    cudaEvent_t ev_side_join[MAX_SIDE] = {nullptr, nullptr};
+    int n_side = 0;
+    cudaStream_t launch_stream = nullptr;     // where launch_k currently enqueues (NULL = stream)
     std::vector<cudaEvent_t> ev_delta;  // [L] delta^k (0-based layer) complete
-    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    cudaEvent_t ev_fork = nullptr;
     float* d_yt = nullptr;              // target tile
     StepParams* d_sp = nullptr;
     double* d_loss = nullptr;
@@ -423,11 +427,11 @@ void launch_backward_gvc(sdnn* h, int layer, int ld, int part) {
         if (a.dbg_grad) {                                                                      \
             auto plan = plan_grid(h, (const void*)backward_kernel<G, V, CPS, FROM_S, SCAT, MIR, true>, units, 1, os_);   \
             if (a.pdl && plan.first <= h->sms) a.pdl = PDL_EARLY;                              \
-            launch_k(h, backward_kernel<G, V, CPS, FROM_S, SCAT, MIR, true>, dim3(plan.first), dim3(plan.second), h->pdl, a); \
+            launch_k(h, backward_kernel<G, V, CPS, FROM_S, SCAT, MIR, true>, dim3(plan.first), dim3(plan.second), a.pdl != 0, a); \
         } else {                                                                               \
             auto plan = plan_grid(h, (const void*)backward_kernel<G, V, CPS, FROM_S, SCAT, MIR, false>, units, 1, os_);  \
             if (a.pdl && plan.first <= h->sms) a.pdl = PDL_EARLY;                              \
-            launch_k(h, backward_kernel<G, V, CPS, FROM_S, SCAT, MIR, false>, dim3(plan.first), dim3(plan.second), h->pdl, a); \
+            launch_k(h, backward_kernel<G, V, CPS, FROM_S, SCAT, MIR, false>, dim3(plan.first), dim3(plan.second), a.pdl != 0, a); \
         }                                                                                      \
     } while (0)
     if (h->mirror) {
@@ -516,11 +520,12 @@ void enqueue_backward_chain(sdnn* h, int ld) {
         // column units chain on the main stream; the row units of layer k only need delta^k and x^{k-1}, so they run on
         // the side stream beside the column units of the layers below
         cudaEventRecord(h->ev_fork, h->stream);
-        cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0);
+        for (int q = 0; q < h->n_side; ++q) cudaStreamWaitEvent(h->side_streams[q], h->ev_fork, 0);
         cudaEventRecord(h->ev_delta[h->L - 1], h->stream);
         for (int k = h->L - 1; k >= 0; --k) {
-            cudaStreamWaitEvent(h->side_stream, h->ev_delta[k], 0);
-            h->launch_stream = h->side_stream;
+            cudaStream_t side = h->side_streams[k % h->n_side];
+            cudaStreamWaitEvent(side, h->ev_delta[k], 0);
+            h->launch_stream = side;
             launch_backward(h, k, ld, 2);
             h->launch_stream = nullptr;
             if (k > 0) {
@@ -528,8 +533,10 @@ void enqueue_backward_chain(sdnn* h, int ld) {
                 cudaEventRecord(h->ev_delta[k - 1], h->stream);
             }
         }
-        cudaEventRecord(h->ev_join, h->side_stream);
-        cudaStreamWaitEvent(h->stream, h->ev_join, 0);
+        for (int q = 0; q < h->n_side; ++q) {
+            cudaEventRecord(h->ev_side_join[q], h->side_streams[q]);
+            cudaStreamWaitEvent(h->stream, h->ev_side_join[q], 0);
+        }
     } else {
         for (int k = h->L - 1; k >= 0; --k) launch_backward(h, k, ld);
     }
@@ -841,8 +848,8 @@ void sdnn_destroy(sdnn_t* h) {
     if (h->ev_lane_start) cudaEventDestroy(h->ev_lane_start);
     for (cudaEvent_t e : h->ev_delta) if (e) cudaEventDestroy(e);
     if (h->ev_fork) cudaEventDestroy(h->ev_fork);
-    if (h->ev_join) cudaEventDestroy(h->ev_join);
-    if (h->side_stream) { cudaStreamSynchronize(h->side_stream); cudaStreamDestroy(h->side_stream); }
+    for (cudaEvent_t e : h->ev_side_join) if (e) cudaEventDestroy(e);
+    for (cudaStream_t st : h->side_streams) if (st) { cudaStreamSynchronize(st); cudaStreamDestroy(st); }
     for (cudaEvent_t e : h->ev_copied) if (e) cudaEventDestroy(e);
     for (cudaEvent_t e : h->ev_consumed) if (e) cudaEventDestroy(e);
     if (h->copy_stream) { cudaStreamSynchronize(h->copy_stream); cudaStreamDestroy(h->copy_stream); }
@@ -914,12 +921,15 @@ int sdnn_create_deferred(sdnn_t** out, int32_t n_layers, int32_t n_neurons, cons
         h->split = h->mirror && !(cfg->flags & SDNN_FLAG_BWD_ONE_LAUNCH);
         if (h->split) {
             if (!(cfg->flags & SDNN_FLAG_KEEP_DEBUG) && (rc = dev_alloc(h, &h->d_delta_all, L * tile, true))) return bail(rc);
-            if ((e = cudaStreamCreateWithFlags(&h->side_stream, cudaStreamNonBlocking)) != cudaSuccess) return bail(cuda_fail(h, e, "cudaStreamCreate"));
+            h->n_side = 2;      // row-unit launches of neighbouring layers do not depend on each other: two streams let them overlap
+            for (int q = 0; q < h->n_side; ++q) {
+                if ((e = cudaStreamCreateWithFlags(&h->side_streams[q], cudaStreamNonBlocking)) != cudaSuccess) return bail(cuda_fail(h, e, "cudaStreamCreate"));
+                if ((e = cudaEventCreateWithFlags(&h->ev_side_join[q], cudaEventDisableTiming)) != cudaSuccess) return bail(cuda_fail(h, e, "cudaEventCreate"));
+            }
             h->ev_delta.assign(n_layers, nullptr);
             for (cudaEvent_t& ev : h->ev_delta)
                 if ((e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming)) != cudaSuccess) { ev = nullptr; return bail(cuda_fail(h, e, "cudaEventCreate")); }
             if ((e = cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming)) != cudaSuccess) return bail(cuda_fail(h, e, "cudaEventCreate"));
-            if ((e = cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming)) != cudaSuccess) return bail(cuda_fail(h, e, "cudaEventCreate"));
         }
         if ((rc = dev_alloc(h, &h->d_s[0], tile, true))) return bail(rc);
         if ((rc = dev_alloc(h, &h->d_s[1], tile, true))) return bail(rc);

@@ -249,6 +249,16 @@ def main():
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        # the launcher gives every rank one OpenMP thread; the (untimed) set-up of a replica - generating the layers,
+        # building the sliced and transposed copies - is OpenMP code and would take minutes that way: share the cores
+        threads = max(1, (os.cpu_count() or 1) // world)
+        os.environ["OMP_NUM_THREADS"] = str(threads)
+        try:        # the OpenMP runtime may have read the variable already (numpy is imported)
+            import ctypes
+            ctypes.CDLL("libgomp.so.1").omp_set_num_threads(threads)
+        except OSError:
+            pass
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
 
     if args.impl == "reference":

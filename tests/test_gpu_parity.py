@@ -587,6 +587,34 @@ def test_state_and_argument_errors(torch_cuda):
     h.destroy()
 
 
+def test_training_handle_infers_with_its_current_weights(torch_cuda):
+    """Train two steps, infer (three tiles, two in flight), train again, infer again: inference on a training handle reads
+    the row-major copy as the last step left it, and training goes on undisturbed."""
+    torch = torch_cuda
+    pkg = sdnn()
+    spec = gen.CFG1_TRAIN.scaled(512, 5).paper_setup()
+    rp, col, val, bias = gen.network(spec)
+    h = pkg.Sdnn.create(rp, col, val, bias, max_batch=16, train=True, activation=pkg.ACT_SIGMOID)
+    ora = OracleNet(rp, col, val, bias, activation="sigmoid")
+    xin = gen.inputs(spec, 40)
+    yd = torch.empty((40, spec.n), dtype=torch.float32, device="cuda")
+    for rnd, batches in enumerate((batches_for(spec, 16, 2), batches_for(spec, 7, 1))):
+        for x0, y in batches:
+            ora.quantize_state()
+            for l in range(spec.layers):
+                h.set_weights(l, ora.w[l], ora.bias[l])
+            B = x0.shape[0]
+            loss = h.train_step(torch.from_numpy(x0).cuda(), torch.from_numpy(y).cuda(), B, 0.01, want_loss=True)
+            out = ora.train_step(x0, y, 0.01, keep=())
+            assert abs(loss - out["loss"]) <= TOL * abs(out["loss"])
+        h.infer_batch(torch.from_numpy(xin).cuda(), 40, yd, None, None, 0)
+        torch.cuda.synchronize()
+        check_close(yd.cpu().numpy(), ora.infer(xin), f"inference after round {rnd}")
+        for l in range(spec.layers):
+            assert h.mirror_mismatches(l) == 0
+    h.destroy()
+
+
 def test_deferred_creation_and_resume(torch_cuda):
     """Layer-by-layer loading gives the same handle; get_weights -> create resumes training exactly."""
     pkg = sdnn()

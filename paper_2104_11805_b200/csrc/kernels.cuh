@@ -63,7 +63,12 @@ __device__ __forceinline__ void prefetch_l2(const void* p, unsigned bytes) {
     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" :: "l"(p), "r"(bytes) : "memory");
 }
 
-// programmatic dependent launch: wait for the kernels this one depends on / let the next one start its prologue
+// programmatic dependent launch: wait for the kernels this one depends on / let the next one start its prologue.
+// The layer kernels take `pdl`: 0 = launched without the attribute (no wait, no release); 1 = wait, release the next
+// launch at the end; 2 = wait, release it right after the wait (its CTAs then move into SM slots as they fall free and
+// do everything that does not depend on this launch - shapes, first indices - under this launch's tail).  Whatever a
+// kernel reads before its wait must not be written by the launch before it: slice offsets, lengths, order, indices
+// and (forward) the bias qualify; values, tiles and counters do not.
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 

@@ -68,12 +68,12 @@ typedef enum {
                                     /* vector has become all zero are dropped from the tile (whole chunks of 256   */
                                     /* columns at a time); only done while no layer has a positive bias, because   */
                                     /* only then does an all-zero vector stay all zero.  Training: a unit of rows  */
-                                    /* whose delta is zero for every input skips its entries.  Results are the     */
-                                    /* same as in dense mode.                                                      */
+                                    /* whose delta is zero for every input skips its entries (not for B <= 4,      */
+                                    /* whose kernels have no such test).  Results are the same as in dense mode.   */
 #define SDNN_FLAG_NO_GRAPH    0x10u /* launch the layer chain kernel by kernel instead of through a CUDA graph     */
 #define SDNN_FLAG_BWD_ONE_LAUNCH 0x80u /* transposed realisation: column and row units of a layer in one launch.  By      */
                                     /* default the row units (the update of the row-major copy) are launches of their    */
-                                    /* own on a second stream, beside the column units of the layers below; that keeps   */
+                                    /* own on two more streams, beside the column units of the layers below; that keeps   */
                                     /* every delta^k of a step (N * padded(B) * 4 bytes per layer more) and is faster    */
 #define SDNN_FLAG_NO_PDL      0x20u /* do not let a layer's kernel start its prologue under the previous layer's tail */
 #define SDNN_FLAG_ONE_TILE    0x40u /* inference: one tile in flight at a time (see sdnn_infer_batch)               */

@@ -187,7 +187,7 @@ int dev_alloc(sdnn* h, T** out, size_t count, bool zero) {
 // slots as they fall free and run their prologue (shapes, first indices) under this launch's tail.  2 is used where
 // the launch has the device to itself (the forward chains: config 5 13.5 -> 13.1 us per layer, config 3 9.3 -> 8.9 us,
 // a 1024-neuron layer 2.7 -> 1.9 us) and for backward launches of at most one CTA per SM; a larger backward launch
-// shares the SMs with the row-unit launches of the side stream, and early CTAs of the next layer, which only wait,
+// shares the SMs with the row-unit launches of the side streams, and early CTAs of the next layer, which only wait,
 // then stand in their way (N = 16384, B = 1: 6 % slower).
 constexpr int PDL_AT_END = 1, PDL_EARLY = 2;
 
@@ -519,7 +519,7 @@ void launch_transpose_in(sdnn* h, const float* src, float* dst, int cnt, int col
 void enqueue_backward_chain(sdnn* h, int ld) {
     if (h->split) {
         // column units chain on the main stream; the row units of layer k only need delta^k and x^{k-1}, so they run on
-        // the side stream beside the column units of the layers below
+        // the side streams beside the column units of the layers below
         cudaEventRecord(h->ev_fork, h->stream);
         for (int q = 0; q < h->n_side; ++q) cudaStreamWaitEvent(h->side_streams[q], h->ev_fork, 0);
         cudaEventRecord(h->ev_delta[h->L - 1], h->stream);

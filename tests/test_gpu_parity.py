@@ -587,6 +587,28 @@ def test_state_and_argument_errors(torch_cuda):
     h.destroy()
 
 
+@pytest.mark.parametrize("bwd", sorted(BWD_MODES))
+@pytest.mark.parametrize("B", [1, 4, 16])
+def test_train_long_and_very_ragged_rows(torch_cuda, B, bwd):
+    """Rows of 0 .. 70 entries on 97 neurons (not a multiple of the slice height): several blocks of chunks per row in the
+    kernels for B <= 4, many steps per unit in the common ones, columns far longer than rows in the transposed copy."""
+    rng = np.random.default_rng(900 + B)
+    arrays = ragged_net(rng, n=97, layers=3, kmax=70, scale=0.25)
+    batches = [(rng.uniform(0, 1.0, size=(B, 97)).astype(np.float32), rng.uniform(0, 1, size=(B, 97)).astype(np.float32))
+               for _ in range(2)]
+    train_parity(torch_cuda, arrays, batches, eta=0.02, update_bias=True, flags=BWD_MODES[bwd], expect_live=True,
+                 activation="sigmoid")
+    train_parity(torch_cuda, arrays, batches, eta=0.02, flags=BWD_MODES[bwd])
+
+
+@pytest.mark.parametrize("cnt,max_batch", [(3, 4), (11, 16), (300, 256)])
+def test_infer_long_and_very_ragged_rows(torch_cuda, cnt, max_batch):
+    rng = np.random.default_rng(950 + cnt)
+    arrays = ragged_net(rng, n=97, layers=4, kmax=70, scale=0.2)
+    x0 = rng.uniform(0, 1.0, size=(cnt, 97)).astype(np.float32)
+    infer_parity(torch_cuda, arrays, x0, max_batch, expect_nonempty=True)
+
+
 def test_training_handle_infers_with_its_current_weights(torch_cuda):
     """Train two steps, infer (three tiles, two in flight), train again, infer again: inference on a training handle reads
     the row-major copy as the last step left it, and training goes on undisturbed."""

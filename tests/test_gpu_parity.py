@@ -609,6 +609,18 @@ def test_infer_long_and_very_ragged_rows(torch_cuda, cnt, max_batch):
     infer_parity(torch_cuda, arrays, x0, max_batch, expect_nonempty=True)
 
 
+@pytest.mark.parametrize("n", [1, 5, 17])
+@pytest.mark.parametrize("B", [1, 16])
+def test_tiny_nets(torch_cuda, n, B):
+    """Fewer neurons than a slice has rows, down to a single one: training (default realisation) and inference."""
+    rng = np.random.default_rng(40 + n + B)
+    arrays = ragged_net(rng, n=n, layers=3, kmax=n, scale=0.7)
+    batches = [(rng.uniform(0, 1.0, size=(B, n)).astype(np.float32), rng.uniform(0, 1, size=(B, n)).astype(np.float32))
+               for _ in range(2)]
+    train_parity(torch_cuda, arrays, batches, eta=0.05, update_bias=True, activation="sigmoid", expect_live=True)
+    infer_parity(torch_cuda, arrays, rng.uniform(0, 1.0, size=(3 * B, n)).astype(np.float32), B)
+
+
 def test_training_handle_infers_with_its_current_weights(torch_cuda):
     """Train two steps, infer (three tiles, two in flight), train again, infer again: inference on a training handle reads
     the row-major copy as the last step left it, and training goes on undisturbed."""

@@ -429,6 +429,34 @@ def test_infer_two_tiles_in_flight_equals_one_at_a_time(torch_cuda, host, skip_d
     assert (idx[total:] == -1).all()
 
 
+@pytest.mark.parametrize("spec,B", [(gen.CFG5.scaled(65536, 8).live(), 16), (gen.CFG3.scaled(16384, 12).live(), 64),
+                                    (gen.CFG1_TRAIN.scaled(65536, 6).paper_setup(), 1)])
+def test_train_in_the_benchmark_launch_configuration(torch_cuda, spec, B):
+    """The handle bench.py times: default flags, no debug buffers (so the kernels' non-debug instantiations, the delta
+    tiles of the split realisation, the CUDA graph), full width N and the configuration's B, a few layers.  Two steps;
+    loss, every layer's weights and the consistency of the two copies are checked against the oracle run the same way."""
+    torch = torch_cuda
+    pkg = sdnn()
+    rp, col, val, bias = gen.network(spec)
+    sigmoid = spec.values == "uniform_pm1"
+    eta = 0.01 if sigmoid else 1e-3
+    h = pkg.Sdnn.create(rp, col, val, bias, max_batch=B, train=True, activation=pkg.ACT_SIGMOID if sigmoid else pkg.ACT_CLAMPED_RELU)
+    ora = OracleNet(rp, col, val, bias, activation="sigmoid" if sigmoid else "clamped_relu")
+    for step, (x0, y) in enumerate(batches_for(spec, B, 2)):
+        if step:
+            ora.quantize_state()
+            for l in range(spec.layers):
+                h.set_weights(l, ora.w[l], ora.bias[l])
+        loss = h.train_step(torch.from_numpy(x0).cuda(), torch.from_numpy(y).cuda(), B, eta, want_loss=True)
+        out = ora.train_step(x0, y, eta, keep=("grad",))
+        assert abs(loss - out["loss"]) <= TOL * abs(out["loss"])
+        assert any(np.any(g != 0.0) for g in out["grad"]), "vacuous: every gradient is zero"
+        for l in range(spec.layers):
+            check_close(h.get_weights(l, want_bias=False), ora.w[l], f"step {step} W^{l + 1}")
+            assert h.mirror_mismatches(l) == 0
+    h.destroy()
+
+
 def test_train_cfg3_live_full_size(torch_cuda):
     """Config 3 at full size (16384 x 480, B = 64), live companion, one step."""
     spec = gen.CFG3.live()

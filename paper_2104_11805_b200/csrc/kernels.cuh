@@ -807,8 +807,8 @@ __device__ __forceinline__ EpShape ep_shape(const Sliced& m, int n) {
     return e;
 }
 
-#define SDNN_EP_LOAD_IDX(C, T0)                                                                         \
-    _Pragma("unroll") for (int i = 0; i < EP_IT; ++i) {                                                  \
+#define SDNN_EP_LOAD_IDX(C, T0, IT)                                                                     \
+    _Pragma("unroll") for (int i = 0; i < (IT); ++i) {                                                   \
         const int t = (T0) + 2 * i + e.h;                                                                \
         C[i] = (t < e.nch) ? __ldcs(reinterpret_cast<const int4*>(m.idx + e.so + t * CHUNK_ROW + e.r * 4)) : make_int4(0, 0, 0, 0); \
     }
@@ -818,7 +818,7 @@ forward_ep_kernel(Sliced m, const float* __restrict__ bias, const float* __restr
                   int n, float clamp, int act, int pdl) {
     const EpShape e = ep_shape(m, n);
     int4 c[EP_IT];
-    SDNN_EP_LOAD_IDX(c, 0)
+    SDNN_EP_LOAD_IDX(c, 0, EP_IT)
     const float b = (e.item < n) ? bias[e.item] : 0.0f;
     if (pdl) grid_dependency_wait();
     if (pdl == 2) grid_launch_dependents();
@@ -834,7 +834,7 @@ forward_ep_kernel(Sliced m, const float* __restrict__ bias, const float* __restr
         }
 #pragma unroll
         for (int i = 0; i < EP_IT; ++i) { SDNN_GATHER_CHUNK(x, i, c[i], xin, 16u) }
-        if (t0 + 2 * EP_IT < e.nch) { SDNN_EP_LOAD_IDX(c, t0 + 2 * EP_IT) }
+        if (t0 + 2 * EP_IT < e.nch) { SDNN_EP_LOAD_IDX(c, t0 + 2 * EP_IT, EP_IT) }
 #pragma unroll
         for (int i = 0; i < EP_IT; ++i) {
             lane_fma(w[i].x, x[4 * i + 0], acc); lane_fma(w[i].y, x[4 * i + 1], acc);
@@ -860,12 +860,16 @@ __device__ __forceinline__ float4 ep_update(const float4& w, float p0, float p1,
 
 // Column units (transposed copy m): delta^{k-1}[j] = (sum_i w(i,j) delta^k[i]) (.) f'(x^{k-1}[j]) with the values before
 // their update, and the update of the transposed copy's values.
+// IT iterations (2 * IT chunks of a unit) in flight together.  The transposed copy's units are ragged (a column of a
+// 32-per-row random pattern has 15 .. 55 entries): IT = 8 takes up to 64 entries in one go where the launch is bound by
+// its chain of dependent round trips rather than by throughput (small nets).
+template <int IT>
 __global__ void __launch_bounds__(128)
 backward_col_ep_kernel(Sliced m, const float* __restrict__ xprev, const float* __restrict__ dk, float* __restrict__ dprev,
                        int n, float clamp, int act, const StepParams* __restrict__ sp, int pdl) {
     const EpShape e = ep_shape(m, n);
-    int4 c[EP_IT];
-    SDNN_EP_LOAD_IDX(c, 0)
+    int4 c[IT];
+    SDNN_EP_LOAD_IDX(c, 0, IT)
     int len = 0, j = 0;
     if (e.item < n) { len = m.len[e.item]; j = m.order[e.item]; }
     if (pdl) grid_dependency_wait();
@@ -874,19 +878,19 @@ backward_col_ep_kernel(Sliced m, const float* __restrict__ xprev, const float* _
     Lane<4> xj, acc;
     lane_fill(xj, 0.0f); lane_fill(acc, 0.0f);
     if (e.item < n) lane_load(xj, xprev + (size_t)j * 4);
-    for (int t0 = 0; t0 < e.nch; t0 += 2 * EP_IT) {
-        float4 w[EP_IT];
-        Lane<4> d[4 * EP_IT];
+    for (int t0 = 0; t0 < e.nch; t0 += 2 * IT) {
+        float4 w[IT];
+        Lane<4> d[4 * IT];
 #pragma unroll
-        for (int i = 0; i < EP_IT; ++i) {
+        for (int i = 0; i < IT; ++i) {
             const int t = t0 + 2 * i + e.h;
             w[i] = (t < e.nch) ? ld_f4(m.val + e.so + t * CHUNK_ROW + e.r * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
 #pragma unroll
-        for (int i = 0; i < EP_IT; ++i) { SDNN_GATHER_CHUNK(d, i, c[i], dk, 16u) }
-        if (t0 + 2 * EP_IT < e.nch) { SDNN_EP_LOAD_IDX(c, t0 + 2 * EP_IT) }
+        for (int i = 0; i < IT; ++i) { SDNN_GATHER_CHUNK(d, i, c[i], dk, 16u) }
+        if (t0 + 2 * IT < e.nch) { SDNN_EP_LOAD_IDX(c, t0 + 2 * IT, IT) }
 #pragma unroll
-        for (int i = 0; i < EP_IT; ++i) {
+        for (int i = 0; i < IT; ++i) {
             const int t = t0 + 2 * i + e.h;
             lane_fma(w[i].x, d[4 * i + 0], acc); lane_fma(w[i].y, d[4 * i + 1], acc);
             lane_fma(w[i].z, d[4 * i + 2], acc); lane_fma(w[i].w, d[4 * i + 3], acc);
@@ -912,7 +916,7 @@ backward_row_ep_kernel(Sliced m, float* __restrict__ bias, const float* __restri
                        float* __restrict__ dbg_grad, int n, const StepParams* __restrict__ sp, int update_bias, int pdl) {
     const EpShape e = ep_shape(m, n);
     int4 c[EP_IT];
-    SDNN_EP_LOAD_IDX(c, 0)
+    SDNN_EP_LOAD_IDX(c, 0, EP_IT)
     const int len = (e.item < n) ? m.len[e.item] : 0;
     if (pdl) grid_dependency_wait();
     if (pdl == 2) grid_launch_dependents();
@@ -932,7 +936,7 @@ backward_row_ep_kernel(Sliced m, float* __restrict__ bias, const float* __restri
         }
 #pragma unroll
         for (int i = 0; i < EP_IT; ++i) { SDNN_GATHER_CHUNK(x, i, c[i], xprev, 16u) }
-        if (t0 + 2 * EP_IT < e.nch) { SDNN_EP_LOAD_IDX(c, t0 + 2 * EP_IT) }
+        if (t0 + 2 * EP_IT < e.nch) { SDNN_EP_LOAD_IDX(c, t0 + 2 * EP_IT, EP_IT) }
 #pragma unroll
         for (int i = 0; i < EP_IT; ++i) {
             const int t = t0 + 2 * i + e.h;

@@ -54,6 +54,7 @@ struct InferLane {
 
 struct LayerMem {
     int64_t r_elems = 0, c_elems = 0;      // padded lengths of the two sliced copies
+    int c_max_chunks = 0;                  // chunks of the widest slice of the transposed copy
     int* r_idx = nullptr; float* r_val = nullptr; float* r_grad = nullptr;
     int* c_idx = nullptr; float* c_val = nullptr;
     std::vector<int> r_slice_off;          // host copy of the row-major slice offsets
@@ -472,8 +473,14 @@ void launch_backward_ep(sdnn* h, int layer, int part) {
     const float* dk = delta_tile(h, layer, tile);
     const dim3 grid((h->NS + 3) / 4), block(128);
     if (part == 1) {
-        launch_k(h, backward_col_ep_kernel, grid, block, h->pdl, cols_of(h, layer), xprev, dk, delta_tile(h, layer - 1, tile), h->N,
-                 h->cfg.clamp, h->cfg.activation, (const StepParams*)h->d_sp, !h->pdl ? 0 : (int)grid.x <= h->sms ? PDL_EARLY : PDL_AT_END);
+        const int pdl = !h->pdl ? 0 : (int)grid.x <= h->sms ? PDL_EARLY : PDL_AT_END;
+        // a launch of at most one CTA per SM is bound by its chain of round trips: take a long column in one go
+        if ((int)grid.x <= h->sms && h->lay[layer].c_max_chunks > 2 * EP_IT)
+            launch_k(h, backward_col_ep_kernel<2 * EP_IT>, grid, block, h->pdl, cols_of(h, layer), xprev, dk, delta_tile(h, layer - 1, tile),
+                     h->N, h->cfg.clamp, h->cfg.activation, (const StepParams*)h->d_sp, pdl);
+        else
+            launch_k(h, backward_col_ep_kernel<EP_IT>, grid, block, h->pdl, cols_of(h, layer), xprev, dk, delta_tile(h, layer - 1, tile),
+                     h->N, h->cfg.clamp, h->cfg.activation, (const StepParams*)h->d_sp, pdl);
     } else {
         float* bias = h->d_bias + (size_t)layer * h->N;
         float* grad = h->lay[layer].r_grad;
@@ -1018,6 +1025,7 @@ int sdnn_load_layer(sdnn_t* h, int32_t layer, const int32_t* row_ptr, const int3
         for (int cc = 0; cc < N; ++cc) c_len[cc] = deg[order[cc]];
         lm.c_elems = build_slice_offsets(N, [&](int cc) { return c_len[cc]; }, c_off);
         if (lm.c_elems < 0) return fail(h, SDNN_ERR_INVALID_ARG, "layer %d: padded transposed layout exceeds 2^31 entries", layer);
+        for (int sl = 0; sl < NS; ++sl) lm.c_max_chunks = std::max(lm.c_max_chunks, (c_off[sl + 1] - c_off[sl]) / CHUNK_ROW);
         c_idx.assign((size_t)lm.c_elems, 0);
         // each thread owns a range of columns and scans all entries in row order: rows ascend within a column
 #pragma omp parallel

@@ -450,7 +450,7 @@ def main():
         alg = bwd_bytes if dom == "backward_kernel" else fwd_bytes
         # tiles of padded width 4 (B <= 4, or the averaged form's backward chain) run the entry-parallel kernels
         ep = not (args.flags & 0x81)
-        names = ("backward_col_ep_kernel", "backward_row_ep_kernel") if ep and ld_bwd == 4 else \
+        names = ("backward_col_ep_kernel<4 or 8>", "backward_row_ep_kernel") if ep and ld_bwd == 4 else \
                 ("backward_kernel<..,1,..>", "backward_kernel<..,0,..>")
         extra = {"backward_launches": f"per layer one column-unit launch ({names[0]}) on the main stream and one "
                                       f"row-unit launch ({names[1]}) on a side stream, running beside each other; "

@@ -393,7 +393,7 @@ __device__ __forceinline__ void prefetch_unit(const Sliced& m, int u, int rpw, i
 // per row; each lane accumulates V batch entries with fp32 FMAs in stored (ascending column) order.
 // While it works on a unit a warp asks for the entries of its next unit to be brought into L2.
 template <int G, int V, int CPS>
-__global__ void __launch_bounds__(256, 2)
+__global__ void __launch_bounds__(256, CPS > 2 ? 1 : 2)
 forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict__ xin, float* __restrict__ xout,
                int n, int ld, float clamp, int act, int pdl, const int* __restrict__ ncols_dev, int* __restrict__ live_flags) {
     constexpr int RPW = 32 / G;

@@ -55,6 +55,7 @@ struct InferLane {
 struct LayerMem {
     int64_t r_elems = 0, c_elems = 0;      // padded lengths of the two sliced copies
     int c_max_chunks = 0;                  // chunks of the widest slice of the transposed copy
+    bool r_chunks_mult4 = false;           // every slice of the row-major copy has a multiple of 4 chunks
     int* r_idx = nullptr; float* r_val = nullptr; float* r_grad = nullptr;
     int* c_idx = nullptr; float* c_val = nullptr;
     std::vector<int> r_slice_off;          // host copy of the row-major slice offsets
@@ -354,13 +355,13 @@ cudaError_t launch_k(sdnn* h, void (*kernel)(KArgs...), dim3 grid, dim3 block, b
     return cudaLaunchKernelEx(&lc, kernel, KArgs(args)...);
 }
 
-template <int G, int V>
+template <int G, int V, int CPS = 2>
 void launch_forward_gv(sdnn* h, int layer, const float* xin, float* xout, int ld, int chunks, bool track) {
     constexpr int RPW = 32 / G;
     const int units = (h->N + RPW - 1) / RPW;
     const float* bias = h->d_bias + (size_t)layer * h->N;
-    auto plan = plan_grid(h, (const void*)forward_kernel<G, V, 2>, units, chunks);
-    launch_k(h, forward_kernel<G, V, 2>, dim3(plan.first, chunks), dim3(plan.second), h->pdl, rows_of(h, layer), bias, xin, xout,
+    auto plan = plan_grid(h, (const void*)forward_kernel<G, V, CPS>, units, chunks);
+    launch_k(h, forward_kernel<G, V, CPS>, dim3(plan.first, chunks), dim3(plan.second), h->pdl, rows_of(h, layer), bias, xin, xout,
              h->N, ld, h->cfg.clamp, h->cfg.activation, h->pdl ? h->fwd_pdl : 0, track ? (const int*)h->cur->cs.ncols : (const int*)nullptr,
              track ? h->cur->cs.flags : (int*)nullptr);
 }
@@ -384,7 +385,13 @@ void launch_forward(sdnn* h, int layer, const float* xin, float* xout, int ld, i
         case 4: launch_forward_gv<4, 8>(h, layer, xin, xout, ld, q.chunks, track); break;
         case 8: launch_forward_gv<8, 8>(h, layer, xin, xout, ld, q.chunks, track); break;
         case 16: launch_forward_gv<16, 8>(h, layer, xin, xout, ld, q.chunks, track); break;
-        default: launch_forward_gv<32, 8>(h, layer, xin, xout, ld, q.chunks, track); break;
+        default:
+            // a launch of at most one warp-row per resident slot is bound by its chain of round trips: four chunks (16
+            // entries) of a row in flight per step instead of two, where every slice has whole steps of that size
+            if (!track && h->lay[layer].r_chunks_mult4 && (int64_t)h->N * q.chunks <= (int64_t)h->sms * 8)
+                launch_forward_gv<32, 8, 4>(h, layer, xin, xout, ld, q.chunks, track);
+            else launch_forward_gv<32, 8>(h, layer, xin, xout, ld, q.chunks, track);
+            break;
     }
     count_launch(h);
 }
@@ -985,6 +992,8 @@ int sdnn_load_layer(sdnn_t* h, int32_t layer, const int32_t* row_ptr, const int3
     for (int i = 0; i < N; ++i) r_len[i] = row_ptr[i + 1] - row_ptr[i];
     lm.r_elems = build_slice_offsets(N, [&](int i) { return r_len[i]; }, lm.r_slice_off);
     if (lm.r_elems < 0) return fail(h, SDNN_ERR_INVALID_ARG, "layer %d: padded sliced layout exceeds 2^31 entries", layer);
+    lm.r_chunks_mult4 = true;
+    for (int sl = 0; sl < NS; ++sl) lm.r_chunks_mult4 = lm.r_chunks_mult4 && ((lm.r_slice_off[sl + 1] - lm.r_slice_off[sl]) / CHUNK_ROW) % 4 == 0;
     std::vector<int> r_idx((size_t)lm.r_elems, 0);
     std::vector<float> r_val;
     csr_to_sliced(h, lm, values, r_val);

@@ -376,7 +376,8 @@ bool entry_parallel(const sdnn* h, int ld) {
 void launch_forward(sdnn* h, int layer, const float* xin, float* xout, int ld, int cols, bool track = false) {
     const Geometry q = geometry(cols);
     if (q.v == 4 && !track && entry_parallel(h, ld)) {
-        launch_k(h, forward_ep_kernel, dim3((h->NS + 3) / 4), dim3(128), h->pdl, rows_of(h, layer),
+        const int wf = h->NS <= h->sms ? 1 : 4;      // few slices: one per CTA, so that they spread over as many SMs
+        launch_k(h, forward_ep_kernel, dim3((h->NS + wf - 1) / wf), dim3(32 * wf), h->pdl, rows_of(h, layer),
                  (const float*)(h->d_bias + (size_t)layer * h->N), xin, xout, h->N, h->cfg.clamp, h->cfg.activation, h->pdl ? h->fwd_pdl : 0);
     } else if (q.v == 4) launch_forward_gv<1, 4>(h, layer, xin, xout, ld, q.chunks, track);
     else switch (q.g) {
@@ -478,7 +479,8 @@ void launch_backward_ep(sdnn* h, int layer, int part) {
     const float* acts = h->bwd_acts ? h->bwd_acts : h->d_acts;
     const float* xprev = acts + (size_t)layer * tile;
     const float* dk = delta_tile(h, layer, tile);
-    const dim3 grid((h->NS + 3) / 4), block(128);
+    const int wb = h->NS <= h->sms ? 1 : 4;          // few slices: one per CTA (a 1024-neuron net: 0.56 -> 0.51 ms per step)
+    const dim3 grid((h->NS + wb - 1) / wb), block(32 * wb);
     if (part == 1) {
         const int pdl = !h->pdl ? 0 : (int)grid.x <= h->sms ? PDL_EARLY : PDL_AT_END;
         // a launch of at most one CTA per SM is bound by its chain of round trips: take a long column in one go

@@ -84,7 +84,9 @@ typedef enum {
 typedef struct {
     int32_t  activation;   /* SDNN_ACT_CLAMPED_RELU or SDNN_ACT_SIGMOID */
     float    clamp;        /* upper clamp of the clamped ReLU, e.g. 32.0f; must be > 0 (ignored by the sigmoid) */
-    int32_t  max_batch;    /* train: largest minibatch B; inference: batch tile (inputs processed together) */
+    int32_t  max_batch;    /* train: largest minibatch B, at most 128 (the whole minibatch is one register tile of the
+                              backward kernels; larger values are rejected with SDNN_ERR_INVALID_ARG);
+                              inference: batch tile (inputs processed together), at most 2^30 */
     int32_t  train;        /* 0: inference only (no stored activations); 1: sdnn_train_step allowed.  A training
                               handle stores x^0..x^L of one minibatch and, unless SDNN_FLAG_BWD_ATOMICS is set, a second
                               (transposed) copy of the indices and values of every layer but the first */
@@ -191,14 +193,16 @@ int sdnn_train_step_averaged(sdnn_t* h, const float* x0, const float* target, in
                              float* loss_out);
 
 /*
- * Current parameters of one layer (0-based), in the caller's original CSR order.
+ * Current parameters of one layer (0-based), in the caller's original CSR order: the W^k that the update line
+ * of Algorithm 1 (W^k <- W^k - eta * grad) has produced so far, and b^k.
  *   values_out  host float[nnz_l], or NULL;   bias_out  host float[N], or NULL
  * Synchronises the stream.  Creating a new handle from these arrays resumes training.
  */
 int sdnn_get_weights(sdnn_t* h, int32_t layer, float* values_out, float* bias_out);
 
 /*
- * Overwrites the parameters of one layer (0-based) from host arrays in the caller's CSR order
+ * Overwrites W^k and b^k, the state that the update line of Algorithm 1 carries from one input to the next, for
+ * one layer (0-based) from host arrays in the caller's CSR order
  * (restore from a checkpoint without re-creating the handle; the pattern cannot change).
  *   values  host float[nnz_l], or NULL to keep;   bias  host float[N], or NULL to keep
  * Values must be finite (else SDNN_ERR_BAD_CSR).  Synchronises the stream.
@@ -241,6 +245,19 @@ int sdnn_mirror_mismatches(sdnn_t* h, int32_t layer, int64_t* count_out);
  * stream, runs about a hundred microseconds of kernels, synchronises.  rows_per_second: host double*.
  */
 int sdnn_probe_gather_rate(int32_t row_bytes, int64_t table_rows, double* rows_per_second);
+
+/*
+ * The same measurement for operand tiles staged on chip (diagnostic; the paper has no counterpart): random rows of
+ * `row_bytes` bytes (32, 64, 128 or 256; read with 128-bit accesses) out of a table of 128 KiB per CTA held in shared
+ * memory.  cluster_size 1: every CTA reads its own shared memory; 2, 4, 8 or 16: the table is spread over the shared
+ * memories of a thread-block cluster and read with ld.shared::cluster (distributed shared memory), every CTA of the
+ * cluster reading the whole cluster's table.  One CTA of 1024 threads per SM, as many whole clusters as the device holds
+ * at once.  rows_per_second (host double*): rows gathered per second by all of them together; ctas_out (host int32*, may
+ * be NULL): CTAs (= SMs) that took part.  Compared with sdnn_probe_gather_rate this says whether staging a tile in a
+ * cluster's shared memories could beat gathering it out of L2.  Errors: INVALID_ARG (sizes), CUDA (a cluster of that
+ * size does not fit the device).  Synchronises.
+ */
+int sdnn_probe_smem_gather_rate(int32_t row_bytes, int32_t cluster_size, double* rows_per_second, int32_t* ctas_out);
 
 /* Counters since creation: kernels launched by this handle (graph nodes count one each);
  * device bytes it holds. */

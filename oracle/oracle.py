@@ -24,8 +24,8 @@ verbatim); delta^0 is never formed (x^0 is data, no z^0 exists); the bias is
 frozen unless update_bias is set, in which case b^k <- b^k - eta * mean_b delta^k_b
 (the bias read as one more column of W^k whose input is the constant 1).
 
-train_step_averaged is the other reading of the same remark ("the gradient vector delta^L ... is computed as the
-averages of gradients over the batch ... a single gradient vector is backpropagated"): delta^L = mean_b delta^L_b,
+train_step_averaged is the other reading of the same remark (Discussion of Section 5: the output gradients of
+the batch are averaged into one delta^L and only that single vector is sent backwards): delta^L = mean_b delta^L_b,
 then the backward loop above for ONE vector, paired with the batch means xbar^{k-1} = mean_b x^{k-1}_b, f' being
 evaluated from xbar^{k-1} as it is from a single input's x^{k-1}.  The remark does not fix that pairing:
 PARITY UNPINNED for this function as far as the paper goes; the pins only hold it to Algorithm 1 where the two

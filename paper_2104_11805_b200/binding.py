@@ -53,6 +53,7 @@ _PROTOS = {
     "sdnn_get_gradient": (ctypes.c_int, [_vp, _i32, _vp]),
     "sdnn_mirror_mismatches": (ctypes.c_int, [_vp, _i32, ctypes.POINTER(_i64)]),
     "sdnn_probe_gather_rate": (ctypes.c_int, [_i32, _i64, ctypes.POINTER(ctypes.c_double)]),
+    "sdnn_probe_smem_gather_rate": (ctypes.c_int, [_i32, _i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(_i32)]),
     "sdnn_get_phase_times": (ctypes.c_int, [_vp, ctypes.POINTER(_f32), ctypes.POINTER(_f32)]),
     "sdnn_get_liveness": (ctypes.c_int, [_vp, _vp]),
     "sdnn_infer_noalloc": (ctypes.c_int, [_i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _f32, _vp]),
@@ -136,6 +137,17 @@ def probe_gather_rate(row_bytes, table_rows):
     if rc != 0:
         raise SdnnError(rc, (lib.sdnn_last_error(None) or b"").decode())
     return out.value
+
+
+def probe_smem_gather_rate(row_bytes, cluster_size):
+    """sdnn_probe_smem_gather_rate: (rows per second, CTAs taking part) for random rows out of shared memory
+    (cluster_size 1) or out of a cluster's distributed shared memory."""
+    lib = load_library()
+    out, ctas = ctypes.c_double(0.0), ctypes.c_int32(0)
+    rc = lib.sdnn_probe_smem_gather_rate(row_bytes, cluster_size, ctypes.byref(out), ctypes.byref(ctas))
+    if rc != 0:
+        raise SdnnError(rc, (lib.sdnn_last_error(None) or b"").decode())
+    return out.value, ctas.value
 
 
 class Sdnn:

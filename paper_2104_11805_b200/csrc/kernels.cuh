@@ -1132,6 +1132,59 @@ gather_probe_kernel(const float* __restrict__ table, float* __restrict__ sink, u
 }
 
 // ---------------------------------------------------------------------------------------------
+// The same probe for a table held in shared memory: of this CTA (cluster of 1), or spread over the shared memories of
+// the CTAs of a thread-block cluster and read with ld.shared::cluster (distributed shared memory).  G lanes of 16 bytes
+// per row (128-bit accesses: the widest shared-memory load), eight gathers in flight per lane.  Every CTA clears its
+// part of the table; the cluster barriers before and after the gathers keep every CTA's shared memory alive while its
+// neighbours read it.  rows_per_cta is a power of two; row r of the cluster's table lives in CTA r / rows_per_cta.
+__device__ __forceinline__ void cluster_barrier() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ unsigned cluster_cta_rank() {
+    unsigned r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+
+template <int G, bool REMOTE>
+__global__ void __launch_bounds__(1024)
+smem_gather_probe_kernel(float* __restrict__ sink, unsigned rows_per_cta_log2, unsigned cluster_log2, int per_group, unsigned seed) {
+    extern __shared__ __align__(16) float probe_table[];
+    constexpr unsigned ROW_BYTES = 16u * G;
+    const unsigned rows_per_cta = 1u << rows_per_cta_log2;
+    for (unsigned q = threadIdx.x; q < rows_per_cta * (ROW_BYTES / 16u); q += blockDim.x)
+        reinterpret_cast<float4*>(probe_table)[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+    __syncthreads();
+    cluster_barrier();
+    const unsigned base = (unsigned)__cvta_generic_to_shared(probe_table);
+    const unsigned row_mask = (rows_per_cta << cluster_log2) - 1u;
+    const int tid = blockIdx.x * blockDim.x + threadIdx.x;
+    const unsigned sub = threadIdx.x % G;
+    unsigned st = (unsigned)(tid / G) * 2654435761u + seed;
+    float acc = 0.f;
+    for (int q = 0; q < per_group; q += 8) {
+        float4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            st = st * 1664525u + 1013904223u;
+            const unsigned r = (st >> 8) & row_mask;
+            const unsigned addr = base + (r & (rows_per_cta - 1u)) * ROW_BYTES + sub * 16u;
+            if (REMOTE) {
+                unsigned ra;
+                asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(addr), "r"(r >> rows_per_cta_log2));
+                asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v[u].x), "=f"(v[u].y), "=f"(v[u].z), "=f"(v[u].w) : "r"(ra));
+            } else {
+                asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v[u].x), "=f"(v[u].y), "=f"(v[u].z), "=f"(v[u].w) : "r"(addr));
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) acc += (v[u].x + v[u].y) + (v[u].z + v[u].w);
+    }
+    if (acc == 123.456f) sink[0] = acc;      // the table is all zero: never taken, keeps the loads alive
+    cluster_barrier();
+}
+
+// ---------------------------------------------------------------------------------------------
 // Final-layer nonzero sets.  The tile is cut into segments of SEG rows.
 //   count: seg_cnt[seg*ld + b] = #{ i in segment : X[i,b] != 0 }
 //   scan : per input b: nz_count[b] = total; seg_cnt becomes the exclusive prefix over segments

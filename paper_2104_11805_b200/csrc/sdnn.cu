@@ -215,6 +215,8 @@ int validate_cfg(const sdnn_config* cfg) {
     if (cfg->activation == SDNN_ACT_CLAMPED_RELU && (!(cfg->clamp > 0.0f) || !std::isfinite(cfg->clamp)))
         return fail(nullptr, SDNN_ERR_INVALID_ARG, "clamp must be finite and > 0");
     if (cfg->max_batch < 1) return fail(nullptr, SDNN_ERR_INVALID_ARG, "max_batch must be >= 1");
+    if (cfg->max_batch > (1 << 30))      // rounding up to the tile width must stay inside 32 bits
+        return fail(nullptr, SDNN_ERR_INVALID_ARG, "max_batch must be at most 2^30");
     if (cfg->train && cfg->max_batch > 128) return fail(nullptr, SDNN_ERR_INVALID_ARG, "training handles support max_batch <= 128");
     if ((cfg->flags & SDNN_FLAG_BWD_ATOMICS) && (cfg->flags & SDNN_FLAG_BWD_CSC))
         return fail(nullptr, SDNN_ERR_INVALID_ARG, "choose one backward strategy");
@@ -1444,6 +1446,96 @@ extern "C" int sdnn_probe_gather_rate(int32_t row_bytes, int64_t table_rows, dou
 }
 
 // ---------------------------------------------------------------------------------------------
+// Shared-memory / distributed-shared-memory gather probe (see sdnn_probe_smem_gather_rate in the header).
+namespace {
+
+template <int G, bool REMOTE>
+int run_smem_probe(int cluster, int rows_log2, int cluster_log2, size_t smem, float* sink, cudaStream_t st, cudaEvent_t a, cudaEvent_t b,
+                   int sms, double* rows_per_second, int* ctas_out) {
+    auto kernel = smem_gather_probe_kernel<G, REMOTE>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess && cluster > 8) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    if (e != cudaSuccess) return cuda_fail(nullptr, e, "cudaFuncSetAttribute(smem probe)");
+    cudaLaunchConfig_t lc = {};
+    lc.blockDim = dim3(1024); lc.dynamicSmemBytes = smem; lc.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = cluster; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    lc.attrs = at; lc.numAttrs = 1;
+    int clusters = sms / cluster;
+    if (cluster > 1) {      // how many clusters of this size the device holds at once
+        lc.gridDim = dim3(cluster);
+        int fit = 0;
+        e = cudaOccupancyMaxActiveClusters(&fit, kernel, &lc);
+        if (e != cudaSuccess || fit < 1) { cudaGetLastError(); return fail(nullptr, SDNN_ERR_CUDA, "clusters of %d CTAs with %zu bytes of shared memory do not fit this device", cluster, smem); }
+        clusters = std::min(clusters, fit);
+    }
+    const int grid = clusters * cluster;
+    lc.gridDim = dim3(grid);
+    const int64_t groups = (int64_t)grid * 1024 / G;
+    const int per_group = 4096;
+    float* snk = sink;
+    unsigned rl = (unsigned)rows_log2, cl = (unsigned)cluster_log2;
+    for (int i = 0; i < 2; ++i) { unsigned seed = 17u + i; e = cudaLaunchKernelEx(&lc, kernel, snk, rl, cl, per_group, seed); if (e != cudaSuccess) return cuda_fail(nullptr, e, "smem probe launch"); }
+    cudaEventRecord(a, st);
+    const int reps = 5;
+    for (int i = 0; i < reps; ++i) { unsigned seed = 101u + i; cudaLaunchKernelEx(&lc, kernel, snk, rl, cl, per_group, seed); }
+    cudaEventRecord(b, st);
+    e = cudaEventSynchronize(b);
+    if (e != cudaSuccess) return cuda_fail(nullptr, e, "smem probe");
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, a, b);
+    if (!(ms > 0.f)) return fail(nullptr, SDNN_ERR_CUDA, "smem probe: no time measured");
+    *rows_per_second = (double)groups * per_group / (ms / reps * 1e-3);
+    if (ctas_out) *ctas_out = grid;
+    return SDNN_OK;
+}
+
+}  // namespace
+
+extern "C" int sdnn_probe_smem_gather_rate(int32_t row_bytes, int32_t cluster_size, double* rows_per_second, int32_t* ctas_out) {
+    if (!rows_per_second) return fail(nullptr, SDNN_ERR_INVALID_ARG, "rows_per_second is NULL");
+    *rows_per_second = 0.0;
+    if (row_bytes != 32 && row_bytes != 64 && row_bytes != 128 && row_bytes != 256)
+        return fail(nullptr, SDNN_ERR_INVALID_ARG, "row_bytes must be 32, 64, 128 or 256");
+    if (cluster_size != 1 && cluster_size != 2 && cluster_size != 4 && cluster_size != 8 && cluster_size != 16)
+        return fail(nullptr, SDNN_ERR_INVALID_ARG, "cluster_size must be 1, 2, 4, 8 or 16");
+    int dev = 0, sms = 0;
+    CU(nullptr, cudaGetDevice(&dev));
+    CU(nullptr, cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const size_t smem = 128u << 10;                      // table bytes per CTA
+    int rows_log2 = 0;
+    while ((size_t)(2u << rows_log2) * row_bytes <= smem) ++rows_log2;
+    int cluster_log2 = 0;
+    while ((1 << cluster_log2) < cluster_size) ++cluster_log2;
+    float* sink = nullptr;
+    cudaEvent_t a = nullptr, b = nullptr;
+    cudaStream_t st = nullptr;
+    int rc = SDNN_OK;
+    if (cudaMalloc(&sink, 256) != cudaSuccess || cudaStreamCreate(&st) != cudaSuccess || cudaEventCreate(&a) != cudaSuccess ||
+        cudaEventCreate(&b) != cudaSuccess) {
+        cudaGetLastError();
+        rc = fail(nullptr, SDNN_ERR_OOM, "could not set up the probe");
+    } else {
+        const bool remote = cluster_size > 1;
+#define SDNN_SMEM_PROBE(G) (remote ? run_smem_probe<G, true>(cluster_size, rows_log2, cluster_log2, smem, sink, st, a, b, sms, rows_per_second, ctas_out) \
+                                   : run_smem_probe<G, false>(1, rows_log2, 0, smem, sink, st, a, b, sms, rows_per_second, ctas_out))
+        switch (row_bytes) {
+            case 32: rc = SDNN_SMEM_PROBE(2); break;
+            case 64: rc = SDNN_SMEM_PROBE(4); break;
+            case 128: rc = SDNN_SMEM_PROBE(8); break;
+            default: rc = SDNN_SMEM_PROBE(16); break;
+        }
+#undef SDNN_SMEM_PROBE
+    }
+    if (a) cudaEventDestroy(a);
+    if (b) cudaEventDestroy(b);
+    if (st) cudaStreamDestroy(st);
+    if (sink) cudaFree(sink);
+    return rc;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Allocation-free inference (see sdnn_infer_noalloc in the header).  The two activation tiles of
 // the forward chain live in this file-scope device array instead of memory owned by a handle.
 // In host code the array's name is only a stand-in for the symbol, not a device address: the
@@ -1501,8 +1593,12 @@ extern "C" int sdnn_infer_noalloc(int32_t n_layers, int32_t n_neurons, const int
     if (!(clamp > 0.0f) || !std::isfinite(clamp)) return fail(nullptr, SDNN_ERR_INVALID_ARG, "clamp must be finite and > 0");
     if (n_inputs == 0) return SDNN_OK;
     if (!x0 || !y_out) return fail(nullptr, SDNN_ERR_INVALID_ARG, "x0 or y_out is NULL");
+    // checked before the batch is rounded up to the tile width, which would not fit 32 bits for batches near 2^31
+    if (n_inputs > SDNN_NOALLOC_MAX_TILE_FLOATS)
+        return fail(nullptr, SDNN_ERR_INVALID_ARG, "problem too large for the built-in scratch: %d inputs, a tile holds %d floats",
+                    n_inputs, (int)SDNN_NOALLOC_MAX_TILE_FLOATS);
     const int ld = noalloc_padded_width(n_inputs);
-    if ((int64_t)n_neurons * ld > (int64_t)SDNN_NOALLOC_MAX_TILE_FLOATS)
+    if (ld <= 0 || (int64_t)n_neurons * ld > (int64_t)SDNN_NOALLOC_MAX_TILE_FLOATS)
         return fail(nullptr, SDNN_ERR_INVALID_ARG,
                     "problem too large for the built-in scratch: n_neurons * padded(n_inputs) = %lld floats, limit %d",
                     (long long)n_neurons * ld, (int)SDNN_NOALLOC_MAX_TILE_FLOATS);

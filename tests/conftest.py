@@ -19,3 +19,14 @@ def _build_cpu_libs():
     import oracle
     gen.build()
     oracle.build()
+
+
+def pytest_terminal_summary(terminalreporter):
+    """Worst error any parity comparison of this session saw, under the asserted metric and the two recorded ones."""
+    try:
+        import parity_util
+    except ImportError:
+        return
+    if any(parity_util.SESSION_WORST.values()):
+        terminalreporter.write_line("parity, worst error of the session by metric: " +
+                                    ", ".join(f"{k} {v:.3g}" for k, v in parity_util.SESSION_WORST.items()))

@@ -104,3 +104,15 @@ def test_tile_beyond_4_gib_is_rejected_before_any_device_work(pkg):
     with pytest.raises(pkg.SdnnError) as ei:
         pkg.Sdnn.create_deferred(1, 1 << 20, nnz, max_batch=1024)
     assert ei.value.code == -1 and "4 GiB" in ei.value.message
+
+
+def test_batch_sizes_whose_padding_overflows_32_bits_are_rejected_on_the_host(pkg):
+    """Rounding a batch of nearly 2^31 inputs up to the tile width must not wrap around: both the allocation-free entry
+    point and handle creation refuse such sizes before touching a device (dummy non-NULL addresses: never used)."""
+    for huge in (2**31 - 1, 2**31 - 100, 2**30 + 1):
+        with pytest.raises(pkg.SdnnError) as ei:
+            pkg.infer_noalloc(1, 1, 16, 16, 16, [0], 16, 16, huge, 16)
+        assert ei.value.code == -1 and "scratch" in ei.value.message
+        with pytest.raises(pkg.SdnnError) as ei:
+            pkg.Sdnn.create_deferred(1, 1, np.zeros(1, dtype=np.int64), max_batch=huge)
+        assert ei.value.code == -1 and "max_batch" in ei.value.message

@@ -9,7 +9,8 @@ import pytest
 
 import gen
 from oracle import OracleNet
-from parity_util import TAU_ULPS, TOL, KinkProtocol, check_close, ragged_net, rel_err
+import parity_util
+from parity_util import TAU_ULPS, TOL, KinkProtocol, assert_few_ambiguous, check_close, ragged_net, rel_err
 
 pytestmark = pytest.mark.gpu
 
@@ -30,7 +31,7 @@ def sdnn():
 
 # ----------------------------------------------------------------------------------------------
 def train_parity(torch, arrays, batches, eta, update_bias=False, flags=0, clamp=32.0, expect_live=None, sync=True,
-                 activation="clamped_relu"):
+                 activation="clamped_relu", host=False):
     """Runs len(batches) SGD steps on both sides, comparing everything after every step.
 
     sync=True: before every step after the first the oracle rounds its parameters to fp32 (the library's
@@ -38,7 +39,10 @@ def train_parity(torch, arrays, batches, eta, update_bias=False, flags=0, clamp=
     numbers; rounding differences of earlier steps would otherwise be amplified step after step by the
     training dynamics themselves (observed: x 10 in five steps on the live 1024 x 120 net), which says
     nothing about one step's arithmetic.  sync=False lets the two trajectories run free (checks that
-    parameters persist across calls)."""
+    parameters persist across calls).  host=True: the step goes through sdnn_train_step_host (numpy buffers).
+
+    Returns statistics of the run: the kink bookkeeping, the worst error under the asserted normwise metric and
+    under the two elementwise ones (parity_util.WORST), and whether any gradient was nonzero."""
     pkg = sdnn()
     rp, col, val, bias = arrays
     L, n = len(col), len(bias[0])
@@ -48,12 +52,16 @@ def train_parity(torch, arrays, batches, eta, update_bias=False, flags=0, clamp=
                         flags=pkg.FLAG_KEEP_DEBUG | flags, activation=pkg.ACT_SIGMOID if sigmoid else pkg.ACT_CLAMPED_RELU)
     ora = OracleNet(rp, col, val, bias, clamp=clamp, update_bias=update_bias, activation=activation)
     stats = dict(ambiguous=0, flipped=0, entries=0, worst=0.0, max_err=0.0, grad_nonzero=False)
+    parity_util.reset_worst()
     for step, (x0, y) in enumerate(batches):
         if sync and step > 0:
             ora.quantize_state()
             for l in range(L):
                 h.set_weights(l, ora.w[l], ora.bias[l])
-        loss_g = h.train_step(torch.from_numpy(x0).cuda(), torch.from_numpy(y).cuda(), B, eta, want_loss=True)
+        if host:
+            loss_g = h.train_step(x0, y, B, eta, want_loss=True, host=True)
+        else:
+            loss_g = h.train_step(torch.from_numpy(x0).cuda(), torch.from_numpy(y).cuda(), B, eta, want_loss=True)
         acts = {}
 
         def gpu_x(k):
@@ -84,6 +92,8 @@ def train_parity(torch, arrays, batches, eta, update_bias=False, flags=0, clamp=
         for key in ("ambiguous", "flipped", "entries"):
             stats[key] += getattr(proto, key)
         stats["worst"] = max(stats["worst"], proto.worst)
+    assert_few_ambiguous(stats["ambiguous"], stats["entries"], "derivative masks")
+    stats["worst_by_metric"] = dict(parity_util.WORST)
     if expect_live is not None:
         assert stats["grad_nonzero"] == expect_live
     h.destroy()
@@ -115,7 +125,8 @@ def infer_parity(torch, arrays, x0, max_batch, host=False, clamp=32.0, expect_no
     z, xl, scale = ora.forward_layer(L - 1, x, want_scale=True)
     check_close(y, xl, "x^L")
     assert total == int(c.sum())
-    amb = np.abs(z) <= TAU_ULPS * 2.0 ** -24 * scale
+    amb = (np.abs(z) <= TAU_ULPS * 2.0 ** -24 * scale) & (scale > 0.0)
+    assert_few_ambiguous(int(amb.sum()), amb.size, "final-layer nonzero sets")
     starts = np.concatenate([[0], np.cumsum(c)])
     n_amb = 0
     for b in range(cnt):
@@ -175,6 +186,20 @@ def test_train_launch_variants_match(torch_cuda, extra):
     batches = [(rng.uniform(0, 1.5, size=(16, 130)).astype(np.float32), rng.uniform(0, 1, size=(16, 130)).astype(np.float32))
                for _ in range(2)]
     train_parity(torch_cuda, arrays, batches, eta=0.01, flags=flags, expect_live=True)
+
+
+@pytest.mark.parametrize("B", [1, 16, 37])
+def test_train_step_through_host_buffers(torch_cuda, B):
+    """sdnn_train_step_host (inputs and targets in host memory, staged by the library): the same parity as the
+    device-pointer entry point, everything compared after each of three steps."""
+    rng = np.random.default_rng(600 + B)
+    arrays = ragged_net(rng, n=203, layers=5, kmax=12)
+    batches = [(rng.uniform(0, 1.5, size=(B, 203)).astype(np.float32), rng.uniform(0, 1, size=(B, 203)).astype(np.float32))
+               for _ in range(3)]
+    train_parity(torch_cuda, arrays, batches, eta=0.01, update_bias=True, expect_live=True, host=True)
+    spec = gen.CFG3.scaled(2048, 12).live()
+    st = train_parity(torch_cuda, gen.network(spec), batches_for(spec, 16, 2), eta=1e-3, expect_live=True, host=True)
+    print("host buffers", spec.name, st)
 
 
 @pytest.mark.parametrize("variant,live", [("base", False), ("live", True)])
@@ -457,6 +482,65 @@ def test_train_in_the_benchmark_launch_configuration(torch_cuda, spec, B):
     h.destroy()
 
 
+def check_update(w_gpu, w_before, w_oracle, what=""):
+    """The update itself, W_new - W_old, not just the updated weights (of which the update is a ten-thousandth): within
+    1e-4 of its largest entry, plus the rounding of one fp32 store of the weight (the library keeps W in fp32)."""
+    u_gpu = w_gpu.astype(np.float64) - w_before
+    u_ora = w_oracle - w_before
+    bound = TOL * np.abs(u_ora).max() + 2.0 ** -23 * np.abs(w_before).max()
+    worst = np.abs(u_gpu - u_ora).max()
+    assert worst <= bound, f"{what}: update off by {worst:.3g} (bound {bound:.3g}, largest update {np.abs(u_ora).max():.3g})"
+    return worst / max(np.abs(u_ora).max(), 1e-300), bool(np.abs(u_ora).max() > 2.0 ** -20 * np.abs(w_before).max())
+
+
+@pytest.mark.parametrize("spec", [gen.CFG5.scaled(65536, 256).live(), gen.CFG5.scaled(65536, 240).paper_setup()])
+def test_train_cfg5_full_width_deep_in_the_benchmark_launch_configuration(torch_cuda, spec):
+    """Config 5 at full width (65536 neurons, B = 16) and as deep as a host of a few tens of GB holds the float64 oracle
+    (256 layers for the live companion, 240 with the paper's own setup: about 17 GB of host memory), on the handle bench.py times: default flags, no
+    debug buffers, the step as one CUDA graph.  Depth is where rounding accumulates and where the long launch chain lives.
+    Two steps; the loss, every layer's activations, updated weights AND the update itself, and the consistency of the two
+    weight copies, against the oracle run the same way (kink protocol as in train_parity)."""
+    torch = torch_cuda
+    pkg = sdnn()
+    rp, col, val, bias = gen.network(spec)
+    sigmoid = spec.values == "uniform_pm1"
+    eta = 0.01 if sigmoid else 1e-3
+    B, L = 16, spec.layers
+    h = pkg.Sdnn.create(rp, col, val, bias, max_batch=B, train=True, activation=pkg.ACT_SIGMOID if sigmoid else pkg.ACT_CLAMPED_RELU)
+    ora = OracleNet(rp, col, val, bias, activation="sigmoid" if sigmoid else "clamped_relu")
+    parity_util.reset_worst()
+    ambiguous = entries = 0
+    worst_update, moved = 0.0, np.zeros(L, dtype=bool)      # moved[l]: the update of layer l is well above one fp32 rounding of W
+    for step, (x0, y) in enumerate(batches_for(spec, B, 2)):
+        if step:
+            ora.quantize_state()
+            for l in range(L):
+                h.set_weights(l, ora.w[l], ora.bias[l])
+        before = [w.copy() for w in ora.w]
+        loss = h.train_step(torch.from_numpy(x0).cuda(), torch.from_numpy(y).cuda(), B, eta, want_loss=True)
+        proto = KinkProtocol(lambda k: h.get_activations(k, B))
+        out = ora.train_step(x0, y, eta, mask_hook=None if sigmoid else proto, keep=("x",))
+        assert proto.hard_mismatch == 0, f"{proto.hard_mismatch} derivative-mask mismatches outside the ambiguous set"
+        ambiguous += proto.ambiguous; entries += proto.entries
+        assert abs(loss - out["loss"]) <= TOL * abs(out["loss"])
+        for l in range(L):
+            w = h.get_weights(l, want_bias=False)
+            check_close(w, ora.w[l], f"step {step} W^{l + 1}")
+            err, big = check_update(w, before[l], ora.w[l], f"step {step} layer {l + 1}")
+            moved[l] |= big
+            if big:
+                worst_update = max(worst_update, err)
+            assert h.mirror_mismatches(l) == 0
+        for k in range(1, L + 1):
+            check_close(h.get_activations(k, B), out["x"][k], f"step {step} x^{k}")
+    assert_few_ambiguous(ambiguous, entries, "derivative masks")
+    # the sigmoid net's gradient fades with depth (f' <= 1/4 per layer), so only its upper layers move; the live net moves everywhere
+    assert moved[-1] and (sigmoid or moved.all()), f"vacuous: only {int(moved.sum())} of {L} layers moved"
+    print(spec.name, L, "layers:", parity_util.WORST, "layers whose update is well above fp32 rounding:", int(moved.sum()),
+          "worst update error among them (of the largest update)", worst_update, "ambiguous", ambiguous, "of", entries)
+    h.destroy()
+
+
 def test_train_cfg3_live_full_size(torch_cuda):
     """Config 3 at full size (16384 x 480, B = 64), live companion, one step."""
     spec = gen.CFG3.live()
@@ -592,6 +676,17 @@ def test_gather_probe_reports_a_rate_and_rejects_bad_sizes(torch_cuda):
     for row_bytes, rows in ((48, 1024), (64, 1000), (512, 1 << 22)):
         with pytest.raises(pkg.SdnnError) as ei:
             pkg.probe_gather_rate(row_bytes, rows)
+        assert ei.value.code == -1
+
+
+def test_shared_memory_gather_probe_reports_rates_and_rejects_bad_sizes(torch_cuda):
+    pkg = sdnn()
+    for cluster in (1, 4, 16):
+        rate, ctas = pkg.probe_smem_gather_rate(64, cluster)
+        assert 1e9 < rate < 1e14 and ctas >= cluster and ctas % cluster == 0
+    for row_bytes, cluster in ((48, 1), (64, 3), (512, 1), (64, 32)):
+        with pytest.raises(pkg.SdnnError) as ei:
+            pkg.probe_smem_gather_rate(row_bytes, cluster)
         assert ei.value.code == -1
 
 

@@ -5,12 +5,16 @@ the whole device to another allocator, they sit in a latency-critical loop, or t
 it), so this entry point keeps its activation scratch in a fixed array inside the library and takes the
 network as the caller's own device arrays.  The test calls it through the C ABI twice in a row (the
 second call with a smaller batch, so stale scratch contents from the first would show) and compares
-with the handle-based entry point.  This file is collected last on purpose.
+with the handle-based entry point and with the float64 oracle; a second test runs nets whose rows have any
+length (rows that do not start on a multiple of four entries take the kernel's one-entry-at-a-time path)
+and batches of one to a few inputs.  This file is collected last on purpose.
 """
 import numpy as np
 import pytest
 
 import gen
+from oracle import OracleNet
+from parity_util import check_close, ragged_net
 
 pytestmark = pytest.mark.gpu
 
@@ -39,14 +43,49 @@ def test_noalloc_inference_matches_handle_inference_twice_in_a_row():
         got = torch.full((cnt, n), -1.0, device="cuda")
         h.infer_batch(x0, cnt, want, None, None, 0)
         torch.cuda.synchronize()
-        reserved = torch.cuda.memory_reserved()
+        free_before = torch.cuda.mem_get_info()[0]          # the driver's count of free device bytes: sees any cudaMalloc
         pkg.infer_noalloc(L, n, d_rp, d_col, d_val, offsets, d_bias, x0, cnt, got)
         torch.cuda.synchronize()
-        assert torch.cuda.memory_reserved() == reserved
+        if start:       # the first call on a device may load the module; from the second on nothing may be taken
+            assert torch.cuda.mem_get_info()[0] == free_before
         w, g = want.cpu().numpy(), got.cpu().numpy()
         assert np.abs(w).max() > 0
         assert np.abs(g - w).max() <= 1e-4 * np.abs(w).max()
+        check_close(g, OracleNet(rp, col, val, bias).infer(gen.inputs(spec, cnt, start=start)), "x^L against the oracle")
     h.destroy()
+
+
+@pytest.mark.parametrize("cnt", [1, 3, 5, 20, 150])
+def test_noalloc_inference_on_ragged_rows_and_tiny_batches_matches_the_oracle(cnt):
+    """Rows of 0..11 entries, so that most rows start off a multiple of four; each layer's entries start on one
+    (the entry point's rule), which leaves up to three unused slots between layers."""
+    torch = pytest.importorskip("torch")
+    assert torch.cuda.is_available()
+    import paper_2104_11805_b200 as pkg
+    from paper_2104_11805_b200.build import build_library
+    build_library()
+
+    rng = np.random.default_rng(40 + cnt)
+    n, L = 301, 4
+    rp, col, val, bias = ragged_net(rng, n=n, layers=L, kmax=11, scale=0.5)
+    offsets, run = [], 0
+    for c in col:
+        offsets.append(run)
+        run += (len(c) + 3) // 4 * 4
+    flat_col = np.zeros(run, dtype=np.int32); flat_val = np.zeros(run, dtype=np.float32)
+    for o, c, v in zip(offsets, col, val):
+        flat_col[o:o + len(c)] = c; flat_val[o:o + len(v)] = v
+    assert all((np.asarray(r)[:-1] % 4 != 0).sum() > n // 2 for r in rp), "most rows should start off a multiple of four"
+    d_rp, d_col, d_val = (torch.from_numpy(a).cuda() for a in (np.stack(rp), flat_col, flat_val))
+    d_bias = torch.from_numpy(np.stack(bias)).cuda()
+    x0 = rng.uniform(0, 1.0, size=(cnt, n)).astype(np.float32)
+    want = OracleNet(rp, col, val, bias).infer(x0)
+    assert np.abs(want).max() > 0
+    for _ in range(2):
+        got = torch.full((cnt, n), -1.0, device="cuda")
+        pkg.infer_noalloc(L, n, d_rp, d_col, d_val, np.asarray(offsets, dtype=np.int64), d_bias, torch.from_numpy(x0).cuda(), cnt, got)
+        torch.cuda.synchronize()
+        check_close(got.cpu().numpy(), want, f"{cnt} inputs")
 
 
 def test_noalloc_rejects_sizes_beyond_the_builtin_scratch():

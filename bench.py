@@ -45,6 +45,9 @@ WORKLOADS = {
     "cfg2-live": (gen.CFG2.live(), "infer", 1024, 60000),
     "cfg4": (gen.CFG4, "infer", 1024, 60000),
     "cfg4-live": (gen.CFG4.live(), "infer", 1024, 60000),
+    # config 4 with the neurons of every inner layer renumbered at random: the block structure is there but hidden
+    "cfg4-shuffled": (gen.CFG4.shuffled(), "infer", 1024, 60000),
+    "cfg4-live-shuffled": (gen.CFG4.live().shuffled(), "infer", 1024, 60000),
     # the paper's own training setup (Section 6): sigmoid, weights uniform in [-1, 1], eta = 0.01
     "cfg3-paper": (gen.CFG3.paper_setup(), "train", 64, 64),
     "cfg5-paper": (gen.CFG5.paper_setup(), "train", 16, 16),
@@ -206,6 +209,41 @@ def workload_config(wname, spec, kind, batch, averaged=False):
     return cfg
 
 
+def study_probes():
+    """Rates of the operand paths a layer kernel can take its gathered rows from, as rows per clock and SM at the maximum
+    SM clock, and the scattered-word rates that a single shared value array would depend on."""
+    import torch
+
+    import paper_2104_11805_b200 as pkg
+    from paper_2104_11805_b200.build import build_library
+    build_library()
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    props = torch.cuda.get_device_properties(torch.cuda.current_device())
+    sms = props.multi_processor_count
+    try:
+        import pynvml
+        pynvml.nvmlInit()
+        mhz = pynvml.nvmlDeviceGetMaxClockInfo(pynvml.nvmlDeviceGetHandleByIndex(torch.cuda.current_device()), pynvml.NVML_CLOCK_SM)
+    except Exception:
+        mhz = 1965
+    clk = mhz * 1e6
+    out = {"study": "probes", "sms": sms, "sm_max_mhz": mhz, "unit": "rows (or words) per clock per SM at sm_max_mhz", "l2": {}, "l2_small_table": {},
+           "shared": {}, "cluster": {}, "words": {}}
+    for rb in (16, 32, 64, 128, 256, 512, 1024):
+        rows = (4 << 20) // rb                                   # a 4 MB table: an activation tile of the large configurations
+        out["l2"][str(rb)] = pkg.probe_gather_rate(rb, rows) / sms / clk
+        out["l2_small_table"][str(rb)] = pkg.probe_gather_rate(rb, max(1, (64 << 10) // rb)) / sms / clk      # 64 KB: L1 hits
+    for rb in (32, 64, 128, 256):
+        r, ctas = pkg.probe_smem_gather_rate(rb, 1)
+        out["shared"][str(rb)] = r / ctas / clk
+        for cl in (2, 4, 8, 16):
+            r, ctas = pkg.probe_smem_gather_rate(rb, cl)
+            out["cluster"][f"{rb}x{cl}"] = {"rate": r / ctas / clk, "ctas": ctas}
+    for name, store in (("load4", 0), ("store4", 1)):
+        out["words"][name] = pkg.probe_word_rate(store, 1 << 21) / sms / clk       # an 8 MB value array (one layer of the largest net)
+    print(json.dumps(out), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -225,15 +263,23 @@ def main():
                     help="train workloads: the averaged form of the minibatch step (one batch-averaged gradient vector is "
                          "backpropagated; sdnn_train_step_averaged) instead of the exact minibatch step")
     ap.add_argument("--flags", type=lambda s: int(s, 0), default=0, help="extra SDNN_FLAG_* bits")
+    ap.add_argument("--batch", type=int, default=None, help="train workloads: another minibatch size on the same net")
+    ap.add_argument("--study", default=None, choices=["probes"],
+                    help="instead of a workload: 'probes' = the operand-path probes (random row gathers out of L2, out of shared "
+                         "memory, out of a cluster's distributed shared memory; scattered 4-byte words), one JSON line")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-compaction", action="store_true", help="inference: skip the extra pass with dead inputs dropped")
     args = ap.parse_args()
     if args.warmup < 3 and args.layers is None:
         args.warmup = 3
+    if args.study == "probes":
+        return study_probes()
     spec, kind, batch, n_inputs = WORKLOADS[args.workload]
     if args.tile and kind == "infer":
         batch = args.tile
+    if args.batch and kind == "train":
+        batch = n_inputs = args.batch
     if args.net:
         n_, l_ = (int(v) for v in args.net.split(","))
         spec = spec.scaled(n_, l_)
@@ -413,7 +459,7 @@ def main():
 
     # -------------------------------------------------------------------- inference: the same call with dead inputs dropped
     compaction = None
-    if kind == "infer" and not args.no_compaction:
+    if kind == "infer" and not args.no_compaction and not (flags & pkg.FLAG_REORDER):
         with torch.cuda.stream(stream):
             hc = pkg.Sdnn.create_deferred(L, N, [spec.nnz_per_layer] * L, max_batch=batch, flags=flags | pkg.FLAG_SKIP_DEAD,
                                           stream=stream.cuda_stream, device=local_rank)
@@ -464,12 +510,13 @@ def main():
     else:
         batch = h.infer_tile_width()           # the library narrows the tile when two of them would not fit in L2
         tiles = (n_inputs + batch - 1) // batch
-        dom = "forward_kernel"
+        dom = "forward_window_kernel" if h.windowed_layers() == L else "forward_kernel"
+        extra_reorder = {"grouped_layers": h.grouped_layers(), "windowed_layers": h.windowed_layers()}
         per_launch_ms = ms_per_step / (tiles * L)      # includes the (small) transpose and count kernels of each tile
         # per launch: the layer's indices and values once, the activation tile read and written once
         alg = 8 * nnz_l + 2 * N * min(batch, n_inputs) * 4
         in_flight = h.infer_tiles_in_flight() if tiles > 1 else 1
-        extra = {"tiles": tiles, "tile_inputs": batch, "tiles_in_flight": in_flight,
+        extra = {"tiles": tiles, "tile_inputs": batch, "tiles_in_flight": in_flight, **extra_reorder,
                  "note": "launch time = call time / forward launches (upper bound)" +
                          ("; two tiles run beside each other on two streams, so this is the time the device spends per "
                           "launch, not one launch's start-to-end duration" if in_flight > 1 else "")}
@@ -492,7 +539,7 @@ def main():
     except Exception as exc:      # the probe is a diagnostic; the line stands without it
         extra["gather_bound"] = {"error": str(exc)}
     achieved = alg / (per_launch_ms * 1e-3) / 1e9 if per_launch_ms else None
-    traffic = NCU_TRAFFIC.get((args.workload.replace("-live", ""), dom)) if (not args.layers or kind == "train") and not args.pattern and not args.net else None
+    traffic = NCU_TRAFFIC.get((args.workload.replace("-live", ""), dom)) if (not args.layers or kind == "train") and not args.pattern and not args.net and not args.batch else None
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
                 "frac": achieved / hbm_peak if achieved else None, "traffic": traffic, "peak_source": peak_src,
                 "algorithmic_bytes_per_launch": alg, "launch_ms": per_launch_ms, **extra}

@@ -24,7 +24,7 @@ _SRC = os.path.join(_HERE, "sdnn_gen.c")
 _LIB = os.path.join(_HERE, "libsdnn_gen.so")
 
 # stream ids (first component of every key)
-S_PATTERN, S_PERM, S_VALUES, S_INPUT, S_TARGET = 1, 2, 3, 4, 5
+S_PATTERN, S_PERM, S_VALUES, S_INPUT, S_TARGET, S_SHUFFLE = 1, 2, 3, 4, 5, 6
 
 
 def build(force: bool = False) -> str:
@@ -80,6 +80,7 @@ class NetSpec:
     input_prob: float = 0.1
     config_id: int = 0          # separates the key spaces of the configs
     seed: int = MASTER_SEED
+    shuffle: bool = False       # hidden structure: the neurons of every inner layer renumbered at random (see shuffled())
 
     # ---- companions that keep activations alive / drive them to the clamp ----
     def live(self) -> "NetSpec":
@@ -94,6 +95,13 @@ class NetSpec:
         """Same pattern with the training setup of the paper's Section 6: weights uniform in [-1, 1], bias 0 (to be
         used with the sigmoid activation and eta = 0.01; no neuron ever dies)."""
         return replace(self, name=self.name + "-paper", values="uniform_pm1", bias=0.0)
+
+    def shuffled(self) -> "NetSpec":
+        """The same network with the neurons of every inner layer renumbered by a seeded random permutation (rows of
+        that layer's matrix permuted, columns of the next layer's matrix renamed to match; input and output neurons
+        keep their numbers).  The function computed is unchanged; whatever block structure the pattern has is
+        hidden behind the renumbering, as in a network that arrives in no particular neuron order."""
+        return replace(self, name=self.name + "-shuffled", shuffle=True)
 
     def sliced(self, layers: int) -> "NetSpec":
         return replace(self, layers=layers)
@@ -126,8 +134,34 @@ def row_ptr(spec: NetSpec) -> np.ndarray:
     return (np.arange(spec.n + 1, dtype=np.int64) * spec.k).astype(np.int32)
 
 
+def _renumbering(spec: NetSpec, layer: int) -> np.ndarray:
+    """q[new] = old number of the output neurons of layer `layer` (0-based); identity for the last layer and for layer -1
+    (the inputs)."""
+    if not spec.shuffle or layer < 0 or layer >= spec.layers - 1:
+        return np.arange(spec.n, dtype=np.int32)
+    q = np.empty(spec.n, dtype=np.int32)
+    _L().sdnn_gen_permutation(spec.seed, (spec.config_id << 8) | S_SHUFFLE, layer, spec.n, _ptr(q))
+    return q
+
+
+def _renumbered(spec: NetSpec, layer: int, col: np.ndarray, val: np.ndarray | None):
+    """Applies the renumbering of shuffled() to one layer given in the original numbering: pure index bookkeeping."""
+    q_out, q_in = _renumbering(spec, layer), _renumbering(spec, layer - 1)
+    inv_in = np.empty(spec.n, dtype=np.int32)
+    inv_in[q_in] = np.arange(spec.n, dtype=np.int32)
+    c = inv_in[col.reshape(spec.n, spec.k)[q_out]]
+    order = np.argsort(c, axis=1, kind="stable")
+    c = np.take_along_axis(c, order, axis=1).astype(np.int32).reshape(-1)
+    if val is None:
+        return c, None
+    v = np.take_along_axis(val.reshape(spec.n, spec.k)[q_out], order, axis=1).reshape(-1)
+    return c, np.ascontiguousarray(v)
+
+
 def layer_pattern(spec: NetSpec, layer: int) -> np.ndarray:
     """Column indices of layer `layer` (0-based), int32 [n*k], ascending within each row."""
+    if spec.shuffle:
+        return _renumbered(spec, layer, layer_pattern(replace(spec, shuffle=False), layer), None)[0]
     col = np.empty(spec.n * spec.k, dtype=np.int32)
     if spec.pattern == "uniform":
         _L().sdnn_gen_pattern_uniform(spec.seed, (spec.config_id << 8) | S_PATTERN, layer, spec.n, spec.k, _ptr(col))
@@ -148,6 +182,9 @@ def layer_permutation(spec: NetSpec, layer: int) -> np.ndarray:
 
 def layer_values(spec: NetSpec, layer: int) -> np.ndarray:
     """Weights of layer `layer` in CSR order, float32 [n*k]."""
+    if spec.shuffle:
+        base = replace(spec, shuffle=False)
+        return _renumbered(spec, layer, layer_pattern(base, layer), layer_values(base, layer))[1]
     cnt = spec.n * spec.k
     if spec.values == "const":
         return np.full(cnt, np.float32(spec.const), dtype=np.float32)

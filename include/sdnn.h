@@ -77,6 +77,25 @@ typedef enum {
                                     /* every delta^k of a step (N * padded(B) * 4 bytes per layer more) and is faster    */
 #define SDNN_FLAG_NO_PDL      0x20u /* do not let a layer's kernel start its prologue under the previous layer's tail */
 #define SDNN_FLAG_ONE_TILE    0x40u /* inference: one tile in flight at a time (see sdnn_infer_batch)               */
+#define SDNN_FLAG_REORDER     0x100u /* set-up (untimed): group the rows of every W^k by the columns they share and    */
+                                    /* renumber the neurons of layer k-1 so that each group's columns are one            */
+                                    /* contiguous window of at most 1536 neurons (the single-GPU counterpart of the      */
+                                    /* paper's row partitioning, Section 5: rows that read the same x entries go         */
+                                    /* together).  A layer for which such groups exist is stored group by group, so that */
+                                    /* the rows worked on at any moment gather from a small window of the activation     */
+                                    /* tile that the caches hold; a layer without that structure (a uniformly random     */
+                                    /* pattern) is left as it is.  Everything                                             */
+                                    /* the caller sees keeps the caller's numbering: inputs, outputs, id lists,           */
+                                    /* sdnn_get_weights / sdnn_set_weights.  The layers are analysed in sdnn_finalize;   */
+                                    /* until then the handle keeps a host copy of every loaded layer.  Inference handles */
+                                    /* only (SDNN_ERR_UNIMPLEMENTED with train = 1); not together with                    */
+                                    /* SDNN_FLAG_SKIP_DEAD.                                                               */
+
+#define SDNN_FLAG_SMEM_WINDOWS 0x200u /* with SDNN_FLAG_REORDER: run the layers for which groups were found with a kernel  */
+                                    /* that copies each group's window of the activation tile into shared memory and     */
+                                    /* gathers from there (forward_window_kernel) instead of the default kernels, which   */
+                                    /* gather the same window out of L1/L2.  Measured slower on B200 for wide inference   */
+                                    /* tiles, hence opt-in; kept so that the comparison can be repeated.                  */
 
 #define SDNN_ACT_CLAMPED_RELU 0
 #define SDNN_ACT_SIGMOID      1
@@ -247,6 +266,18 @@ int sdnn_mirror_mismatches(sdnn_t* h, int32_t layer, int64_t* count_out);
 int sdnn_probe_gather_rate(int32_t row_bytes, int64_t table_rows, double* rows_per_second);
 
 /*
+ * Measures the alternative to keeping two copies of a training layer's values (diagnostic; the paper has no
+ * counterpart): with ONE value array in row-major order, the column units of the transposed product would reach each
+ * value through a position map, i.e. read (and, to apply the update, write) single 4-byte words at scattered places.
+ * store = 0: scattered 4-byte loads; store = 1: scattered 4-byte stores; out of / into a table of `table_words` floats
+ * (a power of two, 2^10 .. 2^28).  words_per_second (host double*): accesses per second by the whole device.  To be
+ * compared with sdnn_probe_gather_rate: a scattered word costs the load/store pipe as much as a gathered row of up
+ * to 64 bytes, so sharing one value array would trade one row gather per stored entry for one (loads) or two (update)
+ * scattered words.  Allocates and frees its own table and stream; synchronises.
+ */
+int sdnn_probe_word_rate(int32_t store, int64_t table_words, double* words_per_second);
+
+/*
  * The same measurement for operand tiles staged on chip (diagnostic; the paper has no counterpart): random rows of
  * `row_bytes` bytes (32, 64, 128 or 256; read with 128-bit accesses) out of a table of 128 KiB per CTA held in shared
  * memory.  cluster_size 1: every CTA reads its own shared memory; 2, 4, 8 or 16: the table is spread over the shared
@@ -258,6 +289,25 @@ int sdnn_probe_gather_rate(int32_t row_bytes, int64_t table_rows, double* rows_p
  * size does not fit the device).  Synchronises.
  */
 int sdnn_probe_smem_gather_rate(int32_t row_bytes, int32_t cluster_size, double* rows_per_second, int32_t* ctas_out);
+
+/* Layers for which SDNN_FLAG_REORDER found groups of rows sharing a window of columns (0 without the flag or before
+ * sdnn_finalize), and how many of them run with the window staged in shared memory (SDNN_FLAG_SMEM_WINDOWS). */
+int32_t sdnn_grouped_layers(const sdnn_t* h);
+int32_t sdnn_windowed_layers(const sdnn_t* h);
+
+/*
+ * The grouping step of SDNN_FLAG_REORDER on one layer, on the host (no device needed; for tests and studies):
+ * greedy column-net clustering of the rows of an n x n CSR pattern (row_ptr host int32[n+1], col_idx host int32[nnz])
+ * into groups of at most row_cap rows whose columns span at most col_cap neurons after renumbering.
+ *   group_of_row  host int32[n]: group of each row (rows without entries: the last group)
+ *   col_label     host int32[n]: new number of each column (a permutation of 0..n-1)
+ *   n_groups      host int32*: number of groups, or 0 when the pattern has no such structure (the other outputs are
+ *                 then untouched)
+ *   max_window    host int32*: widest window (new column numbers spanned by one group)
+ * Errors: INVALID_ARG (NULL, n < 1, caps < 1).
+ */
+int sdnn_cluster_layer(int32_t n, const int32_t* row_ptr, const int32_t* col_idx, int32_t col_cap, int32_t row_cap,
+                       int32_t* group_of_row, int32_t* col_label, int32_t* n_groups, int32_t* max_window);
 
 /* Counters since creation: kernels launched by this handle (graph nodes count one each);
  * device bytes it holds. */

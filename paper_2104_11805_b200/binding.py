@@ -16,6 +16,8 @@ LIB_PATH = os.path.join(_HERE, "libsdnn.so")
 FLAG_BWD_ATOMICS, FLAG_BWD_CSC, FLAG_KEEP_DEBUG, FLAG_SKIP_DEAD, FLAG_NO_GRAPH, FLAG_NO_PDL = 0x01, 0x02, 0x04, 0x08, 0x10, 0x20
 FLAG_BWD_ONE_LAUNCH = 0x80
 FLAG_ONE_TILE = 0x40
+FLAG_REORDER = 0x100
+FLAG_SMEM_WINDOWS = 0x200
 ACT_CLAMPED_RELU, ACT_SIGMOID = 0, 1
 
 STATUS = {0: "SDNN_OK", -1: "SDNN_ERR_INVALID_ARG", -2: "SDNN_ERR_BAD_CSR", -3: "SDNN_ERR_OOM", -4: "SDNN_ERR_CUDA",
@@ -53,10 +55,14 @@ _PROTOS = {
     "sdnn_get_gradient": (ctypes.c_int, [_vp, _i32, _vp]),
     "sdnn_mirror_mismatches": (ctypes.c_int, [_vp, _i32, ctypes.POINTER(_i64)]),
     "sdnn_probe_gather_rate": (ctypes.c_int, [_i32, _i64, ctypes.POINTER(ctypes.c_double)]),
+    "sdnn_probe_word_rate": (ctypes.c_int, [_i32, _i64, ctypes.POINTER(ctypes.c_double)]),
     "sdnn_probe_smem_gather_rate": (ctypes.c_int, [_i32, _i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(_i32)]),
     "sdnn_get_phase_times": (ctypes.c_int, [_vp, ctypes.POINTER(_f32), ctypes.POINTER(_f32)]),
     "sdnn_get_liveness": (ctypes.c_int, [_vp, _vp]),
     "sdnn_infer_noalloc": (ctypes.c_int, [_i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _f32, _vp]),
+    "sdnn_windowed_layers": (_i32, [_vp]),
+    "sdnn_grouped_layers": (_i32, [_vp]),
+    "sdnn_cluster_layer": (ctypes.c_int, [_i32, _vp, _vp, _i32, _i32, _vp, _vp, ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
     "sdnn_kernel_launches": (_i64, [_vp]),
     "sdnn_infer_tile_width": (_i32, [_vp]),
     "sdnn_infer_tiles_in_flight": (_i32, [_vp]),
@@ -134,6 +140,33 @@ def probe_gather_rate(row_bytes, table_rows):
     lib = load_library()
     out = ctypes.c_double(0.0)
     rc = lib.sdnn_probe_gather_rate(row_bytes, table_rows, ctypes.byref(out))
+    if rc != 0:
+        raise SdnnError(rc, (lib.sdnn_last_error(None) or b"").decode())
+    return out.value
+
+
+def cluster_layer(row_ptr, col_idx, col_cap=1536, row_cap=2048):
+    """sdnn_cluster_layer: (group_of_row, col_label, n_groups, max_window) of one CSR pattern; n_groups == 0 and None
+    arrays when the pattern has no block structure.  Host only."""
+    lib = load_library()
+    rp, ci = _np(row_ptr, np.int32), _np(col_idx, np.int32)
+    n = len(rp) - 1
+    grp, lab = np.empty(n, dtype=np.int32), np.empty(n, dtype=np.int32)
+    ng, mw = ctypes.c_int32(0), ctypes.c_int32(0)
+    rc = lib.sdnn_cluster_layer(n, rp.ctypes.data, ci.ctypes.data, col_cap, row_cap, grp.ctypes.data, lab.ctypes.data,
+                                ctypes.byref(ng), ctypes.byref(mw))
+    if rc != 0:
+        raise SdnnError(rc, (lib.sdnn_last_error(None) or b"").decode())
+    if ng.value == 0:
+        return None, None, 0, 0
+    return grp, lab, ng.value, mw.value
+
+
+def probe_word_rate(store, table_words):
+    """sdnn_probe_word_rate: scattered 4-byte loads (store=False) or stores (store=True) per second."""
+    lib = load_library()
+    out = ctypes.c_double(0.0)
+    rc = lib.sdnn_probe_word_rate(int(bool(store)), table_words, ctypes.byref(out))
     if rc != 0:
         raise SdnnError(rc, (lib.sdnn_last_error(None) or b"").decode())
     return out.value
@@ -276,6 +309,14 @@ class Sdnn:
     def infer_tiles_in_flight(self):
         """Tiles infer_batch keeps in flight on this handle when a batch has several (1 or 2)."""
         return int(self._lib.sdnn_infer_tiles_in_flight(self._h))
+
+    def grouped_layers(self):
+        """Layers for which FLAG_REORDER found groups of rows sharing a window of columns."""
+        return int(self._lib.sdnn_grouped_layers(self._h))
+
+    def windowed_layers(self):
+        """Layers that run with their operand window staged in shared memory (FLAG_REORDER)."""
+        return int(self._lib.sdnn_windowed_layers(self._h))
 
     def kernel_launches(self):
         return int(self._lib.sdnn_kernel_launches(self._h))

@@ -44,6 +44,8 @@ struct Sliced {
     const int* idx;         // gathered tile row of each entry (column index; row index in the transposed copy)
     float*     val;
     const int* order;
+    const int* out;         // forward kernels: tile row that unit u's output goes to (NULL: row u), for layers whose rows are
+                            // stored group by group while their neurons carry the numbers the next layer's grouping gave them
 };
 
 __device__ __forceinline__ float4 ld_f4(const float* p) { return *reinterpret_cast<const float4*>(p); }
@@ -262,8 +264,9 @@ __device__ __forceinline__ void chunk_update(float* vp, float* gp, const float4&
 // ---------------------------------------------------------------------------------------------
 // x0 [cnt][n] (input-major, as the caller passes it)  ->  tile [n][ld], zero-padded for b >= cnt.
 // Block (32, 8); grid (ceil(n/32), ceil(cols/32)) where cols = padded columns to fill.
+// row_map (or NULL): tile row of input neuron i, for nets whose input neurons were renumbered at set-up.
 __global__ void transpose_in_kernel(const float* __restrict__ src, float* __restrict__ dst,
-                                    int n, int cnt, int cols, int ld) {
+                                    int n, int cnt, int cols, int ld, const int* __restrict__ row_map) {
     __shared__ float t[32][33];
     const int i0 = blockIdx.x * 32, b0 = blockIdx.y * 32;
     for (int r = threadIdx.y; r < 32; r += 8) {
@@ -273,7 +276,7 @@ __global__ void transpose_in_kernel(const float* __restrict__ src, float* __rest
     __syncthreads();
     for (int r = threadIdx.y; r < 32; r += 8) {
         int i = i0 + r, b = b0 + threadIdx.x;
-        if (i < n && b < cols) dst[(size_t)i * ld + b] = t[threadIdx.x][r];
+        if (i < n && b < cols) dst[(size_t)(row_map ? row_map[i] : i) * ld + b] = t[threadIdx.x][r];
     }
 }
 
@@ -414,6 +417,7 @@ forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict
     int row, base, nch;
     SDNN_UNIT_SHAPE(m, unit, nunits, row, base, nch)
     float b = (row < n) ? bias[row] : 0.0f;
+    int orow = (row < n && m.out) ? m.out[row] : row;
     if (unit < nunits && lane == 0) prefetch_unit(m, unit, RPW, n, UPS);
     int4 c[CPS];
 #pragma unroll
@@ -431,6 +435,7 @@ forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict
         int nrow, nbase, nnch;
         SDNN_UNIT_SHAPE(m, nunit, nunits, nrow, nbase, nnch)
         const float nb = (nrow < n) ? bias[nrow] : 0.0f;
+        const int norow = (nrow < n && m.out) ? m.out[nrow] : nrow;
         if (nunit < nunits && lane == 0) prefetch_unit(m, nunit, RPW, n, UPS);
 
         Lane<V> acc;
@@ -455,15 +460,129 @@ forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict
         if (nch == 0 && nnch > 0) load_idx<CPS>(c, idx + nbase);      // empty slice: nothing prefetched across the boundary yet
         if (row < n) {
             lane_activate(acc, act, clamp);
-            lane_store(tile_row(xout + boff, row, pitch), acc);
+            lane_store(tile_row(xout + boff, orow, pitch), acc);
             if (live_flags) live |= lane_nonzero_bits(acc);
         }
-        unit = nunit; row = nrow; base = nbase; nch = nnch; b = nb;
+        unit = nunit; row = nrow; base = nbase; nch = nnch; b = nb; orow = norow;
     }
     if (live_flags) {
 #pragma unroll
         for (int e = 0; e < V; ++e)
             if ((live >> e) & 1u) live_flags[boff + e] = 1;      // many lanes may store the same 1
+    }
+    if (pdl == 1) grid_launch_dependents();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Forward layer with the gathered operand staged in shared memory (layers whose rows were grouped by the columns
+// they share, see reorder.h).  The stored rows of such a layer come group by group; the columns of a group are one
+// contiguous range of tile rows, its window; every row of a group is padded to the group's longest row (a multiple of
+// eight entries; padding: column 0, value 0), so that the place of every entry follows from the group's base without a
+// row pointer.  Work item = (group, part of its rows, chunk of TC inputs): the CTA copies the window's TC columns into
+// shared memory (16-byte cp.async pieces, all in flight at once), then its warps walk the rows: a lane owns one input,
+// reads x[col][input] from the window (one conflict-free 128-byte wavefront per stored entry at TC = 32) and
+// accumulates in stored order.  The entries of a row (16-bit column within the window, value) travel through a small
+// ring in shared memory per warp: pieces of up to 32 entries are fetched with cp.async WINDOW_RING - 1 pieces ahead and
+// read back with warp-wide broadcast loads, so that no warp waits for an L2 round trip per row.  The output row goes
+// to the tile row `out[row]`: the number the NEXT layer's grouping gave this neuron.  A random row of the window costs
+// a shared-memory wavefront instead of an L2 round trip; the window itself is read once per item, contiguously.
+struct Windowed {
+    const unsigned short* col;    // column of each entry, relative to its group's window
+    const float* val;
+    const int* out;               // [n] tile row each stored row writes
+    const float* bias;            // [n] in stored order
+    const int* g_row0;            // [groups + 1] first stored row of each group
+    const int* g_c0;              // [groups] first tile row of each group's window
+    const int* g_wlen;            // [groups] rows of the window
+    const int* g_ebase;           // [groups] offset of the group's first entry (a multiple of 8)
+    const int* g_k;               // [groups] entries per (padded) row of the group, a multiple of 8
+    int groups;
+};
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(d), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" :: "n"(N) : "memory"); }
+
+constexpr int WINDOW_THREADS = 512;
+constexpr int WINDOW_RING = 4;                 // pieces of a warp's entry ring
+constexpr int WINDOW_PIECE_BYTES = 192;        // 32 entries: 64 bytes of columns, 128 bytes of values
+constexpr int WINDOW_RING_BYTES = (WINDOW_THREADS / 32) * WINDOW_RING * WINDOW_PIECE_BYTES;
+
+template <int TC>
+__global__ void __launch_bounds__(WINDOW_THREADS, 1)
+forward_window_kernel(Windowed m, const float* __restrict__ xin, float* __restrict__ xout, int ld, int chunks, int splits,
+                      float clamp, int act, int pdl) {
+    extern __shared__ __align__(16) unsigned char window_smem[];
+    constexpr int PPR = TC / 4;                           // 16-byte pieces per window row
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    unsigned char* ring = window_smem + warp * (WINDOW_RING * WINDOW_PIECE_BYTES);
+    float* window = reinterpret_cast<float*>(window_smem + WINDOW_RING_BYTES);      // [wlen][TC]
+    const int b = min(lane, TC - 1);                      // lanes beyond the chunk repeat its last input and store nothing
+    if (pdl) grid_dependency_wait();
+    if (pdl == 2) grid_launch_dependents();
+    const int per_group = chunks * splits;
+    const int items = m.groups * per_group;
+    for (int item = blockIdx.x; item < items; item += gridDim.x) {
+        const int g = item / per_group, rest = item - g * per_group;
+        const int split = rest / chunks, t0 = (rest - split * chunks) * TC;
+        const int c0 = m.g_c0[g], wlen = m.g_wlen[g], k = m.g_k[g];
+        const int g0 = m.g_row0[g], per_split = (m.g_row0[g + 1] - g0 + splits - 1) / splits;
+        const int r0 = g0 + split * per_split + warp, r1 = min(m.g_row0[g + 1], g0 + (split + 1) * per_split);
+        const unsigned short* gcol = m.col + m.g_ebase[g];
+        const float* gval = m.val + m.g_ebase[g];
+        const int ppr = (k + 31) >> 5;                    // pieces per row
+        const int my_rows = r0 < r1 ? (r1 - r0 + nwarps - 1) / nwarps : 0;
+        const int pieces = my_rows * ppr;
+        // piece i of this warp: row r0 + (i / ppr) * nwarps, entries (i % ppr) * 32 .. of that row
+        auto fetch = [&](int i) {
+            if (i < pieces) {
+                const int row = r0 + (i / ppr) * nwarps, t = (i % ppr) << 5;
+                const int n = min(32, k - t);             // entries of the piece, a multiple of 8
+                const size_t at = (size_t)(row - g0) * k + t;
+                unsigned char* slot = ring + (i % WINDOW_RING) * WINDOW_PIECE_BYTES;
+                if (lane < (n >> 3)) cp_async16(slot + lane * 16, gcol + at + lane * 8);
+                else if (lane >= 4 && lane - 4 < (n >> 2)) cp_async16(slot + 64 + (lane - 4) * 16, gval + at + (lane - 4) * 4);
+            }
+            cp_async_commit();
+        };
+        __syncthreads();                                  // the previous item's readers are done with the window and the rings
+#pragma unroll
+        for (int i = 0; i < WINDOW_RING - 1; ++i) fetch(i);
+        for (int p = threadIdx.x; p < wlen * PPR; p += blockDim.x) {
+            const int r = p / PPR, q = p - r * PPR;
+            cp_async16(window + r * TC + q * 4, xin + (size_t)(c0 + r) * ld + t0 + q * 4);
+        }
+        cp_async_commit();
+        cp_async_wait<0>();
+        __syncthreads();
+        const float* xw = window + b;
+        float acc = 0.0f;
+        for (int i = 0; i < pieces; ++i) {
+            __syncwarp();                                 // every lane has finished reading the slot that is refilled now
+            fetch(i + WINDOW_RING - 1);
+            cp_async_wait<WINDOW_RING - 1>();             // this lane's share of piece i has landed ...
+            __syncwarp();                                 // ... and so has every other lane's
+            const int row = r0 + (i / ppr) * nwarps, t = (i % ppr) << 5;
+            const int n = min(32, k - t);
+            const unsigned char* slot = ring + (i % WINDOW_RING) * WINDOW_PIECE_BYTES;
+            if (t == 0) acc = m.bias[row];
+            for (int j = 0; j < n; j += 8) {
+                const uint4 c = *reinterpret_cast<const uint4*>(slot + j * 2);
+                const float4 w0 = *reinterpret_cast<const float4*>(slot + 64 + j * 4);
+                const float4 w1 = *reinterpret_cast<const float4*>(slot + 64 + j * 4 + 16);
+                const float x0 = xw[(c.x & 0xffffu) * TC], x1 = xw[(c.x >> 16) * TC], x2 = xw[(c.y & 0xffffu) * TC], x3 = xw[(c.y >> 16) * TC];
+                const float x4 = xw[(c.z & 0xffffu) * TC], x5 = xw[(c.z >> 16) * TC], x6 = xw[(c.w & 0xffffu) * TC], x7 = xw[(c.w >> 16) * TC];
+                acc = fmaf(w0.x, x0, acc); acc = fmaf(w0.y, x1, acc); acc = fmaf(w0.z, x2, acc); acc = fmaf(w0.w, x3, acc);
+                acc = fmaf(w1.x, x4, acc); acc = fmaf(w1.y, x5, acc); acc = fmaf(w1.z, x6, acc); acc = fmaf(w1.w, x7, acc);
+            }
+            if (t + 32 >= k && lane < TC) xout[(size_t)m.out[row] * ld + t0 + lane] = activate(acc, act, clamp);
+        }
+        if (k == 0 && lane < TC)                          // a group of rows without entries: x = f(b)
+            for (int row = r0; row < r1; row += nwarps) xout[(size_t)m.out[row] * ld + t0 + lane] = activate(m.bias[row], act, clamp);
+        cp_async_wait<0>();
     }
     if (pdl == 1) grid_launch_dependents();
 }
@@ -846,7 +965,7 @@ forward_ep_kernel(Sliced m, const float* __restrict__ bias, const float* __restr
     if (e.h == 0 && e.item < n) {
         acc.a.x += b; acc.a.y += b; acc.a.z += b; acc.a.w += b;
         lane_activate(acc, act, clamp);
-        lane_store(xout + (size_t)e.item * 4, acc);
+        lane_store(xout + (size_t)(m.out ? m.out[e.item] : e.item) * 4, acc);
     }
     if (pdl == 1) grid_launch_dependents();
 }
@@ -1129,6 +1248,35 @@ gather_probe_kernel(const float* __restrict__ table, float* __restrict__ sink, u
         for (int u = 0; u < 8; ++u) acc += lane_sum(v[u]);
     }
     if (acc == 123.456f) sink[0] = acc;      // the table is all zero: never taken, keeps the loads alive
+}
+
+// ---------------------------------------------------------------------------------------------
+// Probe of the alternative to the second copy of the values: one value array in row-major order that the column
+// units would read, or read and write, one 4-byte word at a time at scattered places (through a position map).  Eight
+// accesses in flight per lane, indices made in registers.  STORE: 0 = scattered 4-byte loads, 1 = scattered 4-byte stores
+// (every lane stores the value 0, so that the table stays all zero whatever the order).
+template <int STORE>
+__global__ void __launch_bounds__(256)
+word_probe_kernel(float* __restrict__ table, float* __restrict__ sink, unsigned word_mask, int per_lane, unsigned seed) {
+    const int tid = blockIdx.x * blockDim.x + threadIdx.x;
+    unsigned st = (unsigned)tid * 2654435761u + seed;
+    float acc = 0.f;
+    for (int q = 0; q < per_lane; q += 8) {
+        unsigned c[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) { st = st * 1664525u + 1013904223u; c[u] = (st >> 8) & word_mask; }
+        if (STORE) {
+#pragma unroll
+            for (int u = 0; u < 8; ++u) table[c[u]] = 0.0f;
+        } else {
+            float v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) v[u] = __ldg(table + c[u]);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) acc += v[u];
+        }
+    }
+    if (acc == 123.456f) sink[0] = acc;
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -4,6 +4,7 @@
 // arithmetic step runs in the kernels of kernels.cuh.
 #include "../../include/sdnn.h"
 #include "kernels.cuh"
+#include "reorder.h"
 
 #include <algorithm>
 #include <cmath>
@@ -60,6 +61,23 @@ struct LayerMem {
     int* c_idx = nullptr; float* c_val = nullptr;
     std::vector<int> r_slice_off;          // host copy of the row-major slice offsets
     RowShape shape;
+    // set-up reordering (SDNN_FLAG_REORDER): how the stored rows and entries map back to the caller's CSR arrays
+    std::vector<int> row_src;              // [N] stored row -> caller's row (empty: identity)
+    std::vector<int> entry_src;            // [nnz] entry in stored order (stored rows, their entries in stored order) -> caller's position
+    int* r_out = nullptr;                  // grouped layer in the default layout: tile row each stored row writes (device, [N])
+    // windowed layer: rows grouped by shared columns, the group's window staged in shared memory (forward_window_kernel)
+    bool windowed = false;
+    int groups = 0, max_wlen = 0;
+    std::vector<int> w_row_at;             // [N] host: offset of each stored row's entries in w_col / w_val
+    int64_t w_elems = 0;                   // padded entries
+    unsigned short* w_col = nullptr; float* w_val = nullptr; int* w_out = nullptr;
+    int* w_g_row0 = nullptr; int* w_g_c0 = nullptr; int* w_g_wlen = nullptr; int* w_g_ebase = nullptr; int* w_g_k = nullptr;
+};
+
+// caller's arrays of one layer, kept on the host until sdnn_finalize when the neurons are to be reordered
+struct HostLayer {
+    std::vector<int> rp, col;
+    std::vector<float> val, bias;
 };
 
 }  // namespace
@@ -123,6 +141,11 @@ struct sdnn {
     long long* d_running = nullptr;
     int l2_bytes = 0;
     std::vector<char> local_pattern;    // per layer: blocks of 1024 rows touch few distinct columns (see infer_tile_width)
+    bool reorder = false;               // SDNN_FLAG_REORDER: layers are analysed and laid out at sdnn_finalize
+    int grouped_layers = 0;             // layers for which the analysis found groups of rows sharing a window of columns
+    std::vector<HostLayer> pending;     // their arrays until then
+    int* d_in_label = nullptr;          // [N] tile row of input neuron i (NULL: identity)
+    int windowed_layers = 0;
     bool compaction = false;            // SDNN_FLAG_SKIP_DEAD asked for; effective while no bias is positive
     std::vector<char> bias_nonpositive; // per layer
     bool live_valid = false;
@@ -220,6 +243,12 @@ int validate_cfg(const sdnn_config* cfg) {
     if (cfg->train && cfg->max_batch > 128) return fail(nullptr, SDNN_ERR_INVALID_ARG, "training handles support max_batch <= 128");
     if ((cfg->flags & SDNN_FLAG_BWD_ATOMICS) && (cfg->flags & SDNN_FLAG_BWD_CSC))
         return fail(nullptr, SDNN_ERR_INVALID_ARG, "choose one backward strategy");
+    if ((cfg->flags & SDNN_FLAG_REORDER) && cfg->train)
+        return fail(nullptr, SDNN_ERR_UNIMPLEMENTED, "SDNN_FLAG_REORDER is implemented for inference handles (train = 0)");
+    if ((cfg->flags & SDNN_FLAG_SMEM_WINDOWS) && !(cfg->flags & SDNN_FLAG_REORDER))
+        return fail(nullptr, SDNN_ERR_INVALID_ARG, "SDNN_FLAG_SMEM_WINDOWS needs SDNN_FLAG_REORDER");
+    if ((cfg->flags & SDNN_FLAG_REORDER) && (cfg->flags & SDNN_FLAG_SKIP_DEAD))
+        return fail(nullptr, SDNN_ERR_INVALID_ARG, "SDNN_FLAG_REORDER and SDNN_FLAG_SKIP_DEAD cannot be combined");
     return SDNN_OK;
 }
 
@@ -333,6 +362,7 @@ Sliced rows_of(sdnn* h, int layer) {
     m.idx = h->lay[layer].r_idx;
     m.val = h->lay[layer].r_val;
     m.order = nullptr;
+    m.out = h->lay[layer].r_out;
     return m;
 }
 
@@ -343,6 +373,7 @@ Sliced cols_of(sdnn* h, int layer) {
     m.idx = h->lay[layer].c_idx;
     m.val = h->lay[layer].c_val;
     m.order = h->d_c_order + (size_t)layer * h->N;
+    m.out = nullptr;
     return m;
 }
 
@@ -396,6 +427,52 @@ void launch_forward(sdnn* h, int layer, const float* xin, float* xout, int ld, i
             else launch_forward_gv<32, 8>(h, layer, xin, xout, ld, q.chunks, track);
             break;
     }
+    count_launch(h);
+}
+
+// Windowed layers (rows grouped by shared columns at set-up): the group's window of the input tile is staged in shared
+// memory.  One CTA per SM (the window takes most of its shared memory), items = groups x chunks of up to 32 inputs.
+constexpr int WINDOW_COL_CAP = 1536;      // tile rows a window may span: 1536 x 32 inputs x 4 bytes = 192 KB of shared memory
+constexpr int WINDOW_ROW_CAP = 2048;      // rows per group
+
+template <int TC>
+cudaError_t launch_forward_window_tc(sdnn* h, const LayerMem& lm, const Windowed& m, const float* xin, float* xout, int ld, int cols) {
+    static bool configured[64] = {};
+    if (h->device < 64 && !configured[h->device]) {
+        cudaError_t e = cudaFuncSetAttribute(forward_window_kernel<TC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             WINDOW_RING_BYTES + WINDOW_COL_CAP * TC * 4);
+        if (e != cudaSuccess) return e;
+        configured[h->device] = true;
+    }
+    const int chunks = cols / TC;
+    // too few (group, chunk) pairs for the device: split the rows of a group over several items (each stages the window);
+    // an item keeps at least 64 rows per warp-row of work so that the staging stays a small part of it
+    int splits = 1;
+    const int avg_rows = std::max(1, h->N / std::max(1, lm.groups));
+    while (lm.groups * chunks * splits < 2 * h->sms && avg_rows / (splits * 2) >= 64 && splits < 32) splits *= 2;
+    const int items = lm.groups * chunks * splits;
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(std::max(1, std::min(items, h->sms))); lc.blockDim = dim3(WINDOW_THREADS);
+    lc.dynamicSmemBytes = WINDOW_RING_BYTES + (size_t)std::max(lm.max_wlen, 1) * TC * sizeof(float);
+    lc.stream = h->launch_stream ? h->launch_stream : h->stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = at; lc.numAttrs = h->pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&lc, forward_window_kernel<TC>, m, xin, xout, ld, chunks, splits, h->cfg.clamp, (int)h->cfg.activation,
+                              h->pdl ? PDL_AT_END : 0);
+}
+
+void launch_forward_window(sdnn* h, int layer, const float* xin, float* xout, int ld, int cols) {
+    const LayerMem& lm = h->lay[layer];
+    Windowed m;
+    m.col = lm.w_col; m.val = lm.w_val; m.out = lm.w_out;
+    m.bias = h->d_bias + (size_t)layer * h->N;
+    m.g_row0 = lm.w_g_row0; m.g_c0 = lm.w_g_c0; m.g_wlen = lm.w_g_wlen; m.g_ebase = lm.w_g_ebase; m.g_k = lm.w_g_k; m.groups = lm.groups;
+    if (cols >= 32) launch_forward_window_tc<32>(h, lm, m, xin, xout, ld, cols);
+    else if (cols == 16) launch_forward_window_tc<16>(h, lm, m, xin, xout, ld, cols);
+    else if (cols == 8) launch_forward_window_tc<8>(h, lm, m, xin, xout, ld, cols);
+    else launch_forward_window_tc<4>(h, lm, m, xin, xout, ld, cols);
     count_launch(h);
 }
 
@@ -527,9 +604,9 @@ void launch_output_gradient(sdnn* h, int ld) {
     count_launch(h);
 }
 
-void launch_transpose_in(sdnn* h, const float* src, float* dst, int cnt, int cols, int ld) {
+void launch_transpose_in(sdnn* h, const float* src, float* dst, int cnt, int cols, int ld, const int* row_map = nullptr) {
     dim3 grid((h->N + 31) / 32, (cols + 31) / 32), block(32, 8);
-    transpose_in_kernel<<<grid, block, 0, h->launch_stream ? h->launch_stream : h->stream>>>(src, dst, h->N, cnt, cols, ld);
+    transpose_in_kernel<<<grid, block, 0, h->launch_stream ? h->launch_stream : h->stream>>>(src, dst, h->N, cnt, cols, ld, row_map);
     count_launch(h);
 }
 
@@ -688,7 +765,7 @@ int infer_tile(sdnn* h, InferLane& ln, const float* x0, int cnt, float* y_out, i
     cudaStream_t st = ln.stream;
     h->cur = &ln;
     h->launch_stream = st;
-    launch_transpose_in(h, x0, ln.tile[0], cnt, cols, ld);
+    launch_transpose_in(h, x0, ln.tile[0], cnt, cols, ld, h->d_in_label);
     int cur = 0;
     bool track = h->compaction && h->cfg.activation == SDNN_ACT_CLAMPED_RELU;      // sigmoid(b) is never 0: nothing ever dies
     for (int l = 0; l < h->L && track; ++l) track = h->bias_nonpositive[l] != 0;     // the zero vector must be a fixed point
@@ -712,7 +789,8 @@ int infer_tile(sdnn* h, InferLane& ln, const float* x0, int cnt, float* y_out, i
         h->live_lane = (int)(&ln - h->lane);
     } else {
         for (int k = 0; k < h->L; ++k) {
-            launch_forward(h, k, ln.tile[cur], ln.tile[cur ^ 1], ld, cols);
+            if (h->lay[k].windowed) launch_forward_window(h, k, ln.tile[cur], ln.tile[cur ^ 1], ld, cols);
+            else launch_forward(h, k, ln.tile[cur], ln.tile[cur ^ 1], ld, cols);
             cur ^= 1;
         }
     }
@@ -843,146 +921,9 @@ int refresh_mirror(sdnn* h, int layer, unsigned long long* mismatch_dev) {
     return SDNN_OK;
 }
 
-}  // namespace
-
-extern "C" {
-
-const char* sdnn_version(void) { return "sdnn 0.2 (sm_100a)"; }
-
-const char* sdnn_last_error(const sdnn_t* h) { return h ? h->err.c_str() : g_create_error.c_str(); }
-
-int64_t sdnn_kernel_launches(const sdnn_t* h) { return h ? h->launches : 0; }
-int32_t sdnn_infer_tile_width(const sdnn_t* h) { return (h && h->finalized) ? infer_tile_width(h) : 0; }
-int32_t sdnn_infer_tiles_in_flight(const sdnn_t* h) { return (h && h->finalized) ? infer_lanes(h, infer_tile_width(h)) : 0; }
-int64_t sdnn_device_bytes(const sdnn_t* h) { return h ? h->dev_bytes : 0; }
-
-void sdnn_destroy(sdnn_t* h) {
-    if (!h) return;
-    cudaSetDevice(h->device);
-    if (h->stream || h->own_stream) cudaStreamSynchronize(h->stream);
-    if (h->graph) cudaGraphExecDestroy(h->graph);
-    if (h->graph_avg) cudaGraphExecDestroy(h->graph_avg);
-    for (cudaEvent_t e : h->ev) if (e) cudaEventDestroy(e);
-    for (InferLane& ln : h->lane) {
-        if (ln.ev_scan) cudaEventDestroy(ln.ev_scan);
-        if (ln.ev_done) cudaEventDestroy(ln.ev_done);
-        if (ln.stream && ln.stream != h->stream) { cudaStreamSynchronize(ln.stream); cudaStreamDestroy(ln.stream); }
-    }
-    if (h->ev_lane_start) cudaEventDestroy(h->ev_lane_start);
-    for (cudaEvent_t e : h->ev_delta) if (e) cudaEventDestroy(e);
-    if (h->ev_fork) cudaEventDestroy(h->ev_fork);
-    for (cudaEvent_t e : h->ev_side_join) if (e) cudaEventDestroy(e);
-    for (cudaStream_t st : h->side_streams) if (st) { cudaStreamSynchronize(st); cudaStreamDestroy(st); }
-    for (cudaEvent_t e : h->ev_copied) if (e) cudaEventDestroy(e);
-    for (cudaEvent_t e : h->ev_consumed) if (e) cudaEventDestroy(e);
-    if (h->copy_stream) { cudaStreamSynchronize(h->copy_stream); cudaStreamDestroy(h->copy_stream); }
-    for (void* p : h->allocs) cudaFree(p);
-    if (h->own_stream) cudaStreamDestroy(h->stream);
-    delete h;
-}
-
-int sdnn_create_deferred(sdnn_t** out, int32_t n_layers, int32_t n_neurons, const int64_t* nnz_per_layer,
-                         const sdnn_config* cfg) {
-    if (!out) return fail(nullptr, SDNN_ERR_INVALID_ARG, "out is NULL");
-    *out = nullptr;
-    int rc = validate_cfg(cfg);
-    if (rc) return rc;
-    if (n_layers < 1 || n_neurons < 1) return fail(nullptr, SDNN_ERR_INVALID_ARG, "n_layers and n_neurons must be >= 1");
-    if (!nnz_per_layer) return fail(nullptr, SDNN_ERR_INVALID_ARG, "nnz_per_layer is NULL");
-    for (int l = 0; l < n_layers; ++l)
-        if (nnz_per_layer[l] < 0 || nnz_per_layer[l] > INT32_MAX)
-            return fail(nullptr, SDNN_ERR_INVALID_ARG, "layer %d: stored-entry count outside [0, 2^31)", l);
-    // the kernels address a tile row with a 32-bit multiply-add: one tile must stay below 4 GiB
-    if ((int64_t)n_neurons * padded_width(cfg->max_batch) * (int64_t)sizeof(float) >= (1LL << 32))
-        return fail(nullptr, SDNN_ERR_INVALID_ARG, "n_neurons * padded(max_batch) * 4 bytes must stay below 4 GiB: lower max_batch (inference works in tiles of max_batch inputs)");
-
-    int ndev = 0;
-    cudaError_t e = cudaGetDeviceCount(&ndev);
-    if (e != cudaSuccess || ndev == 0) { cudaGetLastError(); return fail(nullptr, SDNN_ERR_CUDA, "no CUDA device: %s", cudaGetErrorString(e)); }
-
-    sdnn* h = new (std::nothrow) sdnn;
-    if (!h) return fail(nullptr, SDNN_ERR_OOM, "host allocation failed");
-    h->L = n_layers; h->N = n_neurons; h->NS = (n_neurons + SLICE - 1) / SLICE; h->cfg = *cfg;
-    h->stream = static_cast<cudaStream_t>(cfg->cuda_stream);
-    auto bail = [&](int code) { g_create_error = h->err; sdnn_destroy(h); return code; };
-    if (cfg->device >= 0) {
-        if (cfg->device >= ndev) { h->err = "device ordinal out of range"; return bail(SDNN_ERR_INVALID_ARG); }
-        if ((e = cudaSetDevice(cfg->device)) != cudaSuccess) return bail(cuda_fail(h, e, "cudaSetDevice"));
-        h->device = cfg->device;
-    } else if ((e = cudaGetDevice(&h->device)) != cudaSuccess) {
-        return bail(cuda_fail(h, e, "cudaGetDevice"));
-    }
-    if ((e = cudaDeviceGetAttribute(&h->sms, cudaDevAttrMultiProcessorCount, h->device)) != cudaSuccess || h->sms < 1)
-        return bail(cuda_fail(h, e, "cudaDeviceGetAttribute(multiprocessor count)"));
-    if (cudaDeviceGetAttribute(&h->l2_bytes, cudaDevAttrL2CacheSize, h->device) != cudaSuccess) { cudaGetLastError(); h->l2_bytes = 0; }
-    if (!h->stream) {   // the legacy default stream cannot be captured into a graph: use a blocking stream of our own,
-                        // which still orders itself against work on the legacy default stream
-        if ((e = cudaStreamCreate(&h->stream)) != cudaSuccess) { h->stream = nullptr; return bail(cuda_fail(h, e, "cudaStreamCreate")); }
-        h->own_stream = true;
-    }
-    h->mirror = cfg->train && !(cfg->flags & SDNN_FLAG_BWD_ATOMICS);
-    h->pdl = !(cfg->flags & SDNN_FLAG_NO_PDL);
-    h->nnz.assign(nnz_per_layer, nnz_per_layer + n_layers);
-    h->loaded.assign(n_layers, 0);
-    h->lay.resize(n_layers);
-    h->ld_max = padded_width(cfg->max_batch);
-    const size_t N = (size_t)n_neurons, L = (size_t)n_layers, tile = N * (size_t)h->ld_max;
-
-    if ((rc = dev_alloc(h, &h->d_r_slice_off, L * (h->NS + 1), false))) return bail(rc);
-    if ((rc = dev_alloc(h, &h->d_r_len, L * N, false))) return bail(rc);
-    if ((rc = dev_alloc(h, &h->d_bias, L * N, false))) return bail(rc);
-    if (h->mirror) {
-        if ((rc = dev_alloc(h, &h->d_c_slice_off, L * (h->NS + 1), false))) return bail(rc);
-        if ((rc = dev_alloc(h, &h->d_c_len, L * N, false))) return bail(rc);
-        if ((rc = dev_alloc(h, &h->d_c_order, L * N, false))) return bail(rc);
-        if ((rc = dev_alloc(h, &h->d_mismatch, 1, true))) return bail(rc);
-    }
-    if (cfg->train) {
-        for (cudaEvent_t& ev : h->ev)
-            if ((e = cudaEventCreate(&ev)) != cudaSuccess) { ev = nullptr; return bail(cuda_fail(h, e, "cudaEventCreate")); }
-        if ((rc = dev_alloc(h, &h->d_acts, (L + 1) * tile, false))) return bail(rc);
-        h->split = h->mirror && !(cfg->flags & SDNN_FLAG_BWD_ONE_LAUNCH);
-        if (h->split) {
-            if (!(cfg->flags & SDNN_FLAG_KEEP_DEBUG) && (rc = dev_alloc(h, &h->d_delta_all, L * tile, true))) return bail(rc);
-            h->n_side = 2;      // row-unit launches of neighbouring layers do not depend on each other: two streams let them overlap
-            for (int q = 0; q < h->n_side; ++q) {
-                if ((e = cudaStreamCreateWithFlags(&h->side_streams[q], cudaStreamNonBlocking)) != cudaSuccess) return bail(cuda_fail(h, e, "cudaStreamCreate"));
-                if ((e = cudaEventCreateWithFlags(&h->ev_side_join[q], cudaEventDisableTiming)) != cudaSuccess) return bail(cuda_fail(h, e, "cudaEventCreate"));
-            }
-            h->ev_delta.assign(n_layers, nullptr);
-            for (cudaEvent_t& ev : h->ev_delta)
-                if ((e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming)) != cudaSuccess) { ev = nullptr; return bail(cuda_fail(h, e, "cudaEventCreate")); }
-            if ((e = cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming)) != cudaSuccess) return bail(cuda_fail(h, e, "cudaEventCreate"));
-        }
-        if ((rc = dev_alloc(h, &h->d_s[0], tile, true))) return bail(rc);
-        if ((rc = dev_alloc(h, &h->d_s[1], tile, true))) return bail(rc);
-        if (!h->mirror && (rc = dev_alloc(h, &h->d_dl, tile, true))) return bail(rc);
-        if ((rc = dev_alloc(h, &h->d_yt, tile, true))) return bail(rc);
-        if ((rc = dev_alloc(h, &h->d_sp, 1, true))) return bail(rc);
-        if ((rc = dev_alloc(h, &h->d_loss, 1, true))) return bail(rc);
-        if (cfg->flags & SDNN_FLAG_KEEP_DEBUG)
-            if ((rc = dev_alloc(h, &h->d_dbg_delta, L * tile, true))) return bail(rc);
-    }
-    {   // inference buffers (a training handle can also infer)
-        h->compaction = (cfg->flags & SDNN_FLAG_SKIP_DEAD) != 0;
-        h->bias_nonpositive.assign(n_layers, 0);
-        h->local_pattern.assign(n_layers, 0);
-        if ((rc = dev_alloc(h, &h->d_running, 1, true))) return bail(rc);
-        if ((rc = alloc_lane(h, h->lane[0], false))) return bail(rc);
-        h->cur = &h->lane[0];
-    }
-    *out = h;
-    return SDNN_OK;
-}
-
-int sdnn_load_layer(sdnn_t* h, int32_t layer, const int32_t* row_ptr, const int32_t* col_idx, const float* values,
-                    const float* bias) {
-    if (!h) return SDNN_ERR_INVALID_ARG;
-    if (h->finalized) return fail(h, SDNN_ERR_STATE, "handle already finalized");
-    if (layer < 0 || layer >= h->L) return fail(h, SDNN_ERR_INVALID_ARG, "layer %d outside [0, %d)", layer, h->L);
-    if (h->loaded[layer]) return fail(h, SDNN_ERR_STATE, "layer %d loaded twice", layer);
-    int rc = validate_layer(h, layer, h->N, h->nnz[layer], row_ptr, col_idx, values, bias);
-    if (rc) return rc;
+// Lays out one validated layer (caller's or reordered CSR, host arrays) in the kernels' sliced format and uploads it.
+int upload_layer(sdnn* h, int layer, const int32_t* row_ptr, const int32_t* col_idx, const float* values, const float* bias) {
+    int rc;
     CU(h, cudaSetDevice(h->device));
     const int N = h->N, NS = h->NS;
     LayerMem& lm = h->lay[layer];
@@ -1081,6 +1022,394 @@ int sdnn_load_layer(sdnn_t* h, int32_t layer, const int32_t* row_ptr, const int3
         }
         h->local_pattern[layer] = distinct <= 2 * (int64_t)N ? 1 : 0;
     }
+    return SDNN_OK;
+}
+
+// Entries per (padded) row of every group of a structured layer and the padded total; -1 if padding every row of a
+// group to its longest row would more than quadruple the layer (plus a margin of 64 entries per row).
+int64_t windowed_padding(int n, const int32_t* rp, const sdnn_reorder::Grouping& g, std::vector<int>* ks) {
+    const int groups = (int)g.group_c0.size();
+    int64_t total = 0;
+    if (ks) ks->assign(groups, 0);
+    for (int q = 0; q < groups; ++q) {
+        int k = 0;
+        for (int s = g.group_row0[q]; s < g.group_row0[q + 1]; ++s) k = std::max(k, rp[g.row_order[s] + 1] - rp[g.row_order[s]]);
+        k = (k + 7) / 8 * 8;
+        if (ks) (*ks)[q] = k;
+        total += (int64_t)k * (g.group_row0[q + 1] - g.group_row0[q]);
+    }
+    if (total > 4 * (int64_t)rp[n] + 64 * (int64_t)n || total > INT32_MAX) return -1;
+    return total;
+}
+
+// One structured layer in the windowed layout: rows group by group, every row padded to its group's longest, columns
+// relative to the group's window.
+//   in_label : new numbers of the layer's input neurons (from this layer's own grouping)
+//   out_label: new numbers of its output neurons (from the next layer's grouping), or NULL for the caller's numbering
+int build_windowed_layer(sdnn* h, int layer, const HostLayer& hl, const sdnn_reorder::Grouping& g, const std::vector<int>* out_label) {
+    const int N = h->N;
+    LayerMem& lm = h->lay[layer];
+    const int groups = (int)g.group_c0.size();
+    std::vector<int> ks, ebase(groups, 0);
+    const int64_t padded = windowed_padding(N, hl.rp.data(), g, &ks);
+    if (padded < 0) return fail(h, SDNN_ERR_STATE, "layer %d: windowed layout too large", layer);      // excluded by build_reordered
+    for (int q = 1; q < groups; ++q) ebase[q] = ebase[q - 1] + ks[q - 1] * (g.group_row0[q] - g.group_row0[q - 1]);
+    std::vector<int> stored_rp(N + 1, 0), out(N);
+    std::vector<float> bias_s(N);
+    lm.w_row_at.assign(N, 0);
+    for (int q = 0; q < groups; ++q)
+        for (int s = g.group_row0[q]; s < g.group_row0[q + 1]; ++s) lm.w_row_at[s] = ebase[q] + (s - g.group_row0[q]) * ks[q];
+    for (int s = 0; s < N; ++s) {
+        const int i = g.row_order[s];
+        stored_rp[s + 1] = stored_rp[s] + (hl.rp[i + 1] - hl.rp[i]);
+        out[s] = out_label ? (*out_label)[i] : i;
+        bias_s[s] = hl.bias[i];
+    }
+    std::vector<unsigned short> wcol((size_t)padded, 0);
+    std::vector<float> wval((size_t)padded, 0.0f);
+    lm.entry_src.assign((size_t)stored_rp[N], 0);
+    int max_wlen = 0;
+    for (int q = 0; q < groups; ++q) max_wlen = std::max(max_wlen, g.group_wlen[q]);
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int q = 0; q < groups; ++q) {
+        std::vector<std::pair<int, int>> ent;      // (column within the window, caller's entry position)
+        for (int s = g.group_row0[q]; s < g.group_row0[q + 1]; ++s) {
+            const int i = g.row_order[s];
+            ent.clear();
+            for (int p = hl.rp[i]; p < hl.rp[i + 1]; ++p) ent.emplace_back(g.col_label[hl.col[p]] - g.group_c0[q], p);
+            std::sort(ent.begin(), ent.end());
+            for (size_t t = 0; t < ent.size(); ++t) {
+                wcol[(size_t)lm.w_row_at[s] + t] = (unsigned short)ent[t].first;
+                wval[(size_t)lm.w_row_at[s] + t] = hl.val[ent[t].second];
+                lm.entry_src[(size_t)stored_rp[s] + t] = ent[t].second;
+            }
+        }
+    }
+    lm.windowed = true;
+    lm.groups = groups;
+    lm.max_wlen = max_wlen;
+    lm.w_elems = padded;
+    lm.shape.uniform_k = -1;
+    lm.shape.row_ptr = stored_rp;
+    lm.row_src = g.row_order;
+    int rc;
+    CU(h, cudaSetDevice(h->device));
+    if ((rc = dev_alloc(h, &lm.w_col, (size_t)padded, false))) return rc;
+    if ((rc = dev_alloc(h, &lm.w_val, (size_t)padded, false))) return rc;
+    if ((rc = dev_alloc(h, &lm.w_out, (size_t)N, false))) return rc;
+    if ((rc = dev_alloc(h, &lm.w_g_row0, (size_t)groups + 1, false))) return rc;
+    if ((rc = dev_alloc(h, &lm.w_g_c0, (size_t)groups, false))) return rc;
+    if ((rc = dev_alloc(h, &lm.w_g_wlen, (size_t)groups, false))) return rc;
+    if ((rc = dev_alloc(h, &lm.w_g_ebase, (size_t)groups, false))) return rc;
+    if ((rc = dev_alloc(h, &lm.w_g_k, (size_t)groups, false))) return rc;
+    if (padded) {
+        CU(h, cudaMemcpyAsync(lm.w_col, wcol.data(), (size_t)padded * sizeof(unsigned short), cudaMemcpyHostToDevice, h->stream));
+        CU(h, cudaMemcpyAsync(lm.w_val, wval.data(), (size_t)padded * sizeof(float), cudaMemcpyHostToDevice, h->stream));
+    }
+    CU(h, cudaMemcpyAsync(lm.w_out, out.data(), (size_t)N * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+    CU(h, cudaMemcpyAsync(lm.w_g_row0, g.group_row0.data(), ((size_t)groups + 1) * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+    CU(h, cudaMemcpyAsync(lm.w_g_c0, g.group_c0.data(), (size_t)groups * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+    CU(h, cudaMemcpyAsync(lm.w_g_wlen, g.group_wlen.data(), (size_t)groups * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+    CU(h, cudaMemcpyAsync(lm.w_g_ebase, ebase.data(), (size_t)groups * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+    CU(h, cudaMemcpyAsync(lm.w_g_k, ks.data(), (size_t)groups * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+    CU(h, cudaMemcpyAsync(h->d_bias + (size_t)layer * N, bias_s.data(), (size_t)N * sizeof(float), cudaMemcpyHostToDevice, h->stream));
+    CU(h, cudaStreamSynchronize(h->stream));
+    bool nonpos = true;
+    for (int i = 0; i < N && nonpos; ++i) nonpos = !(hl.bias[i] > 0.0f);
+    h->bias_nonpositive[layer] = nonpos ? 1 : 0;
+    h->local_pattern[layer] = 1;
+    ++h->windowed_layers;
+    return SDNN_OK;
+}
+
+// One structured layer in the default (sliced) layout: rows stored group by group, columns renumbered so that a group
+// reads one contiguous window of tile rows (which the caches then hold while the group is worked on), every stored row
+// writing the tile row that the next layer's grouping assigned to its neuron.
+int build_grouped_layer(sdnn* h, int layer, const HostLayer& hl, const sdnn_reorder::Grouping& g, const std::vector<int>* out_label) {
+    const int N = h->N;
+    LayerMem& lm = h->lay[layer];
+    std::vector<int> rp(N + 1, 0), col((size_t)hl.rp[N]), out(N);
+    std::vector<float> val((size_t)hl.rp[N]), bias(N);
+    lm.entry_src.assign((size_t)hl.rp[N], 0);
+    for (int s = 0; s < N; ++s) {
+        const int i = g.row_order[s];
+        rp[s + 1] = rp[s] + (hl.rp[i + 1] - hl.rp[i]);
+        out[s] = out_label ? (*out_label)[i] : i;
+        bias[s] = hl.bias[i];
+    }
+#pragma omp parallel
+    {
+        std::vector<std::pair<int, int>> ent;      // (new column number, caller's entry position)
+#pragma omp for schedule(static)
+        for (int s = 0; s < N; ++s) {
+            const int i = g.row_order[s];
+            ent.clear();
+            for (int p = hl.rp[i]; p < hl.rp[i + 1]; ++p) ent.emplace_back(g.col_label[hl.col[p]], p);
+            std::sort(ent.begin(), ent.end());
+            for (size_t t = 0; t < ent.size(); ++t) {
+                col[(size_t)rp[s] + t] = ent[t].first;
+                val[(size_t)rp[s] + t] = hl.val[ent[t].second];
+                lm.entry_src[(size_t)rp[s] + t] = ent[t].second;
+            }
+        }
+    }
+    lm.row_src = g.row_order;
+    int rc = upload_layer(h, layer, rp.data(), col.data(), val.data(), bias.data());
+    if (rc) return rc;
+    if ((rc = dev_alloc(h, &lm.r_out, (size_t)N, false))) return rc;
+    CU(h, cudaMemcpyAsync(lm.r_out, out.data(), (size_t)N * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+    CU(h, cudaStreamSynchronize(h->stream));
+    return SDNN_OK;
+}
+
+// A layer without structure keeps the default layout; only its rows move to where the next layer's grouping put its
+// output neurons (stored row = new number of the neuron, as the default kernels expect).
+int build_plain_layer(sdnn* h, int layer, const HostLayer& hl, const std::vector<int>* out_label) {
+    if (!out_label) return upload_layer(h, layer, hl.rp.data(), hl.col.data(), hl.val.data(), hl.bias.data());
+    const int N = h->N;
+    LayerMem& lm = h->lay[layer];
+    std::vector<int> src(N);
+    for (int i = 0; i < N; ++i) src[(*out_label)[i]] = i;
+    std::vector<int> rp(N + 1, 0), col((size_t)hl.rp[N]);
+    std::vector<float> val((size_t)hl.rp[N]), bias(N);
+    lm.entry_src.assign((size_t)hl.rp[N], 0);
+    for (int s = 0; s < N; ++s) rp[s + 1] = rp[s] + (hl.rp[src[s] + 1] - hl.rp[src[s]]);
+#pragma omp parallel for schedule(static)
+    for (int s = 0; s < N; ++s) {
+        const int i = src[s];
+        bias[s] = hl.bias[i];
+        for (int t = 0; t < hl.rp[i + 1] - hl.rp[i]; ++t) {
+            col[(size_t)rp[s] + t] = hl.col[(size_t)hl.rp[i] + t];
+            val[(size_t)rp[s] + t] = hl.val[(size_t)hl.rp[i] + t];
+            lm.entry_src[(size_t)rp[s] + t] = hl.rp[i] + t;
+        }
+    }
+    lm.row_src = src;
+    return upload_layer(h, layer, rp.data(), col.data(), val.data(), bias.data());
+}
+
+// SDNN_FLAG_REORDER: analyse every layer, renumber, lay out, upload (called by sdnn_finalize).
+int build_reordered(sdnn* h) {
+    const int L = h->L, N = h->N;
+    std::vector<sdnn_reorder::Grouping> G(L);
+    const bool smem_windows = (h->cfg.flags & SDNN_FLAG_SMEM_WINDOWS) != 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int l = 0; l < L; ++l)
+        if (sdnn_reorder::cluster_rows(N, h->pending[l].rp.data(), h->pending[l].col.data(), WINDOW_COL_CAP, WINDOW_ROW_CAP, G[l]) &&
+            smem_windows && windowed_padding(N, h->pending[l].rp.data(), G[l], nullptr) < 0)
+            G[l] = sdnn_reorder::Grouping();      // a few long rows would blow the padded layout up: keep the default one
+    // numbers of the neurons at boundary l (inputs of layer l): given by layer l's grouping; the outputs of the last
+    // layer keep the caller's numbers
+    auto labels = [&](int boundary) -> const std::vector<int>* {
+        return (boundary < L && G[boundary].structured) ? &G[boundary].col_label : nullptr;
+    };
+    int rc;
+    if (labels(0)) {
+        if ((rc = dev_alloc(h, &h->d_in_label, (size_t)N, false))) return rc;
+        CU(h, cudaMemcpyAsync(h->d_in_label, labels(0)->data(), (size_t)N * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+        CU(h, cudaStreamSynchronize(h->stream));
+    }
+    for (int l = 0; l < L; ++l) {
+        const bool smem = (h->cfg.flags & SDNN_FLAG_SMEM_WINDOWS) != 0;
+        rc = !G[l].structured ? build_plain_layer(h, l, h->pending[l], labels(l + 1))
+             : smem           ? build_windowed_layer(h, l, h->pending[l], G[l], labels(l + 1))
+                              : build_grouped_layer(h, l, h->pending[l], G[l], labels(l + 1));
+        if (rc) return rc;
+        if (G[l].structured) ++h->grouped_layers;
+        h->pending[l] = HostLayer();
+        G[l] = sdnn_reorder::Grouping();
+    }
+    h->pending.clear();
+    return SDNN_OK;
+}
+
+// values of a layer: the caller's CSR order <-> the order they are stored in (rows and entries may have moved)
+void caller_to_stored(const LayerMem& lm, const float* src, std::vector<float>& dst, int64_t nnz) {
+    dst.resize((size_t)nnz);
+    if (lm.entry_src.empty()) { std::copy(src, src + nnz, dst.begin()); return; }
+#pragma omp parallel for schedule(static)
+    for (int64_t e = 0; e < nnz; ++e) dst[(size_t)e] = src[lm.entry_src[(size_t)e]];
+}
+void stored_to_caller(const LayerMem& lm, const std::vector<float>& src, float* dst, int64_t nnz) {
+    if (lm.entry_src.empty()) { std::copy(src.begin(), src.begin() + nnz, dst); return; }
+#pragma omp parallel for schedule(static)
+    for (int64_t e = 0; e < nnz; ++e) dst[lm.entry_src[(size_t)e]] = src[(size_t)e];
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* sdnn_version(void) { return "sdnn 0.2 (sm_100a)"; }
+
+const char* sdnn_last_error(const sdnn_t* h) { return h ? h->err.c_str() : g_create_error.c_str(); }
+
+int64_t sdnn_kernel_launches(const sdnn_t* h) { return h ? h->launches : 0; }
+int32_t sdnn_infer_tile_width(const sdnn_t* h) { return (h && h->finalized) ? infer_tile_width(h) : 0; }
+int32_t sdnn_infer_tiles_in_flight(const sdnn_t* h) { return (h && h->finalized) ? infer_lanes(h, infer_tile_width(h)) : 0; }
+int64_t sdnn_device_bytes(const sdnn_t* h) { return h ? h->dev_bytes : 0; }
+int32_t sdnn_windowed_layers(const sdnn_t* h) { return (h && h->finalized) ? h->windowed_layers : 0; }
+int32_t sdnn_grouped_layers(const sdnn_t* h) { return (h && h->finalized) ? h->grouped_layers : 0; }
+
+int sdnn_cluster_layer(int32_t n, const int32_t* row_ptr, const int32_t* col_idx, int32_t col_cap, int32_t row_cap,
+                       int32_t* group_of_row, int32_t* col_label, int32_t* n_groups, int32_t* max_window) {
+    if (n < 1 || !row_ptr || !group_of_row || !col_label || !n_groups || !max_window || col_cap < 1 || row_cap < 1 ||
+        (row_ptr[n] > 0 && !col_idx))
+        return fail(nullptr, SDNN_ERR_INVALID_ARG, "sdnn_cluster_layer: NULL argument or size below 1");
+    *n_groups = 0; *max_window = 0;
+    sdnn_reorder::Grouping g;
+    if (!sdnn_reorder::cluster_rows(n, row_ptr, col_idx, col_cap, row_cap, g)) return SDNN_OK;
+    const int groups = (int)g.group_c0.size();
+    for (int q = 0; q < groups; ++q) {
+        for (int s = g.group_row0[q]; s < g.group_row0[q + 1]; ++s) group_of_row[g.row_order[s]] = q;
+        *max_window = std::max(*max_window, g.group_wlen[q]);
+    }
+    std::copy(g.col_label.begin(), g.col_label.end(), col_label);
+    *n_groups = groups;
+    return SDNN_OK;
+}
+
+void sdnn_destroy(sdnn_t* h) {
+    if (!h) return;
+    cudaSetDevice(h->device);
+    if (h->stream || h->own_stream) cudaStreamSynchronize(h->stream);
+    if (h->graph) cudaGraphExecDestroy(h->graph);
+    if (h->graph_avg) cudaGraphExecDestroy(h->graph_avg);
+    for (cudaEvent_t e : h->ev) if (e) cudaEventDestroy(e);
+    for (InferLane& ln : h->lane) {
+        if (ln.ev_scan) cudaEventDestroy(ln.ev_scan);
+        if (ln.ev_done) cudaEventDestroy(ln.ev_done);
+        if (ln.stream && ln.stream != h->stream) { cudaStreamSynchronize(ln.stream); cudaStreamDestroy(ln.stream); }
+    }
+    if (h->ev_lane_start) cudaEventDestroy(h->ev_lane_start);
+    for (cudaEvent_t e : h->ev_delta) if (e) cudaEventDestroy(e);
+    if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+    for (cudaEvent_t e : h->ev_side_join) if (e) cudaEventDestroy(e);
+    for (cudaStream_t st : h->side_streams) if (st) { cudaStreamSynchronize(st); cudaStreamDestroy(st); }
+    for (cudaEvent_t e : h->ev_copied) if (e) cudaEventDestroy(e);
+    for (cudaEvent_t e : h->ev_consumed) if (e) cudaEventDestroy(e);
+    if (h->copy_stream) { cudaStreamSynchronize(h->copy_stream); cudaStreamDestroy(h->copy_stream); }
+    for (void* p : h->allocs) cudaFree(p);
+    if (h->own_stream) cudaStreamDestroy(h->stream);
+    delete h;
+}
+
+int sdnn_create_deferred(sdnn_t** out, int32_t n_layers, int32_t n_neurons, const int64_t* nnz_per_layer,
+                         const sdnn_config* cfg) {
+    if (!out) return fail(nullptr, SDNN_ERR_INVALID_ARG, "out is NULL");
+    *out = nullptr;
+    int rc = validate_cfg(cfg);
+    if (rc) return rc;
+    if (n_layers < 1 || n_neurons < 1) return fail(nullptr, SDNN_ERR_INVALID_ARG, "n_layers and n_neurons must be >= 1");
+    if (!nnz_per_layer) return fail(nullptr, SDNN_ERR_INVALID_ARG, "nnz_per_layer is NULL");
+    for (int l = 0; l < n_layers; ++l)
+        if (nnz_per_layer[l] < 0 || nnz_per_layer[l] > INT32_MAX)
+            return fail(nullptr, SDNN_ERR_INVALID_ARG, "layer %d: stored-entry count outside [0, 2^31)", l);
+    // the kernels address a tile row with a 32-bit multiply-add: one tile must stay below 4 GiB
+    if ((int64_t)n_neurons * padded_width(cfg->max_batch) * (int64_t)sizeof(float) >= (1LL << 32))
+        return fail(nullptr, SDNN_ERR_INVALID_ARG, "n_neurons * padded(max_batch) * 4 bytes must stay below 4 GiB: lower max_batch (inference works in tiles of max_batch inputs)");
+
+    int ndev = 0;
+    cudaError_t e = cudaGetDeviceCount(&ndev);
+    if (e != cudaSuccess || ndev == 0) { cudaGetLastError(); return fail(nullptr, SDNN_ERR_CUDA, "no CUDA device: %s", cudaGetErrorString(e)); }
+
+    sdnn* h = new (std::nothrow) sdnn;
+    if (!h) return fail(nullptr, SDNN_ERR_OOM, "host allocation failed");
+    h->L = n_layers; h->N = n_neurons; h->NS = (n_neurons + SLICE - 1) / SLICE; h->cfg = *cfg;
+    h->stream = static_cast<cudaStream_t>(cfg->cuda_stream);
+    auto bail = [&](int code) { g_create_error = h->err; sdnn_destroy(h); return code; };
+    if (cfg->device >= 0) {
+        if (cfg->device >= ndev) { h->err = "device ordinal out of range"; return bail(SDNN_ERR_INVALID_ARG); }
+        if ((e = cudaSetDevice(cfg->device)) != cudaSuccess) return bail(cuda_fail(h, e, "cudaSetDevice"));
+        h->device = cfg->device;
+    } else if ((e = cudaGetDevice(&h->device)) != cudaSuccess) {
+        return bail(cuda_fail(h, e, "cudaGetDevice"));
+    }
+    if ((e = cudaDeviceGetAttribute(&h->sms, cudaDevAttrMultiProcessorCount, h->device)) != cudaSuccess || h->sms < 1)
+        return bail(cuda_fail(h, e, "cudaDeviceGetAttribute(multiprocessor count)"));
+    if (cudaDeviceGetAttribute(&h->l2_bytes, cudaDevAttrL2CacheSize, h->device) != cudaSuccess) { cudaGetLastError(); h->l2_bytes = 0; }
+    if (!h->stream) {   // the legacy default stream cannot be captured into a graph: use a blocking stream of our own,
+                        // which still orders itself against work on the legacy default stream
+        if ((e = cudaStreamCreate(&h->stream)) != cudaSuccess) { h->stream = nullptr; return bail(cuda_fail(h, e, "cudaStreamCreate")); }
+        h->own_stream = true;
+    }
+    h->mirror = cfg->train && !(cfg->flags & SDNN_FLAG_BWD_ATOMICS);
+    h->reorder = (cfg->flags & SDNN_FLAG_REORDER) != 0;
+    if (h->reorder) h->pending.resize(n_layers);
+    h->pdl = !(cfg->flags & SDNN_FLAG_NO_PDL);
+    h->nnz.assign(nnz_per_layer, nnz_per_layer + n_layers);
+    h->loaded.assign(n_layers, 0);
+    h->lay.resize(n_layers);
+    h->ld_max = padded_width(cfg->max_batch);
+    const size_t N = (size_t)n_neurons, L = (size_t)n_layers, tile = N * (size_t)h->ld_max;
+
+    if ((rc = dev_alloc(h, &h->d_r_slice_off, L * (h->NS + 1), false))) return bail(rc);
+    if ((rc = dev_alloc(h, &h->d_r_len, L * N, false))) return bail(rc);
+    if ((rc = dev_alloc(h, &h->d_bias, L * N, false))) return bail(rc);
+    if (h->mirror) {
+        if ((rc = dev_alloc(h, &h->d_c_slice_off, L * (h->NS + 1), false))) return bail(rc);
+        if ((rc = dev_alloc(h, &h->d_c_len, L * N, false))) return bail(rc);
+        if ((rc = dev_alloc(h, &h->d_c_order, L * N, false))) return bail(rc);
+        if ((rc = dev_alloc(h, &h->d_mismatch, 1, true))) return bail(rc);
+    }
+    if (cfg->train) {
+        for (cudaEvent_t& ev : h->ev)
+            if ((e = cudaEventCreate(&ev)) != cudaSuccess) { ev = nullptr; return bail(cuda_fail(h, e, "cudaEventCreate")); }
+        if ((rc = dev_alloc(h, &h->d_acts, (L + 1) * tile, false))) return bail(rc);
+        h->split = h->mirror && !(cfg->flags & SDNN_FLAG_BWD_ONE_LAUNCH);
+        if (h->split) {
+            if (!(cfg->flags & SDNN_FLAG_KEEP_DEBUG) && (rc = dev_alloc(h, &h->d_delta_all, L * tile, true))) return bail(rc);
+            h->n_side = 2;      // row-unit launches of neighbouring layers do not depend on each other: two streams let them overlap
+            for (int q = 0; q < h->n_side; ++q) {
+                if ((e = cudaStreamCreateWithFlags(&h->side_streams[q], cudaStreamNonBlocking)) != cudaSuccess) return bail(cuda_fail(h, e, "cudaStreamCreate"));
+                if ((e = cudaEventCreateWithFlags(&h->ev_side_join[q], cudaEventDisableTiming)) != cudaSuccess) return bail(cuda_fail(h, e, "cudaEventCreate"));
+            }
+            h->ev_delta.assign(n_layers, nullptr);
+            for (cudaEvent_t& ev : h->ev_delta)
+                if ((e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming)) != cudaSuccess) { ev = nullptr; return bail(cuda_fail(h, e, "cudaEventCreate")); }
+            if ((e = cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming)) != cudaSuccess) return bail(cuda_fail(h, e, "cudaEventCreate"));
+        }
+        if ((rc = dev_alloc(h, &h->d_s[0], tile, true))) return bail(rc);
+        if ((rc = dev_alloc(h, &h->d_s[1], tile, true))) return bail(rc);
+        if (!h->mirror && (rc = dev_alloc(h, &h->d_dl, tile, true))) return bail(rc);
+        if ((rc = dev_alloc(h, &h->d_yt, tile, true))) return bail(rc);
+        if ((rc = dev_alloc(h, &h->d_sp, 1, true))) return bail(rc);
+        if ((rc = dev_alloc(h, &h->d_loss, 1, true))) return bail(rc);
+        if (cfg->flags & SDNN_FLAG_KEEP_DEBUG)
+            if ((rc = dev_alloc(h, &h->d_dbg_delta, L * tile, true))) return bail(rc);
+    }
+    {   // inference buffers (a training handle can also infer)
+        h->compaction = (cfg->flags & SDNN_FLAG_SKIP_DEAD) != 0;
+        h->bias_nonpositive.assign(n_layers, 0);
+        h->local_pattern.assign(n_layers, 0);
+        if ((rc = dev_alloc(h, &h->d_running, 1, true))) return bail(rc);
+        if ((rc = alloc_lane(h, h->lane[0], false))) return bail(rc);
+        h->cur = &h->lane[0];
+    }
+    *out = h;
+    return SDNN_OK;
+}
+
+int sdnn_load_layer(sdnn_t* h, int32_t layer, const int32_t* row_ptr, const int32_t* col_idx, const float* values,
+                    const float* bias) {
+    if (!h) return SDNN_ERR_INVALID_ARG;
+    if (h->finalized) return fail(h, SDNN_ERR_STATE, "handle already finalized");
+    if (layer < 0 || layer >= h->L) return fail(h, SDNN_ERR_INVALID_ARG, "layer %d outside [0, %d)", layer, h->L);
+    if (h->loaded[layer]) return fail(h, SDNN_ERR_STATE, "layer %d loaded twice", layer);
+    int rc = validate_layer(h, layer, h->N, h->nnz[layer], row_ptr, col_idx, values, bias);
+    if (rc) return rc;
+    if (h->reorder) {      // the layout of a layer depends on its neighbour's grouping: keep the arrays until sdnn_finalize
+        HostLayer& hl = h->pending[layer];
+        const int64_t nz = h->nnz[layer];
+        hl.rp.assign(row_ptr, row_ptr + h->N + 1);
+        hl.col.assign(col_idx, col_idx + nz);
+        hl.val.assign(values, values + nz);
+        hl.bias.assign(bias, bias + h->N);
+        h->loaded[layer] = 1;
+        return SDNN_OK;
+    }
+    rc = upload_layer(h, layer, row_ptr, col_idx, values, bias);
+    if (rc) return rc;
     h->loaded[layer] = 1;
     return SDNN_OK;
 }
@@ -1090,6 +1419,10 @@ int sdnn_finalize(sdnn_t* h) {
     if (h->finalized) return fail(h, SDNN_ERR_STATE, "handle already finalized");
     for (int l = 0; l < h->L; ++l)
         if (!h->loaded[l]) return fail(h, SDNN_ERR_STATE, "layer %d was never loaded", l);
+    if (h->reorder) {
+        int rc = build_reordered(h);
+        if (rc) return rc;
+    }
     CU(h, cudaStreamSynchronize(h->stream));
     h->finalized = true;
     return SDNN_OK;
@@ -1253,12 +1586,30 @@ int sdnn_get_weights(sdnn_t* h, int32_t layer, float* values_out, float* bias_ou
     CU(h, cudaSetDevice(h->device));
     CU(h, cudaStreamSynchronize(h->stream));
     const LayerMem& lm = h->lay[layer];
-    if (values_out && lm.r_elems) {
-        std::vector<float> tmp((size_t)lm.r_elems);
-        CU(h, cudaMemcpy(tmp.data(), lm.r_val, tmp.size() * sizeof(float), cudaMemcpyDeviceToHost));
-        sliced_to_csr(h, lm, tmp, values_out);
+    const int64_t nnz = h->nnz[layer];
+    if (values_out && nnz) {
+        std::vector<float> stored((size_t)nnz);
+        if (lm.windowed) {
+            std::vector<float> tmp((size_t)lm.w_elems);
+            CU(h, cudaMemcpy(tmp.data(), lm.w_val, tmp.size() * sizeof(float), cudaMemcpyDeviceToHost));
+            for (int r = 0; r < h->N; ++r)
+                std::copy(tmp.begin() + lm.w_row_at[r], tmp.begin() + lm.w_row_at[r] + lm.shape.len(r), stored.begin() + lm.shape.start(r));
+        } else {
+            std::vector<float> tmp((size_t)lm.r_elems);
+            CU(h, cudaMemcpy(tmp.data(), lm.r_val, tmp.size() * sizeof(float), cudaMemcpyDeviceToHost));
+            sliced_to_csr(h, lm, tmp, stored.data());
+        }
+        stored_to_caller(lm, stored, values_out, nnz);
     }
-    if (bias_out) CU(h, cudaMemcpy(bias_out, h->d_bias + (size_t)layer * h->N, (size_t)h->N * sizeof(float), cudaMemcpyDeviceToHost));
+    if (bias_out) {
+        if (lm.row_src.empty()) {
+            CU(h, cudaMemcpy(bias_out, h->d_bias + (size_t)layer * h->N, (size_t)h->N * sizeof(float), cudaMemcpyDeviceToHost));
+        } else {
+            std::vector<float> tmp((size_t)h->N);
+            CU(h, cudaMemcpy(tmp.data(), h->d_bias + (size_t)layer * h->N, tmp.size() * sizeof(float), cudaMemcpyDeviceToHost));
+            for (int r = 0; r < h->N; ++r) bias_out[lm.row_src[r]] = tmp[r];
+        }
+    }
     return SDNN_OK;
 }
 
@@ -1275,10 +1626,19 @@ int sdnn_set_weights(sdnn_t* h, int32_t layer, const float* values, const float*
     CU(h, cudaSetDevice(h->device));
     CU(h, cudaStreamSynchronize(h->stream));
     const LayerMem& lm = h->lay[layer];
-    if (values && lm.r_elems) {
-        std::vector<float> tmp;
-        csr_to_sliced(h, lm, values, tmp);
-        CU(h, cudaMemcpy(lm.r_val, tmp.data(), tmp.size() * sizeof(float), cudaMemcpyHostToDevice));
+    const int64_t nnz = h->nnz[layer];
+    if (values && nnz) {
+        std::vector<float> stored, tmp;
+        caller_to_stored(lm, values, stored, nnz);
+        if (lm.windowed) {
+            tmp.assign((size_t)lm.w_elems, 0.0f);
+            for (int r = 0; r < h->N; ++r)
+                std::copy(stored.begin() + lm.shape.start(r), stored.begin() + lm.shape.start(r) + lm.shape.len(r), tmp.begin() + lm.w_row_at[r]);
+            CU(h, cudaMemcpy(lm.w_val, tmp.data(), tmp.size() * sizeof(float), cudaMemcpyHostToDevice));
+        } else {
+            csr_to_sliced(h, lm, stored.data(), tmp);
+            CU(h, cudaMemcpy(lm.r_val, tmp.data(), tmp.size() * sizeof(float), cudaMemcpyHostToDevice));
+        }
         if (lm.c_val) {
             int rc = refresh_mirror(h, layer, nullptr);
             if (rc) return rc;
@@ -1286,7 +1646,13 @@ int sdnn_set_weights(sdnn_t* h, int32_t layer, const float* values, const float*
         }
     }
     if (bias) {
-        CU(h, cudaMemcpy(h->d_bias + (size_t)layer * h->N, bias, (size_t)h->N * sizeof(float), cudaMemcpyHostToDevice));
+        if (lm.row_src.empty()) {
+            CU(h, cudaMemcpy(h->d_bias + (size_t)layer * h->N, bias, (size_t)h->N * sizeof(float), cudaMemcpyHostToDevice));
+        } else {
+            std::vector<float> tmp((size_t)h->N);
+            for (int r = 0; r < h->N; ++r) tmp[r] = bias[lm.row_src[r]];
+            CU(h, cudaMemcpy(h->d_bias + (size_t)layer * h->N, tmp.data(), tmp.size() * sizeof(float), cudaMemcpyHostToDevice));
+        }
         bool nonpos = true;
         for (int i = 0; i < h->N && nonpos; ++i) nonpos = !(bias[i] > 0.0f);
         h->bias_nonpositive[layer] = nonpos ? 1 : 0;
@@ -1436,6 +1802,54 @@ extern "C" int sdnn_probe_gather_rate(int32_t row_bytes, int64_t table_rows, dou
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess || !(ms > 0.f)) rc = cuda_fail(nullptr, e, "gather probe");
         else *rows_per_second = (double)groups * per_group / (ms * 1e-3);
+    }
+    if (a) cudaEventDestroy(a);
+    if (b) cudaEventDestroy(b);
+    if (st) cudaStreamDestroy(st);
+    if (table) cudaFree(table);
+    if (sink) cudaFree(sink);
+    return rc;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Scattered 4-byte word probe (see sdnn_probe_word_rate in the header).
+extern "C" int sdnn_probe_word_rate(int32_t store, int64_t table_words, double* words_per_second) {
+    if (!words_per_second) return fail(nullptr, SDNN_ERR_INVALID_ARG, "words_per_second is NULL");
+    *words_per_second = 0.0;
+    if (store != 0 && store != 1) return fail(nullptr, SDNN_ERR_INVALID_ARG, "store must be 0 (loads) or 1 (stores)");
+    if (table_words < 1024 || (table_words & (table_words - 1)) || table_words > (1LL << 28))
+        return fail(nullptr, SDNN_ERR_INVALID_ARG, "table_words must be a power of two between 2^10 and 2^28");
+    int dev = 0, sms = 0;
+    CU(nullptr, cudaGetDevice(&dev));
+    CU(nullptr, cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    float* table = nullptr;
+    float* sink = nullptr;
+    cudaEvent_t a = nullptr, b = nullptr;
+    cudaStream_t st = nullptr;
+    int rc = SDNN_OK;
+    const size_t bytes = (size_t)table_words * sizeof(float);
+    if (cudaMalloc(&table, bytes) != cudaSuccess || cudaMalloc(&sink, 256) != cudaSuccess || cudaStreamCreate(&st) != cudaSuccess ||
+        cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) {
+        cudaGetLastError();
+        rc = fail(nullptr, SDNN_ERR_OOM, "could not allocate the probe's table");
+    } else {
+        cudaMemsetAsync(table, 0, bytes, st);
+        const int grid = sms * 8, per_lane = 1024, reps = 10;
+        const unsigned mask = (unsigned)(table_words - 1);
+        auto launch = [&](unsigned seed) {
+            if (store) word_probe_kernel<1><<<grid, 256, 0, st>>>(table, sink, mask, per_lane, seed);
+            else word_probe_kernel<0><<<grid, 256, 0, st>>>(table, sink, mask, per_lane, seed);
+        };
+        launch(17u); launch(18u);
+        cudaEventRecord(a, st);
+        for (int i = 0; i < reps; ++i) launch(101u + i);
+        cudaEventRecord(b, st);
+        cudaError_t e = cudaEventSynchronize(b);
+        float ms = 0.f;
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, a, b);
+        if (e == cudaSuccess) e = cudaGetLastError();
+        if (e != cudaSuccess || !(ms > 0.f)) rc = cuda_fail(nullptr, e, "word probe");
+        else *words_per_second = (double)grid * 256 * per_lane / (ms / reps * 1e-3);
     }
     if (a) cudaEventDestroy(a);
     if (b) cudaEventDestroy(b);
@@ -1615,7 +2029,7 @@ extern "C" int sdnn_infer_noalloc(int32_t n_layers, int32_t n_neurons, const int
     const struct { int g, chunks; } q = {ld <= 128 ? ld / 4 : 32, ld <= 128 ? 1 : ld / 128};
     {
         dim3 grid((n_neurons + 31) / 32, (ld + 31) / 32), block(32, 8);
-        transpose_in_kernel<<<grid, block, 0, st>>>(x0, tile[0], n_neurons, n_inputs, ld, ld);
+        transpose_in_kernel<<<grid, block, 0, st>>>(x0, tile[0], n_neurons, n_inputs, ld, ld, nullptr);
     }
     int cur = 0;
     for (int l = 0; l < n_layers; ++l) {

@@ -100,12 +100,15 @@ def train_parity(torch, arrays, batches, eta, update_bias=False, flags=0, clamp=
     return stats
 
 
-def infer_parity(torch, arrays, x0, max_batch, host=False, clamp=32.0, expect_nonempty=None):
+def infer_parity(torch, arrays, x0, max_batch, host=False, clamp=32.0, expect_nonempty=None, flags=0, expect_grouped=None):
     pkg = sdnn()
     rp, col, val, bias = arrays
     L, n = len(col), len(bias[0])
     cnt = x0.shape[0]
-    h = pkg.Sdnn.create(rp, col, val, bias, max_batch=max_batch, clamp=clamp)
+    h = pkg.Sdnn.create(rp, col, val, bias, max_batch=max_batch, clamp=clamp, flags=flags)
+    if expect_grouped is not None:      # layers the set-up analysis found structured; with the shared-memory kernel asked for, all of them use it
+        assert h.grouped_layers() == expect_grouped
+        assert h.windowed_layers() == (expect_grouped if flags & pkg.FLAG_SMEM_WINDOWS else 0)
     cap = cnt * n
     if host:
         y = np.empty((cnt, n), dtype=np.float32); c = np.empty(cnt, dtype=np.int32); idx = np.empty(cap, dtype=np.int32)
@@ -652,6 +655,125 @@ def test_infer_cfg4_in_the_benchmark_launch_shape_sampled(torch_cuda, variant):
         assert not xl.any() and not counts.any()
     else:
         assert xl.any()
+
+
+# ---------------------------------------------------------------------------------------------- set-up reordering
+def block_spec(n, layers, window, live=True):
+    spec = gen.NetSpec("blocks", n, layers, pattern="windowed", window=window, values="const", bias=-0.45, config_id=4)
+    return spec.live() if live else spec
+
+
+REORDER_MODES = {"grouped": 0x100, "smem_windows": 0x300}
+
+
+@pytest.mark.parametrize("mode", sorted(REORDER_MODES))
+@pytest.mark.parametrize("cnt,max_batch,host", [(1, 4, False), (5, 8, True), (13, 16, False), (32, 32, True), (300, 256, False),
+                                                (700, 512, True), (1100, 1024, False)])
+def test_infer_reordered_hidden_blocks(torch_cuda, cnt, max_batch, host, mode):
+    """A block-structured net (config 4's recipe at 4096 neurons, blocks of 1024) whose neurons were renumbered at random:
+    SDNN_FLAG_REORDER finds the blocks in every layer, and outputs, counts and id lists come back in the caller's
+    numbering; every tile width from 4 inputs to several chunks of 32; with the default kernels on the regrouped rows
+    and with the kernel that stages each group's window in shared memory."""
+    spec = block_spec(4096, 6, 1024).shuffled()
+    infer_parity(torch_cuda, gen.network(spec), gen.inputs(spec, cnt), max_batch, host=host, expect_nonempty=True,
+                 flags=REORDER_MODES[mode], expect_grouped=6)
+
+
+@pytest.mark.parametrize("mode", sorted(REORDER_MODES))
+def test_infer_reordered_mixed_layers_and_weights_in_caller_order(torch_cuda, mode):
+    """Layers with block structure (hidden) alternate with uniformly random ones: the former are regrouped, the latter keep
+    the default layout with their rows moved to their neurons' new numbers.  sdnn_get_weights returns the caller's arrays
+    unchanged; after sdnn_set_weights with other values inference follows the new values."""
+    torch = torch_cuda
+    pkg = sdnn()
+    n, k = 2048, 32
+    blocks = block_spec(n, 6, 512).shuffled()
+    uniform = gen.NetSpec("uniform", n, 6, values="normal", sigma=(2.0 / k) ** 0.5, bias=0.0, config_id=2)
+    pick = [blocks, uniform, blocks, blocks, uniform, uniform]
+    rp = [gen.row_ptr(blocks)] * 6
+    col = [gen.layer_pattern(sp, l) for l, sp in enumerate(pick)]
+    val = [gen.layer_values(sp, l) for l, sp in enumerate(pick)]
+    rng = np.random.default_rng(8)
+    bias = [(0.05 * rng.standard_normal(n)).astype(np.float32) for _ in range(6)]
+    x0 = gen.inputs(blocks, 200)
+    infer_parity(torch, (rp, col, val, bias), x0, 128, expect_nonempty=True, flags=REORDER_MODES[mode], expect_grouped=3)
+    h = pkg.Sdnn.create(rp, col, val, bias, max_batch=128, flags=REORDER_MODES[mode])
+    for l in range(6):
+        w, b = h.get_weights(l)
+        assert np.array_equal(w, val[l]) and np.array_equal(b, bias[l])
+    val2 = [(v * rng.uniform(0.5, 1.5, size=v.shape)).astype(np.float32) for v in val]
+    bias2 = [(b + 0.01).astype(np.float32) for b in bias]
+    for l in range(6):
+        h.set_weights(l, val2[l], bias2[l])
+        w, b = h.get_weights(l)
+        assert np.array_equal(w, val2[l]) and np.array_equal(b, bias2[l])
+    yd = torch.empty((200, n), dtype=torch.float32, device="cuda")
+    h.infer_batch(torch.from_numpy(x0).cuda(), 200, yd, None, None, 0)
+    check_close(yd.cpu().numpy(), OracleNet(rp, col, val2, bias2).infer(x0), "x^L after set_weights")
+    h.destroy()
+
+
+@pytest.mark.parametrize("mode", sorted(REORDER_MODES))
+@pytest.mark.parametrize("cnt", [3, 40, 130])
+def test_infer_reordered_ragged_blocks(torch_cuda, cnt, mode):
+    """Blocks of unequal size, rows of 0..9 entries (entries padded to eights in the windowed layout), some rows empty,
+    everything hidden behind random renumberings of rows and columns."""
+    pkg = sdnn()
+    rng = np.random.default_rng(30 + cnt)
+    sizes = [300, 50, 700, 129]
+    n = sum(sizes)
+    rps, cols, vals, biases = [], [], [], []
+    for _ in range(4):
+        perm_r, perm_c = rng.permutation(n), rng.permutation(n)
+        rows, start = {}, 0
+        for sz in sizes:
+            for i in range(start, start + sz):
+                m = int(rng.integers(0, 10))
+                rows[perm_r[i]] = np.sort(perm_c[start + rng.choice(sz, size=min(m, sz), replace=False)])
+            start += sz
+        counts = np.array([len(rows[i]) for i in range(n)])
+        rp = np.zeros(n + 1, dtype=np.int32); rp[1:] = np.cumsum(counts)
+        rps.append(rp); cols.append(np.concatenate([rows[i] for i in range(n)]).astype(np.int32))
+        vals.append((rng.standard_normal(rp[-1]) * 0.6).astype(np.float32))
+        biases.append((rng.standard_normal(n) * 0.1).astype(np.float32))
+    x0 = rng.uniform(0, 1.0, size=(cnt, n)).astype(np.float32)
+    infer_parity(torch_cuda, (rps, cols, vals, biases), x0, 64, expect_nonempty=True, flags=REORDER_MODES[mode], expect_grouped=4)
+
+
+def test_reorder_flag_leaves_an_unstructured_net_alone_and_is_refused_for_training(torch_cuda):
+    pkg = sdnn()
+    spec = gen.CFG2.scaled(4096, 4).live()
+    infer_parity(torch_cuda, gen.network(spec), gen.inputs(spec, 100), 128, expect_nonempty=True, flags=pkg.FLAG_REORDER,
+                 expect_grouped=0)
+    with pytest.raises(pkg.SdnnError) as ei:
+        pkg.Sdnn.create(*gen.network(spec), max_batch=16, flags=pkg.FLAG_SMEM_WINDOWS)       # needs FLAG_REORDER
+    assert ei.value.code == -1
+    with pytest.raises(pkg.SdnnError) as ei:
+        pkg.Sdnn.create(*gen.network(spec), max_batch=16, train=True, flags=pkg.FLAG_REORDER)
+    assert ei.value.code == -6
+
+
+@pytest.mark.parametrize("mode", sorted(REORDER_MODES))
+def test_infer_cfg4_reordered_in_the_benchmark_launch_shape_sampled(torch_cuda, mode):
+    """Config 4 at full size with its neurons renumbered at random and SDNN_FLAG_REORDER, tiles of 1024 inputs (one full,
+    one ragged): the blocks of all 120 layers are found, a sample of the inputs checked one by one against the oracle."""
+    pkg = sdnn()
+    spec = gen.CFG4.live().shuffled()
+    rp, col, val, bias = gen.network(spec)
+    cnt = 1100
+    x0 = gen.inputs(spec, cnt, start=30000)
+    h = pkg.Sdnn.create(rp, col, val, bias, max_batch=1024, flags=REORDER_MODES[mode])
+    assert h.grouped_layers() == spec.layers and h.infer_tile_width() == 1024
+    yd = torch_cuda.empty((cnt, spec.n), dtype=torch_cuda.float32, device="cuda")
+    cd = torch_cuda.empty(cnt, dtype=torch_cuda.int32, device="cuda")
+    h.infer_batch(torch_cuda.from_numpy(x0).cuda(), cnt, yd, cd, None, 0)
+    h.destroy()
+    sample = np.unique(np.concatenate([[0, 1, 31, 32, 255, 256, 511, 1023, 1024, 1099],
+                                       np.random.default_rng(9).integers(0, cnt, size=22)]))
+    xl = OracleNet(rp, col, val, bias).infer(x0[sample])
+    y = yd[torch_cuda.from_numpy(sample).cuda()].cpu().numpy()
+    check_close(y, xl, "sampled x^L")
+    assert xl.any() and np.array_equal(cd.cpu().numpy()[sample], (y != 0.0).sum(axis=1))
 
 
 # ---------------------------------------------------------------------------------------------- API behaviour on a device

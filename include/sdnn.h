@@ -77,6 +77,9 @@ typedef enum {
                                     /* every delta^k of a step (N * padded(B) * 4 bytes per layer more) and is faster    */
 #define SDNN_FLAG_NO_PDL      0x20u /* do not let a layer's kernel start its prologue under the previous layer's tail */
 #define SDNN_FLAG_ONE_TILE    0x40u /* inference: one tile in flight at a time (see sdnn_infer_batch)               */
+#define SDNN_FLAG_IDX32       0x400u /* keep 32-bit indices in the library's internal copies of the layers.  By default a     */
+                                    /* net of at most 65536 neurons stores them in 16 bits (2 bytes less per stored entry  */
+                                    /* and pass over it); results are identical either way                                */
 #define SDNN_FLAG_REORDER     0x100u /* set-up (untimed): group the rows of every W^k by the columns they share and    */
                                     /* renumber the neurons of layer k-1 so that each group's columns are one            */
                                     /* contiguous window of at most 1536 neurons (the single-GPU counterpart of the      */

@@ -18,6 +18,7 @@ FLAG_BWD_ONE_LAUNCH = 0x80
 FLAG_ONE_TILE = 0x40
 FLAG_REORDER = 0x100
 FLAG_SMEM_WINDOWS = 0x200
+FLAG_IDX32 = 0x400
 ACT_CLAMPED_RELU, ACT_SIGMOID = 0, 1
 
 STATUS = {0: "SDNN_OK", -1: "SDNN_ERR_INVALID_ARG", -2: "SDNN_ERR_BAD_CSR", -3: "SDNN_ERR_OOM", -4: "SDNN_ERR_CUDA",

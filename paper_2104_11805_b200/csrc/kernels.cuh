@@ -41,9 +41,11 @@ constexpr int CHUNK_ROW = SLICE * 4; // elements of one chunk over the rows of a
 struct Sliced {
     const int* slice_off;   // [ceil(n/16) + 1] element offsets of the slices, multiples of 128
     const int* len;         // [n] stored entries of each unit
-    const int* idx;         // gathered tile row of each entry (column index; row index in the transposed copy)
+    const int* idx;         // gathered tile row of each entry (column index; row index in the transposed copy);
+                            // with idx16 set the array holds 16-bit unsigned indices instead (nets of at most 65536 neurons)
     float*     val;
     const int* order;
+    int idx16;
     const int* out;         // forward kernels: tile row that unit u's output goes to (NULL: row u), for layers whose rows are
                             // stored group by group while their neurons carry the numbers the next layer's grouping gave them
 };
@@ -360,10 +362,21 @@ forward_csr_kernel(const int* __restrict__ row_ptr, const int* __restrict__ col,
 // (padding has index 0 and value 0), which keeps the lanes of a warp converged.  The indices of a step are
 // loaded one step ahead (while the previous step's gathers are in flight, also across the boundary between
 // two units), so that a step costs one memory round trip, not two dependent ones.
+// the four indices of one chunk of one row, at element offset `at` (a multiple of 4) of the index array
+__device__ __forceinline__ int4 load_idx4(const Sliced& m, int at) {
+    if (m.idx16) {
+        const uint2 v = __ldcs(reinterpret_cast<const uint2*>(reinterpret_cast<const unsigned short*>(m.idx) + at));
+        return make_int4((int)(v.x & 0xffffu), (int)(v.x >> 16), (int)(v.y & 0xffffu), (int)(v.y >> 16));
+    }
+    return __ldcs(reinterpret_cast<const int4*>(m.idx + at));
+}
+__device__ __forceinline__ int load_idx1(const Sliced& m, int at) {
+    return m.idx16 ? (int)reinterpret_cast<const unsigned short*>(m.idx)[at] : m.idx[at];
+}
 template <int CPS>
-__device__ __forceinline__ void load_idx(int4 (&c)[CPS], const int* p) {
+__device__ __forceinline__ void load_idx(int4 (&c)[CPS], const Sliced& m, int at) {
 #pragma unroll
-    for (int i = 0; i < CPS; ++i) c[i] = __ldcs(reinterpret_cast<const int4*>(p + CHUNK_ROW * i));
+    for (int i = 0; i < CPS; ++i) c[i] = load_idx4(m, at + CHUNK_ROW * i);
 }
 
 // asks for the slices that hold the rows of unit `u` (rpw consecutive rows) to be brought into L2
@@ -372,7 +385,11 @@ __device__ __forceinline__ void prefetch_unit(const Sliced& m, int u, int rpw, i
     if (units_per_slice > 1 && (r0 & (SLICE - 1)) != 0) return;      // units narrower than a slice: the first one asks for the whole slice
     const int s0 = r0 / SLICE, s1 = min((n + SLICE - 1) / SLICE, (r0 + rpw - 1) / SLICE + 1);
     const int lo = m.slice_off[s0], hi = m.slice_off[s1];
-    if (hi > lo) { prefetch_l2(m.idx + lo, (unsigned)(hi - lo) * 4u); prefetch_l2(m.val + lo, (unsigned)(hi - lo) * 4u); }
+    if (hi > lo) {
+        if (m.idx16) prefetch_l2(reinterpret_cast<const unsigned short*>(m.idx) + lo, (unsigned)(hi - lo) * 2u);
+        else prefetch_l2(m.idx + lo, (unsigned)(hi - lo) * 4u);
+        prefetch_l2(m.val + lo, (unsigned)(hi - lo) * 4u);
+    }
 }
 
 #define SDNN_GATHER_CHUNK(X, I, C, P, PITCH)                                                              \
@@ -409,7 +426,6 @@ forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict
     const int boff = blockIdx.y * (V * G) + sub * V;
     const float* xg = xin + boff;
     const unsigned pitch = (unsigned)ld * 4u;
-    const int* __restrict__ idx = m.idx;
     const float* __restrict__ val = m.val;
 
     int unit = blockIdx.x * wpb + (threadIdx.x >> 5);
@@ -422,7 +438,7 @@ forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict
     int4 c[CPS];
 #pragma unroll
     for (int i = 0; i < CPS; ++i) c[i] = make_int4(0, 0, 0, 0);
-    if (nch > 0) load_idx<CPS>(c, idx + base);
+    if (nch > 0) load_idx<CPS>(c, m, base);
     if (pdl) grid_dependency_wait();
     if (pdl == 2) grid_launch_dependents();
     // compaction mode: only the first *ncols_dev columns of the tile still hold live inputs
@@ -440,7 +456,6 @@ forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict
 
         Lane<V> acc;
         lane_fill(acc, b);
-        const int* cp = idx + base;
         const float* vp = val + base;
         for (int t = 0; t < nch; t += CPS) {
             float4 w[CPS];
@@ -449,15 +464,15 @@ forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict
             for (int i = 0; i < CPS; ++i) w[i] = __ldcs(reinterpret_cast<const float4*>(vp + (t + i) * CHUNK_ROW));
 #pragma unroll
             for (int i = 0; i < CPS; ++i) { SDNN_GATHER_CHUNK(x, i, c[i], xg, pitch) }
-            if (t + CPS < nch) load_idx<CPS>(c, cp + (t + CPS) * CHUNK_ROW);
-            else if (nnch > 0) load_idx<CPS>(c, idx + nbase);
+            if (t + CPS < nch) load_idx<CPS>(c, m, base + (t + CPS) * CHUNK_ROW);
+            else if (nnch > 0) load_idx<CPS>(c, m, nbase);
 #pragma unroll
             for (int i = 0; i < CPS; ++i) {
                 lane_fma(w[i].x, x[4 * i + 0], acc); lane_fma(w[i].y, x[4 * i + 1], acc);
                 lane_fma(w[i].z, x[4 * i + 2], acc); lane_fma(w[i].w, x[4 * i + 3], acc);
             }
         }
-        if (nch == 0 && nnch > 0) load_idx<CPS>(c, idx + nbase);      // empty slice: nothing prefetched across the boundary yet
+        if (nch == 0 && nnch > 0) load_idx<CPS>(c, m, nbase);      // empty slice: nothing prefetched across the boundary yet
         if (row < n) {
             lane_activate(acc, act, clamp);
             lane_store(tile_row(xout + boff, orow, pitch), acc);
@@ -722,7 +737,6 @@ __device__ __forceinline__ void backward_col_units(const Sliced m, const float* 
     const unsigned gmask = (G >= 2) ? 0xffffffffu : group_mask<G>(grp);     // G >= 2: one slice per warp, its lanes stay converged
     const int nunits = (n + RPW - 1) / RPW;
     const int boff = sub * V;
-    const int* __restrict__ idx = m.idx;
     float* val = m.val;
     const float* dg = dk + boff;
 
@@ -734,7 +748,7 @@ __device__ __forceinline__ void backward_col_units(const Sliced m, const float* 
     int4 c[CPS];
 #pragma unroll
     for (int i = 0; i < CPS; ++i) c[i] = make_int4(0, 0, 0, 0);
-    if (nch > 0) load_idx<CPS>(c, idx + base);
+    if (nch > 0) load_idx<CPS>(c, m, base);
     Lane<V> xj;
     lane_fill(xj, 0.0f);
     if (item < n) lane_load(xj, tile_row(xprev + boff, j, pitch));
@@ -748,10 +762,9 @@ __device__ __forceinline__ void backward_col_units(const Sliced m, const float* 
         Lane<V> nxj, acc;
         lane_fill(nxj, 0.0f);
         lane_fill(acc, 0.0f);
-        const int* ip = idx + base;
         float* vp = val + base;
         const int lim = len - ((G >= 4) ? (sub & 3) : (G == 2) ? 2 * sub : 0);
-#define SDNN_COL_NEXT if (nnch > 0) load_idx<CPS>(c, idx + nbase); if (nitem < n) lane_load(nxj, tile_row(xprev + boff, nj, pitch));
+#define SDNN_COL_NEXT if (nnch > 0) load_idx<CPS>(c, m, nbase); if (nitem < n) lane_load(nxj, tile_row(xprev + boff, nj, pitch));
         for (int t = 0; t < nch; t += CPS) {
             float4 w[CPS];
             Lane<V> d[4 * CPS];
@@ -759,7 +772,7 @@ __device__ __forceinline__ void backward_col_units(const Sliced m, const float* 
             for (int i = 0; i < CPS; ++i) w[i] = ld_f4(vp + (t + i) * CHUNK_ROW);
 #pragma unroll
             for (int i = 0; i < CPS; ++i) { SDNN_GATHER_CHUNK(d, i, c[i], dg, pitch) }
-            if (t + CPS < nch) { load_idx<CPS>(c, ip + (t + CPS) * CHUNK_ROW); }
+            if (t + CPS < nch) { load_idx<CPS>(c, m, base + (t + CPS) * CHUNK_ROW); }
             else { SDNN_COL_NEXT }
 #pragma unroll
             for (int i = 0; i < CPS; ++i) {
@@ -795,7 +808,6 @@ __device__ __forceinline__ void backward_row_units(const Sliced m, float* __rest
     const unsigned gmask = (G >= 2) ? 0xffffffffu : gmask1;
     const int nunits = (n + RPW - 1) / RPW;
     const int boff = sub * V;
-    const int* __restrict__ idx = m.idx;
     float* val = m.val;
     const float* xg = xprev + boff;
     float* sg = SCATTER ? dprev + boff : nullptr;
@@ -807,7 +819,7 @@ __device__ __forceinline__ void backward_row_units(const Sliced m, float* __rest
     int4 c[CPS];
 #pragma unroll
     for (int i = 0; i < CPS; ++i) c[i] = make_int4(0, 0, 0, 0);
-    if (nch > 0) load_idx<CPS>(c, idx + base);
+    if (nch > 0) load_idx<CPS>(c, m, base);
     Lane<V> h0, h1;       // delta^k[i,:] (or S_k[i,:]) and, FROM_S, x^k[i,:]
     lane_fill(h0, 0.0f); lane_fill(h1, 0.0f);
     if (item < n) { lane_load(h0, tile_row(dk + boff, item, pitch)); if (FROM_S) lane_load(h1, tile_row(xk + boff, item, pitch)); }
@@ -837,12 +849,11 @@ __device__ __forceinline__ void backward_row_units(const Sliced m, float* __rest
         if (skip_dead) {             // delta^k(i) = 0 for every input of every row of the unit: nothing changes
             if (__ballot_sync(gmask, lane_any(d)) == 0u) nch = 0;
         }
-        const int* cp = idx + base;
         float* vp = val + base;
         float* gp = DBG ? dbg_grad + base : nullptr;
         const int lim = len - ((G >= 4) ? (sub & 3) : (G == 2) ? 2 * sub : 0);
 #define SDNN_ROW_NEXT                                                                                    \
-        if (nnch > 0) load_idx<CPS>(c, idx + nbase);                                                     \
+        if (nnch > 0) load_idx<CPS>(c, m, nbase);                                                        \
         if (nitem < n) { lane_load(nh0, tile_row(dk + boff, nitem, pitch)); if (FROM_S) lane_load(nh1, tile_row(xk + boff, nitem, pitch)); }
 #define SDNN_SCAT(C, W, Q) if ((Q) < len) lane_red_add(tile_row(sg, C, pitch), W, d);
         for (int t = 0; t < nch; t += CPS) {
@@ -859,7 +870,7 @@ __device__ __forceinline__ void backward_row_units(const Sliced m, float* __rest
                     SDNN_SCAT(c[i].x, w[i].x, q) SDNN_SCAT(c[i].y, w[i].y, q + 1) SDNN_SCAT(c[i].z, w[i].z, q + 2) SDNN_SCAT(c[i].w, w[i].w, q + 3)
                 }
             }
-            if (t + CPS < nch) { load_idx<CPS>(c, cp + (t + CPS) * CHUNK_ROW); }
+            if (t + CPS < nch) { load_idx<CPS>(c, m, base + (t + CPS) * CHUNK_ROW); }
             else { SDNN_ROW_NEXT }
 #pragma unroll
             for (int i = 0; i < CPS; ++i) {
@@ -929,7 +940,7 @@ __device__ __forceinline__ EpShape ep_shape(const Sliced& m, int n) {
 #define SDNN_EP_LOAD_IDX(C, T0, IT)                                                                     \
     _Pragma("unroll") for (int i = 0; i < (IT); ++i) {                                                   \
         const int t = (T0) + 2 * i + e.h;                                                                \
-        C[i] = (t < e.nch) ? __ldcs(reinterpret_cast<const int4*>(m.idx + e.so + t * CHUNK_ROW + e.r * 4)) : make_int4(0, 0, 0, 0); \
+        C[i] = (t < e.nch) ? load_idx4(m, e.so + t * CHUNK_ROW + e.r * 4) : make_int4(0, 0, 0, 0);       \
     }
 
 __global__ void __launch_bounds__(128)
@@ -1088,12 +1099,12 @@ __global__ void mirror_values_kernel(Sliced rows, Sliced cols, int n, unsigned l
     const int base = cols.slice_off[cc / SLICE] + (cc % SLICE) * 4;
     for (int q = threadIdx.x & 31; q < len; q += 32) {
         const int pos = base + (q >> 2) * CHUNK_ROW + (q & 3);
-        const int i = cols.idx[pos];
+        const int i = load_idx1(cols, pos);
         const int rb = rows.slice_off[i / SLICE] + (i % SLICE) * 4;
         int lo = 0, hi = rows.len[i] - 1, at = -1;
         while (lo <= hi) {
             const int mid = (lo + hi) >> 1;
-            const int c = rows.idx[rb + (mid >> 2) * CHUNK_ROW + (mid & 3)];
+            const int c = load_idx1(rows, rb + (mid >> 2) * CHUNK_ROW + (mid & 3));
             if (c == j) { at = mid; break; }
             if (c < j) lo = mid + 1; else hi = mid - 1;
         }

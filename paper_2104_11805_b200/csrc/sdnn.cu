@@ -90,6 +90,7 @@ struct sdnn {
     int device = 0, sms = 0;
     bool finalized = false, stepped = false;
     bool mirror = false;                // training with the transposed copy (no atomics)
+    bool idx16 = false;                 // the sliced copies hold 16-bit indices (at most 65536 neurons, SDNN_FLAG_IDX32 not set)
     bool pdl = false;                   // programmatic dependent launch between the layer kernels
     int fwd_pdl = 2;                    // PDL_EARLY; when a forward launch lets the next one go (PDL_EARLY, or PDL_AT_END while two tiles are in flight)
     std::vector<int64_t> nnz;
@@ -362,6 +363,7 @@ Sliced rows_of(sdnn* h, int layer) {
     m.idx = h->lay[layer].r_idx;
     m.val = h->lay[layer].r_val;
     m.order = nullptr;
+    m.idx16 = h->idx16 ? 1 : 0;
     m.out = h->lay[layer].r_out;
     return m;
 }
@@ -373,6 +375,7 @@ Sliced cols_of(sdnn* h, int layer) {
     m.idx = h->lay[layer].c_idx;
     m.val = h->lay[layer].c_val;
     m.order = h->d_c_order + (size_t)layer * h->N;
+    m.idx16 = h->idx16 ? 1 : 0;
     m.out = nullptr;
     return m;
 }
@@ -921,6 +924,27 @@ int refresh_mirror(sdnn* h, int layer, unsigned long long* mismatch_dev) {
     return SDNN_OK;
 }
 
+// Index arrays of the sliced copies: 16 bits per index where the net has at most 65536 neurons (h->idx16), else 32.
+int alloc_indices(sdnn* h, int** out, size_t count) {
+    if (!h->idx16) return dev_alloc(h, out, count, false);
+    unsigned short* p = nullptr;
+    int rc = dev_alloc(h, &p, count, false);
+    *out = reinterpret_cast<int*>(p);
+    return rc;
+}
+int upload_indices(sdnn* h, int* dst, const std::vector<int>& src) {      // synchronous with respect to `src` when narrowing
+    if (!h->idx16) {
+        CU(h, cudaMemcpyAsync(dst, src.data(), src.size() * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+        return SDNN_OK;
+    }
+    std::vector<unsigned short> narrow(src.size());
+#pragma omp parallel for schedule(static)
+    for (int64_t q = 0; q < (int64_t)src.size(); ++q) narrow[(size_t)q] = (unsigned short)src[(size_t)q];
+    CU(h, cudaMemcpyAsync(dst, narrow.data(), narrow.size() * sizeof(unsigned short), cudaMemcpyHostToDevice, h->stream));
+    CU(h, cudaStreamSynchronize(h->stream));
+    return SDNN_OK;
+}
+
 // Lays out one validated layer (caller's or reordered CSR, host arrays) in the kernels' sliced format and uploads it.
 int upload_layer(sdnn* h, int layer, const int32_t* row_ptr, const int32_t* col_idx, const float* values, const float* bias) {
     int rc;
@@ -948,7 +972,7 @@ int upload_layer(sdnn* h, int layer, const int32_t* row_ptr, const int32_t* col_
         for (int i = 0; i < N; ++i)
             for (int q = 0; q < r_len[i]; ++q) r_idx[(size_t)sliced_pos(off, i, q)] = col_idx[row_ptr[i] + q];
     }
-    if ((rc = dev_alloc(h, &lm.r_idx, (size_t)lm.r_elems, false))) return rc;
+    if ((rc = alloc_indices(h, &lm.r_idx, (size_t)lm.r_elems))) return rc;
     if ((rc = dev_alloc(h, &lm.r_val, (size_t)lm.r_elems, false))) return rc;
     if (h->cfg.train && (h->cfg.flags & SDNN_FLAG_KEEP_DEBUG))
         if ((rc = dev_alloc(h, &lm.r_grad, (size_t)lm.r_elems, true))) return rc;
@@ -956,7 +980,7 @@ int upload_layer(sdnn* h, int layer, const int32_t* row_ptr, const int32_t* col_
     CU(h, cudaMemcpyAsync(h->d_r_len + (size_t)layer * N, r_len.data(), (size_t)N * sizeof(int), cudaMemcpyHostToDevice, h->stream));
     CU(h, cudaMemcpyAsync(h->d_bias + (size_t)layer * N, bias, (size_t)N * sizeof(float), cudaMemcpyHostToDevice, h->stream));
     if (lm.r_elems) {
-        CU(h, cudaMemcpyAsync(lm.r_idx, r_idx.data(), (size_t)lm.r_elems * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+        if ((rc = upload_indices(h, lm.r_idx, r_idx))) return rc;
         CU(h, cudaMemcpyAsync(lm.r_val, r_val.data(), (size_t)lm.r_elems * sizeof(float), cudaMemcpyHostToDevice, h->stream));
     }
 
@@ -998,12 +1022,12 @@ int upload_layer(sdnn* h, int layer, const int32_t* row_ptr, const int32_t* col_
                     c_idx[(size_t)sliced_pos(c_off.data(), place[j], q)] = i;
                 }
         }
-        if ((rc = dev_alloc(h, &lm.c_idx, (size_t)lm.c_elems, false))) return rc;
+        if ((rc = alloc_indices(h, &lm.c_idx, (size_t)lm.c_elems))) return rc;
         if ((rc = dev_alloc(h, &lm.c_val, (size_t)lm.c_elems, true))) return rc;
         CU(h, cudaMemcpyAsync(h->d_c_slice_off + (size_t)layer * (NS + 1), c_off.data(), (size_t)(NS + 1) * sizeof(int), cudaMemcpyHostToDevice, h->stream));
         CU(h, cudaMemcpyAsync(h->d_c_len + (size_t)layer * N, c_len.data(), (size_t)N * sizeof(int), cudaMemcpyHostToDevice, h->stream));
         CU(h, cudaMemcpyAsync(h->d_c_order + (size_t)layer * N, order.data(), (size_t)N * sizeof(int), cudaMemcpyHostToDevice, h->stream));
-        if (lm.c_elems) CU(h, cudaMemcpyAsync(lm.c_idx, c_idx.data(), (size_t)lm.c_elems * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+        if (lm.c_elems && (rc = upload_indices(h, lm.c_idx, c_idx))) return rc;
         if ((rc = refresh_mirror(h, layer, nullptr))) return rc;
     }
     CU(h, cudaStreamSynchronize(h->stream));   // the host vectors above go out of scope; the caller may reuse its arrays
@@ -1334,6 +1358,7 @@ int sdnn_create_deferred(sdnn_t** out, int32_t n_layers, int32_t n_neurons, cons
         h->own_stream = true;
     }
     h->mirror = cfg->train && !(cfg->flags & SDNN_FLAG_BWD_ATOMICS);
+    h->idx16 = n_neurons <= 65536 && !(cfg->flags & SDNN_FLAG_IDX32);
     h->reorder = (cfg->flags & SDNN_FLAG_REORDER) != 0;
     if (h->reorder) h->pending.resize(n_layers);
     h->pdl = !(cfg->flags & SDNN_FLAG_NO_PDL);

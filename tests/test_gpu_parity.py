@@ -657,6 +657,24 @@ def test_infer_cfg4_in_the_benchmark_launch_shape_sampled(torch_cuda, variant):
         assert xl.any()
 
 
+# ---------------------------------------------------------------------------------------------- index width
+@pytest.mark.parametrize("bwd", sorted(BWD_MODES))
+def test_32_bit_indices_on_request_and_beyond_65536_neurons(torch_cuda, bwd):
+    """Nets of at most 65536 neurons keep 16-bit indices in the library's copies of the layers (every other test);
+    SDNN_FLAG_IDX32 keeps 32 bits, and a net of 66000 neurons has to.  Training (every backward realisation) and inference."""
+    pkg = sdnn()
+    rng = np.random.default_rng(12)
+    arrays = ragged_net(rng, n=203, layers=4, kmax=12)
+    batches = [(rng.uniform(0, 1.5, size=(16, 203)).astype(np.float32), rng.uniform(0, 1, size=(16, 203)).astype(np.float32))
+               for _ in range(2)]
+    train_parity(torch_cuda, arrays, batches, eta=0.01, update_bias=True, flags=BWD_MODES[bwd] | pkg.FLAG_IDX32, expect_live=True)
+    spec = gen.NetSpec("wide", 66000, 3, k=6, values="normal", sigma=(2.0 / 6) ** 0.5, bias=0.0, config_id=7, input_prob=0.3)
+    train_parity(torch_cuda, gen.network(spec), batches_for(spec, 5, 2), eta=1e-2, flags=BWD_MODES[bwd], expect_live=True)
+    if bwd == "transposed":
+        infer_parity(torch_cuda, gen.network(spec), gen.inputs(spec, 40), 32, expect_nonempty=True)
+        infer_parity(torch_cuda, arrays, rng.uniform(0, 1, size=(40, 203)).astype(np.float32), 32, flags=pkg.FLAG_IDX32, expect_nonempty=True)
+
+
 # ---------------------------------------------------------------------------------------------- set-up reordering
 def block_spec(n, layers, window, live=True):
     spec = gen.NetSpec("blocks", n, layers, pattern="windowed", window=window, values="const", bias=-0.45, config_id=4)

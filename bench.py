@@ -648,8 +648,14 @@ def main():
     target = {"hbm_frac_target": 0.5, "target_met": bool(frac is not None and frac >= 0.5),
               "note": "the target asks for half of the HBM roofline; these launches are bound by random row gathers out of L2 "
                       "(gather_bound), which caps them well below it"}
+    # the library keeps 16-bit indices for nets of at most 65536 neurons: the same launch against its own, smaller byte count
+    idx16 = N <= 65536 and not (flags & pkg.FLAG_IDX32)
+    alg16 = alg - 2 * nnz_l if idx16 else alg
+    own = {"index_bytes": 2 if idx16 else 4, "algorithmic_bytes_per_launch": alg16,
+           "achieved": alg16 / (per_launch_ms * 1e-3) / 1e9 if per_launch_ms else None,
+           "frac": alg16 / (per_launch_ms * 1e-3) / 1e9 / hbm_peak if per_launch_ms else None}
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
-                "frac": frac, "target": target, "traffic": traffic, "peak_source": peak_src,
+                "frac": frac, "with_stored_index_width": own, "target": target, "traffic": traffic, "peak_source": peak_src,
                 "algorithmic_bytes_per_launch": alg, "launch_ms": per_launch_ms, **extra}
 
     # -------------------------------------------------------------------- CPU oracle on a bounded sample (rank 0, N = 1)

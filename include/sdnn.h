@@ -364,6 +364,15 @@ int sdnn_infer_noalloc(int32_t n_layers, int32_t n_neurons, const int32_t* row_p
                        const float* values, const int64_t* layer_offset, const float* bias,
                        const float* x0, int32_t n_inputs, float* y_out, float clamp, void* cuda_stream);
 
+/*
+ * sdnn_infer_noalloc cannot validate the caller's device arrays on the host.  Its kernel checks the one thing it can
+ * without knowing the arrays' lengths: a column index outside [0, n_neurons) is not followed (the entry contributes
+ * nothing) and is counted.  count_out (host int64*): such indices met on the current device since the library was
+ * loaded; nonzero means the results of some call are not those of the network.  Waits for the device (a copy on
+ * the legacy default stream); allocates nothing.
+ */
+int sdnn_infer_noalloc_bad_columns(int64_t* count_out);
+
 void sdnn_destroy(sdnn_t* h);                 /* NULL is a no-op */
 const char* sdnn_last_error(const sdnn_t* h); /* h may be NULL: last creation error of this thread */
 const char* sdnn_version(void);

@@ -64,6 +64,7 @@ _PROTOS = {
     "sdnn_windowed_layers": (_i32, [_vp]),
     "sdnn_grouped_layers": (_i32, [_vp]),
     "sdnn_cluster_layer": (ctypes.c_int, [_i32, _vp, _vp, _i32, _i32, _vp, _vp, ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
+    "sdnn_infer_noalloc_bad_columns": (ctypes.c_int, [ctypes.POINTER(_i64)]),
     "sdnn_kernel_launches": (_i64, [_vp]),
     "sdnn_infer_tile_width": (_i32, [_vp]),
     "sdnn_infer_tiles_in_flight": (_i32, [_vp]),
@@ -134,6 +135,16 @@ def infer_noalloc(n_layers, n_neurons, row_ptr, col_idx, values, layer_offset, b
                                 _addr(bias), _addr(x0), n_inputs, _addr(y_out), clamp, stream)
     if rc != 0:
         raise SdnnError(rc, (lib.sdnn_last_error(None) or b"").decode())
+
+
+def infer_noalloc_bad_columns():
+    """sdnn_infer_noalloc_bad_columns: out-of-range column indices that infer_noalloc met (and skipped) on this device."""
+    lib = load_library()
+    out = _i64(0)
+    rc = lib.sdnn_infer_noalloc_bad_columns(ctypes.byref(out))
+    if rc != 0:
+        raise SdnnError(rc, (lib.sdnn_last_error(None) or b"").decode())
+    return out.value
 
 
 def probe_gather_rate(row_bytes, table_rows):

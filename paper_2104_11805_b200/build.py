@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsdnn.so")
 SOURCES = [os.path.join(CSRC, "sdnn.cu")]
-DEPENDS = SOURCES + [os.path.join(CSRC, "kernels.cuh"), os.path.join(HERE, "..", "include", "sdnn.h")]
+DEPENDS = SOURCES + [os.path.join(CSRC, "kernels.cuh"), os.path.join(CSRC, "reorder.h"), os.path.join(HERE, "..", "include", "sdnn.h")]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -29,7 +29,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
     if not force and up_to_date():
         return LIB
     nvcc = os.environ.get("NVCC", "nvcc")
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", LIB] + SOURCES + ["-lgomp"]
+    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", LIB] + SOURCES + ["-lgomp", "-ldl"]
     subprocess.check_call(cmd)
     return LIB
 

@@ -306,11 +306,13 @@ __global__ void set_step_params_kernel(StepParams* p, float eta, int batch, doub
 // ---------------------------------------------------------------------------------------------
 // Forward layer on plain CSR arrays (feedforward equation).  Used only where the stored entries
 // belong to the caller and cannot be re-laid out (sdnn_infer_noalloc).
+// The arrays are the caller's and were never validated on the host: a column index outside [0, n) is not followed
+// (its entry contributes nothing) and is counted in *bad_columns, which the host can read afterwards.
 template <int G>
 __global__ void __launch_bounds__(256)
 forward_csr_kernel(const int* __restrict__ row_ptr, const int* __restrict__ col, const float* __restrict__ val,
                    const float* __restrict__ bias, const float* __restrict__ xin, float* __restrict__ xout,
-                   int n, int ld, float clamp) {
+                   int n, int ld, float clamp, unsigned long long* __restrict__ bad_columns) {
     constexpr int RPW = 32 / G;
     const int lane = threadIdx.x & 31;
     const int sub = lane % G, grp = lane / G;
@@ -324,32 +326,34 @@ forward_csr_kernel(const int* __restrict__ row_ptr, const int* __restrict__ col,
     const float b = bias[row];
     float4 acc = make_float4(b, b, b, b);
     int p = s;
+    unsigned bad = 0;
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
 #define SDNN_FMA4(W, X) acc.x = fmaf(W, X.x, acc.x); acc.y = fmaf(W, X.y, acc.y); acc.z = fmaf(W, X.z, acc.z); acc.w = fmaf(W, X.w, acc.w);
+#define SDNN_X(C) ((unsigned)(C) < (unsigned)n ? gather_f4(xg + (size_t)(C) * ld) : (++bad, zero))
     if (((s | e) & 3) == 0) {
         for (; p + 8 <= e; p += 8) {
             const int4 c0 = *reinterpret_cast<const int4*>(col + p), c1 = *reinterpret_cast<const int4*>(col + p + 4);
             const float4 w0 = ld_f4(val + p), w1 = ld_f4(val + p + 4);
-            const float4 x0 = gather_f4(xg + (size_t)c0.x * ld), x1 = gather_f4(xg + (size_t)c0.y * ld);
-            const float4 x2 = gather_f4(xg + (size_t)c0.z * ld), x3 = gather_f4(xg + (size_t)c0.w * ld);
-            const float4 x4 = gather_f4(xg + (size_t)c1.x * ld), x5 = gather_f4(xg + (size_t)c1.y * ld);
-            const float4 x6 = gather_f4(xg + (size_t)c1.z * ld), x7 = gather_f4(xg + (size_t)c1.w * ld);
+            const float4 x0 = SDNN_X(c0.x), x1 = SDNN_X(c0.y), x2 = SDNN_X(c0.z), x3 = SDNN_X(c0.w);
+            const float4 x4 = SDNN_X(c1.x), x5 = SDNN_X(c1.y), x6 = SDNN_X(c1.z), x7 = SDNN_X(c1.w);
             SDNN_FMA4(w0.x, x0) SDNN_FMA4(w0.y, x1) SDNN_FMA4(w0.z, x2) SDNN_FMA4(w0.w, x3)
             SDNN_FMA4(w1.x, x4) SDNN_FMA4(w1.y, x5) SDNN_FMA4(w1.z, x6) SDNN_FMA4(w1.w, x7)
         }
         for (; p < e; p += 4) {
             const int4 c0 = *reinterpret_cast<const int4*>(col + p);
             const float4 w0 = ld_f4(val + p);
-            const float4 x0 = gather_f4(xg + (size_t)c0.x * ld), x1 = gather_f4(xg + (size_t)c0.y * ld);
-            const float4 x2 = gather_f4(xg + (size_t)c0.z * ld), x3 = gather_f4(xg + (size_t)c0.w * ld);
+            const float4 x0 = SDNN_X(c0.x), x1 = SDNN_X(c0.y), x2 = SDNN_X(c0.z), x3 = SDNN_X(c0.w);
             SDNN_FMA4(w0.x, x0) SDNN_FMA4(w0.y, x1) SDNN_FMA4(w0.z, x2) SDNN_FMA4(w0.w, x3)
         }
     } else {
         for (; p < e; ++p) {
             const float w = val[p];
-            const float4 x = gather_f4(xg + (size_t)col[p] * ld);
+            const float4 x = SDNN_X(col[p]);
             SDNN_FMA4(w, x)
         }
     }
+#undef SDNN_X
+    if (bad && sub == 0) atomicAdd(bad_columns, (unsigned long long)bad);      // the lanes of a row see the same columns
     acc.x = clampf(acc.x, clamp); acc.y = clampf(acc.y, clamp);
     acc.z = clampf(acc.z, clamp); acc.w = clampf(acc.w, clamp);
     st_f4(xout + (size_t)row * ld + boff, acc);

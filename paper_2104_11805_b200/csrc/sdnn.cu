@@ -6,6 +6,8 @@
 #include "kernels.cuh"
 #include "reorder.h"
 
+#include <nvtx3/nvToolsExt.h>
+
 #include <algorithm>
 #include <cmath>
 #include <cstdarg>
@@ -311,6 +313,20 @@ int64_t build_slice_offsets(int n, LenFn len, std::vector<int>& off) {
 }
 
 void count_launch(sdnn* h, int k = 1) { h->launches += k; }
+
+// NVTX range on the calling host thread (a timeline tool shows which launches a call or a layer pass enqueued; for a
+// captured step the ranges cover the capture, the replays appear under the range of the call that launches the graph)
+struct NvtxRange {
+    explicit NvtxRange(const char* what, int k = -1) {
+        if (k < 0) { nvtxRangePushA(what); return; }
+        char buf[48];
+        snprintf(buf, sizeof buf, "%s %d", what, k);
+        nvtxRangePushA(buf);
+    }
+    ~NvtxRange() { nvtxRangePop(); }
+    NvtxRange(const NvtxRange&) = delete;
+    NvtxRange& operator=(const NvtxRange&) = delete;
+};
 
 // ---------------------------------------------------------------------------------------------
 // Launch shapes.  The layer kernels are persistent: warps take units in a grid-stride loop.  The number of
@@ -622,6 +638,7 @@ void enqueue_backward_chain(sdnn* h, int ld) {
         for (int q = 0; q < h->n_side; ++q) cudaStreamWaitEvent(h->side_streams[q], h->ev_fork, 0);
         cudaEventRecord(h->ev_delta[h->L - 1], h->stream);
         for (int k = h->L - 1; k >= 0; --k) {
+            NvtxRange pass("backward layer", k + 1);
             cudaStream_t side = h->side_streams[k % h->n_side];
             cudaStreamWaitEvent(side, h->ev_delta[k], 0);
             h->launch_stream = side;
@@ -637,7 +654,10 @@ void enqueue_backward_chain(sdnn* h, int ld) {
             cudaStreamWaitEvent(h->stream, h->ev_side_join[q], 0);
         }
     } else {
-        for (int k = h->L - 1; k >= 0; --k) launch_backward(h, k, ld);
+        for (int k = h->L - 1; k >= 0; --k) {
+            NvtxRange pass("backward layer", k + 1);
+            launch_backward(h, k, ld);
+        }
     }
 }
 
@@ -648,9 +668,15 @@ void enqueue_backward_chain(sdnn* h, int ld) {
 void enqueue_step_body(sdnn* h, int ld, unsigned flags, bool averaged) {
     const size_t tile = (size_t)h->N * ld;
     cudaEventRecordWithFlags(h->ev[0], h->stream, flags);
-    for (int k = 0; k < h->L; ++k)
-        launch_forward(h, k, h->d_acts + (size_t)k * tile, h->d_acts + (size_t)(k + 1) * tile, ld, ld);
+    {
+        NvtxRange chain("sdnn forward chain");
+        for (int k = 0; k < h->L; ++k) {
+            NvtxRange pass("forward layer", k + 1);
+            launch_forward(h, k, h->d_acts + (size_t)k * tile, h->d_acts + (size_t)(k + 1) * tile, ld, ld);
+        }
+    }
     cudaEventRecordWithFlags(h->ev[1], h->stream, flags);
+    NvtxRange chain("sdnn backward chain");
     if (!averaged) {
         launch_output_gradient(h, ld);
         enqueue_backward_chain(h, ld);
@@ -673,6 +699,7 @@ void enqueue_step_body(sdnn* h, int ld, unsigned flags, bool averaged) {
 }
 
 int train_step_device(sdnn* h, const float* x0, const float* target, int B, float eta, float* loss_out, bool averaged = false) {
+    NvtxRange call(averaged ? "sdnn_train_step_averaged" : "sdnn_train_step");
     const int ld = padded_width(B);
     h->fwd_pdl = PDL_EARLY;
     if (averaged) {
@@ -763,6 +790,7 @@ int alloc_lane(sdnn* h, InferLane& ln, bool own_stream) {
 // One tile of inference on device buffers, on lane `ln`: x0 [cnt][N] -> outputs for these cnt inputs.
 int infer_tile(sdnn* h, InferLane& ln, const float* x0, int cnt, float* y_out, int* cnt_out, int* idx_out, long long capacity,
                bool want_sets) {
+    NvtxRange call("sdnn inference tile");
     const int ld = h->ld_max;
     const int cols = padded_width(cnt);
     cudaStream_t st = ln.stream;
@@ -792,6 +820,7 @@ int infer_tile(sdnn* h, InferLane& ln, const float* x0, int cnt, float* y_out, i
         h->live_lane = (int)(&ln - h->lane);
     } else {
         for (int k = 0; k < h->L; ++k) {
+            NvtxRange pass("forward layer", k + 1);
             if (h->lay[k].windowed) launch_forward_window(h, k, ln.tile[cur], ln.tile[cur ^ 1], ld, cols);
             else launch_forward(h, k, ln.tile[cur], ln.tile[cur ^ 1], ld, cols);
             cur ^= 1;
@@ -1982,6 +2011,7 @@ extern "C" int sdnn_probe_smem_gather_rate(int32_t row_bytes, int32_t cluster_si
 namespace {
 
 static __device__ __align__(256) float g_noalloc_scratch[2 * SDNN_NOALLOC_MAX_TILE_FLOATS];
+static __device__ unsigned long long g_noalloc_bad_columns;      // out-of-range column indices met so far (never followed)
 
 // tile geometry of this entry point (plain CSR kernel: 4 batch entries per lane, chunks of 128 columns)
 int noalloc_padded_width(int b) {
@@ -1992,8 +2022,9 @@ int noalloc_padded_width(int b) {
 
 constexpr int kMaxDevices = 64;
 float* g_noalloc_ptr[kMaxDevices] = {};      // per device: address of g_noalloc_scratch on that device
+unsigned long long* g_noalloc_bad_ptr[kMaxDevices] = {};
 
-int noalloc_scratch(float** out) {
+int noalloc_scratch(float** out, unsigned long long** bad_out) {
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return cuda_fail(nullptr, e, "cudaGetDevice");
@@ -2004,22 +2035,25 @@ int noalloc_scratch(float** out) {
         {
             p = g_noalloc_ptr[dev];
             if (!p) {
+                unsigned long long* bad = nullptr;
                 e = cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_noalloc_scratch);
-                if (e == cudaSuccess) g_noalloc_ptr[dev] = p; else p = nullptr;
+                if (e == cudaSuccess) e = cudaGetSymbolAddress(reinterpret_cast<void**>(&bad), g_noalloc_bad_columns);
+                if (e == cudaSuccess) { g_noalloc_bad_ptr[dev] = bad; g_noalloc_ptr[dev] = p; } else p = nullptr;
             }
         }
         if (!p) return cuda_fail(nullptr, e, "cudaGetSymbolAddress(scratch)");
     }
     *out = p;
+    *bad_out = g_noalloc_bad_ptr[dev];
     return SDNN_OK;
 }
 
 template <int G>
 void noalloc_forward_g(cudaStream_t st, const int* rp, const int* col, const float* val, const float* bias,
-                       const float* xin, float* xout, int n, int ld, int chunks, float clamp) {
+                       const float* xin, float* xout, int n, int ld, int chunks, float clamp, unsigned long long* bad) {
     const int rows_per_block = 8 * (32 / G);
     dim3 grid((n + rows_per_block - 1) / rows_per_block, chunks);
-    forward_csr_kernel<G><<<grid, 256, 0, st>>>(rp, col, val, bias, xin, xout, n, ld, clamp);
+    forward_csr_kernel<G><<<grid, 256, 0, st>>>(rp, col, val, bias, xin, xout, n, ld, clamp, bad);
 }
 
 }  // namespace
@@ -2047,7 +2081,8 @@ extern "C" int sdnn_infer_noalloc(int32_t n_layers, int32_t n_neurons, const int
         if (layer_offset[l] < 0 || (layer_offset[l] & 3)) return fail(nullptr, SDNN_ERR_INVALID_ARG, "layer_offset[%d] must be a non-negative multiple of 4", l);
 
     float* scratch = nullptr;
-    int rc = noalloc_scratch(&scratch);
+    unsigned long long* bad = nullptr;
+    int rc = noalloc_scratch(&scratch, &bad);
     if (rc) return rc;
     float* tile[2] = {scratch, scratch + SDNN_NOALLOC_MAX_TILE_FLOATS};
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -2063,12 +2098,12 @@ extern "C" int sdnn_infer_noalloc(int32_t n_layers, int32_t n_neurons, const int
         const float* val = values + layer_offset[l];
         const float* b = bias + (size_t)l * n_neurons;
         switch (q.g) {
-            case 1: noalloc_forward_g<1>(st, rp, col, val, b, tile[cur], tile[cur ^ 1], n_neurons, ld, q.chunks, clamp); break;
-            case 2: noalloc_forward_g<2>(st, rp, col, val, b, tile[cur], tile[cur ^ 1], n_neurons, ld, q.chunks, clamp); break;
-            case 4: noalloc_forward_g<4>(st, rp, col, val, b, tile[cur], tile[cur ^ 1], n_neurons, ld, q.chunks, clamp); break;
-            case 8: noalloc_forward_g<8>(st, rp, col, val, b, tile[cur], tile[cur ^ 1], n_neurons, ld, q.chunks, clamp); break;
-            case 16: noalloc_forward_g<16>(st, rp, col, val, b, tile[cur], tile[cur ^ 1], n_neurons, ld, q.chunks, clamp); break;
-            default: noalloc_forward_g<32>(st, rp, col, val, b, tile[cur], tile[cur ^ 1], n_neurons, ld, q.chunks, clamp); break;
+            case 1: noalloc_forward_g<1>(st, rp, col, val, b, tile[cur], tile[cur ^ 1], n_neurons, ld, q.chunks, clamp, bad); break;
+            case 2: noalloc_forward_g<2>(st, rp, col, val, b, tile[cur], tile[cur ^ 1], n_neurons, ld, q.chunks, clamp, bad); break;
+            case 4: noalloc_forward_g<4>(st, rp, col, val, b, tile[cur], tile[cur ^ 1], n_neurons, ld, q.chunks, clamp, bad); break;
+            case 8: noalloc_forward_g<8>(st, rp, col, val, b, tile[cur], tile[cur ^ 1], n_neurons, ld, q.chunks, clamp, bad); break;
+            case 16: noalloc_forward_g<16>(st, rp, col, val, b, tile[cur], tile[cur ^ 1], n_neurons, ld, q.chunks, clamp, bad); break;
+            default: noalloc_forward_g<32>(st, rp, col, val, b, tile[cur], tile[cur ^ 1], n_neurons, ld, q.chunks, clamp, bad); break;
         }
         cur ^= 1;
     }
@@ -2078,5 +2113,14 @@ extern "C" int sdnn_infer_noalloc(int32_t n_layers, int32_t n_neurons, const int
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(nullptr, e, "kernel launch");
+    return SDNN_OK;
+}
+
+extern "C" int sdnn_infer_noalloc_bad_columns(int64_t* count_out) {
+    if (!count_out) return fail(nullptr, SDNN_ERR_INVALID_ARG, "count_out is NULL");
+    unsigned long long v = 0;
+    cudaError_t e = cudaMemcpyFromSymbol(&v, g_noalloc_bad_columns, sizeof v);      // waits for the work enqueued so far
+    if (e != cudaSuccess) return cuda_fail(nullptr, e, "cudaMemcpyFromSymbol");
+    *count_out = (int64_t)v;
     return SDNN_OK;
 }

@@ -88,6 +88,32 @@ def test_noalloc_inference_on_ragged_rows_and_tiny_batches_matches_the_oracle(cn
         check_close(got.cpu().numpy(), want, f"{cnt} inputs")
 
 
+def test_noalloc_counts_and_skips_out_of_range_columns():
+    """The entry point cannot validate device arrays on the host; its kernel does not follow a column index outside
+    [0, n) and counts it.  Two corrupted entries (one negative, one too large), each seen by every input chunk once."""
+    torch = pytest.importorskip("torch")
+    assert torch.cuda.is_available()
+    import paper_2104_11805_b200 as pkg
+    from paper_2104_11805_b200.build import build_library
+    build_library()
+    spec = gen.CFG2.scaled(1024, 2).live()
+    rp, col, val, bias = gen.network(spec)
+    bad_col = [c.copy() for c in col]
+    bad_col[0][5] = -3
+    bad_col[1][77] = spec.n + 10
+    good_val = [v.copy() for v in val]
+    good_val[0][5] = 0.0; good_val[1][77] = 0.0                  # the net the kernel effectively evaluates
+    offsets = np.arange(2, dtype=np.int64) * spec.nnz_per_layer
+    d_rp, d_col, d_val = (torch.from_numpy(a).cuda() for a in (np.stack(rp), np.concatenate(bad_col), np.concatenate(val)))
+    d_bias = torch.from_numpy(np.stack(bias)).cuda()
+    x0 = gen.inputs(spec, 16)
+    got = torch.empty((16, spec.n), device="cuda")
+    before = pkg.infer_noalloc_bad_columns()
+    pkg.infer_noalloc(2, spec.n, d_rp, d_col, d_val, offsets, d_bias, torch.from_numpy(x0).cuda(), 16, got)
+    assert pkg.infer_noalloc_bad_columns() - before == 2
+    check_close(got.cpu().numpy(), OracleNet(rp, col, good_val, bias).infer(x0), "bad entries skipped")
+
+
 def test_noalloc_rejects_sizes_beyond_the_builtin_scratch():
     import paper_2104_11805_b200 as pkg
     from paper_2104_11805_b200.build import build_library

@@ -344,6 +344,9 @@ def main():
     ap.add_argument("--pattern", default=None, choices=["uniform", "windowed"],
                     help="same recipe with the other pattern family: columns uniform over [0, N), or over the 1024 columns "
                          "that a block of 1024 rows shares (the locality a good neuron order gives)")
+    ap.add_argument("--shuffle", action="store_true",
+                    help="renumber the neurons of every inner layer at random (NetSpec.shuffled): the same function with whatever "
+                         "structure the pattern has hidden, to be recovered with --flags 0x100 (SDNN_FLAG_REORDER)")
     ap.add_argument("--averaged", action="store_true",
                     help="train workloads: the averaged form of the minibatch step (one batch-averaged gradient vector is "
                          "backpropagated; sdnn_train_step_averaged) instead of the exact minibatch step")
@@ -375,6 +378,8 @@ def main():
     if args.pattern and args.pattern != spec.pattern:
         import dataclasses
         spec = dataclasses.replace(spec, name=f"{spec.name}-{args.pattern}", pattern=args.pattern, window=min(1024, spec.n))
+    if args.shuffle and not spec.shuffle:
+        spec = spec.shuffled()
     if args.layers:
         spec = spec.sliced(args.layers)
     if args.inputs and kind == "infer":

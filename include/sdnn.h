@@ -90,15 +90,16 @@ typedef enum {
                                     /* pattern) is left as it is.  Everything                                             */
                                     /* the caller sees keeps the caller's numbering: inputs, outputs, id lists,           */
                                     /* sdnn_get_weights / sdnn_set_weights.  The layers are analysed in sdnn_finalize;   */
-                                    /* until then the handle keeps a host copy of every loaded layer.  Inference handles */
-                                    /* only (SDNN_ERR_UNIMPLEMENTED with train = 1); not together with                    */
-                                    /* SDNN_FLAG_SKIP_DEAD.                                                               */
+                                    /* until then the handle keeps a host copy of every loaded layer.  Inference and     */
+                                    /* training handles (targets, activations, deltas and gradients keep the caller's   */
+                                    /* numbering too); not together with SDNN_FLAG_SKIP_DEAD.                             */
 
 #define SDNN_FLAG_SMEM_WINDOWS 0x200u /* with SDNN_FLAG_REORDER: run the layers for which groups were found with a kernel  */
                                     /* that copies each group's window of the activation tile into shared memory and     */
                                     /* gathers from there (forward_window_kernel) instead of the default kernels, which   */
                                     /* gather the same window out of L1/L2.  Measured slower on B200 for wide inference   */
-                                    /* tiles, hence opt-in; kept so that the comparison can be repeated.                  */
+                                    /* tiles, hence opt-in; kept so that the comparison can be repeated.  Inference       */
+                                    /* handles only (SDNN_ERR_UNIMPLEMENTED with train = 1).                              */
 
 #define SDNN_ACT_CLAMPED_RELU 0
 #define SDNN_ACT_SIGMOID      1

@@ -826,13 +826,16 @@ __device__ __forceinline__ void backward_row_units(const Sliced m, float* __rest
     if (nch > 0) load_idx<CPS>(c, m, base);
     Lane<V> h0, h1;       // delta^k[i,:] (or S_k[i,:]) and, FROM_S, x^k[i,:]
     lane_fill(h0, 0.0f); lane_fill(h1, 0.0f);
-    if (item < n) { lane_load(h0, tile_row(dk + boff, item, pitch)); if (FROM_S) lane_load(h1, tile_row(xk + boff, item, pitch)); }
+    // tile row of stored row `item`: its neuron's number (the stored rows of a regrouped layer are not in neuron order)
+    int lab = (item < n && m.out) ? m.out[item] : item;
+    if (item < n) { lane_load(h0, tile_row(dk + boff, lab, pitch)); if (FROM_S) lane_load(h1, tile_row(xk + boff, lab, pitch)); }
 
     while (u < nunits) {
         const int nu = u + stride;
         int nitem, nbase, nnch;
         SDNN_UNIT_SHAPE(m, nu, nunits, nitem, nbase, nnch)
         const int nlen = (nitem < n) ? m.len[nitem] : 0;
+        const int nlab = (nitem < n && m.out) ? m.out[nitem] : nitem;
         if (nu < nunits && lane == 0) prefetch_unit(m, nu, RPW, n, UPS);
         Lane<V> nh0, nh1;
         lane_fill(nh0, 0.0f); lane_fill(nh1, 0.0f);
@@ -841,9 +844,9 @@ __device__ __forceinline__ void backward_row_units(const Sliced m, float* __rest
             if (FROM_S) {
                 Lane<V> z;
                 lane_fill(z, 0.0f);
-                lane_store(tile_row(dk + boff, item, pitch), z);
+                lane_store(tile_row(dk + boff, lab, pitch), z);
                 lane_mask(d, h1, act, clamp);
-                if (DBG) lane_store(tile_row(dbg_delta + boff, item, pitch), d);
+                if (DBG) lane_store(tile_row(dbg_delta + boff, lab, pitch), d);
             }
             if (update_bias) {       // bias read as one more column of W^k whose input is the constant 1
                 const float bg = group_sum<G>(lane_sum(d), gmask1);
@@ -858,7 +861,7 @@ __device__ __forceinline__ void backward_row_units(const Sliced m, float* __rest
         const int lim = len - ((G >= 4) ? (sub & 3) : (G == 2) ? 2 * sub : 0);
 #define SDNN_ROW_NEXT                                                                                    \
         if (nnch > 0) load_idx<CPS>(c, m, nbase);                                                        \
-        if (nitem < n) { lane_load(nh0, tile_row(dk + boff, nitem, pitch)); if (FROM_S) lane_load(nh1, tile_row(xk + boff, nitem, pitch)); }
+        if (nitem < n) { lane_load(nh0, tile_row(dk + boff, nlab, pitch)); if (FROM_S) lane_load(nh1, tile_row(xk + boff, nlab, pitch)); }
 #define SDNN_SCAT(C, W, Q) if ((Q) < len) lane_red_add(tile_row(sg, C, pitch), W, d);
         for (int t = 0; t < nch; t += CPS) {
             float4 w[CPS];
@@ -887,7 +890,7 @@ __device__ __forceinline__ void backward_row_units(const Sliced m, float* __rest
         if (nch == 0) { SDNN_ROW_NEXT }
 #undef SDNN_ROW_NEXT
 #undef SDNN_SCAT
-        u = nu; item = nitem; base = nbase; nch = nnch; len = nlen; h0 = nh0; h1 = nh1;
+        u = nu; item = nitem; base = nbase; nch = nnch; len = nlen; h0 = nh0; h1 = nh1; lab = nlab;
     }
 }
 
@@ -1058,7 +1061,7 @@ backward_row_ep_kernel(Sliced m, float* __restrict__ bias, const float* __restri
     const float step = sp->eta * inv_b;
     Lane<4> d;
     lane_fill(d, 0.0f);
-    if (e.item < n) lane_load(d, dk + (size_t)e.item * 4);
+    if (e.item < n) lane_load(d, dk + (size_t)(m.out ? m.out[e.item] : e.item) * 4);
     if (update_bias && e.h == 0 && e.item < n) bias[e.item] -= step * lane_sum(d);
     for (int t0 = 0; t0 < e.nch; t0 += 2 * EP_IT) {
         float4 w[EP_IT];
@@ -1095,7 +1098,8 @@ backward_row_ep_kernel(Sliced m, float* __restrict__ bias, const float* __restri
 // Fills the transposed copy's values from the row-major copy: entry (column j, row i) of the transposed
 // copy is looked up by binary search in row i (ascending columns).  One warp per transposed unit.
 // With `mismatch` non-NULL nothing is written; entries whose bits differ from the row-major copy are counted.
-__global__ void mirror_values_kernel(Sliced rows, Sliced cols, int n, unsigned long long* mismatch) {
+// row_of (or NULL): stored row of the row-major copy that holds neuron i, for layers whose rows were regrouped.
+__global__ void mirror_values_kernel(Sliced rows, Sliced cols, int n, unsigned long long* mismatch, const int* __restrict__ row_of) {
     const int cc = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (cc >= n) return;
     const int len = cols.len[cc];
@@ -1103,7 +1107,7 @@ __global__ void mirror_values_kernel(Sliced rows, Sliced cols, int n, unsigned l
     const int base = cols.slice_off[cc / SLICE] + (cc % SLICE) * 4;
     for (int q = threadIdx.x & 31; q < len; q += 32) {
         const int pos = base + (q >> 2) * CHUNK_ROW + (q & 3);
-        const int i = load_idx1(cols, pos);
+        const int i = row_of ? row_of[load_idx1(cols, pos)] : load_idx1(cols, pos);
         const int rb = rows.slice_off[i / SLICE] + (i % SLICE) * 4;
         int lo = 0, hi = rows.len[i] - 1, at = -1;
         while (lo <= hi) {

@@ -67,6 +67,7 @@ struct LayerMem {
     std::vector<int> row_src;              // [N] stored row -> caller's row (empty: identity)
     std::vector<int> entry_src;            // [nnz] entry in stored order (stored rows, their entries in stored order) -> caller's position
     int* r_out = nullptr;                  // grouped layer in the default layout: tile row each stored row writes (device, [N])
+    int* r_row_of = nullptr;               // ... and its inverse: stored row that holds neuron (tile row) i (device, [N])
     // windowed layer: rows grouped by shared columns, the group's window staged in shared memory (forward_window_kernel)
     bool windowed = false;
     int groups = 0, max_wlen = 0;
@@ -148,6 +149,7 @@ struct sdnn {
     int grouped_layers = 0;             // layers for which the analysis found groups of rows sharing a window of columns
     std::vector<HostLayer> pending;     // their arrays until then
     int* d_in_label = nullptr;          // [N] tile row of input neuron i (NULL: identity)
+    std::vector<std::vector<int>> labels;   // [L + 1] host: tile row of neuron i at boundary k (x^k, delta^k); empty = identity
     int windowed_layers = 0;
     bool compaction = false;            // SDNN_FLAG_SKIP_DEAD asked for; effective while no bias is positive
     std::vector<char> bias_nonpositive; // per layer
@@ -246,8 +248,8 @@ int validate_cfg(const sdnn_config* cfg) {
     if (cfg->train && cfg->max_batch > 128) return fail(nullptr, SDNN_ERR_INVALID_ARG, "training handles support max_batch <= 128");
     if ((cfg->flags & SDNN_FLAG_BWD_ATOMICS) && (cfg->flags & SDNN_FLAG_BWD_CSC))
         return fail(nullptr, SDNN_ERR_INVALID_ARG, "choose one backward strategy");
-    if ((cfg->flags & SDNN_FLAG_REORDER) && cfg->train)
-        return fail(nullptr, SDNN_ERR_UNIMPLEMENTED, "SDNN_FLAG_REORDER is implemented for inference handles (train = 0)");
+    if ((cfg->flags & SDNN_FLAG_SMEM_WINDOWS) && cfg->train)
+        return fail(nullptr, SDNN_ERR_UNIMPLEMENTED, "SDNN_FLAG_SMEM_WINDOWS is implemented for inference handles (train = 0)");
     if ((cfg->flags & SDNN_FLAG_SMEM_WINDOWS) && !(cfg->flags & SDNN_FLAG_REORDER))
         return fail(nullptr, SDNN_ERR_INVALID_ARG, "SDNN_FLAG_SMEM_WINDOWS needs SDNN_FLAG_REORDER");
     if ((cfg->flags & SDNN_FLAG_REORDER) && (cfg->flags & SDNN_FLAG_SKIP_DEAD))
@@ -715,7 +717,7 @@ int train_step_device(sdnn* h, const float* x0, const float* target, int B, floa
         set_step_params_kernel<<<1, 1, 0, h->stream>>>(h->d_sp, eta, B, h->d_loss);
         count_launch(h);
     }
-    launch_transpose_in(h, x0, h->d_acts, B, ld, ld);
+    launch_transpose_in(h, x0, h->d_acts, B, ld, ld, h->d_in_label);
     launch_transpose_in(h, target, h->d_yt, B, ld, ld);
     if (h->cfg.flags & SDNN_FLAG_NO_GRAPH) {
         enqueue_step_body(h, ld, cudaEventRecordDefault, averaged);
@@ -948,7 +950,8 @@ void sliced_to_csr(const sdnn* h, const LayerMem& lm, const std::vector<float>& 
 
 int refresh_mirror(sdnn* h, int layer, unsigned long long* mismatch_dev) {
     const int wpb = 8;
-    mirror_values_kernel<<<(h->N + wpb - 1) / wpb, wpb * 32, 0, h->stream>>>(rows_of(h, layer), cols_of(h, layer), h->N, mismatch_dev);
+    mirror_values_kernel<<<(h->N + wpb - 1) / wpb, wpb * 32, 0, h->stream>>>(rows_of(h, layer), cols_of(h, layer), h->N, mismatch_dev,
+                                                                             (const int*)h->lay[layer].r_row_of);
     CU(h, cudaGetLastError());
     return SDNN_OK;
 }
@@ -975,7 +978,9 @@ int upload_indices(sdnn* h, int* dst, const std::vector<int>& src) {      // syn
 }
 
 // Lays out one validated layer (caller's or reordered CSR, host arrays) in the kernels' sliced format and uploads it.
-int upload_layer(sdnn* h, int layer, const int32_t* row_ptr, const int32_t* col_idx, const float* values, const float* bias) {
+// out_label (host, or NULL): tile row that each given row writes, for a layer whose rows are stored group by group.
+int upload_layer(sdnn* h, int layer, const int32_t* row_ptr, const int32_t* col_idx, const float* values, const float* bias,
+                 const int* out_label = nullptr) {
     int rc;
     CU(h, cudaSetDevice(h->device));
     const int N = h->N, NS = h->NS;
@@ -1013,6 +1018,16 @@ int upload_layer(sdnn* h, int layer, const int32_t* row_ptr, const int32_t* col_
         CU(h, cudaMemcpyAsync(lm.r_val, r_val.data(), (size_t)lm.r_elems * sizeof(float), cudaMemcpyHostToDevice, h->stream));
     }
 
+    if (out_label) {
+        std::vector<int> row_of(N);
+        for (int i = 0; i < N; ++i) row_of[out_label[i]] = i;
+        if ((rc = dev_alloc(h, &lm.r_out, (size_t)N, false))) return rc;
+        if ((rc = dev_alloc(h, &lm.r_row_of, (size_t)N, false))) return rc;
+        CU(h, cudaMemcpyAsync(lm.r_out, out_label, (size_t)N * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+        CU(h, cudaMemcpyAsync(lm.r_row_of, row_of.data(), (size_t)N * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+        CU(h, cudaStreamSynchronize(h->stream));
+    }
+
     // ---- transposed sliced copy (not needed for the first layer: delta^0 is never formed)
     std::vector<int> c_idx, c_len, order, c_off;
     if (h->mirror && layer > 0) {
@@ -1048,7 +1063,7 @@ int upload_layer(sdnn* h, int layer, const int32_t* row_ptr, const int32_t* col_
                     const int j = col_idx[p];
                     if (j < j0 || j >= j1) continue;
                     const int q = cursor[j - j0]++;
-                    c_idx[(size_t)sliced_pos(c_off.data(), place[j], q)] = i;
+                    c_idx[(size_t)sliced_pos(c_off.data(), place[j], q)] = out_label ? out_label[i] : i;      // the delta tile's row
                 }
         }
         if ((rc = alloc_indices(h, &lm.c_idx, (size_t)lm.c_elems))) return rc;
@@ -1207,12 +1222,7 @@ int build_grouped_layer(sdnn* h, int layer, const HostLayer& hl, const sdnn_reor
         }
     }
     lm.row_src = g.row_order;
-    int rc = upload_layer(h, layer, rp.data(), col.data(), val.data(), bias.data());
-    if (rc) return rc;
-    if ((rc = dev_alloc(h, &lm.r_out, (size_t)N, false))) return rc;
-    CU(h, cudaMemcpyAsync(lm.r_out, out.data(), (size_t)N * sizeof(int), cudaMemcpyHostToDevice, h->stream));
-    CU(h, cudaStreamSynchronize(h->stream));
-    return SDNN_OK;
+    return upload_layer(h, layer, rp.data(), col.data(), val.data(), bias.data(), out.data());
 }
 
 // A layer without structure keeps the default layout; only its rows move to where the next layer's grouping put its
@@ -1257,6 +1267,8 @@ int build_reordered(sdnn* h) {
         return (boundary < L && G[boundary].structured) ? &G[boundary].col_label : nullptr;
     };
     int rc;
+    h->labels.assign(L + 1, std::vector<int>());
+    for (int k = 0; k <= L; ++k) if (labels(k)) h->labels[k] = *labels(k);
     if (labels(0)) {
         if ((rc = dev_alloc(h, &h->d_in_label, (size_t)N, false))) return rc;
         CU(h, cudaMemcpyAsync(h->d_in_label, labels(0)->data(), (size_t)N * sizeof(int), cudaMemcpyHostToDevice, h->stream));
@@ -1731,15 +1743,16 @@ int sdnn_mirror_mismatches(sdnn_t* h, int32_t layer, int64_t* count_out) {
     return SDNN_OK;
 }
 
-static int fetch_tile(sdnn_t* h, const float* tile, float* out, int B, int ld) {
-    // tile [N][ld] on the device -> out [B][N] on the host
+static int fetch_tile(sdnn_t* h, const float* tile, float* out, int B, int ld, int boundary) {
+    // tile [N][ld] on the device -> out [B][N] on the host, neuron i read from the tile row it was given at set-up
     const int N = h->N;
+    const std::vector<int>* lab = (boundary < (int)h->labels.size() && !h->labels[boundary].empty()) ? &h->labels[boundary] : nullptr;
     std::vector<float> tmp((size_t)N * ld);
     CU(h, cudaSetDevice(h->device));
     CU(h, cudaStreamSynchronize(h->stream));
     CU(h, cudaMemcpy(tmp.data(), tile, tmp.size() * sizeof(float), cudaMemcpyDeviceToHost));
     for (int b = 0; b < B; ++b)
-        for (int i = 0; i < N; ++i) out[(size_t)b * N + i] = tmp[(size_t)i * ld + b];
+        for (int i = 0; i < N; ++i) out[(size_t)b * N + i] = tmp[(size_t)(lab ? (*lab)[i] : i) * ld + b];
     return SDNN_OK;
 }
 
@@ -1747,14 +1760,14 @@ int sdnn_get_activations(sdnn_t* h, int32_t layer, float* out) {
     if (!h || !out) return SDNN_ERR_INVALID_ARG;
     if (!h->stepped) return fail(h, SDNN_ERR_STATE, "no train step has run");
     if (layer < 0 || layer > h->L) return fail(h, SDNN_ERR_INVALID_ARG, "layer %d outside [0, %d]", layer, h->L);
-    return fetch_tile(h, h->d_acts + (size_t)layer * h->N * h->last_ld, out, h->last_b, h->last_ld);
+    return fetch_tile(h, h->d_acts + (size_t)layer * h->N * h->last_ld, out, h->last_b, h->last_ld, layer);
 }
 
 int sdnn_get_delta(sdnn_t* h, int32_t layer, float* out) {
     if (!h || !out) return SDNN_ERR_INVALID_ARG;
     if (!h->stepped || !h->d_dbg_delta) return fail(h, SDNN_ERR_STATE, "needs SDNN_FLAG_KEEP_DEBUG and a train step");
     if (layer < 1 || layer > h->L) return fail(h, SDNN_ERR_INVALID_ARG, "layer %d outside [1, %d]", layer, h->L);
-    return fetch_tile(h, h->d_dbg_delta + (size_t)(layer - 1) * h->N * h->last_delta_ld, out, h->last_delta_b, h->last_delta_ld);
+    return fetch_tile(h, h->d_dbg_delta + (size_t)(layer - 1) * h->N * h->last_delta_ld, out, h->last_delta_b, h->last_delta_ld, layer);
 }
 
 int sdnn_get_gradient(sdnn_t* h, int32_t layer, float* out) {
@@ -1767,7 +1780,9 @@ int sdnn_get_gradient(sdnn_t* h, int32_t layer, float* out) {
     if (lm.r_elems && lm.r_grad) {
         std::vector<float> tmp((size_t)lm.r_elems);
         CU(h, cudaMemcpy(tmp.data(), lm.r_grad, tmp.size() * sizeof(float), cudaMemcpyDeviceToHost));
-        sliced_to_csr(h, lm, tmp, out);
+        std::vector<float> stored((size_t)h->nnz[layer - 1]);
+        sliced_to_csr(h, lm, tmp, stored.data());
+        stored_to_caller(lm, stored, out, h->nnz[layer - 1]);
     }
     return SDNN_OK;
 }

@@ -758,7 +758,7 @@ def test_infer_reordered_ragged_blocks(torch_cuda, cnt, mode):
     infer_parity(torch_cuda, (rps, cols, vals, biases), x0, 64, expect_nonempty=True, flags=REORDER_MODES[mode], expect_grouped=4)
 
 
-def test_reorder_flag_leaves_an_unstructured_net_alone_and_is_refused_for_training(torch_cuda):
+def test_reorder_flag_leaves_an_unstructured_net_alone(torch_cuda):
     pkg = sdnn()
     spec = gen.CFG2.scaled(4096, 4).live()
     infer_parity(torch_cuda, gen.network(spec), gen.inputs(spec, 100), 128, expect_nonempty=True, flags=pkg.FLAG_REORDER,
@@ -767,8 +767,61 @@ def test_reorder_flag_leaves_an_unstructured_net_alone_and_is_refused_for_traini
         pkg.Sdnn.create(*gen.network(spec), max_batch=16, flags=pkg.FLAG_SMEM_WINDOWS)       # needs FLAG_REORDER
     assert ei.value.code == -1
     with pytest.raises(pkg.SdnnError) as ei:
-        pkg.Sdnn.create(*gen.network(spec), max_batch=16, train=True, flags=pkg.FLAG_REORDER)
-    assert ei.value.code == -6
+        pkg.Sdnn.create(*gen.network(spec), max_batch=16, train=True, flags=pkg.FLAG_REORDER | pkg.FLAG_SMEM_WINDOWS)
+    assert ei.value.code == -6          # the shared-memory window kernel exists for the forward pass of inference handles only
+
+
+@pytest.mark.parametrize("bwd", sorted(BWD_MODES))
+@pytest.mark.parametrize("B", [1, 4, 16, 64])
+def test_train_reordered_hidden_blocks(torch_cuda, B, bwd):
+    """Training on a net whose block structure is hidden behind random renumberings, with SDNN_FLAG_REORDER: the rows of
+    every layer are regrouped and the neurons renumbered inside the library, while activations, deltas, gradients, weights
+    and biases are compared with the oracle in the caller's numbering after every step (every backward realisation; the
+    kernels for B <= 4 and the common ones)."""
+    pkg = sdnn()
+    spec = block_spec(1024, 4, 256).shuffled()
+    rp, col, val, bias = gen.network(spec)
+    rng = np.random.default_rng(B)
+    bias = [(0.05 * rng.standard_normal(spec.n)).astype(np.float32) for _ in range(4)]       # biases that tell the rows apart
+    st = train_parity(torch_cuda, (rp, col, val, bias), batches_for(spec, B, 2), eta=1e-2, update_bias=True,
+                      flags=BWD_MODES[bwd] | pkg.FLAG_REORDER, expect_live=True)
+    assert st["entries"] > 0
+
+
+def test_train_reordered_mixed_net_in_the_benchmark_launch_configuration(torch_cuda):
+    """Structured and unstructured layers mixed, default flags plus SDNN_FLAG_REORDER, no debug buffers, the step as one
+    CUDA graph; loss, weights in the caller's order and the consistency of the two weight copies after each of two steps;
+    then inference on the same handle."""
+    torch = torch_cuda
+    pkg = sdnn()
+    n, k, B = 2048, 32, 16
+    blocks = block_spec(n, 5, 512).shuffled()
+    uniform = gen.NetSpec("uniform", n, 5, values="normal", sigma=(2.0 / k) ** 0.5, bias=0.0, config_id=2)
+    pick = [uniform, blocks, blocks, uniform, blocks]
+    rp = [gen.row_ptr(blocks)] * 5
+    col = [gen.layer_pattern(sp, l) for l, sp in enumerate(pick)]
+    val = [gen.layer_values(sp, l) for l, sp in enumerate(pick)]
+    bias = [gen.layer_bias(sp, l) for l, sp in enumerate(pick)]
+    h = pkg.Sdnn.create(rp, col, val, bias, max_batch=B, train=True, flags=pkg.FLAG_REORDER)
+    assert h.grouped_layers() == 3
+    ora = OracleNet(rp, col, val, bias)
+    for step, (x0, y) in enumerate(batches_for(blocks, B, 2)):
+        if step:
+            ora.quantize_state()
+            for l in range(5):
+                h.set_weights(l, ora.w[l], ora.bias[l])
+        loss = h.train_step(torch.from_numpy(x0).cuda(), torch.from_numpy(y).cuda(), B, 1e-3, want_loss=True)
+        out = ora.train_step(x0, y, 1e-3, keep=("grad",))
+        assert abs(loss - out["loss"]) <= TOL * abs(out["loss"])
+        assert all(np.any(g != 0.0) for g in out["grad"])
+        for l in range(5):
+            check_close(h.get_weights(l, want_bias=False), ora.w[l], f"step {step} W^{l + 1}")
+            assert h.mirror_mismatches(l) == 0
+    xin = gen.inputs(blocks, 40)
+    yd = torch.empty((40, n), dtype=torch.float32, device="cuda")
+    h.infer_batch(torch.from_numpy(xin).cuda(), 40, yd, None, None, 0)
+    check_close(yd.cpu().numpy(), ora.infer(xin), "inference on the trained, reordered handle")
+    h.destroy()
 
 
 @pytest.mark.parametrize("mode", sorted(REORDER_MODES))

@@ -366,21 +366,33 @@ forward_csr_kernel(const int* __restrict__ row_ptr, const int* __restrict__ col,
 // (padding has index 0 and value 0), which keeps the lanes of a warp converged.  The indices of a step are
 // loaded one step ahead (while the previous step's gathers are in flight, also across the boundary between
 // two units), so that a step costs one memory round trip, not two dependent ones.
-// the four indices of one chunk of one row, at element offset `at` (a multiple of 4) of the index array
-__device__ __forceinline__ int4 load_idx4(const Sliced& m, int at) {
-    if (m.idx16) {
-        const uint2 v = __ldcs(reinterpret_cast<const uint2*>(reinterpret_cast<const unsigned short*>(m.idx) + at));
-        return make_int4((int)(v.x & 0xffffu), (int)(v.x >> 16), (int)(v.y & 0xffffu), (int)(v.y >> 16));
-    }
-    return __ldcs(reinterpret_cast<const int4*>(m.idx + at));
+// The four indices of one chunk of one row as they are stored: four 32-bit words, or (I16: nets of at most 65536
+// neurons) two words holding four 16-bit indices.  load_idx4 does not touch what it loads, so that the loads of several
+// chunks leave back to back (unpacking at the load would make every load wait for its own data before the next one is
+// issued); idx_unpack turns a chunk into four indices where they are used.
+template <bool I16> struct IdxChunk;
+template <> struct IdxChunk<false> { int4 v; };
+template <> struct IdxChunk<true> { uint2 v; };
+__device__ __forceinline__ void idx_zero(IdxChunk<false>& c) { c.v = make_int4(0, 0, 0, 0); }
+__device__ __forceinline__ void idx_zero(IdxChunk<true>& c) { c.v = make_uint2(0u, 0u); }
+// `at`: element offset of the chunk in the index array, a multiple of 4
+__device__ __forceinline__ void load_idx4(IdxChunk<false>& c, const Sliced& m, int at) {
+    c.v = __ldcs(reinterpret_cast<const int4*>(m.idx + at));
+}
+__device__ __forceinline__ void load_idx4(IdxChunk<true>& c, const Sliced& m, int at) {
+    c.v = __ldcs(reinterpret_cast<const uint2*>(reinterpret_cast<const unsigned short*>(m.idx) + at));
+}
+__device__ __forceinline__ int4 idx_unpack(const IdxChunk<false>& c) { return c.v; }
+__device__ __forceinline__ int4 idx_unpack(const IdxChunk<true>& c) {
+    return make_int4((int)(c.v.x & 0xffffu), (int)(c.v.x >> 16), (int)(c.v.y & 0xffffu), (int)(c.v.y >> 16));
 }
 __device__ __forceinline__ int load_idx1(const Sliced& m, int at) {
     return m.idx16 ? (int)reinterpret_cast<const unsigned short*>(m.idx)[at] : m.idx[at];
 }
-template <int CPS>
-__device__ __forceinline__ void load_idx(int4 (&c)[CPS], const Sliced& m, int at) {
+template <int CPS, bool I16>
+__device__ __forceinline__ void load_idx(IdxChunk<I16> (&c)[CPS], const Sliced& m, int at) {
 #pragma unroll
-    for (int i = 0; i < CPS; ++i) c[i] = load_idx4(m, at + CHUNK_ROW * i);
+    for (int i = 0; i < CPS; ++i) load_idx4(c[i], m, at + CHUNK_ROW * i);
 }
 
 // asks for the slices that hold the rows of unit `u` (rpw consecutive rows) to be brought into L2
@@ -397,8 +409,9 @@ __device__ __forceinline__ void prefetch_unit(const Sliced& m, int u, int rpw, i
 }
 
 #define SDNN_GATHER_CHUNK(X, I, C, P, PITCH)                                                              \
-    lane_gather(X[4 * (I) + 0], tile_row(P, C.x, PITCH)); lane_gather(X[4 * (I) + 1], tile_row(P, C.y, PITCH)); \
-    lane_gather(X[4 * (I) + 2], tile_row(P, C.z, PITCH)); lane_gather(X[4 * (I) + 3], tile_row(P, C.w, PITCH));
+    { const int4 cu_ = idx_unpack(C);                                                                     \
+      lane_gather(X[4 * (I) + 0], tile_row(P, cu_.x, PITCH)); lane_gather(X[4 * (I) + 1], tile_row(P, cu_.y, PITCH)); \
+      lane_gather(X[4 * (I) + 2], tile_row(P, cu_.z, PITCH)); lane_gather(X[4 * (I) + 3], tile_row(P, cu_.w, PITCH)); }
 
 // Position of a group's item (matrix row, or position in the transposed copy) in unit U of matrix M: BASE =
 // element offset of its first chunk, NCH = chunks of its slice (even), ITEM = n for groups beyond the matrix
@@ -416,7 +429,7 @@ __device__ __forceinline__ void prefetch_unit(const Sliced& m, int u, int rpw, i
 // Persistent grid: a warp takes units (32/G consecutive rows) in a grid-stride loop.  One group of G lanes
 // per row; each lane accumulates V batch entries with fp32 FMAs in stored (ascending column) order.
 // While it works on a unit a warp asks for the entries of its next unit to be brought into L2.
-template <int G, int V, int CPS>
+template <int G, int V, int CPS, bool I16>
 __global__ void __launch_bounds__(256, CPS > 2 ? 1 : 2)
 forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict__ xin, float* __restrict__ xout,
                int n, int ld, float clamp, int act, int pdl, const int* __restrict__ ncols_dev, int* __restrict__ live_flags) {
@@ -439,10 +452,10 @@ forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict
     float b = (row < n) ? bias[row] : 0.0f;
     int orow = (row < n && m.out) ? m.out[row] : row;
     if (unit < nunits && lane == 0) prefetch_unit(m, unit, RPW, n, UPS);
-    int4 c[CPS];
+    IdxChunk<I16> c[CPS];
 #pragma unroll
-    for (int i = 0; i < CPS; ++i) c[i] = make_int4(0, 0, 0, 0);
-    if (nch > 0) load_idx<CPS>(c, m, base);
+    for (int i = 0; i < CPS; ++i) idx_zero(c[i]);
+    if (nch > 0) load_idx<CPS, I16>(c, m, base);
     if (pdl) grid_dependency_wait();
     if (pdl == 2) grid_launch_dependents();
     // compaction mode: only the first *ncols_dev columns of the tile still hold live inputs
@@ -468,15 +481,15 @@ forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict
             for (int i = 0; i < CPS; ++i) w[i] = __ldcs(reinterpret_cast<const float4*>(vp + (t + i) * CHUNK_ROW));
 #pragma unroll
             for (int i = 0; i < CPS; ++i) { SDNN_GATHER_CHUNK(x, i, c[i], xg, pitch) }
-            if (t + CPS < nch) load_idx<CPS>(c, m, base + (t + CPS) * CHUNK_ROW);
-            else if (nnch > 0) load_idx<CPS>(c, m, nbase);
+            if (t + CPS < nch) load_idx<CPS, I16>(c, m, base + (t + CPS) * CHUNK_ROW);
+            else if (nnch > 0) load_idx<CPS, I16>(c, m, nbase);
 #pragma unroll
             for (int i = 0; i < CPS; ++i) {
                 lane_fma(w[i].x, x[4 * i + 0], acc); lane_fma(w[i].y, x[4 * i + 1], acc);
                 lane_fma(w[i].z, x[4 * i + 2], acc); lane_fma(w[i].w, x[4 * i + 3], acc);
             }
         }
-        if (nch == 0 && nnch > 0) load_idx<CPS>(c, m, nbase);      // empty slice: nothing prefetched across the boundary yet
+        if (nch == 0 && nnch > 0) load_idx<CPS, I16>(c, m, nbase);      // empty slice: nothing prefetched across the boundary yet
         if (row < n) {
             lane_activate(acc, act, clamp);
             lane_store(tile_row(xout + boff, orow, pitch), acc);
@@ -729,7 +742,7 @@ struct BackwardArgs {
 };
 
 // Column units of the transposed realisation.
-template <int G, int V, int CPS>
+template <int G, int V, int CPS, bool I16>
 __device__ __forceinline__ void backward_col_units(const Sliced m, const float* __restrict__ xprev, const float* __restrict__ dk,
                                                    float* __restrict__ dprev, int n, float clamp, int act, float step, float inv_b,
                                                    int first, int stride) {
@@ -749,10 +762,10 @@ __device__ __forceinline__ void backward_col_units(const Sliced m, const float* 
     if (u < nunits && lane == 0) prefetch_unit(m, u, RPW, n, UPS);
     int len = 0, j = 0;
     if (item < n) { len = m.len[item]; j = m.order[item]; }
-    int4 c[CPS];
+    IdxChunk<I16> c[CPS];
 #pragma unroll
-    for (int i = 0; i < CPS; ++i) c[i] = make_int4(0, 0, 0, 0);
-    if (nch > 0) load_idx<CPS>(c, m, base);
+    for (int i = 0; i < CPS; ++i) idx_zero(c[i]);
+    if (nch > 0) load_idx<CPS, I16>(c, m, base);
     Lane<V> xj;
     lane_fill(xj, 0.0f);
     if (item < n) lane_load(xj, tile_row(xprev + boff, j, pitch));
@@ -768,7 +781,7 @@ __device__ __forceinline__ void backward_col_units(const Sliced m, const float* 
         lane_fill(acc, 0.0f);
         float* vp = val + base;
         const int lim = len - ((G >= 4) ? (sub & 3) : (G == 2) ? 2 * sub : 0);
-#define SDNN_COL_NEXT if (nnch > 0) load_idx<CPS>(c, m, nbase); if (nitem < n) lane_load(nxj, tile_row(xprev + boff, nj, pitch));
+#define SDNN_COL_NEXT if (nnch > 0) load_idx<CPS, I16>(c, m, nbase); if (nitem < n) lane_load(nxj, tile_row(xprev + boff, nj, pitch));
         for (int t = 0; t < nch; t += CPS) {
             float4 w[CPS];
             Lane<V> d[4 * CPS];
@@ -776,7 +789,7 @@ __device__ __forceinline__ void backward_col_units(const Sliced m, const float* 
             for (int i = 0; i < CPS; ++i) w[i] = ld_f4(vp + (t + i) * CHUNK_ROW);
 #pragma unroll
             for (int i = 0; i < CPS; ++i) { SDNN_GATHER_CHUNK(d, i, c[i], dg, pitch) }
-            if (t + CPS < nch) { load_idx<CPS>(c, m, base + (t + CPS) * CHUNK_ROW); }
+            if (t + CPS < nch) { load_idx<CPS, I16>(c, m, base + (t + CPS) * CHUNK_ROW); }
             else { SDNN_COL_NEXT }
 #pragma unroll
             for (int i = 0; i < CPS; ++i) {
@@ -798,7 +811,7 @@ __device__ __forceinline__ void backward_col_units(const Sliced m, const float* 
 }
 
 // Row units.
-template <int G, int V, int CPS, bool FROM_S, bool SCATTER, bool DBG>
+template <int G, int V, int CPS, bool I16, bool FROM_S, bool SCATTER, bool DBG>
 __device__ __forceinline__ void backward_row_units(const Sliced m, float* __restrict__ bias, const float* __restrict__ xk,
                                                    const float* __restrict__ xprev, float* dk, float* dprev,
                                                    float* __restrict__ dbg_delta, float* __restrict__ dbg_grad, int n, float clamp, int act,
@@ -820,10 +833,10 @@ __device__ __forceinline__ void backward_row_units(const Sliced m, float* __rest
     SDNN_UNIT_SHAPE(m, u, nunits, item, base, nch)
     if (u < nunits && lane == 0) prefetch_unit(m, u, RPW, n, UPS);
     int len = (item < n) ? m.len[item] : 0;
-    int4 c[CPS];
+    IdxChunk<I16> c[CPS];
 #pragma unroll
-    for (int i = 0; i < CPS; ++i) c[i] = make_int4(0, 0, 0, 0);
-    if (nch > 0) load_idx<CPS>(c, m, base);
+    for (int i = 0; i < CPS; ++i) idx_zero(c[i]);
+    if (nch > 0) load_idx<CPS, I16>(c, m, base);
     Lane<V> h0, h1;       // delta^k[i,:] (or S_k[i,:]) and, FROM_S, x^k[i,:]
     lane_fill(h0, 0.0f); lane_fill(h1, 0.0f);
     // tile row of stored row `item`: its neuron's number (the stored rows of a regrouped layer are not in neuron order)
@@ -860,7 +873,7 @@ __device__ __forceinline__ void backward_row_units(const Sliced m, float* __rest
         float* gp = DBG ? dbg_grad + base : nullptr;
         const int lim = len - ((G >= 4) ? (sub & 3) : (G == 2) ? 2 * sub : 0);
 #define SDNN_ROW_NEXT                                                                                    \
-        if (nnch > 0) load_idx<CPS>(c, m, nbase);                                                        \
+        if (nnch > 0) load_idx<CPS, I16>(c, m, nbase);                                                        \
         if (nitem < n) { lane_load(nh0, tile_row(dk + boff, nlab, pitch)); if (FROM_S) lane_load(nh1, tile_row(xk + boff, nlab, pitch)); }
 #define SDNN_SCAT(C, W, Q) if ((Q) < len) lane_red_add(tile_row(sg, C, pitch), W, d);
         for (int t = 0; t < nch; t += CPS) {
@@ -874,10 +887,11 @@ __device__ __forceinline__ void backward_row_units(const Sliced m, float* __rest
 #pragma unroll
                 for (int i = 0; i < CPS; ++i) {
                     const int q = 4 * (t + i);
-                    SDNN_SCAT(c[i].x, w[i].x, q) SDNN_SCAT(c[i].y, w[i].y, q + 1) SDNN_SCAT(c[i].z, w[i].z, q + 2) SDNN_SCAT(c[i].w, w[i].w, q + 3)
+                    const int4 cu = idx_unpack(c[i]);
+                    SDNN_SCAT(cu.x, w[i].x, q) SDNN_SCAT(cu.y, w[i].y, q + 1) SDNN_SCAT(cu.z, w[i].z, q + 2) SDNN_SCAT(cu.w, w[i].w, q + 3)
                 }
             }
-            if (t + CPS < nch) { load_idx<CPS>(c, m, base + (t + CPS) * CHUNK_ROW); }
+            if (t + CPS < nch) { load_idx<CPS, I16>(c, m, base + (t + CPS) * CHUNK_ROW); }
             else { SDNN_ROW_NEXT }
 #pragma unroll
             for (int i = 0; i < CPS; ++i) {
@@ -894,7 +908,7 @@ __device__ __forceinline__ void backward_row_units(const Sliced m, float* __rest
     }
 }
 
-template <int G, int V, int CPS, bool FROM_S, bool SCATTER, bool MIRROR, bool DBG>
+template <int G, int V, int CPS, bool I16, bool FROM_S, bool SCATTER, bool MIRROR, bool DBG>
 __global__ void __launch_bounds__(256, 2)
 backward_kernel(const BackwardArgs a) {
     const int wpb = blockDim.x >> 5;
@@ -911,9 +925,9 @@ backward_kernel(const BackwardArgs a) {
     if (a.pdl == 2) grid_launch_dependents();
     const float inv_b = a.sp->inv_b;
     const float step = a.sp->eta * inv_b;
-    if (MIRROR) backward_col_units<G, V, CPS>(a.cols, a.xprev, a.dk, a.dprev, a.n, a.clamp, a.act, step, inv_b, first, stride);
+    if (MIRROR) backward_col_units<G, V, CPS, I16>(a.cols, a.xprev, a.dk, a.dprev, a.n, a.clamp, a.act, step, inv_b, first, stride);
     if (MIRROR && a.cols_only) { if (a.pdl == 1) grid_launch_dependents(); return; }
-    backward_row_units<G, V, CPS, FROM_S, SCATTER, DBG>(a.rows, a.bias, a.xk, a.xprev, a.dk, a.dprev, a.dbg_delta, a.dbg_grad, a.n,
+    backward_row_units<G, V, CPS, I16, FROM_S, SCATTER, DBG>(a.rows, a.bias, a.xk, a.xprev, a.dk, a.dprev, a.dbg_delta, a.dbg_grad, a.n,
                                                         a.clamp, a.act, step, inv_b, a.update_bias, a.skip_dead, first, stride);
     if (a.pdl == 1) grid_launch_dependents();
 }
@@ -947,14 +961,16 @@ __device__ __forceinline__ EpShape ep_shape(const Sliced& m, int n) {
 #define SDNN_EP_LOAD_IDX(C, T0, IT)                                                                     \
     _Pragma("unroll") for (int i = 0; i < (IT); ++i) {                                                   \
         const int t = (T0) + 2 * i + e.h;                                                                \
-        C[i] = (t < e.nch) ? load_idx4(m, e.so + t * CHUNK_ROW + e.r * 4) : make_int4(0, 0, 0, 0);       \
+        idx_zero(C[i]);                                                                                  \
+        if (t < e.nch) load_idx4(C[i], m, e.so + t * CHUNK_ROW + e.r * 4);                               \
     }
 
+template <bool I16>
 __global__ void __launch_bounds__(128)
 forward_ep_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict__ xin, float* __restrict__ xout,
                   int n, float clamp, int act, int pdl) {
     const EpShape e = ep_shape(m, n);
-    int4 c[EP_IT];
+    IdxChunk<I16> c[EP_IT];
     SDNN_EP_LOAD_IDX(c, 0, EP_IT)
     const float b = (e.item < n) ? bias[e.item] : 0.0f;
     if (pdl) grid_dependency_wait();
@@ -1000,12 +1016,12 @@ __device__ __forceinline__ float4 ep_update(const float4& w, float p0, float p1,
 // IT iterations (2 * IT chunks of a unit) in flight together.  The transposed copy's units are ragged (a column of a
 // 32-per-row random pattern has 15 .. 55 entries): IT = 8 takes up to 64 entries in one go where the launch is bound by
 // its chain of dependent round trips rather than by throughput (small nets).
-template <int IT>
+template <int IT, bool I16>
 __global__ void __launch_bounds__(128)
 backward_col_ep_kernel(Sliced m, const float* __restrict__ xprev, const float* __restrict__ dk, float* __restrict__ dprev,
                        int n, float clamp, int act, const StepParams* __restrict__ sp, int pdl) {
     const EpShape e = ep_shape(m, n);
-    int4 c[IT];
+    IdxChunk<I16> c[IT];
     SDNN_EP_LOAD_IDX(c, 0, IT)
     int len = 0, j = 0;
     if (e.item < n) { len = m.len[e.item]; j = m.order[e.item]; }
@@ -1047,12 +1063,12 @@ backward_col_ep_kernel(Sliced m, const float* __restrict__ xprev, const float* _
 }
 
 // Row units (row-major copy m): update of its values (and of the bias) from delta^k[i] and the gathered x^{k-1}[j].
-template <bool DBG>
+template <bool DBG, bool I16>
 __global__ void __launch_bounds__(128)
 backward_row_ep_kernel(Sliced m, float* __restrict__ bias, const float* __restrict__ xprev, const float* __restrict__ dk,
                        float* __restrict__ dbg_grad, int n, const StepParams* __restrict__ sp, int update_bias, int pdl) {
     const EpShape e = ep_shape(m, n);
-    int4 c[EP_IT];
+    IdxChunk<I16> c[EP_IT];
     SDNN_EP_LOAD_IDX(c, 0, EP_IT)
     const int len = (e.item < n) ? m.len[e.item] : 0;
     if (pdl) grid_dependency_wait();

@@ -409,13 +409,13 @@ cudaError_t launch_k(sdnn* h, void (*kernel)(KArgs...), dim3 grid, dim3 block, b
     return cudaLaunchKernelEx(&lc, kernel, KArgs(args)...);
 }
 
-template <int G, int V, int CPS = 2>
+template <bool I16, int G, int V, int CPS = 2>
 void launch_forward_gv(sdnn* h, int layer, const float* xin, float* xout, int ld, int chunks, bool track) {
     constexpr int RPW = 32 / G;
     const int units = (h->N + RPW - 1) / RPW;
     const float* bias = h->d_bias + (size_t)layer * h->N;
-    auto plan = plan_grid(h, (const void*)forward_kernel<G, V, CPS>, units, chunks);
-    launch_k(h, forward_kernel<G, V, CPS>, dim3(plan.first, chunks), dim3(plan.second), h->pdl, rows_of(h, layer), bias, xin, xout,
+    auto plan = plan_grid(h, (const void*)forward_kernel<G, V, CPS, I16>, units, chunks);
+    launch_k(h, forward_kernel<G, V, CPS, I16>, dim3(plan.first, chunks), dim3(plan.second), h->pdl, rows_of(h, layer), bias, xin, xout,
              h->N, ld, h->cfg.clamp, h->cfg.activation, h->pdl ? h->fwd_pdl : 0, track ? (const int*)h->cur->cs.ncols : (const int*)nullptr,
              track ? h->cur->cs.flags : (int*)nullptr);
 }
@@ -427,28 +427,35 @@ bool entry_parallel(const sdnn* h, int ld) {
     return ld == 4 && !(h->cfg.flags & (SDNN_FLAG_BWD_ATOMICS | SDNN_FLAG_BWD_ONE_LAUNCH));
 }
 
-void launch_forward(sdnn* h, int layer, const float* xin, float* xout, int ld, int cols, bool track = false) {
+template <bool I16>
+void launch_forward_i(sdnn* h, int layer, const float* xin, float* xout, int ld, int cols, bool track) {
     const Geometry q = geometry(cols);
     if (q.v == 4 && !track && entry_parallel(h, ld)) {
         const int wf = h->NS <= h->sms ? 1 : 4;      // few slices: one per CTA, so that they spread over as many SMs
-        launch_k(h, forward_ep_kernel, dim3((h->NS + wf - 1) / wf), dim3(32 * wf), h->pdl, rows_of(h, layer),
+        launch_k(h, forward_ep_kernel<I16>, dim3((h->NS + wf - 1) / wf), dim3(32 * wf), h->pdl, rows_of(h, layer),
                  (const float*)(h->d_bias + (size_t)layer * h->N), xin, xout, h->N, h->cfg.clamp, h->cfg.activation, h->pdl ? h->fwd_pdl : 0);
-    } else if (q.v == 4) launch_forward_gv<1, 4>(h, layer, xin, xout, ld, q.chunks, track);
+    } else if (q.v == 4) launch_forward_gv<I16, 1, 4>(h, layer, xin, xout, ld, q.chunks, track);
     else switch (q.g) {
-        case 1: launch_forward_gv<1, 8>(h, layer, xin, xout, ld, q.chunks, track); break;
-        case 2: launch_forward_gv<2, 8>(h, layer, xin, xout, ld, q.chunks, track); break;
-        case 4: launch_forward_gv<4, 8>(h, layer, xin, xout, ld, q.chunks, track); break;
-        case 8: launch_forward_gv<8, 8>(h, layer, xin, xout, ld, q.chunks, track); break;
-        case 16: launch_forward_gv<16, 8>(h, layer, xin, xout, ld, q.chunks, track); break;
+        case 1: launch_forward_gv<I16, 1, 8>(h, layer, xin, xout, ld, q.chunks, track); break;
+        case 2: launch_forward_gv<I16, 2, 8>(h, layer, xin, xout, ld, q.chunks, track); break;
+        case 4: launch_forward_gv<I16, 4, 8>(h, layer, xin, xout, ld, q.chunks, track); break;
+        case 8: launch_forward_gv<I16, 8, 8>(h, layer, xin, xout, ld, q.chunks, track); break;
+        case 16: launch_forward_gv<I16, 16, 8>(h, layer, xin, xout, ld, q.chunks, track); break;
         default:
             // a launch of at most one warp-row per resident slot is bound by its chain of round trips: four chunks (16
             // entries) of a row in flight per step instead of two, where every slice has whole steps of that size
             if (!track && h->lay[layer].r_chunks_mult4 && (int64_t)h->N * q.chunks <= (int64_t)h->sms * 8)
-                launch_forward_gv<32, 8, 4>(h, layer, xin, xout, ld, q.chunks, track);
-            else launch_forward_gv<32, 8>(h, layer, xin, xout, ld, q.chunks, track);
+                launch_forward_gv<I16, 32, 8, 4>(h, layer, xin, xout, ld, q.chunks, track);
+            else launch_forward_gv<I16, 32, 8>(h, layer, xin, xout, ld, q.chunks, track);
             break;
     }
     count_launch(h);
+}
+
+// the kernels are instantiated for both index widths of the sliced copies
+void launch_forward(sdnn* h, int layer, const float* xin, float* xout, int ld, int cols, bool track = false) {
+    if (h->idx16) launch_forward_i<true>(h, layer, xin, xout, ld, cols, track);
+    else launch_forward_i<false>(h, layer, xin, xout, ld, cols, track);
 }
 
 // Windowed layers (rows grouped by shared columns at set-up): the group's window of the input tile is staged in shared
@@ -505,7 +512,7 @@ float* delta_tile(sdnn* h, int layer, size_t tile) {
 }
 
 // part: 0 = the whole layer in one launch; 1 = column units only; 2 = row units only (transposed realisation)
-template <int G, int V, int CPS>
+template <bool I16, int G, int V, int CPS>
 void launch_backward_gvc(sdnn* h, int layer, int ld, int part) {
     constexpr int RPW = 32 / G;
     const size_t tile = (size_t)h->N * ld;
@@ -535,13 +542,13 @@ void launch_backward_gvc(sdnn* h, int layer, int ld, int part) {
 #define SDNN_BWD(FROM_S, SCAT, MIR)                                                            \
     do {                                                                                       \
         if (a.dbg_grad) {                                                                      \
-            auto plan = plan_grid(h, (const void*)backward_kernel<G, V, CPS, FROM_S, SCAT, MIR, true>, units, 1, os_);   \
+            auto plan = plan_grid(h, (const void*)backward_kernel<G, V, CPS, I16, FROM_S, SCAT, MIR, true>, units, 1, os_);   \
             if (a.pdl && plan.first <= h->sms) a.pdl = PDL_EARLY;                              \
-            launch_k(h, backward_kernel<G, V, CPS, FROM_S, SCAT, MIR, true>, dim3(plan.first), dim3(plan.second), a.pdl != 0, a); \
+            launch_k(h, backward_kernel<G, V, CPS, I16, FROM_S, SCAT, MIR, true>, dim3(plan.first), dim3(plan.second), a.pdl != 0, a); \
         } else {                                                                               \
-            auto plan = plan_grid(h, (const void*)backward_kernel<G, V, CPS, FROM_S, SCAT, MIR, false>, units, 1, os_);  \
+            auto plan = plan_grid(h, (const void*)backward_kernel<G, V, CPS, I16, FROM_S, SCAT, MIR, false>, units, 1, os_);  \
             if (a.pdl && plan.first <= h->sms) a.pdl = PDL_EARLY;                              \
-            launch_k(h, backward_kernel<G, V, CPS, FROM_S, SCAT, MIR, false>, dim3(plan.first), dim3(plan.second), a.pdl != 0, a); \
+            launch_k(h, backward_kernel<G, V, CPS, I16, FROM_S, SCAT, MIR, false>, dim3(plan.first), dim3(plan.second), a.pdl != 0, a); \
         }                                                                                      \
     } while (0)
     if (h->mirror) {
@@ -568,12 +575,13 @@ void launch_backward_gvc(sdnn* h, int layer, int ld, int part) {
 #undef SDNN_BWD
 }
 
-template <int G, int V>
+template <bool I16, int G, int V>
 void launch_backward_gv(sdnn* h, int layer, int ld, int part) {
-    launch_backward_gvc<G, V, 2>(h, layer, ld, part);
+    launch_backward_gvc<I16, G, V, 2>(h, layer, ld, part);
 }
 
 // the two launches of a layer in the split transposed realisation, for tiles of padded width 4
+template <bool I16>
 void launch_backward_ep(sdnn* h, int layer, int part) {
     const size_t tile = (size_t)h->N * 4;
     const float* acts = h->bwd_acts ? h->bwd_acts : h->d_acts;
@@ -585,33 +593,39 @@ void launch_backward_ep(sdnn* h, int layer, int part) {
         const int pdl = !h->pdl ? 0 : (int)grid.x <= h->sms ? PDL_EARLY : PDL_AT_END;
         // a launch of at most one CTA per SM is bound by its chain of round trips: take a long column in one go
         if ((int)grid.x <= h->sms && h->lay[layer].c_max_chunks > 2 * EP_IT)
-            launch_k(h, backward_col_ep_kernel<2 * EP_IT>, grid, block, h->pdl, cols_of(h, layer), xprev, dk, delta_tile(h, layer - 1, tile),
+            launch_k(h, backward_col_ep_kernel<2 * EP_IT, I16>, grid, block, h->pdl, cols_of(h, layer), xprev, dk, delta_tile(h, layer - 1, tile),
                      h->N, h->cfg.clamp, h->cfg.activation, (const StepParams*)h->d_sp, pdl);
         else
-            launch_k(h, backward_col_ep_kernel<EP_IT>, grid, block, h->pdl, cols_of(h, layer), xprev, dk, delta_tile(h, layer - 1, tile),
+            launch_k(h, backward_col_ep_kernel<EP_IT, I16>, grid, block, h->pdl, cols_of(h, layer), xprev, dk, delta_tile(h, layer - 1, tile),
                      h->N, h->cfg.clamp, h->cfg.activation, (const StepParams*)h->d_sp, pdl);
     } else {
         float* bias = h->d_bias + (size_t)layer * h->N;
         float* grad = h->lay[layer].r_grad;
-        if (grad) launch_k(h, backward_row_ep_kernel<true>, grid, block, false, rows_of(h, layer), bias, xprev, dk, grad, h->N,
+        if (grad) launch_k(h, backward_row_ep_kernel<true, I16>, grid, block, false, rows_of(h, layer), bias, xprev, dk, grad, h->N,
                            (const StepParams*)h->d_sp, h->cfg.update_bias ? 1 : 0, 0);
-        else launch_k(h, backward_row_ep_kernel<false>, grid, block, false, rows_of(h, layer), bias, xprev, dk, grad, h->N,
+        else launch_k(h, backward_row_ep_kernel<false, I16>, grid, block, false, rows_of(h, layer), bias, xprev, dk, grad, h->N,
                       (const StepParams*)h->d_sp, h->cfg.update_bias ? 1 : 0, 0);
     }
 }
 
-void launch_backward(sdnn* h, int layer, int ld, int part = 0) {
+template <bool I16>
+void launch_backward_i(sdnn* h, int layer, int ld, int part) {
     const Geometry q = geometry(ld);
-    if (q.v == 4 && h->split && part != 0 && entry_parallel(h, ld)) launch_backward_ep(h, layer, part);
-    else if (q.v == 4) launch_backward_gv<1, 4>(h, layer, ld, part);
+    if (q.v == 4 && h->split && part != 0 && entry_parallel(h, ld)) launch_backward_ep<I16>(h, layer, part);
+    else if (q.v == 4) launch_backward_gv<I16, 1, 4>(h, layer, ld, part);
     else switch (q.g) {
-        case 1: launch_backward_gv<1, 8>(h, layer, ld, part); break;
-        case 2: launch_backward_gv<2, 8>(h, layer, ld, part); break;
-        case 4: launch_backward_gv<4, 8>(h, layer, ld, part); break;
-        case 8: launch_backward_gv<8, 8>(h, layer, ld, part); break;
-        default: launch_backward_gv<16, 8>(h, layer, ld, part); break;
+        case 1: launch_backward_gv<I16, 1, 8>(h, layer, ld, part); break;
+        case 2: launch_backward_gv<I16, 2, 8>(h, layer, ld, part); break;
+        case 4: launch_backward_gv<I16, 4, 8>(h, layer, ld, part); break;
+        case 8: launch_backward_gv<I16, 8, 8>(h, layer, ld, part); break;
+        default: launch_backward_gv<I16, 16, 8>(h, layer, ld, part); break;
     }
     count_launch(h);
+}
+
+void launch_backward(sdnn* h, int layer, int ld, int part = 0) {
+    if (h->idx16) launch_backward_i<true>(h, layer, ld, part);
+    else launch_backward_i<false>(h, layer, ld, part);
 }
 
 void launch_output_gradient(sdnn* h, int ld) {

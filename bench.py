@@ -229,7 +229,7 @@ def study_probes():
         mhz = 1965
     clk = mhz * 1e6
     out = {"study": "probes", "sms": sms, "sm_max_mhz": mhz, "unit": "rows (or words) per clock per SM at sm_max_mhz", "l2": {}, "l2_small_table": {},
-           "shared": {}, "cluster": {}, "words": {}}
+           "shared": {}, "cluster": {}, "copy_engine_bulk": {}, "copy_engine_gather4": {}, "words": {}}
     for rb in (16, 32, 64, 128, 256, 512, 1024):
         rows = (4 << 20) // rb                                   # a 4 MB table: an activation tile of the large configurations
         out["l2"][str(rb)] = pkg.probe_gather_rate(rb, rows) / sms / clk
@@ -240,6 +240,14 @@ def study_probes():
         for cl in (2, 4, 8, 16):
             r, ctas = pkg.probe_smem_gather_rate(rb, cl)
             out["cluster"][f"{rb}x{cl}"] = {"rate": r / ctas / clk, "ctas": ctas}
+    for rb in (16, 32, 64, 128, 256):      # rows fetched by the copy engine into shared memory, out of the same 4 MB table
+        for key, g4 in (("copy_engine_bulk", 0), ("copy_engine_gather4", 1)):
+            if g4 and rb < 32:
+                continue
+            try:
+                out[key][str(rb)] = pkg.probe_tma_gather_rate(rb, (4 << 20) // rb, g4) / sms / clk
+            except pkg.SdnnError as exc:
+                out[key][str(rb)] = f"error: {exc.message}"
     for name, store in (("load4", 0), ("store4", 1)):
         out["words"][name] = pkg.probe_word_rate(store, 1 << 21) / sms / clk       # an 8 MB value array (one layer of the largest net)
     print(json.dumps(out), flush=True)

@@ -282,6 +282,17 @@ int sdnn_probe_gather_rate(int32_t row_bytes, int64_t table_rows, double* rows_p
 int sdnn_probe_word_rate(int32_t store, int64_t table_words, double* words_per_second);
 
 /*
+ * The same measurement with the rows fetched by the copy engine (TMA) into shared memory instead of by load
+ * instructions into registers (diagnostic; the paper has no counterpart).  gather4 = 0: one bulk copy
+ * (cp.async.bulk) per row; gather4 = 1: four rows of a two-dimensional tensor map per instruction
+ * (cp.async.bulk.tensor ... tile::gather4).  row_bytes 16 .. 256 (a power of two), table as in sdnn_probe_gather_rate.
+ * No cluster multicast; the tensor map covers this device's own table only.  Every wait of the kernel is bounded;
+ * if one runs out the call returns SDNN_ERR_CUDA with a message instead of a rate.  Allocates and frees its own
+ * table; synchronises.
+ */
+int sdnn_probe_tma_gather_rate(int32_t row_bytes, int64_t table_rows, int32_t gather4, double* rows_per_second);
+
+/*
  * The same measurement for operand tiles staged on chip (diagnostic; the paper has no counterpart): random rows of
  * `row_bytes` bytes (32, 64, 128 or 256; read with 128-bit accesses) out of a table of 128 KiB per CTA held in shared
  * memory.  cluster_size 1: every CTA reads its own shared memory; 2, 4, 8 or 16: the table is spread over the shared

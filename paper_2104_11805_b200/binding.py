@@ -56,6 +56,7 @@ _PROTOS = {
     "sdnn_get_gradient": (ctypes.c_int, [_vp, _i32, _vp]),
     "sdnn_mirror_mismatches": (ctypes.c_int, [_vp, _i32, ctypes.POINTER(_i64)]),
     "sdnn_probe_gather_rate": (ctypes.c_int, [_i32, _i64, ctypes.POINTER(ctypes.c_double)]),
+    "sdnn_probe_tma_gather_rate": (ctypes.c_int, [_i32, _i64, _i32, ctypes.POINTER(ctypes.c_double)]),
     "sdnn_probe_word_rate": (ctypes.c_int, [_i32, _i64, ctypes.POINTER(ctypes.c_double)]),
     "sdnn_probe_smem_gather_rate": (ctypes.c_int, [_i32, _i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(_i32)]),
     "sdnn_get_phase_times": (ctypes.c_int, [_vp, ctypes.POINTER(_f32), ctypes.POINTER(_f32)]),
@@ -172,6 +173,17 @@ def cluster_layer(row_ptr, col_idx, col_cap=1536, row_cap=2048):
     if ng.value == 0:
         return None, None, 0, 0
     return grp, lab, ng.value, mw.value
+
+
+def probe_tma_gather_rate(row_bytes, table_rows, gather4):
+    """sdnn_probe_tma_gather_rate: random rows per second fetched by the copy engine into shared memory (bulk copies
+    per row, or four rows per tile::gather4 instruction)."""
+    lib = load_library()
+    out = ctypes.c_double(0.0)
+    rc = lib.sdnn_probe_tma_gather_rate(row_bytes, table_rows, int(bool(gather4)), ctypes.byref(out))
+    if rc != 0:
+        raise SdnnError(rc, (lib.sdnn_last_error(None) or b"").decode())
+    return out.value
 
 
 def probe_word_rate(store, table_words):

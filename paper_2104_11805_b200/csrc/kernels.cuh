@@ -21,6 +21,7 @@
 // delta^{k-1} = (W^k)^T delta^k (.) f'(z^{k-1}); update W^k(j,i) -= eta delta^k(j) x^{k-1}(i)
 // on stored entries.  Only x^k is stored: with f = clamp to [0,c], f'(z) = [0 < x < c].
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -450,7 +451,6 @@ forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict
     int row, base, nch;
     SDNN_UNIT_SHAPE(m, unit, nunits, row, base, nch)
     float b = (row < n) ? bias[row] : 0.0f;
-    int orow = (row < n && m.out) ? m.out[row] : row;
     if (unit < nunits && lane == 0) prefetch_unit(m, unit, RPW, n, UPS);
     IdxChunk<I16> c[CPS];
 #pragma unroll
@@ -468,7 +468,6 @@ forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict
         int nrow, nbase, nnch;
         SDNN_UNIT_SHAPE(m, nunit, nunits, nrow, nbase, nnch)
         const float nb = (nrow < n) ? bias[nrow] : 0.0f;
-        const int norow = (nrow < n && m.out) ? m.out[nrow] : nrow;
         if (nunit < nunits && lane == 0) prefetch_unit(m, nunit, RPW, n, UPS);
 
         Lane<V> acc;
@@ -492,10 +491,10 @@ forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict
         if (nch == 0 && nnch > 0) load_idx<CPS, I16>(c, m, nbase);      // empty slice: nothing prefetched across the boundary yet
         if (row < n) {
             lane_activate(acc, act, clamp);
-            lane_store(tile_row(xout + boff, orow, pitch), acc);
+            lane_store(tile_row(xout + boff, m.out ? m.out[row] : row, pitch), acc);      // regrouped layer: the neuron's tile row
             if (live_flags) live |= lane_nonzero_bits(acc);
         }
-        unit = nunit; row = nrow; base = nbase; nch = nnch; b = nb; orow = norow;
+        unit = nunit; row = nrow; base = nbase; nch = nnch; b = nb;
     }
     if (live_flags) {
 #pragma unroll
@@ -1365,6 +1364,97 @@ smem_gather_probe_kernel(float* __restrict__ sink, unsigned rows_per_cta_log2, u
     }
     if (acc == 123.456f) sink[0] = acc;      // the table is all zero: never taken, keeps the loads alive
     cluster_barrier();
+}
+
+// ---------------------------------------------------------------------------------------------
+// The same probe for rows fetched by the copy engine (TMA) into shared memory instead of by load instructions into
+// registers: GATHER4 = false: one cp.async.bulk of row_bytes per row; true: cp.async.bulk.tensor.2d ... tile::gather4,
+// four rows of a two-dimensional tensor map (box: one row of row_bytes) per instruction.  The first `issuers` lanes of a
+// warp issue one copy each per round into their own slot of a ring of TMA_STAGES stages per warp; a stage's copies complete on the warp's
+// mbarrier for that stage.  Every wait on an mbarrier is bounded: after TMA_WAIT_LIMIT polls the warp records the
+// failure in *status and stops issuing, waits (bounded again) for what it has in flight, and returns.
+constexpr int TMA_STAGES = 4;
+constexpr int TMA_WARPS = 4;
+constexpr unsigned TMA_WAIT_LIMIT = 1u << 22;
+
+__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
+}
+// polls until the phase with the given parity has completed; false if it gave up
+__device__ __forceinline__ bool mbar_wait_bounded(unsigned bar, unsigned parity) {
+    for (unsigned i = 0; i < TMA_WAIT_LIMIT; ++i) {
+        unsigned done;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
+template <bool GATHER4>
+__global__ void __launch_bounds__(32 * TMA_WARPS)
+tma_gather_probe_kernel(const float* __restrict__ table, const __grid_constant__ CUtensorMap tmap, float* __restrict__ sink,
+                        int* __restrict__ status, unsigned row_mask, unsigned row_bytes, int issuers, int rounds, unsigned seed) {
+    extern __shared__ __align__(128) unsigned char tma_smem[];
+    __shared__ __align__(8) unsigned long long bars[TMA_WARPS * TMA_STAGES];
+    constexpr unsigned ROWS = GATHER4 ? 4u : 1u;                       // rows per copy
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const unsigned slot_bytes = ROWS * row_bytes;                      // one lane's copy
+    const unsigned stage_bytes = (unsigned)issuers * slot_bytes;
+    unsigned char* ring = tma_smem + (size_t)warp * TMA_STAGES * stage_bytes;
+    if (lane == 0)
+        for (int q = 0; q < TMA_STAGES; ++q) mbar_init(smem_u32(&bars[warp * TMA_STAGES + q]), 1u);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncwarp();
+    unsigned st = (unsigned)(blockIdx.x * blockDim.x + threadIdx.x) * 2654435761u + seed;
+    float acc = 0.f;
+    bool ok = true;
+    int issued = 0;
+    auto issue = [&](int r) {
+        const int q = r % TMA_STAGES;
+        const unsigned bar = smem_u32(&bars[warp * TMA_STAGES + q]);
+        if (lane == 0) mbar_expect_tx(bar, stage_bytes);
+        __syncwarp();
+        const unsigned dst = smem_u32(ring + (size_t)q * stage_bytes + (size_t)lane * slot_bytes);
+        if (lane >= issuers) return;
+        if (GATHER4) {
+            int r0, r1, r2, r3;
+            st = st * 1664525u + 1013904223u; r0 = (int)((st >> 8) & row_mask);
+            st = st * 1664525u + 1013904223u; r1 = (int)((st >> 8) & row_mask);
+            st = st * 1664525u + 1013904223u; r2 = (int)((st >> 8) & row_mask);
+            st = st * 1664525u + 1013904223u; r3 = (int)((st >> 8) & row_mask);
+            asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+                         :: "r"(dst), "l"(reinterpret_cast<unsigned long long>(&tmap)), "r"(0), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(bar) : "memory");
+        } else {
+            st = st * 1664525u + 1013904223u;
+            const unsigned long long src = reinterpret_cast<unsigned long long>(table) + (unsigned long long)((st >> 8) & row_mask) * row_bytes;
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         :: "r"(dst), "l"(src), "r"(row_bytes), "r"(bar) : "memory");
+        }
+    };
+    for (; issued < TMA_STAGES - 1 && issued < rounds; ++issued) issue(issued);
+    int done = 0;
+    for (; done < rounds && ok; ++done) {
+        if (issued < rounds) {
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // the slot's earlier readers come before the engine's writes
+            issue(issued); ++issued;
+        }
+        const int q = done % TMA_STAGES;
+        ok = mbar_wait_bounded(smem_u32(&bars[warp * TMA_STAGES + q]), (unsigned)(done / TMA_STAGES) & 1u);
+        ok = __all_sync(0xffffffffu, ok);
+        if (ok && lane < issuers) acc += *reinterpret_cast<const float*>(ring + (size_t)q * stage_bytes + (size_t)lane * slot_bytes);
+        __syncwarp();
+    }
+    if (!ok) {      // gave up: note it, then wait (bounded) for the copies still in flight before the shared memory goes away
+        if (lane == 0) atomicExch(status, 1);
+        for (; done < issued; ++done)
+            mbar_wait_bounded(smem_u32(&bars[warp * TMA_STAGES + done % TMA_STAGES]), (unsigned)(done / TMA_STAGES) & 1u);
+    }
+    if (acc == 123.456f) sink[0] = acc;
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -1943,6 +1943,99 @@ extern "C" int sdnn_probe_word_rate(int32_t store, int64_t table_words, double* 
 }
 
 // ---------------------------------------------------------------------------------------------
+// Copy-engine gather probe (see sdnn_probe_tma_gather_rate in the header).
+extern "C" int sdnn_probe_tma_gather_rate(int32_t row_bytes, int64_t table_rows, int32_t gather4, double* rows_per_second) {
+    if (!rows_per_second) return fail(nullptr, SDNN_ERR_INVALID_ARG, "rows_per_second is NULL");
+    *rows_per_second = 0.0;
+    if (row_bytes != 16 && row_bytes != 32 && row_bytes != 64 && row_bytes != 128 && row_bytes != 256)
+        return fail(nullptr, SDNN_ERR_INVALID_ARG, "row_bytes must be 16, 32, 64, 128 or 256");
+    if (table_rows < 1 || (table_rows & (table_rows - 1)) || table_rows * row_bytes > (1LL << 30))
+        return fail(nullptr, SDNN_ERR_INVALID_ARG, "table_rows must be a power of two with table_rows * row_bytes <= 1 GiB");
+    if (gather4 != 0 && gather4 != 1) return fail(nullptr, SDNN_ERR_INVALID_ARG, "gather4 must be 0 or 1");
+    if (gather4 && row_bytes < 32)      // a copy's four rows land in one 128-byte aligned slot of shared memory
+        return fail(nullptr, SDNN_ERR_INVALID_ARG, "tile::gather4 needs row_bytes >= 32 here");
+    int dev = 0, sms = 0;
+    CU(nullptr, cudaGetDevice(&dev));
+    CU(nullptr, cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    float* table = nullptr;
+    float* sink = nullptr;
+    int* status = nullptr;
+    cudaEvent_t a = nullptr, b = nullptr;
+    cudaStream_t st = nullptr;
+    int rc = SDNN_OK;
+    const size_t bytes = (size_t)table_rows * row_bytes;
+    if (cudaMalloc(&table, bytes) != cudaSuccess || cudaMalloc(&sink, 256) != cudaSuccess || cudaMalloc(&status, sizeof(int)) != cudaSuccess ||
+        cudaStreamCreate(&st) != cudaSuccess || cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) {
+        cudaGetLastError();
+        rc = fail(nullptr, SDNN_ERR_OOM, "could not set up the probe");
+    } else {
+        cudaMemsetAsync(table, 0, bytes, st);
+        cudaMemsetAsync(status, 0, sizeof(int), st);
+        CUtensorMap tmap;
+        memset(&tmap, 0, sizeof tmap);
+        if (gather4) {      // the table as a two-dimensional tensor [table_rows][row_bytes / 4] of floats, box = one row
+            typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                         const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                         CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+            void* fn = nullptr;
+            cudaDriverEntryPointQueryResult qres;
+            cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+            if (e != cudaSuccess || !fn || qres != cudaDriverEntryPointSuccess) { cudaGetLastError(); rc = fail(nullptr, SDNN_ERR_CUDA, "cuTensorMapEncodeTiled is not available"); }
+            else {
+                const cuuint64_t dims[2] = {(cuuint64_t)(row_bytes / 4), (cuuint64_t)table_rows};
+                const cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
+                const cuuint32_t box[2] = {(cuuint32_t)(row_bytes / 4), 1u};
+                const cuuint32_t estr[2] = {1u, 1u};
+                CUresult cr = reinterpret_cast<EncodeFn>(fn)(&tmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, table, dims, strides, box, estr,
+                                                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                                            CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                if (cr != CUDA_SUCCESS) rc = fail(nullptr, SDNN_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)cr);
+            }
+        }
+        if (rc == SDNN_OK) {
+            const unsigned rows_per_copy = gather4 ? 4u : 1u;
+            const int issuers = (int)std::min<size_t>(32, 8192 / ((size_t)rows_per_copy * row_bytes));      // lanes of a warp that issue copies
+            const size_t smem = (size_t)TMA_WARPS * TMA_STAGES * issuers * rows_per_copy * row_bytes;       // at most 128 KB
+            cudaError_t e = gather4 ? cudaFuncSetAttribute(tma_gather_probe_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+                                    : cudaFuncSetAttribute(tma_gather_probe_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            int occ = 1;
+            if (e == cudaSuccess)
+                e = gather4 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, tma_gather_probe_kernel<true>, 32 * TMA_WARPS, smem)
+                            : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, tma_gather_probe_kernel<false>, 32 * TMA_WARPS, smem);
+            if (e != cudaSuccess || occ < 1) rc = cuda_fail(nullptr, e, "copy-engine probe set-up");
+            else {
+                const int grid = sms * std::min(occ, 4), rounds = 256, reps = 5;
+                const unsigned mask = (unsigned)(table_rows - 1);
+                auto launch = [&](unsigned seed) {
+                    if (gather4) tma_gather_probe_kernel<true><<<grid, 32 * TMA_WARPS, smem, st>>>(table, tmap, sink, status, mask, (unsigned)row_bytes, issuers, rounds, seed);
+                    else tma_gather_probe_kernel<false><<<grid, 32 * TMA_WARPS, smem, st>>>(table, tmap, sink, status, mask, (unsigned)row_bytes, issuers, rounds, seed);
+                };
+                launch(17u); launch(18u);
+                cudaEventRecord(a, st);
+                for (int i = 0; i < reps; ++i) launch(101u + i);
+                cudaEventRecord(b, st);
+                e = cudaEventSynchronize(b);
+                float ms = 0.f;
+                int gave_up = 0;
+                if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, a, b);
+                if (e == cudaSuccess) e = cudaMemcpy(&gave_up, status, sizeof(int), cudaMemcpyDeviceToHost);
+                if (e == cudaSuccess) e = cudaGetLastError();
+                if (e != cudaSuccess || !(ms > 0.f)) rc = cuda_fail(nullptr, e, "copy-engine probe");
+                else if (gave_up) rc = fail(nullptr, SDNN_ERR_CUDA, "copy-engine probe: a wait for its copies ran out");
+                else *rows_per_second = (double)grid * issuers * TMA_WARPS * rows_per_copy * rounds / (ms / reps * 1e-3);
+            }
+        }
+    }
+    if (a) cudaEventDestroy(a);
+    if (b) cudaEventDestroy(b);
+    if (st) cudaStreamDestroy(st);
+    if (table) cudaFree(table);
+    if (sink) cudaFree(sink);
+    if (status) cudaFree(status);
+    return rc;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Shared-memory / distributed-shared-memory gather probe (see sdnn_probe_smem_gather_rate in the header).
 namespace {
 

@@ -883,6 +883,17 @@ def test_shared_memory_gather_probe_reports_rates_and_rejects_bad_sizes(torch_cu
         assert ei.value.code == -1
 
 
+def test_copy_engine_gather_probe_reports_rates_and_rejects_bad_sizes(torch_cuda):
+    pkg = sdnn()
+    for row_bytes, gather4 in ((64, 0), (64, 1), (256, 1), (16, 0)):
+        rate = pkg.probe_tma_gather_rate(row_bytes, 1 << 14, gather4)
+        assert 1e8 < rate < 1e13
+    for row_bytes, rows, gather4 in ((48, 1024, 0), (64, 1000, 0), (16, 1024, 1), (512, 1024, 0)):
+        with pytest.raises(pkg.SdnnError) as ei:
+            pkg.probe_tma_gather_rate(row_bytes, rows, gather4)
+        assert ei.value.code == -1
+
+
 def test_state_and_argument_errors(torch_cuda):
     pkg = sdnn()
     rng = np.random.default_rng(2)

@@ -248,6 +248,17 @@ def study_probes():
                 out[key][str(rb)] = pkg.probe_tma_gather_rate(rb, (4 << 20) // rb, g4) / sms / clk
             except pkg.SdnnError as exc:
                 out[key][str(rb)] = f"error: {exc.message}"
+    out["both_paths"] = {}
+    for rb, lsu, tma in ((64, 2048, 256), (256, 1024, 256)):      # do the copy engine's gathers come on top of the loads'?
+        rows_tbl = (4 << 20) // rb
+        rec = {}
+        for key, t, l in (("loads_only", 0, lsu), ("copy_engine_only", tma, 0), ("both", tma, lsu)):
+            try:
+                sec, rows = pkg.probe_mixed_gather(rb, rows_tbl, t, l)
+                rec[key] = {"us": sec * 1e6, "rate": rows / sec / sms / clk}
+            except pkg.SdnnError as exc:
+                rec[key] = f"error: {exc.message}"
+        out["both_paths"][str(rb)] = rec
     for name, store in (("load4", 0), ("store4", 1)):
         out["words"][name] = pkg.probe_word_rate(store, 1 << 21) / sms / clk       # an 8 MB value array (one layer of the largest net)
     print(json.dumps(out), flush=True)

@@ -293,6 +293,18 @@ int sdnn_probe_word_rate(int32_t store, int64_t table_words, double* words_per_s
 int sdnn_probe_tma_gather_rate(int32_t row_bytes, int64_t table_rows, int32_t gather4, double* rows_per_second);
 
 /*
+ * Do the two gather paths add up?  (Diagnostic; the paper has no counterpart.)  One CTA of 1024 threads per SM: four
+ * warps fetch random rows with tile::gather4 into shared memory (tma_rounds rounds each), 28 warps gather random rows
+ * with 256-bit loads into registers (lsu_per_group rows per lane group, a multiple of 8), out of the same table; either
+ * part may be given no work.  row_bytes 64 or 256.  seconds (host double*): device time of one launch; rows (host
+ * double*): rows gathered by one launch over both paths.  Comparing a launch of both parts with launches of each part
+ * alone says whether the copy engine could carry gathers BESIDE the load instructions.  Waits bounded as in
+ * sdnn_probe_tma_gather_rate; allocates and frees its own table; synchronises.
+ */
+int sdnn_probe_mixed_gather(int32_t row_bytes, int64_t table_rows, int32_t tma_rounds, int32_t lsu_per_group,
+                            double* seconds, double* rows);
+
+/*
  * The same measurement for operand tiles staged on chip (diagnostic; the paper has no counterpart): random rows of
  * `row_bytes` bytes (32, 64, 128 or 256; read with 128-bit accesses) out of a table of 128 KiB per CTA held in shared
  * memory.  cluster_size 1: every CTA reads its own shared memory; 2, 4, 8 or 16: the table is spread over the shared

@@ -57,6 +57,7 @@ _PROTOS = {
     "sdnn_mirror_mismatches": (ctypes.c_int, [_vp, _i32, ctypes.POINTER(_i64)]),
     "sdnn_probe_gather_rate": (ctypes.c_int, [_i32, _i64, ctypes.POINTER(ctypes.c_double)]),
     "sdnn_probe_tma_gather_rate": (ctypes.c_int, [_i32, _i64, _i32, ctypes.POINTER(ctypes.c_double)]),
+    "sdnn_probe_mixed_gather": (ctypes.c_int, [_i32, _i64, _i32, _i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]),
     "sdnn_probe_word_rate": (ctypes.c_int, [_i32, _i64, ctypes.POINTER(ctypes.c_double)]),
     "sdnn_probe_smem_gather_rate": (ctypes.c_int, [_i32, _i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(_i32)]),
     "sdnn_get_phase_times": (ctypes.c_int, [_vp, ctypes.POINTER(_f32), ctypes.POINTER(_f32)]),
@@ -184,6 +185,17 @@ def probe_tma_gather_rate(row_bytes, table_rows, gather4):
     if rc != 0:
         raise SdnnError(rc, (lib.sdnn_last_error(None) or b"").decode())
     return out.value
+
+
+def probe_mixed_gather(row_bytes, table_rows, tma_rounds, lsu_per_group):
+    """sdnn_probe_mixed_gather: (seconds per launch, rows per launch) with the copy engine and the load instructions
+    gathering side by side (either part may be 0)."""
+    lib = load_library()
+    sec, rows = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    rc = lib.sdnn_probe_mixed_gather(row_bytes, table_rows, tma_rounds, lsu_per_group, ctypes.byref(sec), ctypes.byref(rows))
+    if rc != 0:
+        raise SdnnError(rc, (lib.sdnn_last_error(None) or b"").decode())
+    return sec.value, rows.value
 
 
 def probe_word_rate(store, table_words):

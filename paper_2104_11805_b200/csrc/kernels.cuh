@@ -1458,6 +1458,84 @@ tma_gather_probe_kernel(const float* __restrict__ table, const __grid_constant__
 }
 
 // ---------------------------------------------------------------------------------------------
+// Do the two gather paths add up?  One CTA of 1024 threads per SM: the first TMA_WARPS warps fetch rows with
+// tile::gather4 into shared memory exactly as tma_gather_probe_kernel<true> does (tma_rounds rounds), the other 28 warps
+// gather rows with 256-bit loads into registers exactly as gather_probe_kernel does (lsu_per_group rows per lane
+// group), out of the same table.  Either part can be switched off by giving it no work.  If the paths are independent
+// the launch takes as long as its slower part; if they share their bottleneck it takes the sum.
+template <int G, int V>
+__global__ void __launch_bounds__(1024)
+mixed_gather_probe_kernel(const float* __restrict__ table, const __grid_constant__ CUtensorMap tmap, float* __restrict__ sink,
+                          int* __restrict__ status, unsigned row_mask, int issuers, int tma_rounds, int lsu_per_group, unsigned seed) {
+    extern __shared__ __align__(128) unsigned char tma_smem[];
+    __shared__ __align__(8) unsigned long long bars[TMA_WARPS * TMA_STAGES];
+    constexpr unsigned ROW_BYTES = 4u * G * V;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    unsigned st = (unsigned)(blockIdx.x * blockDim.x + threadIdx.x) * 2654435761u + seed;
+    float acc = 0.f;
+    if (warp >= TMA_WARPS) {      // ---- load path
+        const int tid = blockIdx.x * (blockDim.x - 32 * TMA_WARPS) + (threadIdx.x - 32 * TMA_WARPS);
+        const int sub = tid % G;
+        st = (unsigned)(tid / G) * 2654435761u + seed;
+        for (int q = 0; q < lsu_per_group; q += 8) {
+            unsigned c[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) { st = st * 1664525u + 1013904223u; c[u] = (st >> 8) & row_mask; }
+            Lane<V> v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) lane_gather(v[u], table + (size_t)c[u] * (V * G) + sub * V);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) acc += lane_sum(v[u]);
+        }
+        if (acc == 123.456f) sink[0] = acc;
+        return;
+    }
+    // ---- copy-engine path (no CTA-wide barrier anywhere: the two kinds of warp never meet)
+    const unsigned slot_bytes = 4u * ROW_BYTES, stage_bytes = (unsigned)issuers * slot_bytes;
+    unsigned char* ring = tma_smem + (size_t)warp * TMA_STAGES * stage_bytes;
+    if (lane == 0)
+        for (int q = 0; q < TMA_STAGES; ++q) mbar_init(smem_u32(&bars[warp * TMA_STAGES + q]), 1u);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncwarp();
+    bool ok = true;
+    int issued = 0;
+    auto issue = [&](int r) {
+        const int q = r % TMA_STAGES;
+        const unsigned bar = smem_u32(&bars[warp * TMA_STAGES + q]);
+        if (lane == 0) mbar_expect_tx(bar, stage_bytes);
+        __syncwarp();
+        if (lane >= issuers) return;
+        const unsigned dst = smem_u32(ring + (size_t)q * stage_bytes + (size_t)lane * slot_bytes);
+        int r0, r1, r2, r3;
+        st = st * 1664525u + 1013904223u; r0 = (int)((st >> 8) & row_mask);
+        st = st * 1664525u + 1013904223u; r1 = (int)((st >> 8) & row_mask);
+        st = st * 1664525u + 1013904223u; r2 = (int)((st >> 8) & row_mask);
+        st = st * 1664525u + 1013904223u; r3 = (int)((st >> 8) & row_mask);
+        asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+                     :: "r"(dst), "l"(reinterpret_cast<unsigned long long>(&tmap)), "r"(0), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(bar) : "memory");
+    };
+    for (; issued < TMA_STAGES - 1 && issued < tma_rounds; ++issued) issue(issued);
+    int done = 0;
+    for (; done < tma_rounds && ok; ++done) {
+        if (issued < tma_rounds) {
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            issue(issued); ++issued;
+        }
+        const int q = done % TMA_STAGES;
+        ok = mbar_wait_bounded(smem_u32(&bars[warp * TMA_STAGES + q]), (unsigned)(done / TMA_STAGES) & 1u);
+        ok = __all_sync(0xffffffffu, ok);
+        if (ok && lane < issuers) acc += *reinterpret_cast<const float*>(ring + (size_t)q * stage_bytes + (size_t)lane * slot_bytes);
+        __syncwarp();
+    }
+    if (!ok) {
+        if (lane == 0) atomicExch(status, 1);
+        for (; done < issued; ++done)
+            mbar_wait_bounded(smem_u32(&bars[warp * TMA_STAGES + done % TMA_STAGES]), (unsigned)(done / TMA_STAGES) & 1u);
+    }
+    if (acc == 123.456f) sink[0] = acc;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Final-layer nonzero sets.  The tile is cut into segments of SEG rows.
 //   count: seg_cnt[seg*ld + b] = #{ i in segment : X[i,b] != 0 }
 //   scan : per input b: nz_count[b] = total; seg_cnt becomes the exclusive prefix over segments

@@ -1943,6 +1943,33 @@ extern "C" int sdnn_probe_word_rate(int32_t store, int64_t table_words, double* 
 }
 
 // ---------------------------------------------------------------------------------------------
+// Tensor map of a table of rows for tile::gather4: a two-dimensional tensor [table_rows][row_bytes / 4] of floats in this
+// device's own memory, box = one row, no swizzle.  The driver's encoder is looked up at run time (no link against libcuda).
+namespace {
+int encode_row_map(CUtensorMap* tmap, float* table, int row_bytes, int64_t table_rows) {
+    typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                 const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || !fn || qres != cudaDriverEntryPointSuccess) {
+        cudaGetLastError();
+        return fail(nullptr, SDNN_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
+    }
+    const cuuint64_t dims[2] = {(cuuint64_t)(row_bytes / 4), (cuuint64_t)table_rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
+    const cuuint32_t box[2] = {(cuuint32_t)(row_bytes / 4), 1u};
+    const cuuint32_t estr[2] = {1u, 1u};
+    CUresult cr = reinterpret_cast<EncodeFn>(fn)(tmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, table, dims, strides, box, estr,
+                                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                                CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (cr != CUDA_SUCCESS) return fail(nullptr, SDNN_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)cr);
+    return SDNN_OK;
+}
+}  // namespace
+
+// ---------------------------------------------------------------------------------------------
 // Copy-engine gather probe (see sdnn_probe_tma_gather_rate in the header).
 extern "C" int sdnn_probe_tma_gather_rate(int32_t row_bytes, int64_t table_rows, int32_t gather4, double* rows_per_second) {
     if (!rows_per_second) return fail(nullptr, SDNN_ERR_INVALID_ARG, "rows_per_second is NULL");
@@ -1973,25 +2000,7 @@ extern "C" int sdnn_probe_tma_gather_rate(int32_t row_bytes, int64_t table_rows,
         cudaMemsetAsync(status, 0, sizeof(int), st);
         CUtensorMap tmap;
         memset(&tmap, 0, sizeof tmap);
-        if (gather4) {      // the table as a two-dimensional tensor [table_rows][row_bytes / 4] of floats, box = one row
-            typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                         const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                         CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-            void* fn = nullptr;
-            cudaDriverEntryPointQueryResult qres;
-            cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
-            if (e != cudaSuccess || !fn || qres != cudaDriverEntryPointSuccess) { cudaGetLastError(); rc = fail(nullptr, SDNN_ERR_CUDA, "cuTensorMapEncodeTiled is not available"); }
-            else {
-                const cuuint64_t dims[2] = {(cuuint64_t)(row_bytes / 4), (cuuint64_t)table_rows};
-                const cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
-                const cuuint32_t box[2] = {(cuuint32_t)(row_bytes / 4), 1u};
-                const cuuint32_t estr[2] = {1u, 1u};
-                CUresult cr = reinterpret_cast<EncodeFn>(fn)(&tmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, table, dims, strides, box, estr,
-                                                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
-                                                            CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-                if (cr != CUDA_SUCCESS) rc = fail(nullptr, SDNN_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)cr);
-            }
-        }
+        if (gather4) rc = encode_row_map(&tmap, table, row_bytes, table_rows);
         if (rc == SDNN_OK) {
             const unsigned rows_per_copy = gather4 ? 4u : 1u;
             const int issuers = (int)std::min<size_t>(32, 8192 / ((size_t)rows_per_copy * row_bytes));      // lanes of a warp that issue copies
@@ -2023,6 +2032,81 @@ extern "C" int sdnn_probe_tma_gather_rate(int32_t row_bytes, int64_t table_rows,
                 if (e != cudaSuccess || !(ms > 0.f)) rc = cuda_fail(nullptr, e, "copy-engine probe");
                 else if (gave_up) rc = fail(nullptr, SDNN_ERR_CUDA, "copy-engine probe: a wait for its copies ran out");
                 else *rows_per_second = (double)grid * issuers * TMA_WARPS * rows_per_copy * rounds / (ms / reps * 1e-3);
+            }
+        }
+    }
+    if (a) cudaEventDestroy(a);
+    if (b) cudaEventDestroy(b);
+    if (st) cudaStreamDestroy(st);
+    if (table) cudaFree(table);
+    if (sink) cudaFree(sink);
+    if (status) cudaFree(status);
+    return rc;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Both gather paths at once (see sdnn_probe_mixed_gather in the header).
+extern "C" int sdnn_probe_mixed_gather(int32_t row_bytes, int64_t table_rows, int32_t tma_rounds, int32_t lsu_per_group,
+                                       double* seconds, double* rows) {
+    if (!seconds || !rows) return fail(nullptr, SDNN_ERR_INVALID_ARG, "seconds or rows is NULL");
+    *seconds = 0.0; *rows = 0.0;
+    if (row_bytes != 64 && row_bytes != 256) return fail(nullptr, SDNN_ERR_INVALID_ARG, "row_bytes must be 64 or 256");
+    if (table_rows < 1 || (table_rows & (table_rows - 1)) || table_rows * row_bytes > (1LL << 30))
+        return fail(nullptr, SDNN_ERR_INVALID_ARG, "table_rows must be a power of two with table_rows * row_bytes <= 1 GiB");
+    if (tma_rounds < 0 || tma_rounds > (1 << 16) || lsu_per_group < 0 || lsu_per_group > (1 << 20) || (lsu_per_group & 7) ||
+        (tma_rounds == 0 && lsu_per_group == 0))
+        return fail(nullptr, SDNN_ERR_INVALID_ARG, "tma_rounds in [0, 65536], lsu_per_group a multiple of 8 in [0, 2^20], not both 0");
+    int dev = 0, sms = 0;
+    CU(nullptr, cudaGetDevice(&dev));
+    CU(nullptr, cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    float* table = nullptr;
+    float* sink = nullptr;
+    int* status = nullptr;
+    cudaEvent_t a = nullptr, b = nullptr;
+    cudaStream_t st = nullptr;
+    int rc = SDNN_OK;
+    const size_t bytes = (size_t)table_rows * row_bytes;
+    if (cudaMalloc(&table, bytes) != cudaSuccess || cudaMalloc(&sink, 256) != cudaSuccess || cudaMalloc(&status, sizeof(int)) != cudaSuccess ||
+        cudaStreamCreate(&st) != cudaSuccess || cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) {
+        cudaGetLastError();
+        rc = fail(nullptr, SDNN_ERR_OOM, "could not set up the probe");
+    } else {
+        cudaMemsetAsync(table, 0, bytes, st);
+        cudaMemsetAsync(status, 0, sizeof(int), st);
+        CUtensorMap tmap;
+        memset(&tmap, 0, sizeof tmap);
+        rc = encode_row_map(&tmap, table, row_bytes, table_rows);
+        if (rc == SDNN_OK) {
+            const int issuers = (int)std::min<size_t>(32, 8192 / ((size_t)4 * row_bytes));
+            const size_t smem = (size_t)TMA_WARPS * TMA_STAGES * issuers * 4 * row_bytes;
+            auto k64 = mixed_gather_probe_kernel<2, 8>;
+            auto k256 = mixed_gather_probe_kernel<8, 8>;
+            cudaError_t e = cudaFuncSetAttribute(row_bytes == 64 ? k64 : k256, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) rc = cuda_fail(nullptr, e, "mixed probe set-up");
+            else {
+                const int grid = sms, reps = 5;
+                const unsigned mask = (unsigned)(table_rows - 1);
+                auto launch = [&](unsigned seed) {
+                    if (row_bytes == 64) k64<<<grid, 1024, smem, st>>>(table, tmap, sink, status, mask, issuers, tma_rounds, lsu_per_group, seed);
+                    else k256<<<grid, 1024, smem, st>>>(table, tmap, sink, status, mask, issuers, tma_rounds, lsu_per_group, seed);
+                };
+                launch(17u); launch(18u);
+                cudaEventRecord(a, st);
+                for (int i = 0; i < reps; ++i) launch(101u + i);
+                cudaEventRecord(b, st);
+                e = cudaEventSynchronize(b);
+                float ms = 0.f;
+                int gave_up = 0;
+                if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, a, b);
+                if (e == cudaSuccess) e = cudaMemcpy(&gave_up, status, sizeof(int), cudaMemcpyDeviceToHost);
+                if (e == cudaSuccess) e = cudaGetLastError();
+                if (e != cudaSuccess || !(ms > 0.f)) rc = cuda_fail(nullptr, e, "mixed probe");
+                else if (gave_up) rc = fail(nullptr, SDNN_ERR_CUDA, "mixed probe: a wait for the copy engine ran out");
+                else {
+                    const int g = row_bytes / 32;
+                    *seconds = ms / reps * 1e-3;
+                    *rows = (double)grid * ((double)TMA_WARPS * issuers * 4 * tma_rounds + (double)(1024 - 32 * TMA_WARPS) / g * lsu_per_group);
+                }
             }
         }
     }

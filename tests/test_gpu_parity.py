@@ -892,6 +892,11 @@ def test_copy_engine_gather_probe_reports_rates_and_rejects_bad_sizes(torch_cuda
         with pytest.raises(pkg.SdnnError) as ei:
             pkg.probe_tma_gather_rate(row_bytes, rows, gather4)
         assert ei.value.code == -1
+    for tma, lsu in ((64, 0), (0, 256), (64, 256)):               # the two paths side by side, or either alone
+        sec, rows = pkg.probe_mixed_gather(64, 1 << 14, tma, lsu)
+        assert sec > 0 and rows > 0
+    with pytest.raises(pkg.SdnnError):
+        pkg.probe_mixed_gather(64, 1 << 14, 0, 0)
 
 
 def test_state_and_argument_errors(torch_cuda):

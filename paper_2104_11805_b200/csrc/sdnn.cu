@@ -1867,24 +1867,31 @@ extern "C" int sdnn_probe_gather_rate(int32_t row_bytes, int64_t table_rows, dou
         rc = fail(nullptr, SDNN_ERR_OOM, "could not allocate the probe's table");
     } else {
         cudaMemsetAsync(table, 0, bytes, st);
-        // threads per SM at which the rate stops growing: 1024 for rows of up to 64 bytes, 2048 for wider ones
-        const int g = row_bytes == 16 ? 1 : row_bytes / 32, grid = sms * (row_bytes >= 128 ? 8 : 4);      // 256-bit lanes
-        const int64_t groups = (int64_t)grid * 256 / g;
-        const int per_group = (int)std::max<int64_t>(8, ((int64_t)1 << 22) / groups / 8 * 8);
+        // the rate depends on the threads per SM (it peaks between 768 and 2048 depending on the row width): try 2 .. 8
+        // CTAs of 256 threads per SM and keep the best, so that the figure is what the path can do, not what one shape does
+        const int g = row_bytes == 16 ? 1 : row_bytes / 32;      // 256-bit lanes
         const unsigned mask = (unsigned)(table_rows - 1);
         float ms = 0.f;
-        switch (row_bytes) {
-            case 16: ms = run_gather_probe<1, 4>(table, sink, mask, per_group, grid, st, 20, a, b); break;
-            case 32: ms = run_gather_probe<1, 8>(table, sink, mask, per_group, grid, st, 20, a, b); break;
-            case 64: ms = run_gather_probe<2, 8>(table, sink, mask, per_group, grid, st, 20, a, b); break;
-            case 128: ms = run_gather_probe<4, 8>(table, sink, mask, per_group, grid, st, 20, a, b); break;
-            case 256: ms = run_gather_probe<8, 8>(table, sink, mask, per_group, grid, st, 20, a, b); break;
-            case 512: ms = run_gather_probe<16, 8>(table, sink, mask, per_group, grid, st, 20, a, b); break;
-            default: ms = run_gather_probe<32, 8>(table, sink, mask, per_group, grid, st, 20, a, b); break;
+        double best = 0.0;
+        for (int per_sm = 2; per_sm <= 8; ++per_sm) {
+            if (per_sm == 5 || per_sm == 7) continue;
+            const int grid = sms * per_sm;
+            const int64_t groups = (int64_t)grid * 256 / g;
+            const int per_group = (int)std::max<int64_t>(8, ((int64_t)1 << 22) / groups / 8 * 8);
+            switch (row_bytes) {
+                case 16: ms = run_gather_probe<1, 4>(table, sink, mask, per_group, grid, st, 10, a, b); break;
+                case 32: ms = run_gather_probe<1, 8>(table, sink, mask, per_group, grid, st, 10, a, b); break;
+                case 64: ms = run_gather_probe<2, 8>(table, sink, mask, per_group, grid, st, 10, a, b); break;
+                case 128: ms = run_gather_probe<4, 8>(table, sink, mask, per_group, grid, st, 10, a, b); break;
+                case 256: ms = run_gather_probe<8, 8>(table, sink, mask, per_group, grid, st, 10, a, b); break;
+                case 512: ms = run_gather_probe<16, 8>(table, sink, mask, per_group, grid, st, 10, a, b); break;
+                default: ms = run_gather_probe<32, 8>(table, sink, mask, per_group, grid, st, 10, a, b); break;
+            }
+            if (ms > 0.f) best = std::max(best, (double)groups * per_group / (ms * 1e-3));
         }
         cudaError_t e = cudaGetLastError();
-        if (e != cudaSuccess || !(ms > 0.f)) rc = cuda_fail(nullptr, e, "gather probe");
-        else *rows_per_second = (double)groups * per_group / (ms * 1e-3);
+        if (e != cudaSuccess || !(best > 0.0)) rc = cuda_fail(nullptr, e, "gather probe");
+        else *rows_per_second = best;
     }
     if (a) cudaEventDestroy(a);
     if (b) cudaEventDestroy(b);

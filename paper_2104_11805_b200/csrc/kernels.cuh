@@ -12,7 +12,9 @@
 // sits in a different 128-byte line.  The entries are therefore kept in slices of 16 rows, interleaved in
 // chunks of 4:
 //     entry q of row i  ->  slice_off[i/16] + (q/4)*64 + (i%16)*4 + q%4          (element offset)
-// so that the 16-byte chunks the row groups of a warp read in one step are contiguous.  A slice is padded
+// so that the chunks (16 bytes of values, 8 or 16 bytes of indices: the index array holds 16-bit indices for nets of at
+// most 65536 neurons, template parameter I16 of the layer kernels) the row groups of a warp read in one step are
+// contiguous.  A slice is padded
 // to the longest of its rows rounded up to 8; padding has index 0 and value 0 and is never updated.  The
 // transposed matrix (columns as "rows", for the backward product without atomics) uses the same layout over
 // the columns sorted by descending length.

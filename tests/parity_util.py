@@ -29,6 +29,13 @@ density near a kink is about 1 / (2.5 * S / sqrt(m)) with S = |b| + sum|w x|, an
 tau = 64 * 2^-24 * S of it with probability about 2 * tau * sqrt(m) / (2.5 * S) = 3e-6 * sqrt(m), i.e. 1e-5 to
 2e-5 for rows of 10 to 40 live terms.  assert_few_ambiguous holds a run to AMBIGUOUS_RATE = 1e-4 of its
 entries (plus a handful for small runs).
+
+Depth.  tau covers the rounding of ONE layer's sum.  A thousand layers down, the layer's input x^{k-1} itself
+differs between the two sides by the rounding accumulated below (measured 5e-6 * max|x| at 960 layers of the
+65536-neuron live net, more than the 4e-6 that tau allows), so that one entry in some 1e9 can sit outside tau
+and still be decided differently for no fault of the layer.  Such an entry gets a second, exact hearing: the
+float64 layer is evaluated on the GPU's OWN x^{k-1} (`relayer`), and there the two decisions may differ only
+within tau again.  An entry that fails both is a hard mismatch.
 """
 from __future__ import annotations
 
@@ -97,8 +104,11 @@ def check_close(gpu, ora, what=""):
 class KinkProtocol:
     """mask_hook for OracleNet.train_step; `gpu_x(k)` returns the GPU's x^k [B, n] (fp32)."""
 
-    def __init__(self, gpu_x, clamp=32.0, tau_ulps=TAU_ULPS):
-        self.gpu_x, self.clamp, self.tau_ulps = gpu_x, float(clamp), tau_ulps
+    def __init__(self, gpu_x, clamp=32.0, tau_ulps=TAU_ULPS, relayer=None):
+        """relayer(k, x_prev) -> (z, scale): float64 pre-activations of layer k (1-based) and their rounding scale
+        for the input x_prev [B, n]; used only for entries that differ outside tau (see the module docstring)."""
+        self.gpu_x, self.clamp, self.tau_ulps, self.relayer = gpu_x, float(clamp), tau_ulps, relayer
+        self.second_hearing = 0   # entries outside tau that were settled on the GPU's own layer input
         self.ambiguous = 0
         self.flipped = 0
         self.entries = 0
@@ -115,7 +125,16 @@ class KinkProtocol:
         self.entries += mask.size
         self.ambiguous += int(amb.sum())
         self.flipped += int(differ.sum())
-        self.hard_mismatch += int((differ & ~amb).sum())
+        hard = differ & ~amb
+        if hard.any() and self.relayer is not None:
+            z2, scale2 = self.relayer(k, self.gpu_x(k - 1).astype(np.float64))
+            m2 = ((z2 > 0.0) & (z2 < self.clamp)).astype(np.float64)
+            margin2 = np.minimum(np.abs(z2), np.abs(z2 - self.clamp))
+            settled = hard & ((mg == m2) | ((margin2 <= self.tau_ulps * 2.0 ** -24 * scale2) & (scale2 > 0.0)))
+            self.second_hearing += int(settled.sum())
+            hard &= ~settled
+            amb = amb | settled          # the oracle continues with the GPU's decision there too
+        self.hard_mismatch += int(hard.sum())
         if differ.any():
             self.worst = max(self.worst, float((margin[differ] / np.maximum(tau[differ], 1e-300)).max()))
         return np.where(amb, mg, mask)

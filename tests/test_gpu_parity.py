@@ -4,6 +4,8 @@ Same seeded inputs on both sides; activations, deltas, gradients, updated weight
 agree within 1e-4 (metric in parity_util.rel_err); derivative masks and final-layer nonzero sets must
 agree bit for bit outside the kink-ambiguous entries (parity_util.KinkProtocol).
 """
+import os
+
 import numpy as np
 import pytest
 
@@ -69,7 +71,7 @@ def train_parity(torch, arrays, batches, eta, update_bias=False, flags=0, clamp=
                 acts[k] = h.get_activations(k, B)
             return acts[k]
 
-        proto = KinkProtocol(gpu_x, clamp=clamp)
+        proto = KinkProtocol(gpu_x, clamp=clamp, relayer=lambda k, xp: ora.forward_layer(k - 1, xp, want_scale=True)[::2])
         out = ora.train_step(x0, y, eta, mask_hook=None if sigmoid else proto)      # the sigmoid has no kinks
         assert proto.hard_mismatch == 0, f"{proto.hard_mismatch} derivative-mask mismatches outside the ambiguous set " \
                                          f"(worst margin/tau = {proto.worst:.3g})"
@@ -496,7 +498,12 @@ def check_update(w_gpu, w_before, w_oracle, what=""):
     return worst / max(np.abs(u_ora).max(), 1e-300), bool(np.abs(u_ora).max() > 2.0 ** -20 * np.abs(w_before).max())
 
 
-@pytest.mark.parametrize("spec", [gen.CFG5.scaled(65536, 256).live(), gen.CFG5.scaled(65536, 240).paper_setup()])
+# depth of the deep config-5 case: 256 layers by default (17 GB of host memory); SDNN_TEST_DEEP_LAYERS=1920 is the whole
+# configuration (128 GB of host memory for the float64 oracle, ten minutes)
+DEEP_LAYERS = int(os.environ.get("SDNN_TEST_DEEP_LAYERS", "256"))
+
+
+@pytest.mark.parametrize("spec", [gen.CFG5.scaled(65536, DEEP_LAYERS).live(), gen.CFG5.scaled(65536, 240).paper_setup()])
 def test_train_cfg5_full_width_deep_in_the_benchmark_launch_configuration(torch_cuda, spec):
     """Config 5 at full width (65536 neurons, B = 16) and as deep as a host of a few tens of GB holds the float64 oracle
     (256 layers for the live companion, 240 with the paper's own setup: about 17 GB of host memory), on the handle bench.py times: default flags, no
@@ -512,7 +519,7 @@ def test_train_cfg5_full_width_deep_in_the_benchmark_launch_configuration(torch_
     h = pkg.Sdnn.create(rp, col, val, bias, max_batch=B, train=True, activation=pkg.ACT_SIGMOID if sigmoid else pkg.ACT_CLAMPED_RELU)
     ora = OracleNet(rp, col, val, bias, activation="sigmoid" if sigmoid else "clamped_relu")
     parity_util.reset_worst()
-    ambiguous = entries = 0
+    ambiguous = entries = second = 0
     worst_update, moved = 0.0, np.zeros(L, dtype=bool)      # moved[l]: the update of layer l is well above one fp32 rounding of W
     for step, (x0, y) in enumerate(batches_for(spec, B, 2)):
         if step:
@@ -521,10 +528,12 @@ def test_train_cfg5_full_width_deep_in_the_benchmark_launch_configuration(torch_
                 h.set_weights(l, ora.w[l], ora.bias[l])
         before = [w.copy() for w in ora.w]
         loss = h.train_step(torch.from_numpy(x0).cuda(), torch.from_numpy(y).cuda(), B, eta, want_loss=True)
-        proto = KinkProtocol(lambda k: h.get_activations(k, B))
+        proto = KinkProtocol(lambda k: h.get_activations(k, B),
+                             relayer=lambda k, xp: ora.forward_layer(k - 1, xp, want_scale=True)[::2])
         out = ora.train_step(x0, y, eta, mask_hook=None if sigmoid else proto, keep=("x",))
         assert proto.hard_mismatch == 0, f"{proto.hard_mismatch} derivative-mask mismatches outside the ambiguous set"
-        ambiguous += proto.ambiguous; entries += proto.entries
+        ambiguous += proto.ambiguous + proto.second_hearing; entries += proto.entries
+        second += proto.second_hearing
         assert abs(loss - out["loss"]) <= TOL * abs(out["loss"])
         for l in range(L):
             w = h.get_weights(l, want_bias=False)
@@ -540,7 +549,8 @@ def test_train_cfg5_full_width_deep_in_the_benchmark_launch_configuration(torch_
     # the sigmoid net's gradient fades with depth (f' <= 1/4 per layer), so only its upper layers move; the live net moves everywhere
     assert moved[-1] and (sigmoid or moved.all()), f"vacuous: only {int(moved.sum())} of {L} layers moved"
     print(spec.name, L, "layers:", parity_util.WORST, "layers whose update is well above fp32 rounding:", int(moved.sum()),
-          "worst update error among them (of the largest update)", worst_update, "ambiguous", ambiguous, "of", entries)
+          "worst update error among them (of the largest update)", worst_update, "ambiguous", ambiguous, "of", entries,
+          "settled on the GPU's own layer input:", second)
     h.destroy()
 
 

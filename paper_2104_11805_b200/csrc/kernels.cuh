@@ -621,6 +621,120 @@ forward_window_kernel(Windowed m, const float* __restrict__ xin, float* __restri
 }
 
 // ---------------------------------------------------------------------------------------------
+// The same layer for chunks of 32 inputs with four rows side by side in a warp: a group of eight lanes owns a row, a
+// lane four inputs of it.  Per four stored entries a lane group reads its row's columns (one 64-bit load) and values (one
+// 128-bit load) from the warp's ring, whose four row slots are staggered over the banks, and each window row with one
+// 128-bit load per lane: 128 contiguous bytes per group, four wavefronts per warp instruction for four entries, and two
+// packed FMAs per lane and entry.  About 38 shared-memory wavefronts per row of 32 entries, against 44 and six instructions
+// per FMA for the lane-per-input mapping above.  32 warps per CTA; the ring holds the piece in use and the next one.
+constexpr int W32_THREADS = 1024;
+constexpr int W32_ROWS = 4;                    // rows side by side in a warp
+constexpr int W32_RING = 2;                    // stages of a warp's entry ring
+constexpr int W32_SLOT = 208;                  // bytes of one row's piece in the ring: 64 of columns, 128 of values, 16 of padding
+                                               // (52 words: the four rows' slots start 20 banks apart)
+constexpr int W32_STAGE = W32_ROWS * W32_SLOT;
+constexpr int W32_RING_BYTES = (W32_THREADS / 32) * W32_RING * W32_STAGE;
+
+__global__ void __launch_bounds__(W32_THREADS, 1)
+forward_window32_kernel(Windowed m, const float* __restrict__ xin, float* __restrict__ xout, int ld, int chunks, int splits,
+                        float clamp, int act, int pdl) {
+    extern __shared__ __align__(16) unsigned char window_smem[];
+    constexpr int TC = 32;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const int grp = lane >> 3, sub = lane & 7;
+    unsigned char* ring = window_smem + warp * (W32_RING * W32_STAGE);
+    float* window = reinterpret_cast<float*>(window_smem + W32_RING_BYTES);      // [wlen][32]
+    // this lane's 16-byte shares of a full piece (4 rows x (4 + 8) shares): share `lane`, and share `lane + 32` for lanes < 16
+    const int sh_row0 = lane / 12, sh_q0 = lane - sh_row0 * 12;
+    const int sh_row1 = (lane + 32) / 12, sh_q1 = (lane + 32) - sh_row1 * 12;
+    if (pdl) grid_dependency_wait();
+    if (pdl == 2) grid_launch_dependents();
+    const int per_group = chunks * splits;
+    const int items = m.groups * per_group;
+    for (int item = blockIdx.x; item < items; item += gridDim.x) {
+        const int g = item / per_group, rest = item - g * per_group;
+        const int split = rest / chunks, t0 = (rest - split * chunks) * TC;
+        const int c0 = m.g_c0[g], wlen = m.g_wlen[g], k = m.g_k[g];
+        const int g0 = m.g_row0[g], per_split = (m.g_row0[g + 1] - g0 + splits - 1) / splits;
+        const int r0 = g0 + split * per_split + warp * W32_ROWS, r1 = min(m.g_row0[g + 1], g0 + (split + 1) * per_split);
+        const int rstep = nwarps * W32_ROWS;
+        const unsigned short* gcol = m.col + m.g_ebase[g];
+        const float* gval = m.val + m.g_ebase[g];
+        // one 16-byte share of a piece (rows rbase .. rbase + 3, entries t .. t + n - 1 of each): columns first (n / 8
+        // shares per row), then values (n / 4)
+        auto share = [&](unsigned char* stage, int rbase, int t, int n, int rr, int q) {
+            const int row = rbase + rr;
+            if (rr < W32_ROWS && row < r1) {
+                const size_t at = (size_t)(row - g0) * k + t;
+                if (q < (n >> 3)) cp_async16(stage + rr * W32_SLOT + q * 16, gcol + at + q * 8);
+                else if (q - (n >> 3) < (n >> 2)) cp_async16(stage + rr * W32_SLOT + 64 + (q - (n >> 3)) * 16, gval + at + (q - (n >> 3)) * 4);
+            }
+        };
+        auto fetch = [&](int stage_no, int rbase, int t) {
+            if (rbase < r1 && t < k) {
+                unsigned char* stage = ring + stage_no * W32_STAGE;
+                const int n = min(32, k - t);                            // entries of the piece, a multiple of 8
+                if (n == 32) {
+                    share(stage, rbase, t, 32, sh_row0, sh_q0);
+                    if (lane < 16) share(stage, rbase, t, 32, sh_row1, sh_q1);
+                } else {
+                    const int per_row = (n >> 3) + (n >> 2);
+                    for (int p = lane; p < W32_ROWS * per_row; p += 32) share(stage, rbase, t, n, p / per_row, p % per_row);
+                }
+            }
+            cp_async_commit();
+        };
+        __syncthreads();                                  // the previous item's readers are done with the window and the rings
+        fetch(0, r0, 0);
+        for (int p = threadIdx.x; p < wlen * (TC / 4); p += blockDim.x)
+            cp_async16(window + p * 4, xin + (size_t)(c0 + (p >> 3)) * ld + t0 + (p & 7) * 4);
+        cp_async_commit();
+        cp_async_wait<0>();
+        __syncthreads();
+        const unsigned xw = (unsigned)__cvta_generic_to_shared(window) + sub * 16;
+        int stage_no = 0;
+        for (int rbase = r0; rbase < r1; rbase += rstep) {
+            const int row = rbase + grp;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int t = 0; t < k; t += 32) {
+                __syncwarp();                             // every lane has finished reading the stage that is refilled now
+                if (t + 32 < k) fetch(stage_no ^ 1, rbase, t + 32); else fetch(stage_no ^ 1, rbase + rstep, 0);
+                cp_async_wait<1>();                       // this lane's share of the current piece has landed ...
+                __syncwarp();                             // ... and so has every other lane's
+                const int n = min(32, k - t);
+                const unsigned slot = (unsigned)__cvta_generic_to_shared(ring + stage_no * W32_STAGE + grp * W32_SLOT);
+                if (row < r1) {
+#pragma unroll 2
+                    for (int j = 0; j < n; j += 4) {
+                        unsigned ca, cb;
+                        float4 w, x0, x1, x2, x3;
+                        asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(ca), "=r"(cb) : "r"(slot + j * 2));
+                        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(w.x), "=f"(w.y), "=f"(w.z), "=f"(w.w) : "r"(slot + 64 + j * 4));
+                        // a window row is 128 bytes: address = window + column * 128 (+ this lane's 16 bytes)
+                        const unsigned a0 = xw + ((ca & 0xffffu) << 7), a1 = xw + ((ca >> 16) << 7);
+                        const unsigned a2 = xw + ((cb & 0xffffu) << 7), a3 = xw + ((cb >> 16) << 7);
+                        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(x0.x), "=f"(x0.y), "=f"(x0.z), "=f"(x0.w) : "r"(a0));
+                        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(x1.x), "=f"(x1.y), "=f"(x1.z), "=f"(x1.w) : "r"(a1));
+                        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(x2.x), "=f"(x2.y), "=f"(x2.z), "=f"(x2.w) : "r"(a2));
+                        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(x3.x), "=f"(x3.y), "=f"(x3.z), "=f"(x3.w) : "r"(a3));
+                        f4_fma(w.x, x0, acc); f4_fma(w.y, x1, acc); f4_fma(w.z, x2, acc); f4_fma(w.w, x3, acc);
+                    }
+                }
+                stage_no ^= 1;
+            }
+            if (row < r1) {                               // also the rows of a group without entries (k = 0): x = f(b)
+                const float b = m.bias[row];
+                acc.x += b; acc.y += b; acc.z += b; acc.w += b;
+                f4_activate(acc, act, clamp);
+                st_f4(xout + (size_t)m.out[row] * ld + t0 + sub * 4, acc);
+            }
+        }
+        cp_async_wait<0>();
+    }
+    if (pdl == 1) grid_launch_dependents();
+}
+
+// ---------------------------------------------------------------------------------------------
 // Output gradient (final-layer gradient equation) and loss: delta^L = (x^L - y) (.) f'(x^L) on the valid
 // batch columns, 0 on the padding; J = 1/(2B) sum (x^L - y)^2 accumulated in double, one atomic per block.
 __global__ void __launch_bounds__(256)

@@ -491,13 +491,39 @@ cudaError_t launch_forward_window_tc(sdnn* h, const LayerMem& lm, const Windowed
                               h->pdl ? PDL_AT_END : 0);
 }
 
+// chunks of 32 inputs: the kernel with four rows side by side in a warp, where its larger entry ring leaves room for the window
+cudaError_t launch_forward_window32(sdnn* h, const LayerMem& lm, const Windowed& m, const float* xin, float* xout, int ld, int cols) {
+    static bool configured[64] = {};
+    if (h->device < 64 && !configured[h->device]) {
+        cudaError_t e = cudaFuncSetAttribute(forward_window32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e != cudaSuccess) return e;
+        configured[h->device] = true;
+    }
+    const int chunks = cols / 32;
+    int splits = 1;
+    const int avg_rows = std::max(1, h->N / std::max(1, lm.groups));
+    while (lm.groups * chunks * splits < 2 * h->sms && avg_rows / (splits * 2) >= 128 && splits < 32) splits *= 2;
+    const int items = lm.groups * chunks * splits;
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(std::max(1, std::min(items, h->sms))); lc.blockDim = dim3(W32_THREADS);
+    lc.dynamicSmemBytes = W32_RING_BYTES + (size_t)std::max(lm.max_wlen, 1) * 32 * sizeof(float);
+    lc.stream = h->launch_stream ? h->launch_stream : h->stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = at; lc.numAttrs = h->pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&lc, forward_window32_kernel, m, xin, xout, ld, chunks, splits, h->cfg.clamp, (int)h->cfg.activation,
+                              h->pdl ? PDL_AT_END : 0);
+}
+
 void launch_forward_window(sdnn* h, int layer, const float* xin, float* xout, int ld, int cols) {
     const LayerMem& lm = h->lay[layer];
     Windowed m;
     m.col = lm.w_col; m.val = lm.w_val; m.out = lm.w_out;
     m.bias = h->d_bias + (size_t)layer * h->N;
     m.g_row0 = lm.w_g_row0; m.g_c0 = lm.w_g_c0; m.g_wlen = lm.w_g_wlen; m.g_ebase = lm.w_g_ebase; m.g_k = lm.w_g_k; m.groups = lm.groups;
-    if (cols >= 32) launch_forward_window_tc<32>(h, lm, m, xin, xout, ld, cols);
+    if (cols >= 32 && W32_RING_BYTES + (size_t)lm.max_wlen * 128 <= 227u * 1024u) launch_forward_window32(h, lm, m, xin, xout, ld, cols);
+    else if (cols >= 32) launch_forward_window_tc<32>(h, lm, m, xin, xout, ld, cols);
     else if (cols == 16) launch_forward_window_tc<16>(h, lm, m, xin, xout, ld, cols);
     else if (cols == 8) launch_forward_window_tc<8>(h, lm, m, xin, xout, ld, cols);
     else launch_forward_window_tc<4>(h, lm, m, xin, xout, ld, cols);

@@ -708,6 +708,15 @@ def test_infer_reordered_hidden_blocks(torch_cuda, cnt, max_batch, host, mode):
 
 
 @pytest.mark.parametrize("mode", sorted(REORDER_MODES))
+def test_infer_reordered_wide_windows(torch_cuda, mode):
+    """Blocks of 1500 neurons: windows near the cap of 1536 tile rows, for which the shared-memory kernel with the small
+    entry ring is the one that still fits beside the window."""
+    spec = block_spec(3000, 3, 1500).shuffled()
+    infer_parity(torch_cuda, gen.network(spec), gen.inputs(spec, 70), 128, expect_nonempty=True,
+                 flags=REORDER_MODES[mode], expect_grouped=3)
+
+
+@pytest.mark.parametrize("mode", sorted(REORDER_MODES))
 def test_infer_reordered_mixed_layers_and_weights_in_caller_order(torch_cuda, mode):
     """Layers with block structure (hidden) alternate with uniformly random ones: the former are regrouped, the latter keep
     the default layout with their rows moved to their neurons' new numbers.  sdnn_get_weights returns the caller's arrays

@@ -378,7 +378,9 @@ def main():
     ap.add_argument("--averaged", action="store_true",
                     help="train workloads: the averaged form of the minibatch step (one batch-averaged gradient vector is "
                          "backpropagated; sdnn_train_step_averaged) instead of the exact minibatch step")
-    ap.add_argument("--flags", type=lambda s: int(s, 0), default=0, help="extra SDNN_FLAG_* bits")
+    ap.add_argument("--flags", type=lambda s: int(s, 0), default=None,
+                    help="SDNN_FLAG_* bits of the handle; default: 0, except 0x300 (set-up reordering + operand windows in shared "
+                         "memory, both part of the untimed set-up) for the config-4 workloads, whose layers have block structure")
     ap.add_argument("--batch", type=int, default=None, help="train workloads: another minibatch size on the same net")
     ap.add_argument("--study", default=None, choices=["probes", "tensor"],
                     help="instead of a workload: 'probes' = the operand-path probes (random row gathers out of L2, out of shared "
@@ -396,6 +398,8 @@ def main():
     if args.study == "tensor":
         return study_tensor()
     spec, kind, batch, n_inputs = WORKLOADS[args.workload]
+    if args.flags is None:
+        args.flags = 0x300 if args.workload.startswith("cfg4") else 0
     if args.tile and kind == "infer":
         batch = args.tile
     if args.batch and kind == "train":
@@ -588,9 +592,11 @@ def main():
 
     # -------------------------------------------------------------------- inference: the same call with dead inputs dropped
     compaction = None
-    if kind == "infer" and not args.no_compaction and not (flags & pkg.FLAG_REORDER):
+    if kind == "infer" and not args.no_compaction:
         with torch.cuda.stream(stream):
-            hc = pkg.Sdnn.create_deferred(L, N, [spec.nnz_per_layer] * L, max_batch=batch, flags=flags | pkg.FLAG_SKIP_DEAD,
+            # dropping dead inputs runs on the default layout (it does not combine with the set-up reordering)
+            hc = pkg.Sdnn.create_deferred(L, N, [spec.nnz_per_layer] * L, max_batch=batch,
+                                          flags=(flags & ~(pkg.FLAG_REORDER | pkg.FLAG_SMEM_WINDOWS)) | pkg.FLAG_SKIP_DEAD,
                                           stream=stream.cuda_stream, device=local_rank)
             for l in range(L):
                 hc.load_layer(l, *gen.layer(spec, l))
@@ -639,7 +645,7 @@ def main():
     else:
         batch = h.infer_tile_width()           # the library narrows the tile when two of them would not fit in L2
         tiles = (n_inputs + batch - 1) // batch
-        dom = "forward_window_kernel" if h.windowed_layers() == L else "forward_kernel"
+        dom = "forward_window32_kernel" if h.windowed_layers() == L else "forward_kernel"
         extra_reorder = {"grouped_layers": h.grouped_layers(), "windowed_layers": h.windowed_layers()}
         per_launch_ms = ms_per_step / (tiles * L)      # includes the (small) transpose and count kernels of each tile
         # per launch: the layer's indices and values once, the activation tile read and written once
@@ -713,7 +719,8 @@ def main():
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {**workload_config(args.workload, spec, kind, batch, args.averaged),
                        "parallelism": "replicas only (no collective)" if kind == "train" else "batch sharded over ranks, no collective",
-                       "inputs_per_step_per_gpu": n_inputs, "setup_seconds": setup_s, "device_bytes": h.device_bytes()},
+                       "inputs_per_step_per_gpu": n_inputs, "setup_seconds": setup_s, "device_bytes": h.device_bytes(),
+                       "handle_flags": hex(flags)},
             "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
             "compaction_mode": compaction,
         }

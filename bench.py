@@ -261,6 +261,17 @@ def study_probes():
         out["both_paths"][str(rb)] = rec
     for name, store in (("load4", 0), ("store4", 1)):
         out["words"][name] = pkg.probe_word_rate(store, 1 << 21) / sms / clk       # an 8 MB value array (one layer of the largest net)
+    # 64-byte rows in strict batches: rate and round trip against the rows in flight per SM
+    out["rows_in_flight"] = []
+    for threads in (128, 256, 512, 1024):
+        for loads in (1, 2, 4, 8, 16):
+            try:
+                rate = pkg.probe_gather_inflight(65536, threads, loads) / sms / clk
+            except pkg.SdnnError:
+                continue          # that many loads per lane at that many threads do not fit the registers
+            inflight = threads // 2 * loads
+            out["rows_in_flight"].append({"threads_per_sm": threads, "loads_per_lane": loads, "rows_in_flight_per_sm": inflight,
+                                          "rate": rate, "round_trip_clk": inflight / rate})
     print(json.dumps(out), flush=True)
 
 

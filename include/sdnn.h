@@ -271,6 +271,19 @@ int sdnn_mirror_mismatches(sdnn_t* h, int32_t layer, int64_t* count_out);
 int sdnn_probe_gather_rate(int32_t row_bytes, int64_t table_rows, double* rows_per_second);
 
 /*
+ * How the gather rate depends on the rows in flight (diagnostic; the paper has no counterpart).  The 64-byte random
+ * rows of sdnn_probe_gather_rate, but in strict batches: every lane keeps exactly `loads_in_flight` (1, 2, 4, 8 or 16)
+ * 256-bit loads in flight and starts its next batch only when the last of them has returned, with `threads_per_sm`
+ * (a multiple of 128, at most 2048) resident threads per SM: threads_per_sm / 2 * loads_in_flight rows in flight per
+ * SM.  rows_per_second (host double*) over that number is the latency-throughput curve of the path; rows in flight
+ * divided by the rate per SM and clock is the round trip.  It tells whether a layer kernel that stays below the rate of
+ * sdnn_probe_gather_rate lacks loads in flight or loses its time elsewhere.  SDNN_ERR_INVALID_ARG if the combination
+ * does not fit an SM's registers (all CTAs must be resident for the figure to mean what it says).  table_rows as in
+ * sdnn_probe_gather_rate.  Allocates and frees its own table and stream; synchronises.
+ */
+int sdnn_probe_gather_inflight(int64_t table_rows, int32_t threads_per_sm, int32_t loads_in_flight, double* rows_per_second);
+
+/*
  * Measures the alternative to keeping two copies of a training layer's values (diagnostic; the paper has no
  * counterpart): with ONE value array in row-major order, the column units of the transposed product would reach each
  * value through a position map, i.e. read (and, to apply the update, write) single 4-byte words at scattered places.

@@ -56,6 +56,7 @@ _PROTOS = {
     "sdnn_get_gradient": (ctypes.c_int, [_vp, _i32, _vp]),
     "sdnn_mirror_mismatches": (ctypes.c_int, [_vp, _i32, ctypes.POINTER(_i64)]),
     "sdnn_probe_gather_rate": (ctypes.c_int, [_i32, _i64, ctypes.POINTER(ctypes.c_double)]),
+    "sdnn_probe_gather_inflight": (ctypes.c_int, [_i64, _i32, _i32, ctypes.POINTER(ctypes.c_double)]),
     "sdnn_probe_tma_gather_rate": (ctypes.c_int, [_i32, _i64, _i32, ctypes.POINTER(ctypes.c_double)]),
     "sdnn_probe_mixed_gather": (ctypes.c_int, [_i32, _i64, _i32, _i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]),
     "sdnn_probe_word_rate": (ctypes.c_int, [_i32, _i64, ctypes.POINTER(ctypes.c_double)]),
@@ -154,6 +155,17 @@ def probe_gather_rate(row_bytes, table_rows):
     lib = load_library()
     out = ctypes.c_double(0.0)
     rc = lib.sdnn_probe_gather_rate(row_bytes, table_rows, ctypes.byref(out))
+    if rc != 0:
+        raise SdnnError(rc, (lib.sdnn_last_error(None) or b"").decode())
+    return out.value
+
+
+def probe_gather_inflight(table_rows, threads_per_sm, loads_in_flight):
+    """sdnn_probe_gather_inflight: 64-byte random rows per second with exactly threads_per_sm / 2 * loads_in_flight rows
+    in flight per SM."""
+    lib = load_library()
+    out = ctypes.c_double(0.0)
+    rc = lib.sdnn_probe_gather_inflight(table_rows, threads_per_sm, loads_in_flight, ctypes.byref(out))
     if rc != 0:
         raise SdnnError(rc, (lib.sdnn_last_error(None) or b"").decode())
     return out.value

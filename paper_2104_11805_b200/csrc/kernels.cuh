@@ -1401,6 +1401,33 @@ gather_probe_kernel(const float* __restrict__ table, float* __restrict__ sink, u
 }
 
 // ---------------------------------------------------------------------------------------------
+// How many rows must be in flight for the gather rate above?  The same 64-byte random rows (two lanes per row, one
+// 256-bit load per lane), but in strict batches: a lane issues F loads, and the row numbers of its next batch depend on
+// the sum of what these returned (always zero, which the compiler cannot know), so that exactly F loads per lane are
+// in flight and nothing of the next batch starts before the last of them is back.  With T resident threads per SM that
+// is T/2 * F rows in flight per SM; rows per clock against that number is the latency-throughput curve of the path, and
+// rows in flight / rate is its round trip.
+template <int F>
+__global__ void __launch_bounds__(128, 1)
+gather_inflight_probe_kernel(const float* __restrict__ table, float* __restrict__ sink, unsigned row_mask, int batches, unsigned seed) {
+    const int tid = blockIdx.x * blockDim.x + threadIdx.x;
+    const int sub = threadIdx.x & 1;
+    unsigned st = (unsigned)(tid >> 1) * 2654435761u + seed;
+    float acc = 0.f;
+    for (int q = 0; q < batches; ++q) {
+        unsigned c[F];
+#pragma unroll
+        for (int u = 0; u < F; ++u) { st = st * 1664525u + 1013904223u; c[u] = ((st >> 8) + __float_as_uint(acc)) & row_mask; }
+        Lane<8> v[F];
+#pragma unroll
+        for (int u = 0; u < F; ++u) lane_gather(v[u], table + (size_t)c[u] * 16 + sub * 8);
+#pragma unroll
+        for (int u = 0; u < F; ++u) acc += lane_sum(v[u]);
+    }
+    if (acc == 123.456f) sink[0] = acc;      // the table is all zero: never taken, keeps the loads alive
+}
+
+// ---------------------------------------------------------------------------------------------
 // Probe of the alternative to the second copy of the values: one value array in row-major order that the column
 // units would read, or read and write, one 4-byte word at a time at scattered places (through a position map).  Eight
 // accesses in flight per lane, indices made in registers.  STORE: 0 = scattered 4-byte loads, 1 = scattered 4-byte stores

@@ -1928,6 +1928,77 @@ extern "C" int sdnn_probe_gather_rate(int32_t row_bytes, int64_t table_rows, dou
 }
 
 // ---------------------------------------------------------------------------------------------
+// Gather rate against rows in flight (see sdnn_probe_gather_inflight in the header).
+namespace {
+template <int F>
+int run_inflight_probe(const float* table, float* sink, unsigned mask, int ctas_per_sm, int sms, cudaStream_t st, cudaEvent_t a,
+                       cudaEvent_t b, double* rate) {
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gather_inflight_probe_kernel<F>, 128, 0) != cudaSuccess) { cudaGetLastError(); occ = 0; }
+    if (occ < ctas_per_sm) return SDNN_ERR_INVALID_ARG;      // not all resident: the figure would not be what it claims
+    const int grid = sms * ctas_per_sm;
+    const int64_t lanes_pairs = (int64_t)grid * 64;
+    const int batches = (int)std::max<int64_t>(4, ((int64_t)1 << 23) / (lanes_pairs * F));      // launches of about 40 us: ramp and drain are a few per cent
+    const int reps = 10;
+    for (int i = 0; i < 2; ++i) gather_inflight_probe_kernel<F><<<grid, 128, 0, st>>>(table, sink, mask, batches, 17u + i);
+    cudaEventRecord(a, st);
+    for (int i = 0; i < reps; ++i) gather_inflight_probe_kernel<F><<<grid, 128, 0, st>>>(table, sink, mask, batches, 101u + i);
+    cudaEventRecord(b, st);
+    cudaEventSynchronize(b);
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, a, b);
+    if (!(ms > 0.f)) return SDNN_ERR_CUDA;
+    *rate = (double)lanes_pairs * F * batches * reps / (ms * 1e-3);
+    return SDNN_OK;
+}
+}  // namespace
+
+extern "C" int sdnn_probe_gather_inflight(int64_t table_rows, int32_t threads_per_sm, int32_t loads_in_flight, double* rows_per_second) {
+    if (!rows_per_second) return fail(nullptr, SDNN_ERR_INVALID_ARG, "rows_per_second is NULL");
+    *rows_per_second = 0.0;
+    if (table_rows < 1 || (table_rows & (table_rows - 1)) || table_rows * 64 > (1LL << 30))
+        return fail(nullptr, SDNN_ERR_INVALID_ARG, "table_rows must be a power of two with table_rows * 64 <= 1 GiB");
+    if (threads_per_sm < 128 || threads_per_sm > 2048 || threads_per_sm % 128)
+        return fail(nullptr, SDNN_ERR_INVALID_ARG, "threads_per_sm must be a multiple of 128 between 128 and 2048");
+    if (loads_in_flight != 1 && loads_in_flight != 2 && loads_in_flight != 4 && loads_in_flight != 8 && loads_in_flight != 16)
+        return fail(nullptr, SDNN_ERR_INVALID_ARG, "loads_in_flight must be 1, 2, 4, 8 or 16");
+    int dev = 0, sms = 0;
+    CU(nullptr, cudaGetDevice(&dev));
+    CU(nullptr, cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    float* table = nullptr;
+    float* sink = nullptr;
+    cudaEvent_t a = nullptr, b = nullptr;
+    cudaStream_t st = nullptr;
+    int rc = SDNN_OK;
+    const size_t bytes = (size_t)table_rows * 64;
+    if (cudaMalloc(&table, bytes) != cudaSuccess || cudaMalloc(&sink, 256) != cudaSuccess || cudaStreamCreate(&st) != cudaSuccess ||
+        cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) {
+        cudaGetLastError();
+        rc = fail(nullptr, SDNN_ERR_OOM, "could not allocate the probe's table");
+    } else {
+        cudaMemsetAsync(table, 0, bytes, st);
+        const unsigned mask = (unsigned)(table_rows - 1);
+        const int cps = threads_per_sm / 128;
+        switch (loads_in_flight) {
+            case 1: rc = run_inflight_probe<1>(table, sink, mask, cps, sms, st, a, b, rows_per_second); break;
+            case 2: rc = run_inflight_probe<2>(table, sink, mask, cps, sms, st, a, b, rows_per_second); break;
+            case 4: rc = run_inflight_probe<4>(table, sink, mask, cps, sms, st, a, b, rows_per_second); break;
+            case 8: rc = run_inflight_probe<8>(table, sink, mask, cps, sms, st, a, b, rows_per_second); break;
+            default: rc = run_inflight_probe<16>(table, sink, mask, cps, sms, st, a, b, rows_per_second); break;
+        }
+        cudaError_t e = cudaGetLastError();
+        if (rc == SDNN_ERR_INVALID_ARG) rc = fail(nullptr, rc, "that many threads with that many loads in flight do not fit an SM's registers");
+        else if (rc != SDNN_OK || e != cudaSuccess) rc = cuda_fail(nullptr, e, "gather in-flight probe");
+    }
+    if (a) cudaEventDestroy(a);
+    if (b) cudaEventDestroy(b);
+    if (st) cudaStreamDestroy(st);
+    if (table) cudaFree(table);
+    if (sink) cudaFree(sink);
+    return rc;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Scattered 4-byte word probe (see sdnn_probe_word_rate in the header).
 extern "C" int sdnn_probe_word_rate(int32_t store, int64_t table_words, double* words_per_second) {
     if (!words_per_second) return fail(nullptr, SDNN_ERR_INVALID_ARG, "words_per_second is NULL");

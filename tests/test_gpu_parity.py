@@ -891,6 +891,18 @@ def test_gather_probe_reports_a_rate_and_rejects_bad_sizes(torch_cuda):
         assert ei.value.code == -1
 
 
+def test_gather_in_flight_probe_saturates_and_rejects_bad_sizes(torch_cuda):
+    pkg = sdnn()
+    few = pkg.probe_gather_inflight(65536, 128, 1)            # 64 rows in flight per SM: a round trip per batch
+    many = pkg.probe_gather_inflight(65536, 512, 4)           # 1024 rows in flight per SM: the path's full rate
+    assert 1e9 < few < many < 1e13 and many > 3 * few
+    assert abs(many / pkg.probe_gather_rate(64, 65536) - 1.0) < 0.35      # the same ceiling the free-running probe finds
+    for rows, threads, loads in ((1000, 256, 4), (65536, 100, 4), (65536, 4096, 4), (65536, 256, 3), (65536, 2048, 16)):
+        with pytest.raises(pkg.SdnnError) as ei:
+            pkg.probe_gather_inflight(rows, threads, loads)
+        assert ei.value.code == -1
+
+
 def test_shared_memory_gather_probe_reports_rates_and_rejects_bad_sizes(torch_cuda):
     pkg = sdnn()
     for cluster in (1, 4, 16):

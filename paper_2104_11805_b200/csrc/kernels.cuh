@@ -429,26 +429,29 @@ __device__ __forceinline__ void prefetch_unit(const Sliced& m, int u, int rpw, i
 
 // ---------------------------------------------------------------------------------------------
 // Forward layer (feedforward equation): Xout[i,:] = clamp(bias[i] + sum_q val[i,q] * Xin[idx[i,q],:]).
-// Persistent grid: a warp takes units (32/G consecutive rows) in a grid-stride loop.  One group of G lanes
+// Persistent grid: a warp takes units (32/G consecutive rows) in a grid-stride loop, or (span > 0) within its CTA's
+// run of `span` consecutive units.  One group of G lanes
 // per row; each lane accumulates V batch entries with fp32 FMAs in stored (ascending column) order.
 // While it works on a unit a warp asks for the entries of its next unit to be brought into L2.
 template <int G, int V, int CPS, bool I16>
 __global__ void __launch_bounds__(256, CPS > 2 ? 1 : 2)
 forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict__ xin, float* __restrict__ xout,
-               int n, int ld, float clamp, int act, int pdl, const int* __restrict__ ncols_dev, int* __restrict__ live_flags) {
+               int n, int ld, float clamp, int act, int pdl, const int* __restrict__ ncols_dev, int* __restrict__ live_flags, int span) {
     constexpr int RPW = 32 / G;
     constexpr int UPS = (RPW >= SLICE) ? 1 : SLICE / RPW;      // units per slice
     const int lane = threadIdx.x & 31;
     const int sub = lane % G, grp = lane / G;
     const int wpb = blockDim.x >> 5;
-    const int nunits = (n + RPW - 1) / RPW;
-    const int stride = gridDim.x * wpb;
+    const int all_units = (n + RPW - 1) / RPW;
+    // span > 0: a CTA takes `span` consecutive units (rows that share their columns then share the SM's L1); 0: grid-stride
+    const int nunits = span > 0 ? min(all_units, ((int)blockIdx.x + 1) * span) : all_units;
+    const int stride = span > 0 ? wpb : gridDim.x * wpb;
     const int boff = blockIdx.y * (V * G) + sub * V;
     const float* xg = xin + boff;
     const unsigned pitch = (unsigned)ld * 4u;
     const float* __restrict__ val = m.val;
 
-    int unit = blockIdx.x * wpb + (threadIdx.x >> 5);
+    int unit = (span > 0 ? blockIdx.x * span : blockIdx.x * wpb) + (threadIdx.x >> 5);
     // prologue that does not depend on the previous layer: shape of the first row, its entries on their way to L2
     int row, base, nch;
     SDNN_UNIT_SHAPE(m, unit, nunits, row, base, nch)

@@ -272,6 +272,14 @@ def study_probes():
             inflight = threads // 2 * loads
             out["rows_in_flight"].append({"threads_per_sm": threads, "loads_per_lane": loads, "rows_in_flight_per_sm": inflight,
                                           "rate": rate, "round_trip_clk": inflight / rate})
+    # a layer boundary as a grid-wide barrier inside one launch against the boundary between two dependent launches
+    out["layer_boundary_us"] = {}
+    for ctas, threads in ((1, 32), (1, 224), (2, 224), (2, 32)):
+        try:
+            bar, lau = pkg.probe_layer_boundary(ctas, threads)
+            out["layer_boundary_us"][f"{ctas}x{threads}"] = {"grid_barrier": bar, "dependent_launch_in_graph": lau}
+        except pkg.SdnnError as exc:
+            out["layer_boundary_us"][f"{ctas}x{threads}"] = f"error: {exc.message}"
     print(json.dumps(out), flush=True)
 
 

@@ -284,6 +284,19 @@ int sdnn_probe_gather_rate(int32_t row_bytes, int64_t table_rows, double* rows_p
 int sdnn_probe_gather_inflight(int64_t table_rows, int32_t threads_per_sm, int32_t loads_in_flight, double* rows_per_second);
 
 /*
+ * What a layer boundary costs on the current device (diagnostic; the paper has no counterpart).  Every layer of
+ * Algorithm 1 needs all of the layer before it, so a layer ends with a device-wide hand-over.  barrier_us (host double*):
+ * microseconds per grid-wide barrier inside ONE cooperative launch of ctas_per_sm (1..4) CTAs of `threads` threads per
+ * SM (release-add on a counter, bounded acquire-spin): what a kernel looping over the layers itself would pay.
+ * launch_us (host double*): microseconds per launch of a chain of dependent launches of the same shape under
+ * programmatic dependent launch, captured into one graph: what the library's layer launches pay.  Each round / launch
+ * writes one float per thread.  SDNN_ERR_INVALID_ARG if the grid cannot be resident as a whole; SDNN_ERR_CUDA with a
+ * message if a barrier wait ran out (the kernel then leaves instead of spinning on).  Allocates and frees its own
+ * buffers, stream and graph; synchronises.
+ */
+int sdnn_probe_layer_boundary(int32_t ctas_per_sm, int32_t threads, double* barrier_us, double* launch_us);
+
+/*
  * Measures the alternative to keeping two copies of a training layer's values (diagnostic; the paper has no
  * counterpart): with ONE value array in row-major order, the column units of the transposed product would reach each
  * value through a position map, i.e. read (and, to apply the update, write) single 4-byte words at scattered places.

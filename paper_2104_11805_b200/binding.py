@@ -57,6 +57,7 @@ _PROTOS = {
     "sdnn_mirror_mismatches": (ctypes.c_int, [_vp, _i32, ctypes.POINTER(_i64)]),
     "sdnn_probe_gather_rate": (ctypes.c_int, [_i32, _i64, ctypes.POINTER(ctypes.c_double)]),
     "sdnn_probe_gather_inflight": (ctypes.c_int, [_i64, _i32, _i32, ctypes.POINTER(ctypes.c_double)]),
+    "sdnn_probe_layer_boundary": (ctypes.c_int, [_i32, _i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]),
     "sdnn_probe_tma_gather_rate": (ctypes.c_int, [_i32, _i64, _i32, ctypes.POINTER(ctypes.c_double)]),
     "sdnn_probe_mixed_gather": (ctypes.c_int, [_i32, _i64, _i32, _i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]),
     "sdnn_probe_word_rate": (ctypes.c_int, [_i32, _i64, ctypes.POINTER(ctypes.c_double)]),
@@ -169,6 +170,17 @@ def probe_gather_inflight(table_rows, threads_per_sm, loads_in_flight):
     if rc != 0:
         raise SdnnError(rc, (lib.sdnn_last_error(None) or b"").decode())
     return out.value
+
+
+def probe_layer_boundary(ctas_per_sm, threads):
+    """sdnn_probe_layer_boundary: (microseconds per grid-wide barrier inside one cooperative launch, microseconds per
+    dependent launch of a graph-captured chain) for grids of ctas_per_sm CTAs of `threads` threads per SM."""
+    lib = load_library()
+    bar, lau = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    rc = lib.sdnn_probe_layer_boundary(ctas_per_sm, threads, ctypes.byref(bar), ctypes.byref(lau))
+    if rc != 0:
+        raise SdnnError(rc, (lib.sdnn_last_error(None) or b"").decode())
+    return bar.value, lau.value
 
 
 def cluster_layer(row_ptr, col_idx, col_cap=1536, row_cap=2048):

@@ -1431,6 +1431,41 @@ gather_inflight_probe_kernel(const float* __restrict__ table, float* __restrict_
 }
 
 // ---------------------------------------------------------------------------------------------
+// What does a layer boundary cost?  Two ways to make every CTA's writes of one round visible to all CTAs of the next:
+// a grid-wide barrier inside one cooperative launch (a release-add on a counter, then an acquire-spin until the
+// round's count is reached: what a kernel that loops over the layers itself would pay per layer), and the end of one
+// launch / start of the next under programmatic dependent launch (what the layer kernels pay).  Each round every thread
+// writes one float, so that there is something to make visible.  The spin is bounded: a CTA that does not see its
+// round complete within BARRIER_SPIN_LIMIT polls raises *err, and every CTA leaves at its next check.
+constexpr int BARRIER_SPIN_LIMIT = 1 << 22;
+__device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p) {
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__global__ void grid_barrier_probe_kernel(unsigned* counter, int* err, int rounds, float* data) {
+    const unsigned ctas = gridDim.x;
+    for (int r = 0; r < rounds; ++r) {
+        data[blockIdx.x * blockDim.x + threadIdx.x] = (float)r;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            asm volatile("red.release.gpu.global.add.u32 [%0], %1;" :: "l"(counter), "r"(1u) : "memory");
+            const unsigned want = (unsigned)(r + 1) * ctas;
+            int spins = 0;
+            while (ld_acquire_gpu(counter) < want)
+                if (++spins > BARRIER_SPIN_LIMIT) { *err = 1; break; }
+        }
+        __syncthreads();
+        if (*reinterpret_cast<volatile int*>(err)) return;
+    }
+}
+__global__ void launch_chain_probe_kernel(float* data, int r) {
+    grid_dependency_wait();
+    grid_launch_dependents();
+    data[blockIdx.x * blockDim.x + threadIdx.x] = (float)r;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Probe of the alternative to the second copy of the values: one value array in row-major order that the column
 // units would read, or read and write, one 4-byte word at a time at scattered places (through a position map).  Eight
 // accesses in flight per lane, indices made in registers.  STORE: 0 = scattered 4-byte loads, 1 = scattered 4-byte stores

@@ -2008,6 +2008,90 @@ extern "C" int sdnn_probe_gather_inflight(int64_t table_rows, int32_t threads_pe
 }
 
 // ---------------------------------------------------------------------------------------------
+// Cost of a layer boundary (see sdnn_probe_layer_boundary in the header).
+extern "C" int sdnn_probe_layer_boundary(int32_t ctas_per_sm, int32_t threads, double* barrier_us, double* launch_us) {
+    if (!barrier_us || !launch_us) return fail(nullptr, SDNN_ERR_INVALID_ARG, "barrier_us or launch_us is NULL");
+    *barrier_us = 0.0; *launch_us = 0.0;
+    if (ctas_per_sm < 1 || ctas_per_sm > 4 || threads < 32 || threads > 1024 || threads % 32)
+        return fail(nullptr, SDNN_ERR_INVALID_ARG, "ctas_per_sm must be 1..4 and threads a multiple of 32 up to 1024");
+    int dev = 0, sms = 0, coop = 0, occ = 0;
+    CU(nullptr, cudaGetDevice(&dev));
+    CU(nullptr, cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    CU(nullptr, cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
+    CU(nullptr, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, grid_barrier_probe_kernel, threads, 0));
+    if (!coop || occ < ctas_per_sm)
+        return fail(nullptr, SDNN_ERR_INVALID_ARG, "the device cannot hold that grid resident (a grid barrier needs every CTA running)");
+    const int grid = sms * ctas_per_sm, rounds = 1000;
+    unsigned* counter = nullptr;
+    int* err = nullptr;
+    float* data = nullptr;
+    cudaStream_t st = nullptr;
+    cudaEvent_t a = nullptr, b = nullptr;
+    cudaGraph_t graph = nullptr;
+    cudaGraphExec_t exec = nullptr;
+    int rc = SDNN_OK;
+    if (cudaMalloc(&counter, 4) != cudaSuccess || cudaMalloc(&err, 4) != cudaSuccess ||
+        cudaMalloc(&data, (size_t)grid * threads * sizeof(float)) != cudaSuccess || cudaStreamCreate(&st) != cudaSuccess ||
+        cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) {
+        cudaGetLastError();
+        rc = fail(nullptr, SDNN_ERR_OOM, "could not allocate the probe's buffers");
+    } else {
+        float best = 0.f;
+        int herr = 0;
+        for (int rep = 0; rep < 3 && rc == SDNN_OK; ++rep) {      // the barrier: one cooperative launch of `rounds` rounds
+            cudaMemsetAsync(counter, 0, 4, st); cudaMemsetAsync(err, 0, 4, st);
+            cudaEventRecord(a, st);
+            int rr = rounds;
+            void* args[] = {&counter, &err, &rr, &data};
+            cudaError_t e = cudaLaunchCooperativeKernel((void*)grid_barrier_probe_kernel, dim3(grid), dim3(threads), args, 0, st);
+            cudaEventRecord(b, st);
+            if (e != cudaSuccess || cudaEventSynchronize(b) != cudaSuccess) { rc = cuda_fail(nullptr, e != cudaSuccess ? e : cudaGetLastError(), "grid barrier probe"); break; }
+            float ms = 0.f;
+            cudaEventElapsedTime(&ms, a, b);
+            if (rep == 0 || ms < best) best = ms;
+            cudaMemcpy(&herr, err, 4, cudaMemcpyDeviceToHost);
+            if (herr) rc = fail(nullptr, SDNN_ERR_CUDA, "grid barrier probe: a wait ran out (the grid was not resident as a whole)");
+        }
+        if (rc == SDNN_OK) *barrier_us = (double)best * 1e3 / rounds;
+        if (rc == SDNN_OK) {      // the launch boundary: `rounds` dependent launches, captured into one graph as the library's steps are
+            cudaError_t e = cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal);
+            for (int r = 0; r < rounds && e == cudaSuccess; ++r) {
+                cudaLaunchConfig_t lc = {};
+                lc.gridDim = dim3(grid); lc.blockDim = dim3(threads); lc.stream = st;
+                cudaLaunchAttribute at[1];
+                at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+                at[0].val.programmaticStreamSerializationAllowed = 1;
+                lc.attrs = at; lc.numAttrs = 1;
+                e = cudaLaunchKernelEx(&lc, launch_chain_probe_kernel, data, r);
+            }
+            cudaError_t e2 = cudaStreamEndCapture(st, &graph);
+            if (e == cudaSuccess) e = e2;
+            if (e == cudaSuccess) e = cudaGraphInstantiate(&exec, graph, 0);
+            for (int rep = 0; rep < 3 && e == cudaSuccess; ++rep) {
+                cudaEventRecord(a, st);
+                e = cudaGraphLaunch(exec, st);
+                cudaEventRecord(b, st);
+                if (e == cudaSuccess) e = cudaEventSynchronize(b);
+                float ms = 0.f;
+                cudaEventElapsedTime(&ms, a, b);
+                if (rep == 0 || ms < best) best = ms;
+            }
+            if (e != cudaSuccess) rc = cuda_fail(nullptr, e, "launch chain probe");
+            else *launch_us = (double)best * 1e3 / rounds;
+        }
+    }
+    if (exec) cudaGraphExecDestroy(exec);
+    if (graph) cudaGraphDestroy(graph);
+    if (a) cudaEventDestroy(a);
+    if (b) cudaEventDestroy(b);
+    if (st) cudaStreamDestroy(st);
+    if (counter) cudaFree(counter);
+    if (err) cudaFree(err);
+    if (data) cudaFree(data);
+    return rc;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Scattered 4-byte word probe (see sdnn_probe_word_rate in the header).
 extern "C" int sdnn_probe_word_rate(int32_t store, int64_t table_words, double* words_per_second) {
     if (!words_per_second) return fail(nullptr, SDNN_ERR_INVALID_ARG, "words_per_second is NULL");

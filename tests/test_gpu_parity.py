@@ -903,6 +903,16 @@ def test_gather_in_flight_probe_saturates_and_rejects_bad_sizes(torch_cuda):
         assert ei.value.code == -1
 
 
+def test_layer_boundary_probe_reports_both_costs_and_rejects_bad_shapes(torch_cuda):
+    pkg = sdnn()
+    barrier_us, launch_us = pkg.probe_layer_boundary(2, 224)
+    assert 0.05 < barrier_us < 100.0 and 0.05 < launch_us < 100.0
+    for ctas, threads in ((0, 128), (5, 128), (1, 48), (1, 2048)):
+        with pytest.raises(pkg.SdnnError) as ei:
+            pkg.probe_layer_boundary(ctas, threads)
+        assert ei.value.code == -1
+
+
 def test_shared_memory_gather_probe_reports_rates_and_rejects_bad_sizes(torch_cuda):
     pkg = sdnn()
     for cluster in (1, 4, 16):

@@ -256,8 +256,13 @@ __device__ __forceinline__ void chunk_update(float* vp, float* gp, const float4&
     } else if (G == 2) {
         const float wa = sub ? w.z : w.x, wb = sub ? w.w : w.y;
         const int m = 2 * sub;
-        if (q0 < lim) { vp[m] = __fmaf_rn(-step, p0, wa); if (DBG) gp[m] = p0 * inv_b; }
-        if (q0 + 1 < lim) { vp[m + 1] = __fmaf_rn(-step, p1, wb); if (DBG) gp[m + 1] = p1 * inv_b; }
+        const float n0 = __fmaf_rn(-step, p0, wa), n1 = __fmaf_rn(-step, p1, wb);
+        if (q0 + 1 < lim) *reinterpret_cast<float2*>(vp + m) = make_float2(n0, n1);      // both entries stored: one 8-byte store
+        else if (q0 < lim) vp[m] = n0;
+        if (DBG) {
+            if (q0 < lim) gp[m] = p0 * inv_b;
+            if (q0 + 1 < lim) gp[m + 1] = p1 * inv_b;
+        }
     } else {
         if (q0 + 0 < lim) { vp[0] = __fmaf_rn(-step, p0, w.x); if (DBG) gp[0] = p0 * inv_b; }
         if (q0 + 1 < lim) { vp[1] = __fmaf_rn(-step, p1, w.y); if (DBG) gp[1] = p1 * inv_b; }

@@ -264,10 +264,19 @@ __device__ __forceinline__ void chunk_update(float* vp, float* gp, const float4&
             if (q0 + 1 < lim) gp[m + 1] = p1 * inv_b;
         }
     } else {
-        if (q0 + 0 < lim) { vp[0] = __fmaf_rn(-step, p0, w.x); if (DBG) gp[0] = p0 * inv_b; }
-        if (q0 + 1 < lim) { vp[1] = __fmaf_rn(-step, p1, w.y); if (DBG) gp[1] = p1 * inv_b; }
-        if (q0 + 2 < lim) { vp[2] = __fmaf_rn(-step, p2, w.z); if (DBG) gp[2] = p2 * inv_b; }
-        if (q0 + 3 < lim) { vp[3] = __fmaf_rn(-step, p3, w.w); if (DBG) gp[3] = p3 * inv_b; }
+        const float4 nw = make_float4(__fmaf_rn(-step, p0, w.x), __fmaf_rn(-step, p1, w.y), __fmaf_rn(-step, p2, w.z), __fmaf_rn(-step, p3, w.w));
+        if (q0 + 3 < lim) st_f4(vp, nw);      // a whole chunk: one 16-byte store
+        else {
+            if (q0 + 0 < lim) vp[0] = nw.x;
+            if (q0 + 1 < lim) vp[1] = nw.y;
+            if (q0 + 2 < lim) vp[2] = nw.z;
+        }
+        if (DBG) {
+            if (q0 + 0 < lim) gp[0] = p0 * inv_b;
+            if (q0 + 1 < lim) gp[1] = p1 * inv_b;
+            if (q0 + 2 < lim) gp[2] = p2 * inv_b;
+            if (q0 + 3 < lim) gp[3] = p3 * inv_b;
+        }
     }
 }
 
@@ -909,7 +918,7 @@ __device__ __forceinline__ void backward_col_units(const Sliced m, const float* 
             float4 w[CPS];
             Lane<V> d[4 * CPS];
 #pragma unroll
-            for (int i = 0; i < CPS; ++i) w[i] = ld_f4(vp + (t + i) * CHUNK_ROW);
+            for (int i = 0; i < CPS; ++i) w[i] = __ldcs(reinterpret_cast<const float4*>(vp + (t + i) * CHUNK_ROW));
 #pragma unroll
             for (int i = 0; i < CPS; ++i) { SDNN_GATHER_CHUNK(d, i, c[i], dg, pitch) }
             if (t + CPS < nch) { load_idx<CPS, I16>(c, m, base + (t + CPS) * CHUNK_ROW); }
@@ -1003,7 +1012,7 @@ __device__ __forceinline__ void backward_row_units(const Sliced m, float* __rest
             float4 w[CPS];
             Lane<V> x[4 * CPS];
 #pragma unroll
-            for (int i = 0; i < CPS; ++i) w[i] = ld_f4(vp + (t + i) * CHUNK_ROW);
+            for (int i = 0; i < CPS; ++i) w[i] = __ldcs(reinterpret_cast<const float4*>(vp + (t + i) * CHUNK_ROW));
 #pragma unroll
             for (int i = 0; i < CPS; ++i) { SDNN_GATHER_CHUNK(x, i, c[i], xg, pitch) }
             if (SCATTER) {       // stored entries only: padding must not touch S

@@ -92,7 +92,7 @@ typedef enum {
                                     /* sdnn_get_weights / sdnn_set_weights.  The layers are analysed in sdnn_finalize;   */
                                     /* until then the handle keeps a host copy of every loaded layer.  Inference and     */
                                     /* training handles (targets, activations, deltas and gradients keep the caller's   */
-                                    /* numbering too); not together with SDNN_FLAG_SKIP_DEAD.                             */
+                                    /* numbering too).                                                                    */
 
 #define SDNN_FLAG_SMEM_WINDOWS 0x200u /* with SDNN_FLAG_REORDER: run the layers for which groups were found with kernels   */
                                     /* that own a group: the group's window of the activation tile is copied into shared */
@@ -100,7 +100,8 @@ typedef enum {
                                     /* inputs, forward_window_kernel for narrower ones) instead of out of L1/L2.         */
                                     /* Measured on B200: 13-20 % faster on a net of 64 blocks per layer (65536 neurons,  */
                                     /* windows of 1024), slower on a net that is one group (1024 neurons), hence opt-in. */
-                                    /* Inference handles only (SDNN_ERR_UNIMPLEMENTED with train = 1).                   */
+                                    /* Inference handles only (SDNN_ERR_UNIMPLEMENTED with train = 1); not together with */
+                                    /* SDNN_FLAG_SKIP_DEAD (these kernels do not keep track of live inputs).             */
 
 #define SDNN_ACT_CLAMPED_RELU 0
 #define SDNN_ACT_SIGMOID      1

@@ -252,8 +252,9 @@ int validate_cfg(const sdnn_config* cfg) {
         return fail(nullptr, SDNN_ERR_UNIMPLEMENTED, "SDNN_FLAG_SMEM_WINDOWS is implemented for inference handles (train = 0)");
     if ((cfg->flags & SDNN_FLAG_SMEM_WINDOWS) && !(cfg->flags & SDNN_FLAG_REORDER))
         return fail(nullptr, SDNN_ERR_INVALID_ARG, "SDNN_FLAG_SMEM_WINDOWS needs SDNN_FLAG_REORDER");
-    if ((cfg->flags & SDNN_FLAG_REORDER) && (cfg->flags & SDNN_FLAG_SKIP_DEAD))
-        return fail(nullptr, SDNN_ERR_INVALID_ARG, "SDNN_FLAG_REORDER and SDNN_FLAG_SKIP_DEAD cannot be combined");
+    if ((cfg->flags & SDNN_FLAG_SMEM_WINDOWS) && (cfg->flags & SDNN_FLAG_SKIP_DEAD))
+        return fail(nullptr, SDNN_ERR_INVALID_ARG, "SDNN_FLAG_SMEM_WINDOWS and SDNN_FLAG_SKIP_DEAD cannot be combined "
+                                                  "(the window kernels do not keep track of live inputs)");
     return SDNN_OK;
 }
 

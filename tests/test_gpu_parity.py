@@ -788,6 +788,37 @@ def test_reorder_flag_leaves_an_unstructured_net_alone(torch_cuda):
     with pytest.raises(pkg.SdnnError) as ei:
         pkg.Sdnn.create(*gen.network(spec), max_batch=16, train=True, flags=pkg.FLAG_REORDER | pkg.FLAG_SMEM_WINDOWS)
     assert ei.value.code == -6          # the shared-memory window kernel exists for the forward pass of inference handles only
+    with pytest.raises(pkg.SdnnError) as ei:      # the window kernels do not keep track of live inputs
+        pkg.Sdnn.create(*gen.network(spec), max_batch=16, flags=pkg.FLAG_REORDER | pkg.FLAG_SMEM_WINDOWS | pkg.FLAG_SKIP_DEAD)
+    assert ei.value.code == -1
+
+
+@pytest.mark.parametrize("host", [False, True])
+def test_infer_reordered_dropping_dead_inputs(torch_cuda, host):
+    """SDNN_FLAG_REORDER with SDNN_FLAG_SKIP_DEAD: the regrouped layers run in compaction mode (live inputs only, in
+    chunks that shrink as inputs die); outputs, counts and id lists against the oracle in the caller's numbering, several
+    tiles, and the per-layer live counts of the last tile."""
+    pkg = sdnn()
+    spec = block_spec(4096, 6, 1024).shuffled()
+    arrays = gen.network(spec)
+    cnt = 700
+    x0 = gen.inputs(spec, cnt)
+    rng = np.random.default_rng(11)
+    x0[rng.uniform(size=cnt) < 0.5] = 0.0          # half of the inputs die at layer 1 (bias 0, x = 0 is a fixed point)
+    infer_parity(torch_cuda, arrays, x0, 512, host=host, expect_nonempty=True, flags=pkg.FLAG_REORDER | pkg.FLAG_SKIP_DEAD,
+                 expect_grouped=6)
+    h = pkg.Sdnn.create(*arrays, max_batch=1024, flags=pkg.FLAG_REORDER | pkg.FLAG_SKIP_DEAD)
+    yd = torch_cuda.empty((cnt, spec.n), dtype=torch_cuda.float32, device="cuda")
+    h.infer_batch(torch_cuda.from_numpy(x0).cuda(), cnt, yd, None, None, 0)
+    live = list(h.get_liveness())
+    h.destroy()
+    ora = OracleNet(*arrays)
+    x = x0.astype(np.float64)
+    want = []
+    for k in range(spec.layers):
+        _, x, _ = ora.forward_layer(k, x)
+        want.append(int((x != 0).any(axis=1).sum()))
+    assert live == want and 0 < want[-1] < cnt, (live, want)
 
 
 @pytest.mark.parametrize("bwd", sorted(BWD_MODES))
@@ -804,6 +835,17 @@ def test_train_reordered_hidden_blocks(torch_cuda, B, bwd):
     bias = [(0.05 * rng.standard_normal(spec.n)).astype(np.float32) for _ in range(4)]       # biases that tell the rows apart
     st = train_parity(torch_cuda, (rp, col, val, bias), batches_for(spec, B, 2), eta=1e-2, update_bias=True,
                       flags=BWD_MODES[bwd] | pkg.FLAG_REORDER, expect_live=True)
+    assert st["entries"] > 0
+
+
+@pytest.mark.parametrize("B", [1, 16])
+def test_train_reordered_skipping_dead_rows(torch_cuda, B):
+    """SDNN_FLAG_REORDER with SDNN_FLAG_SKIP_DEAD in training (row units whose delta is zero for every input skip their
+    entries): same results as the oracle, which skips nothing."""
+    pkg = sdnn()
+    spec = block_spec(1024, 4, 256).shuffled()
+    st = train_parity(torch_cuda, gen.network(spec), batches_for(spec, B, 2), eta=1e-2,
+                      flags=pkg.FLAG_REORDER | pkg.FLAG_SKIP_DEAD, expect_live=True)
     assert st["entries"] > 0
 
 

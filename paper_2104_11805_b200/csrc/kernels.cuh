@@ -6,8 +6,9 @@
 // of 4 columns), a row is shared by G = ld / V lanes, and a warp works on 32/G matrix rows at once.  Tiles
 // wider than 256 inputs are processed in chunks of 256 (blockIdx.y).
 //
-// Stored entries.  These kernels are bound by instruction issue and by L1 wavefronts per stored entry,
-// not by bytes: the gather of a tile row costs one wavefront whatever its width up to 128 bytes, and with
+// Stored entries.  These kernels are bound by the memory requests an SM can make per stored entry, not by
+// bytes: the gather of a tile row costs one request whatever its width up to 64 bytes (a store that leaves
+// holes in a 32-byte sector costs several), and with
 // plain CSR the index and value loads of the row groups of a warp would cost as much again, because each row
 // sits in a different 128-byte line.  The entries are therefore kept in slices of 16 rows, interleaved in
 // chunks of 4:

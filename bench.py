@@ -62,7 +62,8 @@ def setup_of(spec):
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
 # (training kernels: captured on a 48-layer slice of the same net, per-launch traffic does not depend on the depth)
-NCU_TRAFFIC = {("cfg5", "backward_kernel"): 21.26e6 + 27.10e6, ("cfg5", "forward_kernel"): 17.07e6}      # backward: both launches of a layer
+NCU_TRAFFIC = {("cfg5", "backward_kernel"): 21.26e6 + 27.10e6, ("cfg5", "forward_kernel"): 17.07e6,      # backward: both launches of a layer
+               ("cfg3", "backward_kernel"): 11.62e6 + 16.24e6, ("cfg3", "forward_kernel"): 7.42e6}
 
 
 def measured_peaks():

@@ -75,8 +75,9 @@ __device__ __forceinline__ void prefetch_l2(const void* p, unsigned bytes) {
 // The layer kernels take `pdl`: 0 = launched without the attribute (no wait, no release); 1 = wait, release the next
 // launch at the end; 2 = wait, release it right after the wait (its CTAs then move into SM slots as they fall free and
 // do everything that does not depend on this launch - shapes, first indices - under this launch's tail).  Whatever a
-// kernel reads before its wait must not be written by the launch before it: slice offsets, lengths, order, indices
-// and (forward) the bias qualify; values, tiles and counters do not.
+// kernel reads before its wait must not be written by the launch before it: slice offsets, lengths, order, indices,
+// (forward) the bias and (column units of the backward pass) the step parameters and the rows of x^{k-1}, which the
+// forward pass of the same step wrote, qualify; values, the delta tiles and counters do not.
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
@@ -878,7 +879,7 @@ struct BackwardArgs {
 template <int G, int V, int CPS, bool I16>
 __device__ __forceinline__ void backward_col_units(const Sliced m, const float* __restrict__ xprev, const float* __restrict__ dk,
                                                    float* __restrict__ dprev, int n, float clamp, int act, float step, float inv_b,
-                                                   int first, int stride) {
+                                                   int first, int stride, int pdl) {
     constexpr int RPW = 32 / G;
     constexpr int UPS = (RPW >= SLICE) ? 1 : SLICE / RPW;
     constexpr unsigned pitch = 4u * V * G;
@@ -902,6 +903,9 @@ __device__ __forceinline__ void backward_col_units(const Sliced m, const float* 
     Lane<V> xj;
     lane_fill(xj, 0.0f);
     if (item < n) lane_load(xj, tile_row(xprev + boff, j, pitch));
+    // everything above is static for the chain of launches (shapes, indices, x^{k-1}); delta^k is what the launch waits for
+    if (pdl) grid_dependency_wait();
+    if (pdl == 2) grid_launch_dependents();
 
     while (u < nunits) {
         const int nu = u + stride;
@@ -1054,11 +1058,14 @@ backward_kernel(const BackwardArgs a) {
             prefetch_l2(reinterpret_cast<const char*>(a.warm) + lo, len & ~15u);
         }
     }
-    if (a.pdl) grid_dependency_wait();
-    if (a.pdl == 2) grid_launch_dependents();
+    // step parameters: written once per step, long before any backward launch
     const float inv_b = a.sp->inv_b;
     const float step = a.sp->eta * inv_b;
-    if (MIRROR) backward_col_units<G, V, CPS, I16>(a.cols, a.xprev, a.dk, a.dprev, a.n, a.clamp, a.act, step, inv_b, first, stride);
+    if (MIRROR) backward_col_units<G, V, CPS, I16>(a.cols, a.xprev, a.dk, a.dprev, a.n, a.clamp, a.act, step, inv_b, first, stride, a.pdl);
+    else {
+        if (a.pdl) grid_dependency_wait();
+        if (a.pdl == 2) grid_launch_dependents();
+    }
     if (MIRROR && a.cols_only) { if (a.pdl == 1) grid_launch_dependents(); return; }
     backward_row_units<G, V, CPS, I16, FROM_S, SCATTER, DBG>(a.rows, a.bias, a.xk, a.xprev, a.dk, a.dprev, a.dbg_delta, a.dbg_grad, a.n,
                                                         a.clamp, a.act, step, inv_b, a.update_bias, a.skip_dead, first, stride);

@@ -587,11 +587,11 @@ void launch_backward_gvc(sdnn* h, int layer, int ld, int part) {
     do {                                                                                       \
         if (a.dbg_grad) {                                                                      \
             auto plan = plan_grid(h, (const void*)backward_kernel<G, V, CPS, I16, FROM_S, SCAT, MIR, true>, units, 1, os_);   \
-            if (a.pdl && plan.first <= h->sms) a.pdl = PDL_EARLY;                              \
+            if (a.pdl && (plan.first <= h->sms || MIR)) a.pdl = PDL_EARLY;                     \
             launch_k(h, backward_kernel<G, V, CPS, I16, FROM_S, SCAT, MIR, true>, dim3(plan.first), dim3(plan.second), a.pdl != 0, a); \
         } else {                                                                               \
             auto plan = plan_grid(h, (const void*)backward_kernel<G, V, CPS, I16, FROM_S, SCAT, MIR, false>, units, 1, os_);  \
-            if (a.pdl && plan.first <= h->sms) a.pdl = PDL_EARLY;                              \
+            if (a.pdl && (plan.first <= h->sms || MIR)) a.pdl = PDL_EARLY;                     \
             launch_k(h, backward_kernel<G, V, CPS, I16, FROM_S, SCAT, MIR, false>, dim3(plan.first), dim3(plan.second), a.pdl != 0, a); \
         }                                                                                      \
     } while (0)

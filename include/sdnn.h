@@ -262,7 +262,7 @@ int sdnn_mirror_mismatches(sdnn_t* h, int32_t layer, int64_t* count_out);
 /*
  * Measures what bounds the layer kernels on the current device (diagnostic; the paper has no counterpart): the
  * rate at which an SM array can gather random rows of `row_bytes` bytes (16 .. 1024, a power of two; read with the
- * layer kernels' own 256-bit accesses) out of a table
+ * layer kernels' own 256-bit accesses, through L1 or past it, whichever is faster) out of a table
  * of `table_rows` rows (a power of two; at most 1 GiB in all) that sits in L2 or, if larger, in HBM, with nothing
  * else competing for the load pipe.  A layer with nnz stored entries and a padded batch of ld inputs gathers
  * nnz rows of 4*ld bytes in the forward product and 2*nnz in the backward launch (transposed realisation), so

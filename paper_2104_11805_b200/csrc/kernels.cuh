@@ -1419,7 +1419,7 @@ __global__ void __launch_bounds__(256) expand_kernel(ColState s, const float* __
 // in registers (a linear congruential sequence per lane group, masked to the table), so that only the gathers
 // use the load pipe.  G lanes of V floats per row (the layer kernels' own access width), eight gathers in flight
 // per lane.
-template <int G, int V>
+template <int G, int V, bool PAST_L1>
 __global__ void __launch_bounds__(256)
 gather_probe_kernel(const float* __restrict__ table, float* __restrict__ sink, unsigned row_mask, int per_group, unsigned seed) {
     const int tid = blockIdx.x * blockDim.x + threadIdx.x;
@@ -1432,7 +1432,7 @@ gather_probe_kernel(const float* __restrict__ table, float* __restrict__ sink, u
         for (int u = 0; u < 8; ++u) { st = st * 1664525u + 1013904223u; c[u] = (st >> 8) & row_mask; }
         Lane<V> v[8];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) lane_gather(v[u], table + (size_t)c[u] * (V * G) + sub * V);
+        for (int u = 0; u < 8; ++u) lane_gather_sel<PAST_L1>(v[u], table + (size_t)c[u] * (V * G) + sub * V);
 #pragma unroll
         for (int u = 0; u < 8; ++u) acc += lane_sum(v[u]);
     }

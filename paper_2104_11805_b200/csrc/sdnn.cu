@@ -1873,17 +1873,26 @@ int sdnn_get_liveness(sdnn_t* h, int32_t* live_inputs_out) {
 // Gather-rate probe (see sdnn_probe_gather_rate in the header).
 namespace {
 
-template <int G, int V>
-float run_gather_probe(const float* table, float* sink, unsigned mask, int per_group, int grid, cudaStream_t st, int reps,
-                       cudaEvent_t a, cudaEvent_t b) {
-    for (int i = 0; i < 2; ++i) gather_probe_kernel<G, V><<<grid, 256, 0, st>>>(table, sink, mask, per_group, 17u + i);
+template <int G, int V, bool PAST_L1>
+float run_gather_probe_path(const float* table, float* sink, unsigned mask, int per_group, int grid, cudaStream_t st, int reps,
+                            cudaEvent_t a, cudaEvent_t b) {
+    for (int i = 0; i < 2; ++i) gather_probe_kernel<G, V, PAST_L1><<<grid, 256, 0, st>>>(table, sink, mask, per_group, 17u + i);
     cudaEventRecord(a, st);
-    for (int i = 0; i < reps; ++i) gather_probe_kernel<G, V><<<grid, 256, 0, st>>>(table, sink, mask, per_group, 101u + i);
+    for (int i = 0; i < reps; ++i) gather_probe_kernel<G, V, PAST_L1><<<grid, 256, 0, st>>>(table, sink, mask, per_group, 101u + i);
     cudaEventRecord(b, st);
     cudaEventSynchronize(b);
     float ms = 0.f;
     cudaEventElapsedTime(&ms, a, b);
     return ms / reps;
+}
+// the faster of the two load paths the layer kernels use: through L1 (read-only path) and past it
+template <int G, int V>
+float run_gather_probe(const float* table, float* sink, unsigned mask, int per_group, int grid, cudaStream_t st, int reps,
+                       cudaEvent_t a, cudaEvent_t b) {
+    const float t0 = run_gather_probe_path<G, V, false>(table, sink, mask, per_group, grid, st, reps, a, b);
+    if (V != 8) return t0;
+    const float t1 = run_gather_probe_path<G, V, true>(table, sink, mask, per_group, grid, st, reps, a, b);
+    return (t1 > 0.f && (t0 <= 0.f || t1 < t0)) ? t1 : t0;
 }
 
 }  // namespace

@@ -88,7 +88,10 @@ __device__ __forceinline__ float dmask(float x, float c) { return (x > 0.0f && x
 // paper's experiments, Section 6), f'(z) = x (1 - x).  Both derivatives are functions of the stored output x.
 constexpr int ACT_CLAMPED_RELU = 0, ACT_SIGMOID = 1;
 __device__ __forceinline__ float activate(float z, int act, float c) {
-    return act == ACT_SIGMOID ? 1.0f / (1.0f + expf(-z)) : clampf(z, c);
+    // sigmoid with the hardware's exp2 and reciprocal approximations (relative error about 1e-6 for |z| <= 20, against a
+    // parity bar of 1e-4): the accurate expf and division cost a forward launch of 16 inputs 10 % of its time, all of it
+    // in the tail of the launch where nothing else runs
+    return act == ACT_SIGMOID ? __fdividef(1.0f, 1.0f + __expf(-z)) : clampf(z, c);
 }
 __device__ __forceinline__ float derivative(float x, int act, float c) {
     return act == ACT_SIGMOID ? x * (1.0f - x) : dmask(x, c);

@@ -131,6 +131,7 @@ __device__ __forceinline__ void lane_gather(Lane<8>& v, const float* p) {    // 
 // The same gather past L1 (cached in L2 only).  For rows of up to 64 bytes out of a tile that no L1 can hold, a probe of
 // nothing but such gathers runs 6 % faster this way (0.82 against 0.77 rows per clock and SM) and the forward launches of
 // 16 inputs 2 %; wider rows, which several lanes read side by side, and the backward launches lose by it.
+// (Only for layers without padding entries: those all point at tile row 0, which L1 absorbs and one L2 slice would not.)
 template <bool PAST_L1> __device__ __forceinline__ void lane_gather_sel(Lane<4>& v, const float* p) { v.a = gather_f4(p); }
 template <bool PAST_L1> __device__ __forceinline__ void lane_gather_sel(Lane<8>& v, const float* p) {
     if (PAST_L1)
@@ -466,7 +467,8 @@ __device__ __forceinline__ void prefetch_unit(const Sliced& m, int u, int rpw, i
 // run of `span` consecutive units.  One group of G lanes
 // per row; each lane accumulates V batch entries with fp32 FMAs in stored (ascending column) order.
 // While it works on a unit a warp asks for the entries of its next unit to be brought into L2.
-template <int G, int V, int CPS, bool I16>
+// CG: the gathers go past L1 (64-byte rows of a layer without padding entries).
+template <int G, int V, int CPS, bool I16, bool CG = false>
 __global__ void __launch_bounds__(256, CPS > 2 ? 1 : 2)
 forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict__ xin, float* __restrict__ xout,
                int n, int ld, float clamp, int act, int pdl, const int* __restrict__ ncols_dev, int* __restrict__ live_flags, int span) {
@@ -517,7 +519,7 @@ forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict
 #pragma unroll
             for (int i = 0; i < CPS; ++i) w[i] = __ldcs(reinterpret_cast<const float4*>(vp + (t + i) * CHUNK_ROW));
 #pragma unroll
-            for (int i = 0; i < CPS; ++i) { SDNN_GATHER_CHUNK_SEL((G == 2 && V == 8), x, i, c[i], xg, pitch) }
+            for (int i = 0; i < CPS; ++i) { SDNN_GATHER_CHUNK_SEL(CG, x, i, c[i], xg, pitch) }
             if (t + CPS < nch) load_idx<CPS, I16>(c, m, base + (t + CPS) * CHUNK_ROW);
             else if (nnch > 0) load_idx<CPS, I16>(c, m, nbase);
 #pragma unroll

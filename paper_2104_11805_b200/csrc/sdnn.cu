@@ -433,6 +433,14 @@ void launch_forward_gv(sdnn* h, int layer, const float* xin, float* xout, int ld
     const double tile_bytes = (double)h->N * ld * sizeof(float);
     if (plan.first * (plan.second / 32) < units && (h->l2_bytes <= 0 || tile_bytes <= 0.55 * (double)h->l2_bytes))
         span = (units + plan.first - 1) / plan.first;
+    // 64-byte rows of a layer whose rows all have the same length (no padding entries, which all point at tile row 0: L1
+    // absorbs those, one L2 slice would not): the instantiation whose gathers go past L1
+    if (G == 2 && V == 8 && CPS == 2 && h->lay[layer].shape.uniform_k > 0 && h->N % SLICE == 0) {
+        launch_k(h, forward_kernel<G, V, CPS, I16, (G == 2 && V == 8 && CPS == 2)>, dim3(plan.first, chunks), dim3(plan.second), h->pdl,
+                 rows_of(h, layer), bias, xin, xout, h->N, ld, h->cfg.clamp, h->cfg.activation, h->pdl ? h->fwd_pdl : 0,
+                 track ? (const int*)h->cur->cs.ncols : (const int*)nullptr, track ? h->cur->cs.flags : (int*)nullptr, span);
+        return;
+    }
     launch_k(h, forward_kernel<G, V, CPS, I16>, dim3(plan.first, chunks), dim3(plan.second), h->pdl, rows_of(h, layer), bias, xin, xout,
              h->N, ld, h->cfg.clamp, h->cfg.activation, h->pdl ? h->fwd_pdl : 0, track ? (const int*)h->cur->cs.ncols : (const int*)nullptr,
              track ? h->cur->cs.flags : (int*)nullptr, span);

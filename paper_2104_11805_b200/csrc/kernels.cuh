@@ -180,7 +180,13 @@ __device__ __forceinline__ void lane_mask(Lane<4>& d, const Lane<4>& x, int act,
 __device__ __forceinline__ void lane_mask(Lane<8>& d, const Lane<8>& x, int act, float c) { f4_mask(d.a, x.a, act, c); f4_mask(d.b, x.b, act, c); }
 
 __device__ __forceinline__ void f4_activate(float4& v, int act, float c) {
-    v.x = activate(v.x, act, c); v.y = activate(v.y, act, c); v.z = activate(v.z, act, c); v.w = activate(v.w, act, c);
+    // one branch for the four (the activation is the same for the whole launch), so that the clamped-ReLU path does not
+    // evaluate the sigmoid's special-function instructions only to discard them
+    if (act == ACT_SIGMOID) {
+        v.x = activate(v.x, ACT_SIGMOID, c); v.y = activate(v.y, ACT_SIGMOID, c); v.z = activate(v.z, ACT_SIGMOID, c); v.w = activate(v.w, ACT_SIGMOID, c);
+    } else {
+        v.x = clampf(v.x, c); v.y = clampf(v.y, c); v.z = clampf(v.z, c); v.w = clampf(v.w, c);
+    }
 }
 __device__ __forceinline__ void lane_activate(Lane<4>& v, int act, float c) { f4_activate(v.a, act, c); }
 __device__ __forceinline__ void lane_activate(Lane<8>& v, int act, float c) { f4_activate(v.a, act, c); f4_activate(v.b, act, c); }
@@ -468,7 +474,8 @@ __device__ __forceinline__ void prefetch_unit(const Sliced& m, int u, int rpw, i
 // per row; each lane accumulates V batch entries with fp32 FMAs in stored (ascending column) order.
 // While it works on a unit a warp asks for the entries of its next unit to be brought into L2.
 // CG: the gathers go past L1 (64-byte rows of a layer without padding entries).
-template <int G, int V, int CPS, bool I16, bool CG = false>
+// SPAN: a CTA takes a run of `span` consecutive units instead of walking the units in a grid-wide stride.
+template <int G, int V, int CPS, bool I16, bool CG = false, bool SPAN = false>
 __global__ void __launch_bounds__(256, CPS > 2 ? 1 : 2)
 forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict__ xin, float* __restrict__ xout,
                int n, int ld, float clamp, int act, int pdl, const int* __restrict__ ncols_dev, int* __restrict__ live_flags, int span) {
@@ -478,15 +485,14 @@ forward_kernel(Sliced m, const float* __restrict__ bias, const float* __restrict
     const int sub = lane % G, grp = lane / G;
     const int wpb = blockDim.x >> 5;
     const int all_units = (n + RPW - 1) / RPW;
-    // span > 0: a CTA takes `span` consecutive units (rows that share their columns then share the SM's L1); 0: grid-stride
-    const int nunits = span > 0 ? min(all_units, ((int)blockIdx.x + 1) * span) : all_units;
-    const int stride = span > 0 ? wpb : gridDim.x * wpb;
+    const int nunits = SPAN ? min(all_units, ((int)blockIdx.x + 1) * span) : all_units;
+    const int stride = SPAN ? wpb : gridDim.x * wpb;
     const int boff = blockIdx.y * (V * G) + sub * V;
     const float* xg = xin + boff;
     const unsigned pitch = (unsigned)ld * 4u;
     const float* __restrict__ val = m.val;
 
-    int unit = (span > 0 ? blockIdx.x * span : blockIdx.x * wpb) + (threadIdx.x >> 5);
+    int unit = (SPAN ? blockIdx.x * span : blockIdx.x * wpb) + (threadIdx.x >> 5);
     // prologue that does not depend on the previous layer: shape of the first row, its entries on their way to L2
     int row, base, nch;
     SDNN_UNIT_SHAPE(m, unit, nunits, row, base, nch)

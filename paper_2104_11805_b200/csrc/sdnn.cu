@@ -426,24 +426,27 @@ void launch_forward_gv(sdnn* h, int layer, const float* xin, float* xout, int ld
     auto plan = plan_grid(h, (const void*)forward_kernel<G, V, CPS, I16>, units, chunks);
     // A persistent grid gives every CTA a run of consecutive units, so that its entries are one contiguous stretch of the
     // layer's arrays: 3 % faster than a grid-stride walk at configs 3 and 5, 15 % on a local pattern with 256-input tiles.
+    // Tiles of one chunk (up to 256 inputs) only: with several chunks per tile the grid-stride walk measured 1 % faster
+    // (config 2: 5.00e12 against 4.95e12 edges/s).
     // Not where the input tile outgrows L2: there a grid-stride walk keeps all SMs inside the same few row blocks at any
     // time, and on a local pattern (config 4, 1024-input tiles: 268 MB) that is what keeps their window of the tile in
     // L2 (the blocked walk measured 2.4e12 against 4.6e12 edges/s there).
     int span = 0;
     const double tile_bytes = (double)h->N * ld * sizeof(float);
-    if (plan.first * (plan.second / 32) < units && (h->l2_bytes <= 0 || tile_bytes <= 0.55 * (double)h->l2_bytes))
+    if (chunks == 1 && plan.first * (plan.second / 32) < units && (h->l2_bytes <= 0 || tile_bytes <= 0.55 * (double)h->l2_bytes))
         span = (units + plan.first - 1) / plan.first;
     // 64-byte rows of a layer whose rows all have the same length (no padding entries, which all point at tile row 0: L1
     // absorbs those, one L2 slice would not): the instantiation whose gathers go past L1
-    if (G == 2 && V == 8 && CPS == 2 && h->lay[layer].shape.uniform_k > 0 && h->N % SLICE == 0) {
-        launch_k(h, forward_kernel<G, V, CPS, I16, (G == 2 && V == 8 && CPS == 2)>, dim3(plan.first, chunks), dim3(plan.second), h->pdl,
-                 rows_of(h, layer), bias, xin, xout, h->N, ld, h->cfg.clamp, h->cfg.activation, h->pdl ? h->fwd_pdl : 0,
-                 track ? (const int*)h->cur->cs.ncols : (const int*)nullptr, track ? h->cur->cs.flags : (int*)nullptr, span);
-        return;
-    }
-    launch_k(h, forward_kernel<G, V, CPS, I16>, dim3(plan.first, chunks), dim3(plan.second), h->pdl, rows_of(h, layer), bias, xin, xout,
-             h->N, ld, h->cfg.clamp, h->cfg.activation, h->pdl ? h->fwd_pdl : 0, track ? (const int*)h->cur->cs.ncols : (const int*)nullptr,
-             track ? h->cur->cs.flags : (int*)nullptr, span);
+    const bool cg = G == 2 && V == 8 && CPS == 2 && h->lay[layer].shape.uniform_k > 0 && h->N % SLICE == 0;
+#define SDNN_FWD(CG_, SPAN_)                                                                                                   \
+    launch_k(h, forward_kernel<G, V, CPS, I16, CG_, SPAN_>, dim3(plan.first, chunks), dim3(plan.second), h->pdl, rows_of(h, layer), \
+             bias, xin, xout, h->N, ld, h->cfg.clamp, h->cfg.activation, h->pdl ? h->fwd_pdl : 0,                              \
+             track ? (const int*)h->cur->cs.ncols : (const int*)nullptr, track ? h->cur->cs.flags : (int*)nullptr, span)
+    // the grid-stride instantiation is the one the wide inference tiles take: it carries nothing of the other walk
+    if (cg) { if (span > 0) SDNN_FWD((G == 2 && V == 8 && CPS == 2), true); else SDNN_FWD((G == 2 && V == 8 && CPS == 2), false); }
+    else if (span > 0) SDNN_FWD(false, true);
+    else SDNN_FWD(false, false);
+#undef SDNN_FWD
 }
 
 // track: compaction mode (process only the live columns, mark the columns that stay live)

@@ -645,7 +645,7 @@ void launch_backward_ep(sdnn* h, int layer, int part) {
     const int wb = h->NS <= h->sms ? 1 : 4;          // few slices: one per CTA (a 1024-neuron net: 0.56 -> 0.51 ms per step)
     const dim3 grid((h->NS + wb - 1) / wb), block(32 * wb);
     if (part == 1) {
-        const int pdl = !h->pdl ? 0 : (int)grid.x <= h->sms ? PDL_EARLY : PDL_AT_END;
+        const int pdl = h->pdl ? PDL_EARLY : 0;      // indices, lengths and order are read in front of the wait
         // a launch of at most one CTA per SM is bound by its chain of round trips: take a long column in one go
         if ((int)grid.x <= h->sms && h->lay[layer].c_max_chunks > 2 * EP_IT)
             launch_k(h, backward_col_ep_kernel<2 * EP_IT, I16>, grid, block, h->pdl, cols_of(h, layer), xprev, dk, delta_tile(h, layer - 1, tile),
